@@ -1,0 +1,18 @@
+"""CPU oracle for the tree-verification hot path.
+
+TEST INFRASTRUCTURE ONLY.  This package is the plain, slow, fp64 statement of
+what the four operations compute, written from the paper's definitions.  It
+shares no code with the CUDA path and must never be imported by the product
+package: only the tests, the smoke check and the benchmark's CPU-baseline leg
+may call it.
+"""
+from .jet_oracle import (  # noqa: F401
+    anc_from_parent,
+    bf16_bits_to_f64,
+    gather_paged_prefix,
+    kv_compact_ref,
+    tree_accept_ref,
+    tree_attn_ref,
+    tree_attn_rows_ref,
+    tree_build_ref,
+)
