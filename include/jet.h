@@ -1,0 +1,193 @@
+/*
+ * jet.h -- C ABI of the tree-verification hot path of parallel-tree-drafting
+ * speculative decoding (sm_100a).
+ *
+ * Four operations, in the order one verification step runs them:
+ *
+ *   jet_tree_build        per-depth draft log-probs -> budgeted candidate tree
+ *   jet_tree_verify_attn  attention of all tree nodes over prefix KV + tree KV
+ *                         under the ancestor mask (once per layer)
+ *   jet_tree_accept       greedy acceptance of the deepest matching path
+ *   jet_kv_compact        commit of the accepted path's K/V into the cache
+ *
+ * Conventions shared by every call
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a comment
+ *     says "host".  The library allocates nothing and frees nothing.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *     return; no call synchronises the host with the device.
+ *   - `workspace` is caller-provided device scratch of at least the size the
+ *     matching *_workspace_bytes() query returns, 256-byte aligned.  Its
+ *     contents need not be initialised and are undefined afterwards.  Two calls
+ *     that may overlap on the device must not share a workspace.
+ *   - Argument errors are detected on the host before anything is launched and
+ *     reported as a negative jet_status; outputs are then untouched.
+ *   - B is the node budget INCLUDING the root (1 <= B <= JET_MAX_NODES).
+ *     Node rows v >= n_nodes[b] are padding: parent = depth = token = -1, mask
+ *     row zero, attention output row zero; acceptance ignores them.
+ *   - Ancestor mask: row v has mask_words = ceil(B/32) uint32 words; bit
+ *     (u mod 32) of word (u div 32) is set iff u is v or an ancestor of v.
+ *   - All element offsets are 64-bit.
+ */
+#ifndef JET_H_
+#define JET_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define JET_API __attribute__((visibility("default")))
+#else
+#define JET_API
+#endif
+
+typedef int32_t jet_status;
+
+enum {
+  JET_OK = 0,
+  JET_ERR_INVALID_ARG = -1, /* null pointer, size out of range, bad alignment */
+  JET_ERR_UNSUPPORTED = -2, /* shape outside the compiled instantiations       */
+  JET_ERR_WORKSPACE = -3,   /* workspace null, misaligned or too small         */
+  JET_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed             */
+  JET_ERR_TIMEOUT = -5      /* a bounded device-side wait gave up              */
+};
+
+#define JET_MAX_NODES 512 /* largest node budget B                      */
+#define JET_MAX_WIDTH 32  /* largest branching width W                  */
+#define JET_MAX_DEPTH 64  /* largest draft depth N                      */
+
+/* Human-readable name of a status code (host pointer to a static string). */
+JET_API const char* jet_status_string(jet_status s);
+
+/* ---------------------------------------------------------------------------
+ * jet_tree_build -- Algorithm 1 (Parallel Tree Drafting) with the accumulated
+ * draft log-probability score of Section 3.3, preceded by the per-depth top-W
+ * extraction that Section 3.3 / Appendix E describe.
+ *
+ * For each sequence b: candidates of depth d are the W largest entries of
+ * logp[b,d,:] (ties -> lowest token id, -0.0 == +0.0).  Node 0 is the root
+ * (token root_token[b], score 0, depth 0).  Repeatedly the pending node with
+ * the largest score (ties -> lowest node index) is taken; if its depth is N it
+ * is dropped, otherwise its min(W,V) children are appended in rank order with
+ * score = fl32(score[parent] + logp[b, depth[parent], token]) until the tree
+ * holds B nodes or no node is pending.  Nodes are numbered in creation order,
+ * so parent[v] < v.
+ *
+ *   logp         fp32 [batch, N, V]; element (b,d,t) at
+ *                b*logp_batch_stride + d*logp_depth_stride + t.  No NaN.
+ *   root_token   i32 [batch]
+ *   parent, depth, token   i32 [batch, B] out
+ *   score        fp32 [batch, B] out, may be NULL
+ *   anc_mask     u32 [batch, B, ceil(B/32)] out
+ *   n_nodes      i32 [batch] out
+ * Limits: 1 <= N <= JET_MAX_DEPTH, 1 <= W <= JET_MAX_WIDTH, V >= 1.
+ */
+JET_API size_t jet_tree_build_workspace_bytes(int batch, int N, int V, int W);
+
+JET_API jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride, int64_t logp_depth_stride,
+                          const int32_t* root_token, int batch, int N, int V, int W, int B,
+                          int32_t* parent, int32_t* depth, int32_t* token, float* score,
+                          uint32_t* anc_mask, int32_t* n_nodes, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * jet_tree_verify_attn -- the masked tree attention of Section 3.2 (tree-causal
+ * mask: a node sees the whole prefix, its ancestors and itself), as used by the
+ * one-pass tree verification of Section 3.3 / Appendix E.  One call = one layer.
+ *
+ * For sequence b, node v < n_nodes[b], query head h (KV head g = h / (Hq/Hkv)):
+ *   out[b,v,h,:] = softmax_j( softmax_scale * <q[b,v,h,:], K_j> ) . V_j
+ * over the seq_len[b] prefix keys (all visible) and the tree keys u whose bit
+ * is set in anc_mask[b,v].  bf16 operands, fp32 accumulation, bf16 output.
+ *
+ *   q            bf16 [batch, B, Hq, D]
+ *   k_cache, v_cache
+ *                bf16.  page_table == NULL: contiguous, position j of sequence
+ *                b at element ((b*kv_batch_stride) + j*Hkv*D + g*D).
+ *                page_table != NULL: paged [num_pages, page_size, Hkv, D];
+ *                position j of sequence b is row (j mod page_size) of page
+ *                page_table[b*max_pages_per_seq + j / page_size].
+ *   num_pages    pages in the pool (paged) -- bounds the tensor map; ignored
+ *                when contiguous.
+ *   max_seq_len  host value, >= every seq_len[b]; sizes the grid and, when
+ *                contiguous, bounds the rows per sequence.
+ *   seq_len      i32 [batch] prefix lengths (0 allowed)
+ *   tree_k, tree_v  bf16 [batch, B, Hkv, D]
+ *   out          bf16 [batch, B, Hq, D]
+ *   lse          fp32 [batch, Hq, B] natural-log sum of exp of the visible
+ *                scaled scores; may be NULL.  Padding rows get -inf.
+ *   device_status  i32[1], may be NULL: set to JET_ERR_TIMEOUT if a bounded
+ *                wait inside the kernel expired (outputs are then undefined).
+ * Limits: D in {64,128}; Hq % Hkv == 0 and Hq/Hkv a power of two <= 16;
+ * page_size == 16 when paged; all base pointers 16-byte aligned.
+ */
+JET_API size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
+                                            int max_seq_len);
+
+JET_API jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
+                                const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                const void* tree_k, const void* tree_v, const uint32_t* anc_mask,
+                                const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D,
+                                int64_t kv_batch_stride, float softmax_scale, void* out, float* lse,
+                                int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                void* stream);
+
+/* ---------------------------------------------------------------------------
+ * jet_tree_accept -- greedy acceptance (Section 3.3, Appendix E): a node is
+ * accepted iff its token equals the target's arg-max prediction at its parent;
+ * the deepest fully accepted root-to-node path is selected and the target's
+ * prediction at its last node is the correction token.
+ *
+ *   logits       fp32, row (b*B + v) at logits + (b*B+v)*logits_row_stride,
+ *                V entries.  Arg-max ties -> lowest index.  No NaN.
+ *   token, parent, depth   i32 [batch, B]  (from jet_tree_build)
+ *   anc_mask, n_nodes      as produced by jet_tree_build
+ *   tgt_argmax   i32 [batch, B] out (-1 on padding rows)
+ *   accept_len   i32 [batch] out: a = number of accepted draft nodes (root not
+ *                counted); end node v* = deepest accepted node, ties -> lowest
+ *                index
+ *   path         i32 [batch, N+1] out: node ids root .. v*, then -1
+ *   out_tokens   i32 [batch, N+1] out: the a accepted tokens, then the
+ *                correction token tgt_argmax[v*], then -1
+ */
+JET_API size_t jet_tree_accept_workspace_bytes(int batch, int B, int V);
+
+JET_API jet_status jet_tree_accept(const float* logits, int64_t logits_row_stride, const int32_t* token,
+                           const int32_t* parent, const int32_t* depth, const uint32_t* anc_mask,
+                           const int32_t* n_nodes, int batch, int B, int V, int N,
+                           int32_t* tgt_argmax, int32_t* accept_len, int32_t* path,
+                           int32_t* out_tokens, void* workspace, size_t workspace_bytes,
+                           void* stream);
+
+/* ---------------------------------------------------------------------------
+ * jet_kv_compact -- commit of the accepted path (Appendix E: "the accepted path
+ * is committed"): for every layer l, sequence b and i in [0, accept_len[b]] the
+ * K and V rows of tree node path[b,i] are copied to cache position
+ * seq_len[b] + i (the root's K/V is committed too); afterwards
+ * seq_len[b] += accept_len[b] + 1.  All layers in one call.
+ *
+ *   tree_k, tree_v  bf16 [layers, batch, B, Hkv, D]
+ *   k_cache, v_cache  bf16; layer l starts cache_layer_stride elements after
+ *                layer l-1.  Within a layer the layout is that of
+ *                jet_tree_verify_attn (contiguous with kv_batch_stride, or
+ *                paged when page_table != NULL).
+ *   page_table   i32 [batch, max_pages_per_seq] or NULL.  The pages covering
+ *                positions seq_len[b] .. seq_len[b]+N must already be assigned.
+ *   path         i32 [batch, N+1], accept_len i32 [batch] (from jet_tree_accept)
+ *   seq_len      i32 [batch], read and then updated in place
+ * Every cache byte outside the written rows is left untouched.
+ */
+JET_API jet_status jet_kv_compact(const void* tree_k, const void* tree_v, void* k_cache, void* v_cache,
+                          int64_t cache_layer_stride, int64_t kv_batch_stride,
+                          const int32_t* page_table, int max_pages_per_seq, int page_size,
+                          const int32_t* path, const int32_t* accept_len, int32_t* seq_len,
+                          int layers, int batch, int B, int Hkv, int D, int N, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JET_H_ */

@@ -1,0 +1,25 @@
+"""B200-native tree-verification kernels (tree build, tree attention, acceptance, KV commit).
+
+The product is ``libjet.so`` (C ABI declared in ``include/jet.h``); this package is the
+thin ctypes binding with the same names.  Importing the package does not need a GPU;
+calling an entry point needs the built library and fails loudly without it.
+"""
+from .binding import (  # noqa: F401
+    JET_ERR_CUDA,
+    JET_ERR_INVALID_ARG,
+    JET_ERR_TIMEOUT,
+    JET_ERR_UNSUPPORTED,
+    JET_ERR_WORKSPACE,
+    JET_OK,
+    JetError,
+    exported_symbols,
+    jet_kv_compact,
+    jet_tree_accept,
+    jet_tree_accept_workspace_bytes,
+    jet_tree_build,
+    jet_tree_build_workspace_bytes,
+    jet_tree_verify_attn,
+    jet_tree_verify_attn_workspace_bytes,
+    load,
+    status_string,
+)

@@ -1,0 +1,76 @@
+// jet_kv_compact: commit of the accepted path.  One launch copies the K and V rows of
+// every accepted node of every layer and sequence behind the prefix (contiguous or paged
+// cache); a second one-block launch then advances seq_len, so that no copy block can see
+// an already advanced length.
+#include "jet_common.cuh"
+
+namespace jet {
+namespace {
+
+__global__ void __launch_bounds__(256)
+kv_compact_kernel(const uint4* __restrict__ tree_k, const uint4* __restrict__ tree_v,
+                  uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                  int64_t layer_stride16, int64_t batch_stride16,
+                  const int32_t* __restrict__ page_table, int max_pages, int page_size,
+                  const int32_t* __restrict__ path, const int32_t* __restrict__ accept_len,
+                  const int32_t* __restrict__ seq_len, int batch, int B, int row16, int N) {
+  const int i = blockIdx.x, b = blockIdx.y, layer = blockIdx.z;
+  if (i > accept_len[b]) return;
+  const int node = path[static_cast<size_t>(b) * (N + 1) + i];
+  if (node < 0 || node >= B) return;
+  const int64_t pos = static_cast<int64_t>(seq_len[b]) + i;
+  int64_t dst_row;
+  if (page_table) {
+    const int page = page_table[static_cast<size_t>(b) * max_pages + pos / page_size];
+    dst_row = static_cast<int64_t>(page) * page_size + pos % page_size;
+    dst_row = layer * layer_stride16 + dst_row * row16;
+  } else {
+    dst_row = layer * layer_stride16 + b * batch_stride16 + pos * row16;
+  }
+  const int64_t src = ((static_cast<int64_t>(layer) * batch + b) * B + node) * row16;
+  for (int t = threadIdx.x; t < 2 * row16; t += blockDim.x) {
+    if (t < row16) k_cache[dst_row + t] = tree_k[src + t];
+    else v_cache[dst_row + t - row16] = tree_v[src + t - row16];
+  }
+}
+
+__global__ void advance_seq_len_kernel(const int32_t* __restrict__ accept_len,
+                                       int32_t* __restrict__ seq_len, int batch) {
+  for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < batch; b += gridDim.x * blockDim.x)
+    seq_len[b] += accept_len[b] + 1;
+}
+
+}  // namespace
+}  // namespace jet
+
+extern "C" jet_status jet_kv_compact(const void* tree_k, const void* tree_v, void* k_cache,
+                                     void* v_cache, int64_t cache_layer_stride,
+                                     int64_t kv_batch_stride, const int32_t* page_table,
+                                     int max_pages_per_seq, int page_size, const int32_t* path,
+                                     const int32_t* accept_len, int32_t* seq_len, int layers,
+                                     int batch, int B, int Hkv, int D, int N, void* stream) {
+  using namespace jet;
+  if (!tree_k || !tree_v || !k_cache || !v_cache || !path || !accept_len || !seq_len)
+    return JET_ERR_INVALID_ARG;
+  if (layers < 1 || layers > 65535 || batch < 1 || batch > 65535 || B < 1 || B > JET_MAX_NODES ||
+      Hkv < 1 || D < 1 || N < 1 || N > JET_MAX_DEPTH)
+    return JET_ERR_INVALID_ARG;
+  const int64_t row_elems = static_cast<int64_t>(Hkv) * D;
+  if (row_elems % 8 != 0 || cache_layer_stride % 8 != 0) return JET_ERR_INVALID_ARG;   // 16-byte rows
+  if (!aligned(tree_k, 16) || !aligned(tree_v, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16))
+    return JET_ERR_INVALID_ARG;
+  if (page_table) {
+    if (page_size < 1 || max_pages_per_seq < 1) return JET_ERR_INVALID_ARG;
+  } else if (kv_batch_stride % 8 != 0 || kv_batch_stride < 0) {
+    return JET_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int row16 = static_cast<int>(row_elems / 8);
+  kv_compact_kernel<<<dim3(N + 1, batch, layers), 256, 0, st>>>(
+      static_cast<const uint4*>(tree_k), static_cast<const uint4*>(tree_v),
+      static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), cache_layer_stride / 8,
+      kv_batch_stride / 8, page_table, max_pages_per_seq, page_size, path, accept_len, seq_len,
+      batch, B, row16, N);
+  advance_seq_len_kernel<<<1, 256, 0, st>>>(accept_len, seq_len, batch);
+  return launch_status();
+}

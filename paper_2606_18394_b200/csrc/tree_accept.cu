@@ -1,0 +1,180 @@
+// jet_tree_accept: greedy acceptance of the deepest matching root-to-node path.
+//
+// Two launches:
+//   argmax_partial_kernel  grid (chunks, batch*B rows): the one HBM pass over the target
+//                          logits; each block reduces a slice of one row to a
+//                          (value, lowest index) key in the workspace.  Padding rows are
+//                          not read.
+//   accept_path_kernel     grid (batch), one thread per node: finishes the arg-max,
+//                          builds the match bit-set, tests every node's ancestor mask
+//                          against it, picks the deepest accepted node and writes the
+//                          path and the output tokens.
+#include "jet_common.cuh"
+
+namespace jet {
+namespace {
+
+constexpr int kArgThreads = 256;
+constexpr int kArgElems = 32;
+constexpr int kArgChunk = kArgThreads * kArgElems;
+
+__global__ void __launch_bounds__(kArgThreads)
+argmax_partial_kernel(const float* __restrict__ logits, int64_t row_stride, int V, int B,
+                      const int32_t* __restrict__ n_nodes, int nchunks, bool vec_ok,
+                      unsigned long long* __restrict__ partial) {
+  const int chunk = blockIdx.x;
+  const int row = blockIdx.y;
+  const int b = row / B, v = row - b * B;
+  if (v >= n_nodes[b]) return;
+  const int tid = threadIdx.x;
+  const float* p = logits + static_cast<int64_t>(row) * row_stride;
+  const int base = chunk * kArgChunk;
+
+  float best = 0.0f;
+  uint32_t best_idx = 0xFFFFFFFFu;     // none yet
+  if (vec_ok && base + kArgChunk <= V) {
+    const float4* p4 = reinterpret_cast<const float4*>(p + base);
+    float4 x[kArgElems / 4];
+#pragma unroll
+    for (int i = 0; i < kArgElems / 4; ++i) x[i] = __ldcs(p4 + i * kArgThreads + tid);
+#pragma unroll
+    for (int i = 0; i < kArgElems / 4; ++i) {
+      const uint32_t idx = base + (i * kArgThreads + tid) * 4;     // ascending in i
+      if (best_idx == 0xFFFFFFFFu || x[i].x > best) { best = x[i].x; best_idx = idx; }
+      if (x[i].y > best) { best = x[i].y; best_idx = idx + 1; }
+      if (x[i].z > best) { best = x[i].z; best_idx = idx + 2; }
+      if (x[i].w > best) { best = x[i].w; best_idx = idx + 3; }
+    }
+  } else {
+#pragma unroll 4
+    for (int i = 0; i < kArgElems; ++i) {
+      const int idx = base + i * kArgThreads + tid;
+      if (idx < V) {
+        const float x = __ldcs(p + idx);
+        if (best_idx == 0xFFFFFFFFu || x > best) { best = x; best_idx = idx; }
+      }
+    }
+  }
+  unsigned long long key = best_idx == 0xFFFFFFFFu ? 0ull : make_key(best, best_idx);
+  key = warp_max_u64(key);
+  __shared__ unsigned long long warp_best[kArgThreads / 32];
+  if ((tid & 31) == 0) warp_best[tid >> 5] = key;
+  __syncthreads();
+  if (tid < 32) {
+    unsigned long long w = tid < kArgThreads / 32 ? warp_best[tid] : 0ull;
+    w = warp_max_u64(w);
+    if (tid == 0) partial[static_cast<size_t>(row) * nchunks + chunk] = w;
+  }
+}
+
+__global__ void __launch_bounds__(JET_MAX_NODES)
+accept_path_kernel(const unsigned long long* __restrict__ partial, int nchunks,
+                   const int32_t* __restrict__ token, const int32_t* __restrict__ parent,
+                   const int32_t* __restrict__ depth, const uint32_t* __restrict__ anc_mask,
+                   const int32_t* __restrict__ n_nodes, int B, int N,
+                   int32_t* __restrict__ tgt_out, int32_t* __restrict__ accept_len,
+                   int32_t* __restrict__ path, int32_t* __restrict__ out_tokens) {
+  __shared__ int32_t s_tgt[JET_MAX_NODES];
+  __shared__ uint32_t s_match[JET_MAX_NODES / 32];
+  __shared__ uint32_t s_best[JET_MAX_NODES / 32];
+  __shared__ uint32_t s_end_row[JET_MAX_NODES / 32];
+  __shared__ int s_end;
+
+  const int b = blockIdx.x, v = threadIdx.x, lane = v & 31, warp = v >> 5;
+  const int n = n_nodes[b];
+  const int words = (B + 31) / 32;
+  const size_t o = static_cast<size_t>(b) * B;
+  const bool live = v < n;              // blockDim.x >= B, n <= B
+
+  int32_t tgt = -1;
+  if (live) {
+    unsigned long long k = 0ull;
+    const unsigned long long* pr = partial + (o + v) * nchunks;
+    for (int c = 0; c < nchunks; ++c) { const unsigned long long x = pr[c]; k = x > k ? x : k; }
+    tgt = static_cast<int32_t>(key_index(k));
+  }
+  s_tgt[v] = tgt;
+  if (v < B) tgt_out[o + v] = tgt;
+  __syncthreads();
+
+  // match[v]: the root always matches; other nodes iff token == target prediction at the parent
+  int my_parent = -1, my_depth = -1, my_token = -1;
+  if (live) { my_parent = parent[o + v]; my_depth = depth[o + v]; my_token = token[o + v]; }
+  const bool match = live && (v == 0 || (my_parent >= 0 && my_parent < n && my_token == s_tgt[my_parent]));
+  const uint32_t mbits = __ballot_sync(0xffffffffu, match);
+  if (lane == 0) s_match[warp] = mbits;
+  __syncthreads();
+
+  // accepted iff every node of Anc(v)+{v} matches
+  bool acc = live;
+  if (live) {
+    const uint32_t* row = anc_mask + (o + v) * words;
+    for (int w = 0; w < words; ++w) acc = acc && ((row[w] & ~s_match[w]) == 0u);
+  }
+  // deepest accepted node, ties -> lowest index
+  uint32_t key = acc ? ((static_cast<uint32_t>(my_depth) << 16) | (0xFFFFu - v)) : 0u;
+  key = __reduce_max_sync(0xffffffffu, key);
+  if (lane == 0) s_best[warp] = key;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t k = lane < blockDim.x / 32 ? s_best[lane] : 0u;
+    k = __reduce_max_sync(0xffffffffu, k);
+    if (lane == 0) s_end = k ? static_cast<int>(0xFFFFu - (k & 0xFFFFu)) : 0;
+  }
+  __syncthreads();
+  const int end = s_end;
+  if (v < words) s_end_row[v] = anc_mask[(o + end) * words + v];
+  __syncthreads();
+
+  const int a = s_tgt[end] >= 0 ? depth[o + end] : 0;
+  int32_t* my_path = path + static_cast<size_t>(b) * (N + 1);
+  int32_t* my_tok = out_tokens + static_cast<size_t>(b) * (N + 1);
+  for (int i = v; i <= N; i += blockDim.x)
+    if (i > a) { my_path[i] = -1; my_tok[i] = -1; }
+  if (live && ((s_end_row[v >> 5] >> (v & 31)) & 1u) && my_depth <= N) {
+    my_path[my_depth] = v;
+    if (my_depth >= 1) my_tok[my_depth - 1] = my_token;
+  }
+  if (v == 0) { accept_len[b] = a; my_tok[a] = s_tgt[end]; }
+}
+
+int chunks_for(int V) { return (V + kArgChunk - 1) / kArgChunk; }
+
+}  // namespace
+}  // namespace jet
+
+extern "C" size_t jet_tree_accept_workspace_bytes(int batch, int B, int V) {
+  if (batch < 1 || B < 1 || V < 1) return 0;
+  return jet::round_up(static_cast<size_t>(batch) * B * jet::chunks_for(V) * sizeof(unsigned long long), 256);
+}
+
+extern "C" jet_status jet_tree_accept(const float* logits, int64_t logits_row_stride,
+                                      const int32_t* token, const int32_t* parent,
+                                      const int32_t* depth, const uint32_t* anc_mask,
+                                      const int32_t* n_nodes, int batch, int B, int V, int N,
+                                      int32_t* tgt_argmax, int32_t* accept_len, int32_t* path,
+                                      int32_t* out_tokens, void* workspace, size_t workspace_bytes,
+                                      void* stream) {
+  using namespace jet;
+  if (!logits || !token || !parent || !depth || !anc_mask || !n_nodes || !tgt_argmax || !accept_len ||
+      !path || !out_tokens)
+    return JET_ERR_INVALID_ARG;
+  if (batch < 1 || B < 1 || B > JET_MAX_NODES || V < 1 || N < 1 || N > JET_MAX_DEPTH ||
+      logits_row_stride < V || static_cast<int64_t>(batch) * B > 65535)
+    return JET_ERR_INVALID_ARG;
+  if (!aligned(logits, 4)) return JET_ERR_INVALID_ARG;
+  const size_t need = jet_tree_accept_workspace_bytes(batch, B, V);
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
+
+  const int nchunks = chunks_for(V);
+  const bool vec_ok = aligned(logits, 16) && logits_row_stride % 4 == 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  auto* partial = static_cast<unsigned long long*>(workspace);
+  argmax_partial_kernel<<<dim3(nchunks, batch * B), kArgThreads, 0, st>>>(
+      logits, logits_row_stride, V, B, n_nodes, nchunks, vec_ok, partial);
+  const int threads = (B + 31) / 32 * 32;
+  accept_path_kernel<<<batch, threads, 0, st>>>(partial, nchunks, token, parent, depth, anc_mask,
+                                                 n_nodes, B, N, tgt_argmax, accept_len, path,
+                                                 out_tokens);
+  return launch_status();
+}

@@ -1,0 +1,209 @@
+// jet_tree_build: per-depth top-W extraction followed by Algorithm 1 (best-first
+// budgeted tree construction with the accumulated log-probability score).
+//
+// Two launches:
+//   topw_partial_kernel  grid (chunks, N, batch): every block scans one slice of one
+//                        vocabulary row and leaves its W best (value, token) keys in
+//                        the workspace -- the only pass over the [N,V] log-probs.
+//   tree_expand_kernel   grid (batch): merges the per-slice candidates, runs the
+//                        sequential pop/expand loop in one warp with the pending
+//                        queue held in shared memory, then emits parent / depth /
+//                        token / score / ancestor bitmask.
+#include "jet_common.cuh"
+
+namespace jet {
+namespace {
+
+constexpr int kTopThreads = 256;
+constexpr int kTopElems = 16;                        // elements per thread
+constexpr int kTopChunk = kTopThreads * kTopElems;   // vocabulary slice per block
+
+__global__ void __launch_bounds__(kTopThreads)
+topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
+                    int V, int Wc, int nchunks, bool vec_ok,
+                    unsigned long long* __restrict__ cand) {
+  const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x;
+  const float* row = logp + b * batch_stride + d * depth_stride;
+  const int base = chunk * kTopChunk;
+
+  unsigned long long keys[kTopElems];
+  if (vec_ok && base + kTopChunk <= V) {
+    const float4* row4 = reinterpret_cast<const float4*>(row + base);
+#pragma unroll
+    for (int i = 0; i < kTopElems / 4; ++i) {
+      float4 x = __ldg(row4 + i * kTopThreads + tid);
+      const uint32_t idx = base + (i * kTopThreads + tid) * 4;
+      keys[i * 4 + 0] = make_key(x.x, idx + 0);
+      keys[i * 4 + 1] = make_key(x.y, idx + 1);
+      keys[i * 4 + 2] = make_key(x.z, idx + 2);
+      keys[i * 4 + 3] = make_key(x.w, idx + 3);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < kTopElems; ++i) {
+      const int idx = base + i * kTopThreads + tid;
+      keys[i] = idx < V ? make_key(__ldg(row + idx), idx) : 0ull;
+    }
+  }
+
+  __shared__ unsigned long long warp_best[kTopThreads / 32];
+  __shared__ unsigned long long winner;
+  unsigned long long* out = cand + ((static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk) * Wc;
+  for (int r = 0; r < Wc; ++r) {
+    unsigned long long best = 0ull;
+#pragma unroll
+    for (int i = 0; i < kTopElems; ++i) best = keys[i] > best ? keys[i] : best;
+    best = warp_max_u64(best);
+    if ((tid & 31) == 0) warp_best[tid >> 5] = best;
+    __syncthreads();
+    if (tid < 32) {
+      unsigned long long w = tid < kTopThreads / 32 ? warp_best[tid] : 0ull;
+      w = warp_max_u64(w);
+      if (tid == 0) { winner = w; out[r] = w; }
+    }
+    __syncthreads();
+    const unsigned long long w = winner;
+#pragma unroll
+    for (int i = 0; i < kTopElems; ++i) if (keys[i] == w) keys[i] = 0ull;   // keys are unique
+  }
+}
+
+constexpr int kExpThreads = 256;
+
+__global__ void __launch_bounds__(kExpThreads)
+tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
+                   const int32_t* __restrict__ root_token, int N, int Wc, int B, int nchunks,
+                   const unsigned long long* __restrict__ cand,
+                   int32_t* __restrict__ parent_out, int32_t* __restrict__ depth_out,
+                   int32_t* __restrict__ token_out, float* __restrict__ score_out,
+                   uint32_t* __restrict__ anc_out, int32_t* __restrict__ n_nodes_out) {
+  __shared__ int32_t s_top_tok[JET_MAX_DEPTH][JET_MAX_WIDTH];
+  __shared__ float s_top_lp[JET_MAX_DEPTH][JET_MAX_WIDTH];
+  __shared__ int32_t s_parent[JET_MAX_NODES], s_depth[JET_MAX_NODES], s_token[JET_MAX_NODES];
+  __shared__ float s_score[JET_MAX_NODES];
+  __shared__ unsigned long long s_qkey[JET_MAX_NODES];
+  __shared__ int s_n;
+
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* lp = logp + b * batch_stride;
+
+  // ---- merge the per-slice candidates: depth d's W best of nchunks*Wc keys (keys are unique,
+  //      so "largest key below the previous winner" walks them in rank order)
+  for (int d = warp; d < N; d += kExpThreads / 32) {
+    const unsigned long long* c = cand + (static_cast<size_t>(b) * N + d) * nchunks * Wc;
+    const int total = nchunks * Wc;
+    unsigned long long prev = ~0ull;
+    for (int r = 0; r < Wc; ++r) {
+      unsigned long long best = 0ull;
+      for (int i = lane; i < total; i += 32) {
+        const unsigned long long k = c[i];
+        if (k < prev && k > best) best = k;
+      }
+      best = warp_max_u64(best);
+      if (lane == 0) {
+        const uint32_t t = key_index(best);
+        s_top_tok[d][r] = static_cast<int32_t>(t);
+        s_top_lp[d][r] = lp[d * depth_stride + t];   // the stored bits, not the canonicalised key
+      }
+      prev = best;
+    }
+  }
+  __syncthreads();
+
+  // ---- Algorithm 1: one warp, pending queue = keys (score, lowest index first) in shared memory
+  if (warp == 0) {
+    if (lane == 0) {
+      s_parent[0] = -1; s_depth[0] = 0; s_token[0] = root_token[b]; s_score[0] = 0.0f;
+      s_qkey[0] = make_key(0.0f, 0);
+    }
+    __syncwarp();
+    int n = 1;
+    while (n < B) {
+      unsigned long long best = 0ull;
+      for (int i = lane; i < n; i += 32) { const unsigned long long k = s_qkey[i]; best = k > best ? k : best; }
+      best = warp_max_u64(best);
+      if (best == 0ull) break;                        // nothing pending
+      const int v = static_cast<int>(key_index(best));
+      const int d = s_depth[v];
+      const float sv = s_score[v];
+      __syncwarp();
+      if (lane == 0) s_qkey[v] = 0ull;                // popped
+      if (d < N) {
+        const int cnt = min(Wc, B - n);
+        if (lane < cnt) {
+          const int u = n + lane;
+          const float s = __fadd_rn(sv, s_top_lp[d][lane]);
+          s_parent[u] = v; s_depth[u] = d + 1; s_token[u] = s_top_tok[d][lane]; s_score[u] = s;
+          s_qkey[u] = make_key(s, u);
+        }
+        n += cnt;
+      }
+      __syncwarp();
+    }
+    if (lane == 0) s_n = n;
+  }
+  __syncthreads();
+
+  // ---- emit
+  const int n = s_n;
+  const size_t o = static_cast<size_t>(b) * B;
+  for (int v = tid; v < B; v += kExpThreads) {
+    const bool live = v < n;
+    parent_out[o + v] = live ? s_parent[v] : -1;
+    depth_out[o + v] = live ? s_depth[v] : -1;
+    token_out[o + v] = live ? s_token[v] : -1;
+    if (score_out) score_out[o + v] = live ? s_score[v] : 0.0f;
+  }
+  if (tid == 0) n_nodes_out[b] = n;
+  const int words = (B + 31) / 32;
+  for (int i = tid; i < B * words; i += kExpThreads) {
+    const int v = i / words, w = i - v * words;
+    uint32_t bits = 0u;
+    if (v < n) {
+      for (int u = v; u >= 0; u = s_parent[u])
+        if ((u >> 5) == w) bits |= 1u << (u & 31);
+    }
+    anc_out[o * words + i] = bits;
+  }
+}
+
+int chunks_for(int V) { return (V + kTopChunk - 1) / kTopChunk; }
+
+}  // namespace
+}  // namespace jet
+
+extern "C" size_t jet_tree_build_workspace_bytes(int batch, int N, int V, int W) {
+  if (batch < 1 || N < 1 || V < 1 || W < 1) return 0;
+  const size_t Wc = static_cast<size_t>(W < V ? W : V);
+  return jet::round_up(static_cast<size_t>(batch) * N * jet::chunks_for(V) * Wc * sizeof(unsigned long long), 256);
+}
+
+extern "C" jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride,
+                                     int64_t logp_depth_stride, const int32_t* root_token,
+                                     int batch, int N, int V, int W, int B, int32_t* parent,
+                                     int32_t* depth, int32_t* token, float* score,
+                                     uint32_t* anc_mask, int32_t* n_nodes, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+  using namespace jet;
+  if (!logp || !root_token || !parent || !depth || !token || !anc_mask || !n_nodes)
+    return JET_ERR_INVALID_ARG;
+  if (batch < 1 || batch > 65535 || N < 1 || N > JET_MAX_DEPTH || W < 1 || W > JET_MAX_WIDTH || V < 1 ||
+      B < 1 || B > JET_MAX_NODES || logp_depth_stride < V || logp_batch_stride < 0)
+    return JET_ERR_INVALID_ARG;
+  if (!aligned(logp, 4)) return JET_ERR_INVALID_ARG;
+  const size_t need = jet_tree_build_workspace_bytes(batch, N, V, W);
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
+
+  const int Wc = W < V ? W : V;
+  const int nchunks = chunks_for(V);
+  const bool vec_ok = aligned(logp, 16) && logp_batch_stride % 4 == 0 && logp_depth_stride % 4 == 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  auto* cand = static_cast<unsigned long long*>(workspace);
+  topw_partial_kernel<<<dim3(nchunks, N, batch), kTopThreads, 0, st>>>(
+      logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand);
+  tree_expand_kernel<<<batch, kExpThreads, 0, st>>>(logp, logp_batch_stride, logp_depth_stride,
+                                                     root_token, N, Wc, B, nchunks, cand, parent,
+                                                     depth, token, score, anc_mask, n_nodes);
+  return launch_status();
+}

@@ -1,0 +1,89 @@
+"""Test-side helpers: run the C-ABI entry points on numpy inputs (device memory via torch)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2606_18394_b200 as jet
+
+DEV = "cuda:0"
+
+
+def dev(x, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.to(DEV)
+
+
+def dev_bf16(bits):
+    """uint16 bit patterns -> device bf16 tensor with the same bits."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(DEV).view(torch.bfloat16)
+
+
+def bf16_to_f64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def workspace(nbytes):
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=DEV)
+
+
+def run_tree_build(logp, root_token, N, W, B, with_score=True):
+    """logp [batch,N,V] fp32 numpy; returns dict of numpy arrays."""
+    batch, _, V = logp.shape
+    d_logp = dev(logp)
+    d_root = dev(np.asarray(root_token, dtype=np.int32))
+    words = (B + 31) // 32
+    parent = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
+    depth = torch.full_like(parent, -7)
+    token = torch.full_like(parent, -7)
+    score = torch.full((batch, B), 123.0, dtype=torch.float32, device=DEV) if with_score else None
+    anc = torch.full((batch, B, words), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
+    n_nodes = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
+    ws = workspace(jet.jet_tree_build_workspace_bytes(batch, N, V, W))
+    jet.jet_tree_build(d_logp, d_root, batch, N, V, W, B, parent, depth, token, score, anc, n_nodes, ws)
+    torch.cuda.synchronize()
+    return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
+                score=score.cpu().numpy() if with_score else None,
+                anc_mask=anc.cpu().numpy().view(np.uint32), n_nodes=n_nodes.cpu().numpy())
+
+
+def run_tree_accept(logits, token, parent, depth, anc_mask, n_nodes, N):
+    """logits [batch,B,V]; tree arrays [batch,B]; returns dict of numpy arrays."""
+    batch, B, V = logits.shape
+    d_logits = dev(logits)
+    tgt = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
+    acc = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
+    path = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
+    toks = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
+    ws = workspace(jet.jet_tree_accept_workspace_bytes(batch, B, V))
+    jet.jet_tree_accept(d_logits, V, dev(token.astype(np.int32)), dev(parent.astype(np.int32)),
+                        dev(depth.astype(np.int32)), dev(anc_mask.view(np.int32)),
+                        dev(np.asarray(n_nodes, dtype=np.int32)), batch, B, V, N, tgt, acc, path, toks, ws)
+    torch.cuda.synchronize()
+    return dict(tgt=tgt.cpu().numpy(), accept_len=acc.cpu().numpy(), path=path.cpu().numpy(),
+                out_tokens=toks.cpu().numpy())
+
+
+def run_kv_compact(tree_k, tree_v, k_cache, v_cache, page_table, path, accept_len, seq_len, N):
+    """bf16-bit numpy arrays laid out as the oracle's kv_compact_ref takes them."""
+    layers, batch, B, Hkv, D = tree_k.shape
+    dk, dv = dev(k_cache.view(np.int16)), dev(v_cache.view(np.int16))
+    d_seq = dev(np.asarray(seq_len, dtype=np.int32))
+    if page_table is None:
+        Lmax = k_cache.shape[2]
+        layer_stride = batch * Lmax * Hkv * D
+        batch_stride = Lmax * Hkv * D
+        pt, max_pages, page_size = None, 0, 0
+    else:
+        num_pages, page_size = k_cache.shape[1], k_cache.shape[2]
+        layer_stride = num_pages * page_size * Hkv * D
+        batch_stride = 0
+        pt = dev(page_table.astype(np.int32))
+        max_pages = page_table.shape[1]
+    jet.jet_kv_compact(dev(tree_k.view(np.int16)), dev(tree_v.view(np.int16)), dk, dv, layer_stride,
+                       batch_stride, pt, max_pages, page_size, dev(path.astype(np.int32)),
+                       dev(np.asarray(accept_len, dtype=np.int32)), d_seq, layers, batch, B, Hkv, D, N)
+    torch.cuda.synchronize()
+    return (dk.cpu().numpy().view(np.uint16), dv.cpu().numpy().view(np.uint16), d_seq.cpu().numpy())

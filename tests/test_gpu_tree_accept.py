@@ -1,0 +1,100 @@
+"""GPU parity: jet_tree_accept against the oracle, bit-exact."""
+import numpy as np
+import pytest
+
+from jet_inputs import (CONFIGS, chain_tree, make_logp, make_target_logits, plant_path, random_tree,
+                        star_tree)
+from oracle import anc_from_parent, tree_accept_ref, tree_build_ref
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare(logits, token, parent, depth, anc, n_nodes, N):
+    import jet_harness as H
+    got = H.run_tree_accept(logits, token, parent, depth, anc, n_nodes, N)
+    for b in range(logits.shape[0]):
+        ref = tree_accept_ref(logits[b], token[b], parent[b], depth[b], int(n_nodes[b]), N)
+        assert np.array_equal(got["tgt"][b], ref["tgt"]), b
+        assert got["accept_len"][b] == ref["accept_len"], (b, got["accept_len"][b], ref["accept_len"])
+        assert np.array_equal(got["path"][b], ref["path"]), (b, got["path"][b], ref["path"])
+        assert np.array_equal(got["out_tokens"][b], ref["out_tokens"]), b
+    return got
+
+
+def _built(rng, batch, N, W, B, V, sigma, peaked=0.7):
+    trees = [tree_build_ref(make_logp(rng, N, V, sigma, peaked_p=peaked), 1, N, W, B) for _ in range(batch)]
+    stack = lambda k: np.stack([t[k] for t in trees])
+    return stack("token"), stack("parent"), stack("depth"), stack("anc_mask"), np.array([t["n_nodes"] for t in trees])
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_tiny_config_planted(seed):
+    c = CONFIGS["tiny"]
+    rng = np.random.default_rng(1000 + seed)
+    token, parent, depth, anc, n = _built(rng, 1, c["N"], c["W"], c["B"], c["V"], c["sigma_draft"])
+    logits = make_target_logits(rng, c["B"], c["V"], c["sigma_target"])[None]
+    end, eff = plant_path(logits[0], token[0], parent[0], depth[0], int(n[0]), c["plant"], rng)
+    got = _compare(logits, token, parent, depth, anc, n, c["N"])
+    assert got["accept_len"][0] == eff
+
+
+@pytest.mark.parametrize("plant", [0, 5, 8])
+def test_qwen3_8b_config_planted(plant):
+    c = CONFIGS["qwen3_8b"]
+    rng = np.random.default_rng(2000 + plant)
+    token, parent, depth, anc, n = _built(rng, 1, c["N"], c["W"], c["B"], c["V"], c["sigma_draft"])
+    logits = make_target_logits(rng, c["B"], c["V"], c["sigma_target"])[None]
+    end, eff = plant_path(logits[0], token[0], parent[0], depth[0], int(n[0]), plant, rng)
+    got = _compare(logits, token, parent, depth, anc, n, c["N"])
+    assert got["accept_len"][0] == eff == min(plant, depth[0].max())
+
+
+def test_batched_ragged_plants_and_padding():
+    rng = np.random.default_rng(4000)
+    batch, N, W, B, V = 6, 8, 7, 64, 20011
+    token, parent, depth, anc, n = _built(rng, batch, N, W, B, V, 3.0)
+    # shrink two trees so that they carry padding rows
+    for b, keep in ((1, 40), (4, 1)):
+        n[b] = keep
+        token[b, keep:] = parent[b, keep:] = depth[b, keep:] = -1
+        anc[b, keep:] = 0
+    logits = np.stack([make_target_logits(rng, B, V, 2.0) for _ in range(batch)])
+    for b in range(batch):
+        plant_path(logits[b], token[b], parent[b], depth[b], int(n[b]), int(rng.integers(1, 9)), rng)
+    _compare(logits, token, parent, depth, anc, n, N)
+
+
+@pytest.mark.parametrize("B,V", [(1, 1), (2, 5), (33, 8191), (512, 300), (100, 8193), (31, 16385)])
+def test_random_trees_small_vocab_many_matches(B, V):
+    rng = np.random.default_rng(B * 7 + V)
+    N = 12
+    parent, depth, token = random_tree(B, rng, V=min(V, 4), max_depth=N)
+    anc = anc_from_parent(parent, B, B)
+    logits = make_target_logits(rng, B, V, 1.0)
+    logits[:, : min(V, 4)] += 6.0                    # predictions fall in the small token range
+    _compare(logits[None], token[None], parent[None], depth[None], anc[None], np.array([B]), N)
+
+
+def test_argmax_ties_take_lowest_index_across_slices():
+    B, V, N = 4, 40000, 3
+    parent, depth, token = chain_tree(B)
+    logits = np.zeros((1, B, V), dtype=np.float32)             # all equal -> index 0
+    logits[0, 1, [39999, 123, 20000]] = 2.0                    # equal maxima in three slices -> 123
+    logits[0, 2, [8192, 8191]] = [1.0, 1.0]
+    logits[0, 3, :] = -np.inf
+    token = np.array([9, 0, 123, 8191], dtype=np.int32)
+    anc = anc_from_parent(parent, B, B)
+    got = _compare(logits, token[None], parent[None], depth[None], anc[None], np.array([B]), N)
+    assert got["tgt"][0].tolist() == [0, 123, 8191, 0]
+    assert got["accept_len"][0] == 3
+
+
+def test_star_and_duplicate_sibling_tokens():
+    B, V, N = 9, 50, 2
+    parent, depth, token = star_tree(B)
+    token = np.array([0, 7, 7, 7, 3, 3, 1, 2, 4], dtype=np.int32)
+    logits = make_target_logits(np.random.default_rng(1), B, V, 1.0)
+    logits[0, 7] = 50.0
+    anc = anc_from_parent(parent, B, B)
+    got = _compare(logits[None], token[None], parent[None], depth[None], anc[None], np.array([B]), N)
+    assert got["path"][0].tolist() == [0, 1, -1]
