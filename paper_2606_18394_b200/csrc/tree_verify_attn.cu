@@ -1,8 +1,747 @@
+// jet_tree_verify_attn: tree attention over prefix KV + tree KV under the ancestor mask.
+//
+// Kernel structure (one CTA per SM, warp-specialised):
+//   work item   = (sequence b, KV head g, group of MT 128-row query tiles, key split s).
+//                 Row r of a query tile is (node v, query head g*G + j) with r = v_local*G + j,
+//                 so all G heads of a KV group share every K/V tile that is loaded.
+//   warp 0      = TMA producer: Q tiles once, then K and V tiles (128 keys) through a ring of
+//                 shared-memory stages; paged caches are fetched one 16-row page per TMA box.
+//   warp 1      = tcgen05 issuer: S = Q K^T into TMEM, later O += P V into TMEM.
+//   warp 2      = TMEM allocation / release.
+//   warps 4..   = one softmax warpgroup per query tile, one thread per row: reads S from TMEM,
+//                 applies the key-validity / ancestor-bit mask, keeps the running maximum and sum
+//                 (online softmax with lazy rescaling of O), writes P (bf16) to shared memory in
+//                 the swizzled operand layout, and finally normalises O.
+//   Split-KV    = when there are fewer work items than SMs the key range is cut into `nsplit`
+//                 slices; each CTA then writes a normalised fp32 partial + log-sum-exp to the
+//                 workspace and tree_attn_merge_kernel combines the slices.
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
+// loops, outstanding TMA loads are drained, TMEM is released and JET_ERR_TIMEOUT is reported.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 #include "jet_common.cuh"
-extern "C" size_t jet_tree_verify_attn_workspace_bytes(int, int, int, int, int, int) { return 256; }
-extern "C" jet_status jet_tree_verify_attn(const void*, const void*, const void*, const int32_t*, int, int,
-                                           int64_t, const int32_t*, int, const void*, const void*,
-                                           const uint32_t*, const int32_t*, int, int, int, int, int,
-                                           int64_t, float, void*, float*, int32_t*, void*, size_t, void*) {
-  return JET_ERR_UNSUPPORTED;
+#include "sm100_ptx.cuh"
+
+namespace jet {
+namespace {
+
+constexpr int kBM = 128;             // query rows per tile
+constexpr int kBN = 128;             // keys per tile
+constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more
+
+struct AttnParams {
+  const int32_t* page_table;
+  const int32_t* seq_len;
+  const int32_t* n_nodes;
+  const uint32_t* anc_mask;
+  __nv_bfloat16* out;
+  float* lse;
+  int32_t* status;
+  float* part_o;
+  float* part_lse;
+  int max_pages, paged;
+  int batch, B, Hq, Hkv, G, words;
+  int nsplit, n_mgroups;
+  float scale_log2;   // softmax_scale * log2(e)
+};
+
+template <int D, int MT>
+struct Cfg {
+  static constexpr int kHalves = D / 64;
+  static constexpr int kQBytes = MT * kHalves * kHalfBytes;
+  static constexpr int kPBytes = MT * 2 * kHalfBytes;
+  static constexpr int kStageBytes = kHalves * kHalfBytes;
+  static constexpr int kStages = (D == 128) ? (MT == 1 ? 4 : 3) : 6;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kSmemBytes = kQBytes + kPBytes + kStages * kStageBytes + kBarBytes + 1024;
+  static constexpr int kThreads = 128 + 128 * MT;
+  static constexpr int kTmemCols = (MT == 1) ? 256 : 512;   // per query tile: S (128) + O (<=128)
+};
+
+struct Bars {       // offsets (in 8-byte units) inside the barrier block
+  enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
+         kCount = 21 };
+};
+
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  bool ok = false;
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (ptx::mbar_test(bar, parity)) { ok = true; break; }
+    if ((i & 1023u) == 1023u && *abort_flag) break;
+  }
+  if (!ok) *abort_flag = 1u;
+  return __all_sync(0xffffffffu, ok);
+}
+
+template <int D, int MT>
+__global__ void __launch_bounds__(Cfg<D, MT>::kThreads, 1)
+tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tk,
+                 const __grid_constant__ CUtensorMap tm_tv, const AttnParams p) {
+  using C = Cfg<D, MT>;
+  constexpr int kHalves = C::kHalves;
+  constexpr int kStages = C::kStages;
+
+  // ---------------- work item
+  const int split = blockIdx.x % p.nsplit;
+  const int unit = blockIdx.x / p.nsplit;
+  const int mgroup = unit % p.n_mgroups;
+  const int bg = unit / p.n_mgroups;
+  const int g = bg % p.Hkv;
+  const int b = bg / p.Hkv;
+  const int G = p.G;
+  const int npt = kBM / G;                       // nodes per query tile
+  const int L = p.seq_len[b];
+  const int n = min(p.n_nodes[b], p.B);
+  const int node_lo = mgroup * MT * npt;
+  const int node_hi = min(p.B, node_lo + MT * npt);
+  const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const int ntree = min(n, node_hi);                         // tree keys any row here can see
+  const int TP = (L + kBN - 1) / kBN;
+  const int TT = (ntree + kBN - 1) / kBN;
+  const int T_all = TP + TT;
+  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split) / p.nsplit);
+  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1)) / p.nsplit);
+  const int T = t_hi - t_lo;
+
+  float* part_o = p.part_o + (static_cast<size_t>(unit) * p.nsplit + split) * MT * kBM * D;
+  float* part_lse = p.part_lse + (static_cast<size_t>(unit) * p.nsplit + split) * MT * kBM;
+
+  if (node_lo >= n || T == 0) {
+    // No live node in this CTA, or an empty key slice (uniform for the whole CTA).
+    if (p.nsplit == 1) {
+      for (int i = tid; i < (node_hi - node_lo) * G * (D / 8); i += C::kThreads) {
+        const int row = i / (D / 8), c8 = i - row * (D / 8);
+        const int v = node_lo + row / G, h = g * G + row % G;
+        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+            make_uint4(0u, 0u, 0u, 0u);
+        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = -INFINITY;
+      }
+    } else {
+      for (int i = tid; i < MT * kBM; i += C::kThreads) part_lse[i] = -INFINITY;
+    }
+    return;
+  }
+
+  // ---------------- shared memory carve-up (1024-byte aligned for the 128-byte swizzle)
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+  const uint32_t sQ = smem_base;
+  const uint32_t sP = sQ + C::kQBytes;
+  const uint32_t sKV = sP + C::kPBytes;
+  const uint32_t sBar = sKV + kStages * C::kStageBytes;
+  uint8_t* gen_kv = smem_gen + C::kQBytes + C::kPBytes;
+  uint8_t* gen_p = smem_gen + C::kQBytes;
+  uint8_t* gen_bar = gen_kv + kStages * C::kStageBytes;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + Bars::kCount * 8);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  auto bar = [&](int idx) { return sBar + 8u * idx; };
+
+  if (tid == 0) {
+    ptx::mbar_init(bar(Bars::kQFull), 1);
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(bar(Bars::kKvFull + s), 1);
+      ptx::mbar_init(bar(Bars::kKvEmpty + s), 1);
+    }
+    for (int mt = 0; mt < MT; ++mt) {
+      ptx::mbar_init(bar(Bars::kSFull + mt), 1);
+      ptx::mbar_init(bar(Bars::kSFree + mt), 128);
+      ptx::mbar_init(bar(Bars::kPFull + mt), 128);
+      ptx::mbar_init(bar(Bars::kODone + mt), 1);
+    }
+    *abort_flag = 0u;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_q);
+    ptx::prefetch_tmap(&tm_k);
+    ptx::prefetch_tmap(&tm_v);
+    ptx::prefetch_tmap(&tm_tk);
+    ptx::prefetch_tmap(&tm_tv);
+  }
+  if (warp == 2) {
+    ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: query tile mt owns [mt*256, mt*256+128) for S and [mt*256+128, mt*256+128+D) for O.
+
+  // Valid keys of tile t (global tile index): prefix tiles first, then tree tiles.
+  auto tile_valid = [&](int t) { return t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN); };
+
+  if (warp == 0) {
+    // =========================================================== TMA producer
+    if (lane == 0) {
+      ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
+      for (int mt = 0; mt < n_mt; ++mt)
+        for (int h = 0; h < kHalves; ++h)
+          ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
+                           b * p.B + node_lo + mt * npt);
+    }
+    int issued = 0;
+    bool ok = true;
+    for (int t = t_lo; t < t_hi && ok; ++t) {
+      for (int kv = 0; kv < 2 && ok; ++kv) {
+        const int stage = issued % kStages;
+        if (issued >= kStages)
+          ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t dst = sKV + stage * C::kStageBytes;
+        const uint32_t full = bar(Bars::kKvFull + stage);
+        if (t < TP) {
+          if (!p.paged) {
+            if (lane == 0) {
+              ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+              for (int h = 0; h < kHalves; ++h)
+                ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v : &tm_k, full, h * 64, g, t * kBN, b);
+            }
+          } else {
+            const int npages = min(8, (L - t * kBN + 15) / 16);
+            if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
+            __syncwarp();
+            if (lane < npages) {
+              const int page = p.page_table[static_cast<size_t>(b) * p.max_pages + t * 8 + lane];
+              for (int h = 0; h < kHalves; ++h)
+                ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g,
+                                 page * 16);
+            }
+          }
+        } else if (lane == 0) {
+          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+          for (int h = 0; h < kHalves; ++h)
+            ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_tv : &tm_tk, full, h * 64, g, (t - TP) * kBN, b);
+        }
+        ++issued;
+        __syncwarp();
+      }
+    }
+    if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
+      // drain: every load that was issued must land before the CTA may exit
+      for (int s = 0; s < kStages; ++s) {
+        if (issued > s) {
+          const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
+          bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag);
+        }
+      }
+      bounded_wait(bar(Bars::kQFull), 0, abort_flag);
+    }
+  } else if (warp == 1) {
+    // =========================================================== tcgen05 issuer
+    constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
+    constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
+    bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag);
+
+    auto issue_qk = [&](int mt, int stage) {      // S[mt] = Q[mt] K^T
+      if (lane == 0) {
+        const uint32_t d_tmem = tmem_base + mt * 256;
+#pragma unroll
+        for (int kd = 0; kd < D / 16; ++kd) {
+          const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
+          const uint64_t a = ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0);
+          const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0);
+          ptx::umma_ss(d_tmem, a, bdesc, idesc_qk, kd > 0 ? 1u : 0u);
+        }
+      }
+    };
+    auto issue_pv = [&](int mt, int stage, bool first) {   // O[mt] (+)= P[mt] V
+      if (lane == 0) {
+        const uint32_t d_tmem = tmem_base + mt * 256 + 128;
+#pragma unroll
+        for (int kk = 0; kk < kBN / 16; ++kk) {
+          const uint64_t a = ptx::smem_desc_sw128(sP + mt * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0);
+          const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes);
+          ptx::umma_ss(d_tmem, a, bdesc, idesc_pv, (first && kk == 0) ? 0u : 1u);
+        }
+      }
+    };
+
+    for (int tl = 0; tl < T && ok; ++tl) {
+      if (tl == 0) {
+        const int stage = 0;
+        ok = bounded_wait(bar(Bars::kKvFull + stage), 0, abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        for (int mt = 0; mt < n_mt; ++mt) {
+          issue_qk(mt, stage);
+          if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
+        }
+        if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+        __syncwarp();
+      }
+      if (tl + 1 < T) {        // next tile's scores as soon as the softmax groups release S
+        const int item = 2 * (tl + 1), stage = item % kStages;
+        ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
+        for (int mt = 0; mt < n_mt && ok; ++mt) {
+          ok = bounded_wait(bar(Bars::kSFree + mt), tl & 1, abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          issue_qk(mt, stage);
+          if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
+          __syncwarp();
+        }
+        if (!ok) break;
+        if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+        __syncwarp();
+      }
+      {
+        const int item = 2 * tl + 1, stage = item % kStages;
+        ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
+        if (!ok) break;
+        const int valid = tile_valid(t_lo + tl);
+        if (valid < kBN) {
+          // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
+          uint8_t* vt = gen_kv + stage * C::kStageBytes;
+          const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
+          for (int h = 0; h < kHalves; ++h)
+            for (int i = lane; i < chunks; i += 32)
+              *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+        }
+        for (int mt = 0; mt < n_mt && ok; ++mt) {
+          ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          issue_pv(mt, stage, tl == 0);
+          if (lane == 0) ptx::umma_commit(bar(Bars::kODone + mt));
+          __syncwarp();
+        }
+        if (!ok) break;
+        if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+        __syncwarp();
+      }
+    }
+  } else if (warp >= 4) {
+    // =========================================================== softmax / epilogue warpgroups
+    const int mt = (warp - 4) >> 2;
+    if (mt < n_mt) {
+      const int r = tid - 128 - mt * 128;                     // row of the query tile = TMEM lane
+      const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      const uint32_t tS = tmem_base + lane_base + mt * 256;
+      const uint32_t tO = tS + 128;
+      const int v = node_lo + mt * npt + r / G;
+      const int h = g * G + r % G;
+      const bool row_live = v < n;
+      const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
+      uint8_t* my_p = gen_p + mt * 2 * kHalfBytes + r * 128;
+      const float sl2 = p.scale_log2;
+
+      float m_used = -INFINITY;     // running reference maximum (raw score units)
+      float l = 0.0f;               // running sum of exp2((s - m_used) * sl2)
+      bool ok = true;
+
+      for (int tl = 0; tl < T && ok; ++tl) {
+        const int t = t_lo + tl;
+        // visibility bits of this row for the four 32-key chunks of the tile
+        uint32_t vis[4];
+        if (t < TP) {
+          const int valid = L - t * kBN;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int nv = valid - c * 32;
+            vis[c] = nv >= 32 ? 0xFFFFFFFFu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+          }
+        } else {
+          const int w0 = (t - TP) * 4;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) vis[c] = (row_live && w0 + c < p.words) ? __ldg(mask_row + w0 + c) : 0u;
+        }
+        const bool all_visible = (vis[0] & vis[1] & vis[2] & vis[3]) == 0xFFFFFFFFu;
+
+        ok = bounded_wait(bar(Bars::kSFull + mt), tl & 1, abort_flag);
+        if (!ok) break;
+        ptx::tc_fence_after();
+
+        // ---- pass 1: row maximum over visible keys
+        float m_tile = -INFINITY;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t s[32];
+          ptx::tmem_ld32(tS + c * 32, s);
+          ptx::tmem_wait_ld();
+          if (all_visible) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) m_tile = fmaxf(m_tile, __uint_as_float(s[j]));
+          } else {
+            const uint32_t bits = vis[c];
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if ((bits >> j) & 1u) m_tile = fmaxf(m_tile, __uint_as_float(s[j]));
+          }
+        }
+        // ---- running maximum with lazy rescaling
+        float factor = 1.0f;
+        if (m_tile > -INFINITY) {
+          if (m_used == -INFINITY) {
+            m_used = m_tile;                       // nothing accumulated yet for this row
+          } else if ((m_tile - m_used) * sl2 > kRescaleThreshold) {
+            factor = exp2f((m_used - m_tile) * sl2);
+            m_used = m_tile;
+          }
+        }
+        const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
+        const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+
+        // P of the previous tile must have been consumed before it is overwritten; the same
+        // completion also makes O safe to rescale.
+        if (tl > 0) {
+          ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag);
+          if (!ok) break;
+          ptx::tc_fence_after();
+        }
+
+        // ---- pass 2: probabilities, row sum, P -> shared memory (swizzled bf16)
+        float row_sum = 0.0f;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t s[32];
+          ptx::tmem_ld32(tS + c * 32, s);
+          ptx::tmem_wait_ld();
+          const uint32_t bits = all_visible ? 0xFFFFFFFFu : vis[c];
+          uint32_t packed[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float p0 = exp2f(fmaf(__uint_as_float(s[j]), sl2, -m_ref));
+            float p1 = exp2f(fmaf(__uint_as_float(s[j + 1]), sl2, -m_ref));
+            if (!((bits >> j) & 1u)) p0 = 0.0f;
+            if (!((bits >> (j + 1)) & 1u)) p1 = 0.0f;
+            row_sum += p0 + p1;
+            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+            packed[j / 2] = *reinterpret_cast<uint32_t*>(&pk);
+          }
+          // chunk c covers keys [32c, 32c+32): 64-key block c/2, 16-byte chunks (c%2)*4 .. +3
+          uint8_t* dst = my_p + (c >> 1) * kHalfBytes;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int ch = ((c & 1) * 4 + q4) ^ (r & 7);
+            *reinterpret_cast<uint4*>(dst + ch * 16) =
+                make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
+          }
+        }
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(bar(Bars::kSFree + mt));          // S may be overwritten by the next Q K^T
+        l = l * factor + row_sum;
+
+        if (need_rescale && tl > 0) {
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            ptx::tmem_ld32(tO + c * 32, o);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+            ptx::tmem_st32(tO + c * 32, o);
+          }
+          ptx::tmem_wait_st();
+        }
+        ptx::fence_proxy_async_smem();
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(bar(Bars::kPFull + mt));
+      }
+
+      // ---- epilogue: O / l
+      if (ok) ok = bounded_wait(bar(Bars::kODone + mt), (T - 1) & 1, abort_flag);
+      if (ok) {
+        ptx::tc_fence_after();
+        const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+        const float lse = l > 0.0f ? (m_used * sl2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        const bool in_range = v < p.B;
+        if (p.nsplit == 1) {
+          __nv_bfloat16* orow = p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D;
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            ptx::tmem_ld32(tO + c * 32, o);
+            ptx::tmem_wait_ld();
+            if (in_range) {
+#pragma unroll
+              for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t w[4];
+#pragma unroll
+                for (int k2 = 0; k2 < 4; ++k2) {
+                  const float a0 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2]) * inv : 0.0f;
+                  const float a1 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2 + 1]) * inv : 0.0f;
+                  __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
+                  w[k2] = *reinterpret_cast<uint32_t*>(&pk);
+                }
+                *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+          }
+          if (p.lse && in_range) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = row_live ? lse : -INFINITY;
+        } else {
+          float* prow = part_o + (static_cast<size_t>(mt) * kBM + r) * D;
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            ptx::tmem_ld32(tO + c * 32, o);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4)
+              *reinterpret_cast<float4*>(prow + c * 32 + q4 * 4) =
+                  make_float4(__uint_as_float(o[q4 * 4]) * inv, __uint_as_float(o[q4 * 4 + 1]) * inv,
+                              __uint_as_float(o[q4 * 4 + 2]) * inv, __uint_as_float(o[q4 * 4 + 3]) * inv);
+          }
+          part_lse[mt * kBM + r] = row_live ? lse : -INFINITY;
+        }
+      }
+    }
+  }
+
+  // ---------------- teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+  if (tid == 0 && *abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
+}
+
+// Combines the key slices: out = sum_s exp(lse_s - lse) * O_s, lse = log sum_s exp(lse_s).
+template <int D, int MT>
+__global__ void __launch_bounds__(256)
+tree_attn_merge_kernel(const AttnParams p) {
+  constexpr int kRowsPerBlock = 256 / (D / 8);
+  const int unit = blockIdx.y;
+  const int mgroup = unit % p.n_mgroups;
+  const int bg = unit / p.n_mgroups;
+  const int g = bg % p.Hkv, b = bg / p.Hkv;
+  const int row = blockIdx.x * kRowsPerBlock + threadIdx.x / (D / 8);   // row within the MT*128 group
+  const int c8 = threadIdx.x % (D / 8);
+  const int npt = kBM / p.G;
+  const int v = mgroup * MT * npt + row / p.G;
+  const int h = g * p.G + row % p.G;
+  if (v >= p.B) return;
+  const int n = min(p.n_nodes[b], p.B);
+  __nv_bfloat16* orow = p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8;
+  float* lse_out = p.lse ? p.lse + (static_cast<size_t>(b) * p.Hq + h) * p.B + v : nullptr;
+  if (v >= n) {
+    *reinterpret_cast<uint4*>(orow) = make_uint4(0u, 0u, 0u, 0u);
+    if (lse_out && c8 == 0) *lse_out = -INFINITY;
+    return;
+  }
+  const size_t base = static_cast<size_t>(unit) * p.nsplit;
+  float m = -INFINITY;
+  for (int s = 0; s < p.nsplit; ++s) m = fmaxf(m, p.part_lse[(base + s) * MT * kBM + row]);
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  float wsum = 0.0f;
+  for (int s = 0; s < p.nsplit; ++s) {
+    const float ls = p.part_lse[(base + s) * MT * kBM + row];
+    if (ls == -INFINITY) continue;
+    const float w = __expf(ls - m);
+    wsum += w;
+    const float4* src = reinterpret_cast<const float4*>(p.part_o + ((base + s) * MT * kBM + row) * D + c8 * 8);
+    const float4 x0 = src[0], x1 = src[1];
+    acc[0] += w * x0.x; acc[1] += w * x0.y; acc[2] += w * x0.z; acc[3] += w * x0.w;
+    acc[4] += w * x1.x; acc[5] += w * x1.y; acc[6] += w * x1.z; acc[7] += w * x1.w;
+  }
+  const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+  uint32_t w4[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    __nv_bfloat162 pk = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
+    w4[k] = *reinterpret_cast<uint32_t*>(&pk);
+  }
+  *reinterpret_cast<uint4*>(orow) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+  if (lse_out && c8 == 0) *lse_out = wsum > 0.0f ? m + __logf(wsum) : -INFINITY;
+}
+
+// ------------------------------------------------------------------------------------------ host
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return static_cast<EncodeFn>(nullptr);
+    return reinterpret_cast<EncodeFn>(sym);
+  }();
+  return fn;
+}
+
+// bf16 tensor map, 128-byte swizzle, innermost box of 64 elements.
+bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+              const uint32_t* box) {
+  EncodeFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[5], gstr[4];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), gdim, gstr, bx, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = [] {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+    return v;
+  }();
+  return n;
+}
+
+struct Plan {
+  int mt;          // query tiles per CTA (1 or 2)
+  int n_mgroups;   // groups of mt query tiles per (sequence, KV head)
+  int units;
+  int nsplit;
+};
+
+Plan make_plan(int batch, int B, int Hq, int Hkv, int max_seq_len) {
+  Plan pl;
+  const int G = Hq / Hkv;
+  const int rows = B * G;
+  pl.mt = rows > kBM ? 2 : 1;
+  pl.n_mgroups = (rows + pl.mt * kBM - 1) / (pl.mt * kBM);
+  pl.units = batch * Hkv * pl.n_mgroups;
+  const int tiles = (max_seq_len + kBN - 1) / kBN + (B + kBN - 1) / kBN;
+  int ns = sm_count() / pl.units;
+  if (ns < 1) ns = 1;
+  if (ns > tiles) ns = tiles;
+  pl.nsplit = ns;
+  return pl;
+}
+
+size_t partial_bytes(const Plan& pl, int D) {
+  if (pl.nsplit == 1) return 0;
+  const size_t rows = static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM;
+  return round_up(rows * D * sizeof(float), 256) + round_up(rows * sizeof(float), 256);
+}
+
+template <int D, int MT>
+jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& ttk,
+                  const CUtensorMap& ttv, const AttnParams& p, const Plan& pl, cudaStream_t st) {
+  using C = Cfg<D, MT>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::kSmemBytes) != cudaSuccess)
+      return JET_ERR_CUDA;
+    configured = true;
+  }
+  tree_attn_kernel<D, MT><<<pl.units * pl.nsplit, C::kThreads, C::kSmemBytes, st>>>(tq, tk, tv, ttk, ttv, p);
+  if (pl.nsplit > 1) {
+    constexpr int kRowsPerBlock = 256 / (D / 8);
+    tree_attn_merge_kernel<D, MT><<<dim3(MT * kBM / kRowsPerBlock, pl.units), 256, 0, st>>>(p);
+  }
+  return launch_status();
+}
+
+}  // namespace
+}  // namespace jet
+
+extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
+                                                       int max_seq_len) {
+  if (batch < 1 || B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0 || D < 1) return 0;
+  const jet::Plan pl = jet::make_plan(batch, B, Hq, Hkv, max_seq_len);
+  return jet::partial_bytes(pl, D) + 256;
+}
+
+extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
+                                           const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                           int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                           const void* tree_k, const void* tree_v, const uint32_t* anc_mask,
+                                           const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D,
+                                           int64_t kv_batch_stride, float softmax_scale, void* out, float* lse,
+                                           int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                           void* stream) {
+  using namespace jet;
+  if (!q || !seq_len || !tree_k || !tree_v || !anc_mask || !n_nodes || !out) return JET_ERR_INVALID_ARG;
+  if (batch < 1 || B < 1 || B > JET_MAX_NODES || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0)
+    return JET_ERR_INVALID_ARG;
+  if (max_seq_len > 0 && (!k_cache || !v_cache)) return JET_ERR_INVALID_ARG;
+  const int G = Hq / Hkv;
+  if (D != 64 && D != 128) return JET_ERR_UNSUPPORTED;
+  if (G > 16 || (G & (G - 1)) != 0) return JET_ERR_UNSUPPORTED;
+  const bool paged = page_table != nullptr;
+  if (paged && (page_size != 16 || max_pages_per_seq < 1 || num_pages < 1)) return JET_ERR_UNSUPPORTED;
+  if (paged && static_cast<int64_t>(max_pages_per_seq) * 16 < max_seq_len) return JET_ERR_INVALID_ARG;
+  if (!paged && batch > 1 && (kv_batch_stride < static_cast<int64_t>(max_seq_len) * Hkv * D || kv_batch_stride % 8 != 0))
+    return JET_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(tree_k, 16) || !aligned(tree_v, 16) || !aligned(out, 16) ||
+      (k_cache && !aligned(k_cache, 16)) || (v_cache && !aligned(v_cache, 16)))
+    return JET_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(batch) * B >= (1ll << 31)) return JET_ERR_INVALID_ARG;
+
+  const Plan pl = make_plan(batch, B, Hq, Hkv, max_seq_len);
+  const size_t need = partial_bytes(pl, D) + 256;
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
+
+  // ---- tensor maps (bf16, 128-byte swizzle, 64-element inner box)
+  CUtensorMap tq, tk, tv, ttk, ttv;
+  const uint64_t eb = 2;
+  {
+    const uint64_t dims[4] = {static_cast<uint64_t>(D), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
+                              static_cast<uint64_t>(batch) * B};
+    const uint64_t str[3] = {D * eb, static_cast<uint64_t>(G) * D * eb, static_cast<uint64_t>(Hq) * D * eb};
+    const uint32_t box[4] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(kBM / G)};
+    if (!make_map(&tq, q, 4, dims, str, box)) return JET_ERR_CUDA;
+  }
+  {
+    const uint64_t dims[4] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Hkv), static_cast<uint64_t>(B),
+                              static_cast<uint64_t>(batch)};
+    const uint64_t str[3] = {D * eb, static_cast<uint64_t>(Hkv) * D * eb, static_cast<uint64_t>(B) * Hkv * D * eb};
+    const uint32_t box[4] = {64, 1, kBN, 1};
+    if (!make_map(&ttk, tree_k, 4, dims, str, box) || !make_map(&ttv, tree_v, 4, dims, str, box))
+      return JET_ERR_CUDA;
+  }
+  if (max_seq_len == 0) {
+    tk = ttk;   // never dereferenced: there are no prefix tiles
+    tv = ttv;
+  } else if (paged) {
+    const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Hkv),
+                              static_cast<uint64_t>(num_pages) * 16};
+    const uint64_t str[2] = {D * eb, static_cast<uint64_t>(Hkv) * D * eb};
+    const uint32_t box[3] = {64, 1, 16};
+    if (!make_map(&tk, k_cache, 3, dims, str, box) || !make_map(&tv, v_cache, 3, dims, str, box))
+      return JET_ERR_CUDA;
+  } else {
+    const uint64_t bstride = batch > 1 ? static_cast<uint64_t>(kv_batch_stride)
+                                       : static_cast<uint64_t>(max_seq_len) * Hkv * D;
+    const uint64_t dims[4] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Hkv),
+                              static_cast<uint64_t>(max_seq_len), static_cast<uint64_t>(batch)};
+    const uint64_t str[3] = {D * eb, static_cast<uint64_t>(Hkv) * D * eb, bstride * eb};
+    const uint32_t box[4] = {64, 1, kBN, 1};
+    if (!make_map(&tk, k_cache, 4, dims, str, box) || !make_map(&tv, v_cache, 4, dims, str, box))
+      return JET_ERR_CUDA;
+  }
+
+  AttnParams p;
+  p.page_table = page_table;
+  p.seq_len = seq_len;
+  p.n_nodes = n_nodes;
+  p.anc_mask = anc_mask;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse = lse;
+  p.status = device_status;
+  const size_t rows = static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM;
+  p.part_o = static_cast<float*>(workspace);
+  p.part_lse = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up(rows * D * sizeof(float), 256));
+  p.max_pages = max_pages_per_seq;
+  p.paged = paged ? 1 : 0;
+  p.batch = batch; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.words = (B + 31) / 32;
+  p.nsplit = pl.nsplit;
+  p.n_mgroups = pl.n_mgroups;
+  p.scale_log2 = softmax_scale * 1.4426950408889634f;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (D == 128) return pl.mt == 1 ? launch<128, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
+                                  : launch<128, 2>(tq, tk, tv, ttk, ttv, p, pl, st);
+  return pl.mt == 1 ? launch<64, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
+                    : launch<64, 2>(tq, tk, tv, ttk, ttv, p, pl, st);
 }

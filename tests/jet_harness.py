@@ -87,3 +87,38 @@ def run_kv_compact(tree_k, tree_v, k_cache, v_cache, page_table, path, accept_le
                        dev(np.asarray(accept_len, dtype=np.int32)), d_seq, layers, batch, B, Hkv, D, N)
     torch.cuda.synchronize()
     return (dk.cpu().numpy().view(np.uint16), dv.cpu().numpy().view(np.uint16), d_seq.cpu().numpy())
+
+
+def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_mask, n_nodes, scale,
+                  max_seq_len=None, want_lse=True):
+    """q [batch,B,Hq,D], tree_k/v [batch,B,Hkv,D] bf16 bits; cache contiguous [batch,Lmax,Hkv,D] or paged
+    [num_pages,16,Hkv,D] (with page_table [batch,max_pages]).  Returns (out fp64, lse fp64, status)."""
+    batch, B, Hq, D = q.shape
+    Hkv = tree_k.shape[2]
+    seq_len = np.asarray(seq_len, dtype=np.int32)
+    if max_seq_len is None:
+        max_seq_len = int(seq_len.max()) if page_table is None else int(seq_len.max())
+    d_q, d_tk, d_tv = dev_bf16(q), dev_bf16(tree_k), dev_bf16(tree_v)
+    if k_cache is not None and k_cache.size:
+        d_k, d_v = dev_bf16(k_cache), dev_bf16(v_cache)
+    else:
+        d_k = d_v = None
+    if page_table is None:
+        pt, max_pages, page_size, num_pages = None, 0, 0, 0
+        kv_batch_stride = int(k_cache.shape[1] * Hkv * D) if k_cache is not None else 0
+        if k_cache is not None:
+            max_seq_len = min(max_seq_len, k_cache.shape[1]) if max_seq_len > k_cache.shape[1] else max_seq_len
+    else:
+        pt = dev(page_table.astype(np.int32))
+        max_pages, page_size, num_pages = page_table.shape[1], k_cache.shape[1], k_cache.shape[0]
+        kv_batch_stride = 0
+    out = torch.full((batch, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((batch, Hq, B), float("nan"), dtype=torch.float32, device=DEV) if want_lse else None
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
+    jet.jet_tree_verify_attn(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
+                             d_tk, d_tv, dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
+                             batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
+    torch.cuda.synchronize()
+    return (bf16_to_f64(out), lse.cpu().numpy().astype(np.float64) if want_lse else None,
+            int(status.cpu()[0]))
