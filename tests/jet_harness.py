@@ -97,7 +97,7 @@ def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_
     Hkv = tree_k.shape[2]
     seq_len = np.asarray(seq_len, dtype=np.int32)
     if max_seq_len is None:
-        max_seq_len = int(seq_len.max()) if page_table is None else int(seq_len.max())
+        max_seq_len = int(seq_len.max())
     d_q, d_tk, d_tv = dev_bf16(q), dev_bf16(tree_k), dev_bf16(tree_v)
     if k_cache is not None and k_cache.size:
         d_k, d_v = dev_bf16(k_cache), dev_bf16(v_cache)
@@ -106,8 +106,6 @@ def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_
     if page_table is None:
         pt, max_pages, page_size, num_pages = None, 0, 0, 0
         kv_batch_stride = int(k_cache.shape[1] * Hkv * D) if k_cache is not None else 0
-        if k_cache is not None:
-            max_seq_len = min(max_seq_len, k_cache.shape[1]) if max_seq_len > k_cache.shape[1] else max_seq_len
     else:
         pt = dev(page_table.astype(np.int32))
         max_pages, page_size, num_pages = page_table.shape[1], k_cache.shape[1], k_cache.shape[0]

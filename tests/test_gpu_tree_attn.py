@@ -1,0 +1,216 @@
+"""GPU parity: jet_tree_verify_attn against the fp64 oracle.
+
+Tolerance (bf16 operands, fp32 accumulation, bf16 output): max |err| <= 2e-2 and
+mean |err| <= 2e-3 against the fp64 oracle; log-sum-exp within 1e-3.
+"""
+import numpy as np
+import pytest
+
+from jet_inputs import (CONFIGS, binary_tree, chain_tree, make_attn_inputs, make_logp, make_paged_cache,
+                        random_tree, star_tree)
+from oracle import anc_from_parent, gather_paged_prefix, tree_attn_ref, tree_attn_rows_ref, tree_build_ref
+
+pytestmark = pytest.mark.gpu
+
+MAX_ERR, MEAN_ERR, LSE_ERR = 2e-2, 2e-3, 1e-3
+NAN_BITS = np.uint16(0x7FC0)
+
+
+def _check(out, lse, ref, rlse, n):
+    assert not np.isnan(out).any()
+    err = np.abs(out - ref)
+    assert err.max() <= MAX_ERR, err.max()
+    assert err.mean() <= MEAN_ERR, err.mean()
+    assert (out[n:] == 0).all()
+    if lse is not None:
+        assert np.abs(lse[:, :n] - rlse[:, :n]).max() <= LSE_ERR
+        assert np.isneginf(lse[:, n:]).all()
+
+
+def _tree(kind, n, rng):
+    return {"random": lambda: random_tree(n, rng), "chain": lambda: chain_tree(n),
+            "star": lambda: star_tree(n), "binary": lambda: binary_tree(n)}[kind]()
+
+
+def _run_contiguous(B, Hq, Hkv, D, L, seed, n=None, kind="random", junk_rows=40, scale=None):
+    import jet_harness as H
+    rng = np.random.default_rng(seed)
+    n = n or B
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = _tree(kind, n, rng)
+    anc = anc_from_parent(parent, n, B)
+    scale = scale or 1.0 / np.sqrt(D)
+    ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, n, scale)
+    # cache rows beyond the prefix hold NaN junk that must never influence the result
+    kc = np.full((1, L + junk_rows, Hkv, D), NAN_BITS, np.uint16)
+    vc = np.full_like(kc, NAN_BITS)
+    kc[0, :L], vc[0, :L] = x["k_prefix"], x["v_prefix"]
+    tk, tv = x["tree_k"].copy(), x["tree_v"].copy()
+    tk[n:], tv[n:] = NAN_BITS, NAN_BITS                       # padding nodes hold junk too
+    out, lse, st = H.run_tree_attn(x["q"][None], kc, vc, None, [L], tk[None], tv[None], anc[None], [n], scale,
+                                   max_seq_len=L + junk_rows)
+    assert st == 0
+    _check(out[0], lse[0], ref, rlse, n)
+    return out[0], ref
+
+
+@pytest.mark.parametrize("seed", range(2))
+def test_tiny_config(seed):
+    c = CONFIGS["tiny"]
+    _run_contiguous(c["B"], c["Hq"], c["Hkv"], c["D"], c["L"], 1000 + seed)
+
+
+def test_tiny_config_with_built_tree():
+    import jet_harness as H
+    c = CONFIGS["tiny"]
+    rng = np.random.default_rng(1000)
+    t = tree_build_ref(make_logp(rng, c["N"], c["V"], c["sigma_draft"]), 1, c["N"], c["W"], c["B"])
+    x = make_attn_inputs(rng, c["B"], c["Hq"], c["Hkv"], c["D"], c["L"])
+    scale = 1.0 / np.sqrt(c["D"])
+    ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], t["anc_mask"],
+                              t["n_nodes"], scale)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [c["L"]],
+                                   x["tree_k"][None], x["tree_v"][None], t["anc_mask"][None], [t["n_nodes"]], scale)
+    assert st == 0
+    _check(out[0], lse[0], ref, rlse, t["n_nodes"])
+
+
+def test_qwen3_8b_config():
+    c = CONFIGS["qwen3_8b"]
+    _run_contiguous(c["B"], c["Hq"], c["Hkv"], c["D"], c["L"], 2000)
+
+
+@pytest.mark.parametrize("L", [0, 1, 127, 128, 129, 255, 257])
+@pytest.mark.parametrize("B", [1, 2, 31, 32, 33])
+def test_tile_boundaries(L, B):
+    _run_contiguous(B, 8, 2, 128, L, 31 * L + B)
+
+
+@pytest.mark.parametrize("kind", ["chain", "star", "binary"])
+def test_tree_shapes(kind):
+    _run_contiguous(48, 8, 2, 128, 200, 5, kind=kind)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,D,L", [(64, 8, 8, 128, 333), (40, 4, 2, 64, 700), (128, 32, 4, 128, 520),
+                                          (200, 16, 1, 64, 130), (512, 8, 2, 128, 140), (512, 8, 1, 128, 260)])
+def test_head_group_and_budget_variants(B, Hq, Hkv, D, L):
+    _run_contiguous(B, Hq, Hkv, D, L, B + L)
+
+
+def test_padding_nodes_give_zero_rows():
+    _run_contiguous(64, 8, 2, 128, 300, 9, n=37)
+    _run_contiguous(300, 8, 2, 128, 100, 10, n=129)
+    _run_contiguous(64, 32, 8, 128, 50, 11, n=1)
+
+
+def test_masked_nodes_have_no_influence_and_output_is_deterministic():
+    out_a, ref = _run_contiguous(64, 8, 2, 128, 500, 77)
+    out_b, _ = _run_contiguous(64, 8, 2, 128, 500, 77)
+    assert np.array_equal(out_a, out_b)
+
+
+def test_large_scores_stay_finite():
+    # scale 1.0 with head_dim 128 gives scores of +-30: exercises the running-max rescaling
+    _run_contiguous(64, 8, 2, 128, 900, 3, scale=1.0)
+
+
+def test_sweep_16k_sampled_rows():
+    """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
+    import jet_harness as H
+    c = CONFIGS["sweep_16k"]
+    B, Hq, Hkv, D, L = 128, c["Hq"], c["Hkv"], c["D"], c["L"]
+    rng = np.random.default_rng(3000)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = random_tree(B, rng, max_depth=12)
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0 / np.sqrt(D)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [L],
+                                   x["tree_k"][None], x["tree_v"][None], anc[None], [B], scale)
+    assert st == 0 and not np.isnan(out).any()
+    rows = [(int(rng.integers(0, B)), int(rng.integers(0, Hq))) for _ in range(96)] + [(0, 0), (B - 1, Hq - 1)]
+    ref, rlse = tree_attn_rows_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale,
+                                   rows)
+    got = np.stack([out[0, v, h] for v, h in rows])
+    err = np.abs(got - ref)
+    assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR
+    assert np.abs(np.array([lse[0, h, v] for v, h in rows]) - rlse).max() <= LSE_ERR
+
+
+@pytest.mark.parametrize("batch,B,Hq,Hkv,D", [(3, 16, 8, 2, 64), (5, 64, 8, 2, 128), (32, 64, 32, 8, 128)])
+def test_batched_paged_ragged(batch, B, Hq, Hkv, D):
+    import jet_harness as H
+    rng = np.random.default_rng(4000 + batch)
+    if batch == 32:
+        seq = rng.integers(100, 600, size=batch).astype(np.int32)      # shape of the serving case, shorter
+    else:
+        seq = rng.integers(0, 400, size=batch).astype(np.int32)
+        seq[0] = 16 * 5
+        seq[1] = 0
+    kp, vp, table = make_paged_cache(rng, seq, 16, Hkv, D, reserve=9)
+    # rows past each sequence's length are junk: poison them
+    for b in range(batch):
+        for pos in range(int(seq[b]), (int(seq[b]) + 9 + 15) // 16 * 16):
+            kp[table[b, pos // 16], pos % 16] = NAN_BITS
+            vp[table[b, pos // 16], pos % 16] = NAN_BITS
+    n_nodes = rng.integers(1, B + 1, size=batch)
+    n_nodes[0] = B
+    qs, tks, tvs, ancs = [], [], [], []
+    for b in range(batch):
+        x = make_attn_inputs(rng, B, Hq, Hkv, D, 0)
+        parent, _, _ = random_tree(int(n_nodes[b]), rng, max_depth=8)
+        qs.append(x["q"]); tks.append(x["tree_k"]); tvs.append(x["tree_v"])
+        ancs.append(anc_from_parent(parent, int(n_nodes[b]), B))
+    scale = 1.0 / np.sqrt(D)
+    out, lse, st = H.run_tree_attn(np.stack(qs), kp, vp, table, seq, np.stack(tks), np.stack(tvs), np.stack(ancs),
+                                   n_nodes, scale)
+    assert st == 0
+    check = range(batch) if batch <= 5 else (0, 7, 31)
+    for b in check:
+        kpre = gather_paged_prefix(kp, table[b], int(seq[b]))
+        vpre = gather_paged_prefix(vp, table[b], int(seq[b]))
+        ref, rlse = tree_attn_ref(qs[b], kpre, vpre, tks[b], tvs[b], ancs[b], int(n_nodes[b]), scale)
+        _check(out[b], lse[b], ref, rlse, int(n_nodes[b]))
+
+
+def test_batched_contiguous_with_batch_stride():
+    import jet_harness as H
+    rng = np.random.default_rng(99)
+    batch, B, Hq, Hkv, D, Lmax = 3, 32, 8, 2, 128, 300
+    seq = np.array([300, 17, 128], dtype=np.int32)
+    kc = np.full((batch, Lmax, Hkv, D), NAN_BITS, np.uint16); vc = np.full_like(kc, NAN_BITS)
+    xs, ancs = [], []
+    for b in range(batch):
+        x = make_attn_inputs(rng, B, Hq, Hkv, D, int(seq[b]))
+        kc[b, :seq[b]], vc[b, :seq[b]] = x["k_prefix"], x["v_prefix"]
+        parent, _, _ = random_tree(B, rng)
+        xs.append(x); ancs.append(anc_from_parent(parent, B, B))
+    scale = 1.0 / np.sqrt(D)
+    out, lse, st = H.run_tree_attn(np.stack([x["q"] for x in xs]), kc, vc, None, seq,
+                                   np.stack([x["tree_k"] for x in xs]), np.stack([x["tree_v"] for x in xs]),
+                                   np.stack(ancs), [B] * batch, scale, max_seq_len=Lmax)
+    assert st == 0
+    for b in range(batch):
+        x = xs[b]
+        ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], ancs[b], B, scale)
+        _check(out[b], lse[b], ref, rlse, B)
+
+
+def test_argument_errors():
+    import torch
+    import jet_harness as H
+    import paper_2606_18394_b200 as jet
+    t = torch.zeros(1 << 16, dtype=torch.bfloat16, device=H.DEV)
+    i32 = torch.ones(64, dtype=torch.int32, device=H.DEV)
+    ws = H.workspace(1 << 20)
+    args = dict(q=t, k_cache=t, v_cache=t, page_table=None, max_pages_per_seq=0, page_size=0, num_pages=0,
+                seq_len=i32, max_seq_len=16, tree_k=t, tree_v=t, anc_mask=i32, n_nodes=i32, batch=1, B=8, Hq=8,
+                Hkv=2, D=128, kv_batch_stride=0, softmax_scale=0.1, out=t, lse=None, device_status=None,
+                workspace=ws, check=False)
+    assert jet.jet_tree_verify_attn(**{**args, "D": 96}) == jet.JET_ERR_UNSUPPORTED
+    assert jet.jet_tree_verify_attn(**{**args, "Hq": 6, "Hkv": 2}) == jet.JET_ERR_UNSUPPORTED
+    assert jet.jet_tree_verify_attn(**{**args, "Hq": 7}) == jet.JET_ERR_INVALID_ARG
+    assert jet.jet_tree_verify_attn(**{**args, "B": 513}) == jet.JET_ERR_INVALID_ARG
+    assert jet.jet_tree_verify_attn(**{**args, "q": None}) == jet.JET_ERR_INVALID_ARG
+    assert jet.jet_tree_verify_attn(**{**args, "workspace": None}) == jet.JET_ERR_WORKSPACE
+    assert jet.jet_tree_verify_attn(**{**args, "page_table": i32, "page_size": 32, "max_pages_per_seq": 4,
+                                       "num_pages": 4}) == jet.JET_ERR_UNSUPPORTED
