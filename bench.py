@@ -1,0 +1,455 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verification hot path (one B200 per rank).
+
+A step = jet_tree_build -> jet_tree_verify_attn for every layer (each layer has its own KV
+buffers, so the K/V stream comes from HBM, not from L2) -> jet_tree_accept -> jet_kv_compact
+on the Qwen3-8B-shaped workload (batch 1, 32/8 heads, head_dim 128, prefix 4096, 64-node tree).
+The metric is microseconds per layer of a whole step (lower is better).  With N > 1 ranks every
+rank verifies its own sequence (no data-path collective: the path shards by sequence).
+
+`--impl reference` times the CPU oracle (test infrastructure, never the product path) on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from jet_inputs import CONFIGS, plant_path  # noqa: E402
+
+METRIC = "tree_verify_us_per_layer"
+UNIT = "us/layer"
+
+# DRAM bytes (read + write) of one tree_attn_kernel launch on the benchmark workload, from the ncu
+# capture summarised under profiles/ (None until a capture exists for the workload).
+NCU_TRAFFIC_BYTES = {"qwen3_8b": None}
+
+
+def workload(name):
+    c = dict(CONFIGS[name])
+    if "B" not in c:
+        raise SystemExit(f"config {name} is a sweep; pick a single-budget config")
+    return c
+
+
+def attn_algorithmic_bytes(c, seq_lens, n_nodes):
+    """K and V prefix + tree K/V + Q in + O out + ancestor mask, per layer (all sequences)."""
+    B, Hq, Hkv, D = c["B"], c["Hq"], c["Hkv"], c["D"]
+    total = 0
+    for L in seq_lens:
+        total += 2 * L * Hkv * D * 2 + 2 * B * Hkv * D * 2 + 2 * B * Hq * D * 2 + B * ((B + 31) // 32) * 4
+    return total
+
+
+def attn_algorithmic_flops(c, seq_lens, depths):
+    B, Hq, Hkv, D = c["B"], c["Hq"], c["Hkv"], c["D"]
+    G = Hq // Hkv
+    total = 0
+    for L, dep in zip(seq_lens, depths):
+        total += 4 * B * Hq * D * L + 4 * G * D * Hkv * int(sum(int(d) + 1 for d in dep if d >= 0))
+    return total
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 6 and r[2 + i].lower() == "active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+def build_inputs(c, name, seed, device):
+    """Seeded synthetic step inputs on the device.  Returns (VerifyStep, info dict)."""
+    import torch
+    from paper_2606_18394_b200.step import VerifyStep
+
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    batch, layers = c["batch"], c["layers"]
+    B, N, W, V, Hq, Hkv, D = c["B"], c["N"], c["W"], c["V"], c["Hq"], c["Hkv"], c["D"]
+    if c.get("paged"):
+        rng = np.random.default_rng(seed)
+        lo, hi = c["L_range"]
+        seq = rng.integers(lo, hi + 1, size=batch).astype(np.int32)
+        need = [(int(L) + N + 1 + 15) // 16 for L in seq]
+        num_pages = sum(need) + 3
+        perm = rng.permutation(num_pages)
+        max_pages = max(need)
+        table = np.full((batch, max_pages), 0, dtype=np.int32)
+        pos = 0
+        for b, cnt in enumerate(need):
+            table[b, :cnt] = perm[pos:pos + cnt]
+            pos += cnt
+        st = VerifyStep(batch=batch, layers=layers, Hq=Hq, Hkv=Hkv, D=D, B=B, N=N, W=W, V=V,
+                        max_seq_len=int(seq.max()), page_size=16, num_pages=num_pages, max_pages=max_pages,
+                        device=device)
+        st.page_table.copy_(torch.from_numpy(table))
+    else:
+        seq = np.full(batch, c["L"], dtype=np.int32)
+        st = VerifyStep(batch=batch, layers=layers, Hq=Hq, Hkv=Hkv, D=D, B=B, N=N, W=W, V=V,
+                        max_seq_len=int(c["L"]), device=device)
+    st.seq_len0.copy_(torch.from_numpy(seq))
+    for t in (st.q, st.tree_k, st.tree_v):
+        t.copy_(torch.randn(t.shape, generator=gen, device=device, dtype=torch.float32))
+    for layer in range(layers):      # layer by layer: bounded temporaries
+        st.k_cache[layer].copy_(torch.randn(st.k_cache[layer].shape, generator=gen, device=device, dtype=torch.float32))
+        st.v_cache[layer].copy_(torch.randn(st.v_cache[layer].shape, generator=gen, device=device, dtype=torch.float32))
+    # draft log-probs: log_softmax of N(0, sigma) logits with one confident token per depth (p = 0.7),
+    # evaluated in fp64 and rounded to fp32
+    for b in range(batch):
+        logits = torch.randn((N, V), generator=gen, device=device, dtype=torch.float32).double() * c["sigma_draft"]
+        top = torch.randint(0, V, (N,), generator=gen, device=device)
+        rest = logits.clone()
+        rest[torch.arange(N, device=device), top] = -float("inf")
+        logits[torch.arange(N, device=device), top] = np.log(0.7 / 0.3) + torch.logsumexp(rest, dim=1)
+        st.logp[b].copy_(torch.log_softmax(logits, dim=1).float())
+    st.root_token.copy_(torch.arange(batch, device=device, dtype=torch.int32) + 1)
+    st.logits.copy_(torch.randn(st.logits.shape, generator=gen, device=device, dtype=torch.float32) * c["sigma_target"])
+    # plant the target arg-max along one random path of the tree that jet_tree_build produces
+    st.seq_len.copy_(st.seq_len0)
+    st.tree_build()
+    torch.cuda.synchronize()
+    parent, depth, token = st.parent.cpu().numpy(), st.depth.cpu().numpy(), st.token.cpu().numpy()
+    n_nodes = st.n_nodes.cpu().numpy()
+    rng = np.random.default_rng(seed + 1)
+    planted = []
+    for b in range(batch):
+        rows = st.logits[b].cpu().numpy()
+        want = c.get("plant", int(rng.integers(1, N + 1)))
+        _, eff = plant_path(rows, token[b], parent[b], depth[b], int(n_nodes[b]), want, rng)
+        st.logits[b].copy_(torch.from_numpy(rows))
+        planted.append(eff)
+    info = dict(seq_lens=[int(x) for x in seq], planted=planted, depth=depth, n_nodes=n_nodes)
+    return st, info
+
+
+def time_step(st, steps, warmup, use_graph):
+    import torch
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        st.run()
+        stream.synchronize()
+        graph = None
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                st.run()
+        run = graph.replay if graph is not None else st.run
+        for _ in range(warmup):
+            run()
+        stream.synchronize()
+    return stream, run
+
+
+def bench_jet(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2606_18394_b200 as jet
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    jet.load()
+    device = f"cuda:{local_rank}"
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    c = workload(args.config)
+    st, info = build_inputs(c, args.config, 1000 * 2 + rank, device)
+    layers = c["layers"]
+
+    stream, run = time_step(st, args.steps, max(args.warmup, 3), not args.no_graph)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- device-resident timing of K whole steps
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(args.steps):
+            run()
+        e1.record(stream)
+    stream.synchronize()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    t = torch.tensor([ms_total], device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    assert int(st.status.item()) == 0, "a bounded device wait expired"
+    acc = st.accept_len.cpu().numpy().tolist()
+    assert acc == info["planted"], (acc, info["planted"])
+
+    # ---------------- per-call timing of the attention layer (events around every call; cold KV)
+    with torch.cuda.stream(stream):
+        st.seq_len.copy_(st.seq_len0)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(layers * args.steps)]
+        for rep in range(2):                       # first repetition warms up
+            i = 0
+            for _ in range(args.steps):
+                for layer in range(layers):
+                    a, b_ = evs[i]
+                    a.record(stream)
+                    st.verify_attn(layer)
+                    b_.record(stream)
+                    i += 1
+            stream.synchronize()
+    attn_us = statistics.mean(a.elapsed_time(b_) for a, b_ in evs) * 1e3
+
+    # ---------------- end to end: host buffers in, result out, every step
+    pinned = {k: getattr(st, k).cpu().pin_memory() for k in ("logp", "root_token", "logits", "q", "tree_k", "tree_v")}
+    host_out = {k: torch.empty_like(getattr(st, k), device="cpu").pin_memory()
+                for k in ("accept_len", "out_tokens", "path")}
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values())
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+
+    def e2e_step():
+        for k, v in pinned.items():
+            getattr(st, k).copy_(v, non_blocking=True)
+        run()
+        for k, v in host_out.items():
+            v.copy_(getattr(st, k), non_blocking=True)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            e2e_step()
+        stream.synchronize()
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        e1.record(stream)
+        stream.synchronize()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms_step = float(t.item()) / args.steps
+    assert host_out["accept_len"].numpy().tolist() == info["planted"]
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---------------- roofline of the dominant kernel (one attention call = attention + slice merge)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peaks, peak_src = json.load(open(peaks_path)), "measured"
+    else:
+        peaks, peak_src = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+    bytes_alg = attn_algorithmic_bytes(c, info["seq_lens"], info["n_nodes"])
+    flops_alg = attn_algorithmic_flops(c, info["seq_lens"], info["depth"])
+    t_bytes = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    t_flops = flops_alg / (peaks["bf16_tflops"] * 1e12)
+    if t_bytes >= t_flops:
+        roof = {"bound": "hbm", "achieved": bytes_alg / (attn_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": flops_alg / (attn_us * 1e-6) / 1e12, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.config)
+    roof.update(kernel="tree_attn_kernel (+ tree_attn_merge_kernel)", peak_source=peak_src, us_per_launch=attn_us,
+                algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
+                roofline_us=max(t_bytes, t_flops) * 1e6)
+
+    cpu = cpu_baseline(st, c, info) if not args.no_cpu_baseline else None
+
+    line = {
+        "metric": METRIC, "value": ms_step * 1e3 / (layers * world), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.config, "batch_per_gpu": c["batch"], "layers": layers, "Hq": c["Hq"],
+                   "Hkv": c["Hkv"], "head_dim": c["D"], "prefix": info["seq_lens"] if c.get("paged") else c["L"],
+                   "tree_nodes": c["B"], "max_depth": c["N"], "width": c["W"], "vocab": c["V"],
+                   "paged": bool(c.get("paged")), "cuda_graph": not args.no_graph,
+                   "l2": "every layer streams its own KV buffers; one step reads far more than the 126 MB L2",
+                   "accepted_len": acc},
+        "attn_us_per_layer": attn_us,
+        "e2e": {"value": e2e_ms_step * 1e3 / (layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step},
+        "gpu_launches": args.steps * st.launches_per_step(2),
+        "clocks": clocks, "roofline": roof,
+    }
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+def _bits(t):
+    import torch
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def oracle_sample(c, x, attn_layers):
+    """The CPU oracle on a bounded sample of one step of one sequence: tree_build and tree_accept in
+    full, `attn_layers` attention layers in full (fp64).  `x` holds numpy inputs: logp, root, logits,
+    planted, scale and per-layer lists q / k / v / tk / tv (bf16 bit patterns).
+    Returns (seconds, description, us/layer)."""
+    import oracle
+    B, N, W, layers = c["B"], c["N"], c["W"], c["layers"]
+    t0 = time.perf_counter()
+    tree = oracle.tree_build_ref(x["logp"], x["root"], N, W, B)
+    t_build = time.perf_counter() - t0
+    t_attn = 0.0
+    for layer in range(attn_layers):
+        t0 = time.perf_counter()
+        oracle.tree_attn_ref(x["q"][layer], x["k"][layer], x["v"][layer], x["tk"][layer], x["tv"][layer],
+                             tree["anc_mask"], tree["n_nodes"], x["scale"])
+        t_attn += time.perf_counter() - t0
+    t0 = time.perf_counter()
+    acc = oracle.tree_accept_ref(x["logits"], tree["token"], tree["parent"], tree["depth"], tree["n_nodes"], N)
+    t_accept = time.perf_counter() - t0
+    per_layer_us = (t_attn / attn_layers + (t_build + t_accept) / layers) * 1e6
+    desc = (f"one sequence of the workload: tree_build + tree_accept in full, attention of {attn_layers} of "
+            f"{layers} layers in full (fp64); us/layer = attention per layer + (build + accept) / layers; "
+            f"commit copies omitted (negligible)")
+    if x.get("planted") is not None:
+        assert acc["accept_len"] == x["planted"], (acc["accept_len"], x["planted"])
+    return t_attn + t_build + t_accept, desc, per_layer_us
+
+
+def _blas_threads():
+    try:
+        import threadpoolctl
+        info = threadpoolctl.threadpool_info()
+        return max(p["num_threads"] for p in info) if info else 1
+    except Exception:
+        return os.cpu_count()
+
+
+def cpu_baseline(st, c, info):
+    """Oracle timing on the benchmark's own inputs (sequence 0, first two layers), copied to the host."""
+    L = info["seq_lens"][0]
+    nl = 2
+    if st.paged:
+        import oracle
+        table = st.page_table[0].cpu().numpy()
+        ks = [oracle.gather_paged_prefix(_bits(st.k_cache[l]), table, L) for l in range(nl)]
+        vs = [oracle.gather_paged_prefix(_bits(st.v_cache[l]), table, L) for l in range(nl)]
+    else:
+        ks = [_bits(st.k_cache[l, 0, :L]) for l in range(nl)]
+        vs = [_bits(st.v_cache[l, 0, :L]) for l in range(nl)]
+    x = dict(logp=st.logp[0].cpu().numpy(), root=int(st.root_token[0].item()), logits=st.logits[0].cpu().numpy(),
+             planted=info["planted"][0], scale=st.scale, q=[_bits(st.q[l, 0]) for l in range(nl)], k=ks, v=vs,
+             tk=[_bits(st.tree_k[l, 0]) for l in range(nl)], tv=[_bits(st.tree_v[l, 0]) for l in range(nl)])
+    secs, desc, per_layer_us = oracle_sample(c, x, attn_layers=nl)
+    return {"value": per_layer_us, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": desc,
+            "seconds": secs, "host_cpus": os.cpu_count()}
+
+
+def reference_inputs(c, seed):
+    """Host-only synthetic inputs of the workload's shape for the reference arm (no GPU, no product code)."""
+    import oracle
+    from jet_inputs import make_attn_inputs, make_logp, make_target_logits
+    rng = np.random.default_rng(seed)
+    L = c["L"] if "L" in c else int(rng.integers(c["L_range"][0], c["L_range"][1] + 1))
+    logp = make_logp(rng, c["N"], c["V"], c["sigma_draft"], peaked_p=0.7)
+    tree = oracle.tree_build_ref(logp, 1, c["N"], c["W"], c["B"])
+    logits = make_target_logits(rng, c["B"], c["V"], c["sigma_target"])
+    _, eff = plant_path(logits, tree["token"], tree["parent"], tree["depth"], tree["n_nodes"], c.get("plant", 4), rng)
+    a = make_attn_inputs(rng, c["B"], c["Hq"], c["Hkv"], c["D"], L)
+    return dict(logp=logp, root=1, logits=logits, planted=eff, scale=1.0 / np.sqrt(c["D"]), q=[a["q"]],
+                k=[a["k_prefix"]], v=[a["v_prefix"]], tk=[a["tree_k"]], tv=[a["tree_v"]])
+
+
+def bench_reference(args):
+    """The reference arm: the CPU oracle as it stands, on the host cores of rank 0 (other ranks idle)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    c = workload(args.config)
+    x = reference_inputs(c, 2000)
+    warm = min(args.warmup, 1)
+    for _ in range(warm):
+        oracle_sample(c, x, attn_layers=1)
+    times, per_layer, desc = [], [], ""
+    for _ in range(args.steps):
+        secs, desc, us = oracle_sample(c, x, attn_layers=1)
+        times.append(secs)
+        per_layer.append(us)
+    value = statistics.mean(per_layer)
+    cpu = {"value": value, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": desc,
+           "host_cpus": os.cpu_count()}
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": warm,
+            "ms_per_step": statistics.mean(times) * 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.config, "sample": desc}, "cpu_baseline": cpu,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["jet", "reference"], default="jet")
+    ap.add_argument("--config", default="qwen3_8b", choices=[k for k, v in CONFIGS.items() if "B" in v])
+    ap.add_argument("--no-graph", action="store_true", help="issue the calls directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        bench_reference(args)
+    else:
+        bench_jet(args)
+
+
+if __name__ == "__main__":
+    main()

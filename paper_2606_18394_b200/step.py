@@ -1,0 +1,120 @@
+"""One verification step = tree_build -> tree_verify_attn per layer -> tree_accept -> kv_compact.
+
+``VerifyStep`` only owns device buffers (torch tensors as memory handles) and issues the four
+C-ABI calls in order on the current stream; it performs no arithmetic of its own.  It is what
+the benchmark, the smoke check and the end-to-end test drive.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+
+from . import binding as jet
+
+
+class VerifyStep:
+    def __init__(self, *, batch, layers, Hq, Hkv, D, B, N, W, V, max_seq_len, page_size=0, num_pages=0,
+                 max_pages=0, device="cuda:0"):
+        self.batch, self.layers, self.Hq, self.Hkv, self.D = batch, layers, Hq, Hkv, D
+        self.B, self.N, self.W, self.V = B, N, W, V
+        self.max_seq_len = max_seq_len
+        self.paged = page_size > 0
+        self.page_size, self.num_pages, self.max_pages = page_size, num_pages, max_pages
+        self.device = torch.device(device)
+        dev = self.device
+        i32 = dict(dtype=torch.int32, device=dev)
+        words = (B + 31) // 32
+        self.words = words
+        # ---- inputs
+        self.logp = torch.zeros((batch, N, V), dtype=torch.float32, device=dev)
+        self.root_token = torch.zeros(batch, **i32)
+        self.logits = torch.zeros((batch, B, V), dtype=torch.float32, device=dev)
+        self.q = torch.zeros((layers, batch, B, Hq, D), dtype=torch.bfloat16, device=dev)
+        self.tree_k = torch.zeros((layers, batch, B, Hkv, D), dtype=torch.bfloat16, device=dev)
+        self.tree_v = torch.zeros_like(self.tree_k)
+        kv_layers = layers
+        self.kv_layers = kv_layers
+        if self.paged:
+            self.k_cache = torch.zeros((kv_layers, num_pages, page_size, Hkv, D), dtype=torch.bfloat16, device=dev)
+            self.page_table = torch.zeros((batch, max_pages), **i32)
+            self.rows_per_seq = 0
+        else:
+            # room for the committed path behind the longest prefix
+            self.rows_per_seq = max_seq_len + N + 1
+            self.k_cache = torch.zeros((kv_layers, batch, self.rows_per_seq, Hkv, D), dtype=torch.bfloat16,
+                                       device=dev)
+            self.page_table = None
+        self.v_cache = torch.zeros_like(self.k_cache)
+        self.seq_len0 = torch.zeros(batch, **i32)      # prefix lengths at the start of a step
+        self.seq_len = torch.zeros(batch, **i32)
+        # ---- outputs
+        self.parent = torch.zeros((batch, B), **i32)
+        self.depth = torch.zeros((batch, B), **i32)
+        self.token = torch.zeros((batch, B), **i32)
+        self.score = torch.zeros((batch, B), dtype=torch.float32, device=dev)
+        self.anc_mask = torch.zeros((batch, B, words), **i32)
+        self.n_nodes = torch.zeros(batch, **i32)
+        self.out = torch.zeros((layers, batch, B, Hq, D), dtype=torch.bfloat16, device=dev)
+        self.status = torch.zeros(1, **i32)
+        self.tgt = torch.zeros((batch, B), **i32)
+        self.accept_len = torch.zeros(batch, **i32)
+        self.path = torch.zeros((batch, N + 1), **i32)
+        self.out_tokens = torch.zeros((batch, N + 1), **i32)
+        # ---- workspaces
+        def ws(nbytes):
+            return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=dev)
+        self.ws_build = ws(jet.jet_tree_build_workspace_bytes(batch, N, V, W))
+        self.ws_attn = ws(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, self.attn_max_len))
+        self.ws_accept = ws(jet.jet_tree_accept_workspace_bytes(batch, B, V))
+        self.scale = 1.0 / math.sqrt(D)
+
+    @property
+    def attn_max_len(self):
+        return self.max_seq_len if self.paged else self.rows_per_seq
+
+    @property
+    def kv_batch_stride(self):
+        return 0 if self.paged else self.rows_per_seq * self.Hkv * self.D
+
+    @property
+    def cache_layer_stride(self):
+        return self.k_cache.stride(0)
+
+    # ------------------------------------------------------------------ the four calls
+    def tree_build(self):
+        jet.jet_tree_build(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, self.parent,
+                           self.depth, self.token, self.score, self.anc_mask, self.n_nodes, self.ws_build)
+
+    def verify_attn(self, layer):
+        jet.jet_tree_verify_attn(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
+                                 self.max_pages, self.page_size, self.num_pages, self.seq_len, self.attn_max_len,
+                                 self.tree_k[layer], self.tree_v[layer], self.anc_mask, self.n_nodes, self.batch,
+                                 self.B, self.Hq, self.Hkv, self.D, self.kv_batch_stride, self.scale,
+                                 self.out[layer], None, self.status, self.ws_attn)
+
+    def tree_accept(self):
+        jet.jet_tree_accept(self.logits, self.V, self.token, self.parent, self.depth, self.anc_mask, self.n_nodes,
+                            self.batch, self.B, self.V, self.N, self.tgt, self.accept_len, self.path,
+                            self.out_tokens, self.ws_accept)
+
+    def kv_compact(self):
+        jet.jet_kv_compact(self.tree_k, self.tree_v, self.k_cache, self.v_cache,
+                           self.cache_layer_stride, self.kv_batch_stride,
+                           self.page_table, self.max_pages, self.page_size, self.path, self.accept_len,
+                           self.seq_len, self.layers, self.batch, self.B, self.Hkv, self.D, self.N)
+
+    def run(self):
+        """The whole hot path once, on the current stream.  seq_len restarts from seq_len0 so that
+        repeated steps (and graph replays) see the same prefix lengths."""
+        self.seq_len.copy_(self.seq_len0)
+        self.tree_build()
+        for layer in range(self.layers):
+            self.verify_attn(layer)
+        self.tree_accept()
+        self.kv_compact()
+
+    LAUNCHES_PER_STEP_FIXED = 6      # tree_build 2, tree_accept 2, kv_compact 2
+
+    def launches_per_step(self, attn_launches_per_layer):
+        return self.LAUNCHES_PER_STEP_FIXED + self.layers * attn_launches_per_layer
