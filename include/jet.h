@@ -164,6 +164,38 @@ JET_API jet_status jet_tree_accept(const float* logits, int64_t logits_row_strid
                            void* stream);
 
 /* ---------------------------------------------------------------------------
+ * jet_tree_accept_static -- the same operation as jet_tree_accept for callers that cannot
+ * provide scratch memory.  (The paper has no counterpart; this is a library convenience.)
+ *
+ * Who needs it: code that runs after all device memory has been handed out (a serving engine
+ * that reserved the rest of the GPU for its KV cache at start-up, so a late cudaMalloc fails or
+ * fragments the pool), and code on a latency-critical decode loop where an allocator call is
+ * forbidden because cudaMalloc / cudaFree may synchronise the whole device.
+ *
+ * Instead of a caller workspace the arg-max partials go to an array built into the library:
+ * JET_STATIC_ACCEPT_SCRATCH_BYTES of device memory that every GPU which loads the library
+ * holds until the process exits.  The call makes no cudaMalloc / cudaFree and uses no
+ * allocating library routine.  Inputs and outputs are exactly those of jet_tree_accept.
+ *
+ * Limit: batch * B * ceil(V / 8192) * 8 bytes must fit in JET_STATIC_ACCEPT_SCRATCH_BYTES
+ * (e.g. 4096 logits rows of a 151936-entry vocabulary); larger problems are rejected on the
+ * host with JET_ERR_WORKSPACE and nothing is launched.
+ * First call on a device: looks up the array's device address (cudaGetSymbolAddress, with the
+ * calling thread's current device); make that first call outside any stream capture.
+ * Sharing: all calls on one GPU use the same array, which keeps the previous call's contents.
+ * Nothing in it has to be cleared between calls, but two calls that can overlap on the GPU
+ * (different streams) race on it -- serialise them, or use jet_tree_accept with separate
+ * workspaces.
+ */
+#define JET_STATIC_ACCEPT_SCRATCH_BYTES (1u << 20)
+
+JET_API jet_status jet_tree_accept_static(const float* logits, int64_t logits_row_stride, const int32_t* token,
+                                  const int32_t* parent, const int32_t* depth, const uint32_t* anc_mask,
+                                  const int32_t* n_nodes, int batch, int B, int V, int N,
+                                  int32_t* tgt_argmax, int32_t* accept_len, int32_t* path,
+                                  int32_t* out_tokens, void* stream);
+
+/* ---------------------------------------------------------------------------
  * jet_kv_compact -- commit of the accepted path (Appendix E: "the accepted path
  * is committed"): for every layer l, sequence b and i in [0, accept_len[b]] the
  * K and V rows of tree node path[b,i] are copied to cache position

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     exported_symbols,
     jet_kv_compact,
     jet_tree_accept,
+    jet_tree_accept_static,
     jet_tree_accept_workspace_bytes,
     jet_tree_build,
     jet_tree_build_workspace_bytes,

@@ -35,6 +35,8 @@ _SIGNATURES = {
     "jet_tree_accept_workspace_bytes": (_sz, [_i, _i, _i]),
     "jet_tree_accept": (_c.c_int32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp,
                                      _vp, _vp, _sz, _vp]),
+    "jet_tree_accept_static": (_c.c_int32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp,
+                                            _vp, _vp]),
     "jet_kv_compact": (_c.c_int32, [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i, _i, _vp, _vp, _vp, _i, _i,
                                     _i, _i, _i, _i, _vp]),
 }
@@ -144,6 +146,20 @@ def jet_tree_accept(logits, logits_row_stride, token, parent, depth, anc_mask, n
                                 _p(out_tokens), _p(workspace), wb, _stream(stream))
     if check:
         _check(st, "jet_tree_accept")
+    return st
+
+
+def jet_tree_accept_static(logits, logits_row_stride, token, parent, depth, anc_mask, n_nodes, batch, B, V, N,
+                           tgt_argmax, accept_len, path, out_tokens, stream=None, check=True):
+    """jet_tree_accept without a caller workspace: the scratch is an array built into libjet.so.
+    For callers that must not allocate device memory (everything already reserved, or no allocator
+    calls allowed on the decode loop).  Problems larger than the built-in array give JET_ERR_WORKSPACE;
+    calls that overlap on one GPU race on the shared array."""
+    st = load().jet_tree_accept_static(_p(logits), logits_row_stride, _p(token), _p(parent), _p(depth),
+                                       _p(anc_mask), _p(n_nodes), batch, B, V, N, _p(tgt_argmax),
+                                       _p(accept_len), _p(path), _p(out_tokens), _stream(stream))
+    if check:
+        _check(st, "jet_tree_accept_static")
     return st
 
 

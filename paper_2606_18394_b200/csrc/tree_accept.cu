@@ -140,6 +140,12 @@ accept_path_kernel(const unsigned long long* __restrict__ partial, int nchunks,
 
 int chunks_for(int V) { return (V + kArgChunk - 1) / kArgChunk; }
 
+// Built-in scratch of jet_tree_accept_static: one 64-bit arg-max key per (logits row, 8192-entry
+// slice).  It lives in every device context that loads the library (1 MiB) until the process exits.
+constexpr size_t kStaticKeys = JET_STATIC_ACCEPT_SCRATCH_BYTES / sizeof(unsigned long long);
+static __device__ __align__(256) unsigned long long g_accept_scratch[kStaticKeys];
+constexpr int kMaxDevices = 64;
+
 }  // namespace
 }  // namespace jet
 
@@ -177,4 +183,34 @@ extern "C" jet_status jet_tree_accept(const float* logits, int64_t logits_row_st
                                                  n_nodes, B, N, tgt_argmax, accept_len, path,
                                                  out_tokens);
   return launch_status();
+}
+
+extern "C" jet_status jet_tree_accept_static(const float* logits, int64_t logits_row_stride,
+                                             const int32_t* token, const int32_t* parent,
+                                             const int32_t* depth, const uint32_t* anc_mask,
+                                             const int32_t* n_nodes, int batch, int B, int V, int N,
+                                             int32_t* tgt_argmax, int32_t* accept_len, int32_t* path,
+                                             int32_t* out_tokens, void* stream) {
+  using namespace jet;
+  if (batch < 1 || B < 1 || V < 1) return JET_ERR_INVALID_ARG;
+  const size_t need = static_cast<size_t>(batch) * B * chunks_for(V) * sizeof(unsigned long long);
+  if (need > JET_STATIC_ACCEPT_SCRATCH_BYTES) return JET_ERR_WORKSPACE;   // beyond the built-in scratch
+
+  // Device address of the built-in array, looked up once per device with that device current.
+  // (In host code the array's name is only a handle; kernels must be given this address.)
+  static unsigned long long* scratch_of_device[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return JET_ERR_CUDA;
+  unsigned long long* scratch = scratch_of_device[dev];
+  if (!scratch) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_accept_scratch) != cudaSuccess || !addr) return JET_ERR_CUDA;
+    scratch = static_cast<unsigned long long*>(addr);
+    scratch_of_device[dev] = scratch;
+  }
+  // Nothing in the scratch has to start at zero: every entry that accept_path_kernel reads was
+  // written by argmax_partial_kernel of the same call.
+  return jet_tree_accept(logits, logits_row_stride, token, parent, depth, anc_mask, n_nodes, batch, B, V,
+                         N, tgt_argmax, accept_len, path, out_tokens, scratch,
+                         JET_STATIC_ACCEPT_SCRATCH_BYTES, stream);
 }
