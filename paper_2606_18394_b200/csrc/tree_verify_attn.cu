@@ -1,7 +1,7 @@
 // jet_tree_verify_attn: tree attention over prefix KV + tree KV under the ancestor mask.
 //
 // Kernel structure (one CTA per SM, warp-specialised):
-//   work item   = (sequence b, KV head g, group of MT 128-row query tiles, key split s).
+//   work item   = (sequence b, KV head g, group of MT 128-row query tiles, key slice s).
 //                 Row r of a query tile is (node v, query head g*G + j) with r = v_local*G + j,
 //                 so all G heads of a KV group share every K/V tile that is loaded.
 //   warp 0      = TMA producer: Q tiles once, then K and V tiles (128 keys) through a ring of
@@ -12,11 +12,14 @@
 //                 applies the key-validity / ancestor-bit mask, keeps the running maximum and sum
 //                 (online softmax with lazy rescaling of O), writes P (bf16) to shared memory in
 //                 the swizzled operand layout, and finally normalises O.
-//   Split-KV    = when there are fewer work items than SMs the key range is cut into `nsplit`
-//                 slices; each CTA then writes a normalised fp32 partial + log-sum-exp to the
-//                 workspace and tree_attn_merge_kernel combines the slices.
+//   key slices  = when there are fewer work items than SMs the key range is cut into `nsplit`
+//                 slices that run as one thread-block cluster.  After the key loop every CTA
+//                 sends its normalised rows and their log-sum-exp to the row's owner CTA through
+//                 distributed shared memory; the owners combine the slices and write the output.
+//                 Nothing goes through global memory and there is no second launch.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
-// loops, outstanding TMA loads are drained, TMEM is released and JET_ERR_TIMEOUT is reported.
+// loops (still taking part in the cluster barriers), outstanding TMA loads are drained, TMEM is
+// released and JET_ERR_TIMEOUT is reported.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -24,12 +27,17 @@
 #include "sm100_ptx.cuh"
 
 namespace jet {
+
+#ifdef JET_TRACE
+long long* g_trace_ptr = nullptr;    // debug builds only
+#endif
+
 namespace {
 
-constexpr int kBM = 128;             // query rows per tile
-constexpr int kBN = 128;             // keys per tile
+constexpr int kBM = 128;               // query rows per tile
+constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr int kMaxSplit = 16;          // largest cluster
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more
 
 struct AttnParams {
@@ -40,13 +48,20 @@ struct AttnParams {
   __nv_bfloat16* out;
   float* lse;
   int32_t* status;
-  float* part_o;
-  float* part_lse;
   int max_pages, paged;
   int batch, B, Hq, Hkv, G, words;
   int nsplit, n_mgroups;
   float scale_log2;   // softmax_scale * log2(e)
+#ifdef JET_TRACE
+  long long* trace;   // 32 clock64() samples per CTA
+#endif
 };
+
+#ifdef JET_TRACE
+#define JET_TR(slot) do { if (p.trace) p.trace[blockIdx.x * 32 + (slot)] = clock64(); } while (0)
+#else
+#define JET_TR(slot) do { } while (0)
+#endif
 
 template <int D, int MT>
 struct Cfg {
@@ -54,26 +69,64 @@ struct Cfg {
   static constexpr int kQBytes = MT * kHalves * kHalfBytes;
   static constexpr int kPBytes = MT * 2 * kHalfBytes;
   static constexpr int kStageBytes = kHalves * kHalfBytes;
-  static constexpr int kStages = (D == 128) ? (MT == 1 ? 4 : 3) : 6;
+  static constexpr int kStages = (D == 128) ? (MT == 1 ? 5 : 3) : 6;
+  static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
   static constexpr int kBarBytes = 256;
-  static constexpr int kSmemBytes = kQBytes + kPBytes + kStages * kStageBytes + kBarBytes + 1024;
+  static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
   static constexpr int kThreads = 128 + 128 * MT;
   static constexpr int kTmemCols = (MT == 1) ? 256 : 512;   // per query tile: S (128) + O (<=128)
+  // slice merge: rows arrive as [source slice][row][D fp32 + lse], padded so that the row-per-thread
+  // stores of a warp spread over all banks
+  static constexpr int kRecvPitch = D * 4 + 16;
+  static constexpr int kStageOff = 0;                              // this CTA's 128 normalised rows
+  static constexpr int kRecvOff = (kBM * kRecvPitch + 1023) / 1024 * 1024;   // rows received from every slice
+  static_assert(kRecvOff + (kBM + kMaxSplit) * kRecvPitch <= kTileBytes, "merge buffers must fit in the tile memory");
 };
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
   enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
-         kCount = 21 };
+         kClusterA = 21, kClusterC = 22, kRecv = 23, kCount = 25 };
 };
+
+// Every wait is bounded: at most kWaitRounds suspensions of kWaitHintNs each (about a second).
+constexpr uint32_t kWaitRounds = 1u << 16;
+constexpr uint32_t kWaitHintNs = 16384;
 
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   bool ok = false;
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (ptx::mbar_test(bar, parity)) { ok = true; break; }
-    if ((i & 1023u) == 1023u && *abort_flag) break;
+  for (uint32_t i = 0; i < kWaitRounds; ++i) {
+    if (ptx::mbar_try_wait(bar, parity, kWaitHintNs)) { ok = true; break; }
+    if (*abort_flag) break;
   }
   if (!ok) *abort_flag = 1u;
   return __all_sync(0xffffffffu, ok);
+}
+
+// The same for a barrier that other CTAs of the cluster arrive on / copy into (acquire at cluster scope);
+// called by every thread of the CTA, returns a CTA-uniform result.
+__device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  bool ok = false;
+  for (uint32_t i = 0; i < kWaitRounds; ++i) {
+    if (ptx::mbar_try_wait_cluster(bar, parity, kWaitHintNs)) { ok = true; break; }
+    if (*abort_flag) break;
+  }
+  if (!ok) *abort_flag = 1u;
+  return __syncthreads_and(ok ? 1 : 0) != 0;
+}
+
+// Cluster-wide rendezvous built from one mbarrier per CTA (count = cluster size): after a CTA-wide
+// barrier one thread arrives on the barrier of every CTA of the cluster, then everybody waits for
+// all `nsplit` arrivals on the local one.
+__device__ __forceinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag) {
+  __syncthreads();
+  if (threadIdx.x == 0)
+    for (int c = 0; c < nsplit; ++c) ptx::mbar_arrive_remote(ptx::map_to_rank(local_bar, c));
+  return bounded_wait_cluster(local_bar, 0, abort_flag);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 pk = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&pk);
 }
 
 template <int D, int MT>
@@ -84,49 +137,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   using C = Cfg<D, MT>;
   constexpr int kHalves = C::kHalves;
   constexpr int kStages = C::kStages;
-
-  // ---------------- work item
-  const int split = blockIdx.x % p.nsplit;
-  const int unit = blockIdx.x / p.nsplit;
-  const int mgroup = unit % p.n_mgroups;
-  const int bg = unit / p.n_mgroups;
-  const int g = bg % p.Hkv;
-  const int b = bg / p.Hkv;
-  const int G = p.G;
-  const int npt = kBM / G;                       // nodes per query tile
-  const int L = p.seq_len[b];
-  const int n = min(p.n_nodes[b], p.B);
-  const int node_lo = mgroup * MT * npt;
-  const int node_hi = min(p.B, node_lo + MT * npt);
-  const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-  const int ntree = min(n, node_hi);                         // tree keys any row here can see
-  const int TP = (L + kBN - 1) / kBN;
-  const int TT = (ntree + kBN - 1) / kBN;
-  const int T_all = TP + TT;
-  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split) / p.nsplit);
-  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1)) / p.nsplit);
-  const int T = t_hi - t_lo;
-
-  float* part_o = p.part_o + (static_cast<size_t>(unit) * p.nsplit + split) * MT * kBM * D;
-  float* part_lse = p.part_lse + (static_cast<size_t>(unit) * p.nsplit + split) * MT * kBM;
-
-  if (node_lo >= n || T == 0) {
-    // No live node in this CTA, or an empty key slice (uniform for the whole CTA).
-    if (p.nsplit == 1) {
-      for (int i = tid; i < (node_hi - node_lo) * G * (D / 8); i += C::kThreads) {
-        const int row = i / (D / 8), c8 = i - row * (D / 8);
-        const int v = node_lo + row / G, h = g * G + row % G;
-        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
-            make_uint4(0u, 0u, 0u, 0u);
-        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = -INFINITY;
-      }
-    } else {
-      for (int i = tid; i < MT * kBM; i += C::kThreads) part_lse[i] = -INFINITY;
-    }
-    return;
-  }
+  if (tid == 0) JET_TR(0);
 
   // ---------------- shared memory carve-up (1024-byte aligned for the 128-byte swizzle)
   extern __shared__ uint8_t smem_raw[];
@@ -143,41 +155,104 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
   auto bar = [&](int idx) { return sBar + 8u * idx; };
 
-  if (tid == 0) {
+  // ---------------- set-up that touches no global memory (overlaps the previous kernel's tail)
+  if (warp == 0 && lane == 0) {
     ptx::mbar_init(bar(Bars::kQFull), 1);
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(bar(Bars::kKvFull + s), 1);
       ptx::mbar_init(bar(Bars::kKvEmpty + s), 1);
     }
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_q);
+    ptx::prefetch_tmap(&tm_k);
+    ptx::prefetch_tmap(&tm_v);
+  } else if (warp == 1 && lane == 0) {
     for (int mt = 0; mt < MT; ++mt) {
       ptx::mbar_init(bar(Bars::kSFull + mt), 1);
       ptx::mbar_init(bar(Bars::kSFree + mt), 128);
       ptx::mbar_init(bar(Bars::kPFull + mt), 128);
       ptx::mbar_init(bar(Bars::kODone + mt), 1);
     }
+    ptx::mbar_init(bar(Bars::kClusterA), p.nsplit);
+    ptx::mbar_init(bar(Bars::kClusterC), p.nsplit);
+    for (int mt = 0; mt < MT; ++mt) {
+      // slice merge: every slice sends this CTA its block of rows of query tile mt
+      const int rows_per = (kBM + p.nsplit - 1) / p.nsplit;
+      const int own_n = max(0, min(rows_per, kBM - static_cast<int>(blockIdx.x % p.nsplit) * rows_per));
+      ptx::mbar_init(bar(Bars::kRecv + mt), 1);
+      if (p.nsplit > 1) ptx::mbar_arrive_expect_tx(bar(Bars::kRecv + mt), p.nsplit * own_n * C::kRecvPitch);
+    }
     *abort_flag = 0u;
     ptx::fence_mbar_init();
-    ptx::prefetch_tmap(&tm_q);
-    ptx::prefetch_tmap(&tm_k);
-    ptx::prefetch_tmap(&tm_v);
     ptx::prefetch_tmap(&tm_tk);
     ptx::prefetch_tmap(&tm_tv);
-  }
-  if (warp == 2) {
+  } else if (warp == 2) {
     ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
     ptx::tmem_relinquish();
   }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  // TMEM columns: query tile mt owns [mt*256, mt*256+128) for S and [mt*256+128, mt*256+128+D) for O.
+  ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
+
+  // ---------------- work item
+  const int split = blockIdx.x % p.nsplit;     // = rank in the cluster
+  const int unit = blockIdx.x / p.nsplit;
+  const int mgroup = unit % p.n_mgroups;
+  const int bg = unit / p.n_mgroups;
+  const int g = bg % p.Hkv;
+  const int b = bg / p.Hkv;
+  const int G = p.G;
+  const int npt = kBM / G;                       // nodes per query tile
+  const int L = p.seq_len[b];
+  const int n = min(p.n_nodes[b], p.B);
+  const int node_lo = mgroup * MT * npt;
+  const int node_hi = min(p.B, node_lo + MT * npt);
+  const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
+  const int ntree = min(n, node_hi);                         // tree keys any row here can see
+  const int TP = (L + kBN - 1) / kBN;
+  const int TT = (ntree + kBN - 1) / kBN;
+  const int T_all = TP + TT;
+  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split) / p.nsplit);
+  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1)) / p.nsplit);
+  const int T = t_hi - t_lo;
+  if (tid == 0) JET_TR(1);
+  const bool dead_unit = node_lo >= n;           // no live node: uniform over the cluster
+  const bool has_work = !dead_unit && T > 0;
 
   // Valid keys of tile t (global tile index): prefix tiles first, then tree tiles.
   auto tile_valid = [&](int t) { return t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN); };
 
-  if (warp == 0) {
-    // =========================================================== TMA producer
+  // One K or V tile into ring slot `item % kStages` (warp 0, all lanes).
+  auto issue_kv = [&](int item) {
+    const int t = t_lo + (item >> 1), kv = item & 1, stage = item % kStages;
+    const uint32_t dst = sKV + stage * C::kStageBytes;
+    const uint32_t full = bar(Bars::kKvFull + stage);
+    if (t < TP) {
+      if (!p.paged) {
+        if (lane == 0) {
+          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+          for (int h = 0; h < kHalves; ++h)
+            ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v : &tm_k, full, h * 64, g, t * kBN, b);
+        }
+      } else {
+        const int npages = min(8, (L - t * kBN + 15) / 16);
+        if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
+        __syncwarp();
+        if (lane < npages) {
+          const int page = p.page_table[static_cast<size_t>(b) * p.max_pages + t * 8 + lane];
+          for (int h = 0; h < kHalves; ++h)
+            ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page * 16);
+        }
+      }
+    } else if (lane == 0) {
+      ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+      for (int h = 0; h < kHalves; ++h)
+        ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_tv : &tm_tk, full, h * 64, g, (t - TP) * kBN, b);
+    }
+    __syncwarp();
+  };
+
+  // The producer starts the first loads before the CTA-wide set-up barrier: its own barriers are ready.
+  int issued = 0;
+  if (warp == 0 && has_work) {
     if (lane == 0) {
       ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
       for (int mt = 0; mt < n_mt; ++mt)
@@ -185,162 +260,156 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
                            b * p.B + node_lo + mt * npt);
     }
-    int issued = 0;
-    bool ok = true;
-    for (int t = t_lo; t < t_hi && ok; ++t) {
-      for (int kv = 0; kv < 2 && ok; ++kv) {
+    __syncwarp();
+    for (; issued < min(kStages, 2 * T); ++issued) issue_kv(issued);
+    if (lane == 0) JET_TR(14);
+  }
+  ptx::tc_fence_before();
+  if (p.nsplit > 1) {
+    // the barriers of every CTA of the cluster must exist before any CTA arrives on them remotely;
+    // this is straight-line code from the kernel entry, so the hardware cluster barrier is safe here
+    __syncwarp();
+    ptx::cluster_sync_all();
+  } else {
+    __syncthreads();
+  }
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // TMEM columns: query tile mt owns [mt*256, mt*256+128) for S and [mt*256+128, mt*256+128+D) for O.
+  if (tid == 0) JET_TR(15);
+
+  // per-row state of the softmax threads, live until the epilogue
+  float m_used = -INFINITY;     // running reference maximum (raw score units)
+  float l = 0.0f;               // running sum of exp2((s - m_used) * sl2)
+  bool row_ok = true;           // false once a bounded wait of this warp expired
+
+  if (has_work) {
+    if (warp == 0) {
+      // =========================================================== TMA producer (remaining tiles)
+      bool ok = true;
+      for (; issued < 2 * T && ok; ++issued) {
         const int stage = issued % kStages;
-        if (issued >= kStages)
-          ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag);
+        ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag);
         if (!ok) break;
-        const uint32_t dst = sKV + stage * C::kStageBytes;
-        const uint32_t full = bar(Bars::kKvFull + stage);
-        if (t < TP) {
-          if (!p.paged) {
-            if (lane == 0) {
-              ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-              for (int h = 0; h < kHalves; ++h)
-                ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v : &tm_k, full, h * 64, g, t * kBN, b);
-            }
-          } else {
-            const int npages = min(8, (L - t * kBN + 15) / 16);
-            if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
-            __syncwarp();
-            if (lane < npages) {
-              const int page = p.page_table[static_cast<size_t>(b) * p.max_pages + t * 8 + lane];
-              for (int h = 0; h < kHalves; ++h)
-                ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g,
-                                 page * 16);
-            }
+        issue_kv(issued);
+      }
+      if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
+        // drain: every load that was issued must land before the CTA may exit
+        for (int s = 0; s < kStages; ++s) {
+          if (issued > s) {
+            const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
+            bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag);
           }
-        } else if (lane == 0) {
-          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-          for (int h = 0; h < kHalves; ++h)
-            ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_tv : &tm_tk, full, h * 64, g, (t - TP) * kBN, b);
         }
-        ++issued;
-        __syncwarp();
+        bounded_wait(bar(Bars::kQFull), 0, abort_flag);
       }
-    }
-    if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
-      // drain: every load that was issued must land before the CTA may exit
-      for (int s = 0; s < kStages; ++s) {
-        if (issued > s) {
-          const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
-          bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag);
-        }
-      }
-      bounded_wait(bar(Bars::kQFull), 0, abort_flag);
-    }
-  } else if (warp == 1) {
-    // =========================================================== tcgen05 issuer
-    constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
-    constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
-    bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag);
+    } else if (warp == 1) {
+      // =========================================================== tcgen05 issuer
+      constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
+      constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
+      bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag);
+      if (lane == 0) JET_TR(2);
 
-    auto issue_qk = [&](int mt, int stage) {      // S[mt] = Q[mt] K^T
-      if (lane == 0) {
-        const uint32_t d_tmem = tmem_base + mt * 256;
+      auto issue_qk = [&](int mt, int stage) {      // S[mt] = Q[mt] K^T
+        if (lane == 0) {
+          const uint32_t d_tmem = tmem_base + mt * 256;
 #pragma unroll
-        for (int kd = 0; kd < D / 16; ++kd) {
-          const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
-          const uint64_t a = ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0);
-          const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0);
-          ptx::umma_ss(d_tmem, a, bdesc, idesc_qk, kd > 0 ? 1u : 0u);
+          for (int kd = 0; kd < D / 16; ++kd) {
+            const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
+            const uint64_t a = ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0);
+            const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0);
+            ptx::umma_ss(d_tmem, a, bdesc, idesc_qk, kd > 0 ? 1u : 0u);
+          }
         }
-      }
-    };
-    auto issue_pv = [&](int mt, int stage, bool first) {   // O[mt] (+)= P[mt] V
-      if (lane == 0) {
-        const uint32_t d_tmem = tmem_base + mt * 256 + 128;
+      };
+      auto issue_pv = [&](int mt, int stage, bool first) {   // O[mt] (+)= P[mt] V
+        if (lane == 0) {
+          const uint32_t d_tmem = tmem_base + mt * 256 + 128;
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk) {
-          const uint64_t a = ptx::smem_desc_sw128(sP + mt * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0);
-          const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes);
-          ptx::umma_ss(d_tmem, a, bdesc, idesc_pv, (first && kk == 0) ? 0u : 1u);
+          for (int kk = 0; kk < kBN / 16; ++kk) {
+            const uint64_t a =
+                ptx::smem_desc_sw128(sP + mt * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0);
+            const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes);
+            ptx::umma_ss(d_tmem, a, bdesc, idesc_pv, (first && kk == 0) ? 0u : 1u);
+          }
         }
-      }
-    };
+      };
 
-    for (int tl = 0; tl < T && ok; ++tl) {
-      if (tl == 0) {
-        const int stage = 0;
-        ok = bounded_wait(bar(Bars::kKvFull + stage), 0, abort_flag);
-        if (!ok) break;
-        ptx::tc_fence_after();
-        for (int mt = 0; mt < n_mt; ++mt) {
-          issue_qk(mt, stage);
-          if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
-        }
-        if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-        __syncwarp();
-      }
-      if (tl + 1 < T) {        // next tile's scores as soon as the softmax groups release S
-        const int item = 2 * (tl + 1), stage = item % kStages;
-        ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
-        for (int mt = 0; mt < n_mt && ok; ++mt) {
-          ok = bounded_wait(bar(Bars::kSFree + mt), tl & 1, abort_flag);
+      for (int tl = 0; tl < T && ok; ++tl) {
+        if (tl == 0) {
+          ok = bounded_wait(bar(Bars::kKvFull + 0), 0, abort_flag);
           if (!ok) break;
+          if (lane == 0) JET_TR(3);
           ptx::tc_fence_after();
-          issue_qk(mt, stage);
-          if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
+          for (int mt = 0; mt < n_mt; ++mt) {
+            issue_qk(mt, 0);
+            if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
+          }
+          if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + 0));
           __syncwarp();
         }
-        if (!ok) break;
-        if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-        __syncwarp();
-      }
-      {
-        const int item = 2 * tl + 1, stage = item % kStages;
-        ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
-        if (!ok) break;
-        const int valid = tile_valid(t_lo + tl);
-        if (valid < kBN) {
-          // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
-          uint8_t* vt = gen_kv + stage * C::kStageBytes;
-          const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
-          for (int h = 0; h < kHalves; ++h)
-            for (int i = lane; i < chunks; i += 32)
-              *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-        }
-        for (int mt = 0; mt < n_mt && ok; ++mt) {
-          ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag);
+        if (tl + 1 < T) {        // next tile's scores as soon as the softmax groups release S
+          const int item = 2 * (tl + 1), stage = item % kStages;
+          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
+          for (int mt = 0; mt < n_mt && ok; ++mt) {
+            ok = bounded_wait(bar(Bars::kSFree + mt), tl & 1, abort_flag);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            issue_qk(mt, stage);
+            if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
+            __syncwarp();
+          }
           if (!ok) break;
-          ptx::tc_fence_after();
-          issue_pv(mt, stage, tl == 0);
-          if (lane == 0) ptx::umma_commit(bar(Bars::kODone + mt));
+          if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
           __syncwarp();
         }
-        if (!ok) break;
-        if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-        __syncwarp();
+        {
+          const int item = 2 * tl + 1, stage = item % kStages;
+          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
+          if (!ok) break;
+          const int valid = tile_valid(t_lo + tl);
+          if (valid < kBN) {
+            // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
+            uint8_t* vt = gen_kv + stage * C::kStageBytes;
+            const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
+            for (int h = 0; h < kHalves; ++h)
+              for (int i = lane; i < chunks; i += 32)
+                *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+          }
+          for (int mt = 0; mt < n_mt && ok; ++mt) {
+            ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            issue_pv(mt, stage, tl == 0);
+            if (lane == 0) ptx::umma_commit(bar(Bars::kODone + mt));
+            __syncwarp();
+          }
+          if (!ok) break;
+          if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+          __syncwarp();
+        }
       }
-    }
-  } else if (warp >= 4) {
-    // =========================================================== softmax / epilogue warpgroups
-    const int mt = (warp - 4) >> 2;
-    if (mt < n_mt) {
+    } else if (warp >= 4 && ((warp - 4) >> 2) < n_mt) {
+      // =========================================================== softmax warpgroups
+      const int mt = (warp - 4) >> 2;
       const int r = tid - 128 - mt * 128;                     // row of the query tile = TMEM lane
       const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
       const uint32_t tS = tmem_base + lane_base + mt * 256;
       const uint32_t tO = tS + 128;
       const int v = node_lo + mt * npt + r / G;
-      const int h = g * G + r % G;
       const bool row_live = v < n;
       const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
       uint8_t* my_p = gen_p + mt * 2 * kHalfBytes + r * 128;
       const float sl2 = p.scale_log2;
-
-      float m_used = -INFINITY;     // running reference maximum (raw score units)
-      float l = 0.0f;               // running sum of exp2((s - m_used) * sl2)
       bool ok = true;
 
       for (int tl = 0; tl < T && ok; ++tl) {
         const int t = t_lo + tl;
         // visibility bits of this row for the four 32-key chunks of the tile
         uint32_t vis[4];
+        const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
         if (t < TP) {
           const int valid = L - t * kBN;
 #pragma unroll
@@ -353,29 +422,37 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
           for (int c = 0; c < 4; ++c) vis[c] = (row_live && w0 + c < p.words) ? __ldg(mask_row + w0 + c) : 0u;
         }
-        const bool all_visible = (vis[0] & vis[1] & vis[2] & vis[3]) == 0xFFFFFFFFu;
 
         ok = bounded_wait(bar(Bars::kSFull + mt), tl & 1, abort_flag);
         if (!ok) break;
         ptx::tc_fence_after();
+        if (tid == 128 && tl < 1) JET_TR(4);
 
-        // ---- pass 1: row maximum over visible keys
-        float m_tile = -INFINITY;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t s[32];
-          ptx::tmem_ld32(tS + c * 32, s);
-          ptx::tmem_wait_ld();
-          if (all_visible) {
+        // ---- scores of this row: all 128 into registers, then S is free for the next Q K^T
+        uint32_t s[4][32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) m_tile = fmaxf(m_tile, __uint_as_float(s[j]));
-          } else {
-            const uint32_t bits = vis[c];
+        for (int c = 0; c < 4; ++c) ptx::tmem_ld32(tS + c * 32, s[c]);
+        ptx::tmem_wait_ld();
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(bar(Bars::kSFree + mt));
+
+        // ---- row maximum over visible keys
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (full_tile) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[c][j]));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              if ((bits >> j) & 1u) m_tile = fmaxf(m_tile, __uint_as_float(s[j]));
-          }
+              if ((vis[c] >> j) & 1u) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[c][j]));
         }
+        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        if (tid == 128 && tl < 1) JET_TR(5);
+
         // ---- running maximum with lazy rescaling
         float factor = 1.0f;
         if (m_tile > -INFINITY) {
@@ -386,6 +463,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             m_used = m_tile;
           }
         }
+        if (tid == 128 && tl < 1) JET_TR(16);
         const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
         const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
 
@@ -397,25 +475,26 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ptx::tc_fence_after();
         }
 
-        // ---- pass 2: probabilities, row sum, P -> shared memory (swizzled bf16)
-        float row_sum = 0.0f;
-#pragma unroll 1
+        // ---- probabilities, row sum, P -> shared memory (swizzled bf16).  Each 32-key chunk is done in
+        //      stages (scale, exp2, mask, sum, pack) so that the 32 independent exp2 are in flight together.
+        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t s[32];
-          ptx::tmem_ld32(tS + c * 32, s);
-          ptx::tmem_wait_ld();
-          const uint32_t bits = all_visible ? 0xFFFFFFFFu : vis[c];
+          float e[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(s[c][j]), sl2, -m_ref);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) e[j] = exp2f(e[j]);
+          if (!full_tile) {
+            const uint32_t bits = vis[c];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) e[j] = ((bits >> j) & 1u) ? e[j] : 0.0f;
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
           uint32_t packed[16];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float p0 = exp2f(fmaf(__uint_as_float(s[j]), sl2, -m_ref));
-            float p1 = exp2f(fmaf(__uint_as_float(s[j + 1]), sl2, -m_ref));
-            if (!((bits >> j) & 1u)) p0 = 0.0f;
-            if (!((bits >> (j + 1)) & 1u)) p1 = 0.0f;
-            row_sum += p0 + p1;
-            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-            packed[j / 2] = *reinterpret_cast<uint32_t*>(&pk);
-          }
+          for (int j = 0; j < 16; ++j) packed[j] = pack_bf16(e[2 * j], e[2 * j + 1]);
           // chunk c covers keys [32c, 32c+32): 64-key block c/2, 16-byte chunks (c%2)*4 .. +3
           uint8_t* dst = my_p + (c >> 1) * kHalfBytes;
 #pragma unroll
@@ -425,9 +504,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
           }
         }
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kSFree + mt));          // S may be overwritten by the next Q K^T
-        l = l * factor + row_sum;
+        l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+        if (tid == 128 && tl < 1) JET_TR(17);
 
         if (need_rescale && tl > 0) {
 #pragma unroll 1
@@ -442,116 +520,184 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ptx::tmem_wait_st();
         }
         ptx::fence_proxy_async_smem();
+        if (tid == 128 && tl < 1) JET_TR(18);
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar(Bars::kPFull + mt));
+        if (tid == 128 && tl < 1) JET_TR(6);
       }
-
-      // ---- epilogue: O / l
+      if (tid == 128) JET_TR(10);
+      // O complete once the last P V has been committed
       if (ok) ok = bounded_wait(bar(Bars::kODone + mt), (T - 1) & 1, abort_flag);
-      if (ok) {
-        ptx::tc_fence_after();
-        const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-        const float lse = l > 0.0f ? (m_used * sl2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
-        const bool in_range = v < p.B;
-        if (p.nsplit == 1) {
-          __nv_bfloat16* orow = p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D;
+      if (ok) ptx::tc_fence_after();
+      row_ok = ok;
+      if (tid == 128) JET_TR(11);
+    }
+  }
+
+  // =============================================================== epilogue
+  const bool softmax_thread = has_work && warp >= 4 && ((warp - 4) >> 2) < n_mt;
+  const int e_mt = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
+  const int e_r = (tid - 128) & 127;                           // its row within the query tile
+  const uint32_t e_tO = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + e_mt * 256 + 128;
+  const float e_inv = l > 0.0f ? 1.0f / l : 0.0f;
+  const float e_lse2 = l > 0.0f ? m_used * p.scale_log2 + log2f(l) : -INFINITY;   // log2 of the row's sum
+
+  if (p.nsplit == 1) {
+    if (dead_unit || !has_work) {
+      // no live node here (or nothing to attend to): the rows of this CTA are zero
+      for (int i = tid; i < (node_hi - node_lo) * G * (D / 8); i += C::kThreads) {
+        const int row = i / (D / 8), c8 = i - row * (D / 8);
+        const int v = node_lo + row / G, h = g * G + row % G;
+        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+            make_uint4(0u, 0u, 0u, 0u);
+        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = -INFINITY;
+      }
+    } else if (softmax_thread && row_ok) {
+      const int v = node_lo + e_mt * npt + e_r / G;
+      const int h = g * G + e_r % G;
+      const bool row_live = v < n, in_range = v < p.B;
+      __nv_bfloat16* orow = p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D;
 #pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            ptx::tmem_ld32(tO + c * 32, o);
-            ptx::tmem_wait_ld();
-            if (in_range) {
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        ptx::tmem_ld32(e_tO + c * 32, o);
+        ptx::tmem_wait_ld();
+        if (in_range) {
 #pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4) {
-                uint32_t w[4];
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t w[4];
 #pragma unroll
-                for (int k2 = 0; k2 < 4; ++k2) {
-                  const float a0 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2]) * inv : 0.0f;
-                  const float a1 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2 + 1]) * inv : 0.0f;
-                  __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
-                  w[k2] = *reinterpret_cast<uint32_t*>(&pk);
-                }
-                *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-              }
+            for (int k2 = 0; k2 < 4; ++k2) {
+              const float a0 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2]) * e_inv : 0.0f;
+              const float a1 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2 + 1]) * e_inv : 0.0f;
+              w[k2] = pack_bf16(a0, a1);
             }
+            *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
-          if (p.lse && in_range) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = row_live ? lse : -INFINITY;
-        } else {
-          float* prow = part_o + (static_cast<size_t>(mt) * kBM + r) * D;
+        }
+      }
+      if (p.lse && in_range)
+        p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = row_live ? e_lse2 * 0.6931471805599453f : -INFINITY;
+    }
+  } else if (dead_unit) {
+    // uniform over the cluster: slice 0 clears the unit's rows, nobody takes part in a cluster barrier
+    if (split == 0) {
+      for (int i = tid; i < (node_hi - node_lo) * G * (D / 8); i += C::kThreads) {
+        const int row = i / (D / 8), c8 = i - row * (D / 8);
+        const int v = node_lo + row / G, h = g * G + row % G;
+        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+            make_uint4(0u, 0u, 0u, 0u);
+        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = -INFINITY;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------- slice merge through DSMEM
+    // One round per query tile.  The tile's 128 rows are dealt out to the slices in blocks of
+    // rows_per (row r belongs to slice r / rows_per).  Every CTA stages its normalised rows --
+    // D fp32 values followed by the row's log2-sum-exp -- in its own shared memory, then sends
+    // each owner its block with one bulk copy that is credited to the owner's kRecv barrier.
+    // Both buffers overlay the tile memory, which is idle once every CTA has left its key loop.
+    const int S = p.nsplit;
+    const int rows_per = (kBM + S - 1) / S;
+    const int own_lo = split * rows_per;
+    const int own_n = max(0, min(rows_per, kBM - own_lo));
+    uint8_t* stage = smem_gen + C::kStageOff;
+    const uint8_t* recv = smem_gen + C::kRecvOff;
+    // A: every CTA of the cluster has left its key loop, so tile memory may be overwritten
+    bool merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag);
+    if (tid == 128) JET_TR(7);
+    for (int mt = 0; mt < MT; ++mt) {
+      if (mt > 0) {
+        // C: everybody has combined the previous tile's rows, so both buffers are free again
+        merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag) && merge_ok;
+      }
+      if (warp >= 4 && ((warp - 4) >> 2) == mt) {
+        uint8_t* srow = stage + e_r * C::kRecvPitch;
+        const bool active = softmax_thread && row_ok;           // warp-uniform
+        if (active) {
 #pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
-            ptx::tmem_ld32(tO + c * 32, o);
+            ptx::tmem_ld32(e_tO + c * 32, o);
             ptx::tmem_wait_ld();
 #pragma unroll
             for (int q4 = 0; q4 < 8; ++q4)
-              *reinterpret_cast<float4*>(prow + c * 32 + q4 * 4) =
-                  make_float4(__uint_as_float(o[q4 * 4]) * inv, __uint_as_float(o[q4 * 4 + 1]) * inv,
-                              __uint_as_float(o[q4 * 4 + 2]) * inv, __uint_as_float(o[q4 * 4 + 3]) * inv);
+              *reinterpret_cast<float4*>(srow + (c * 32 + q4 * 4) * 4) =
+                  make_float4(__uint_as_float(o[q4 * 4]) * e_inv, __uint_as_float(o[q4 * 4 + 1]) * e_inv,
+                              __uint_as_float(o[q4 * 4 + 2]) * e_inv, __uint_as_float(o[q4 * 4 + 3]) * e_inv);
           }
-          part_lse[mt * kBM + r] = row_live ? lse : -INFINITY;
         }
+        // rows this CTA computed nothing for (empty key slice, tile without nodes) are marked absent
+        *reinterpret_cast<float*>(srow + D * 4) = (active && l > 0.0f) ? e_lse2 : -INFINITY;
+        ptx::fence_proxy_async_smem();
+      }
+      __syncthreads();
+      if (tid < S && merge_ok) {
+        const int dst_lo = tid * rows_per;
+        const int dst_n = max(0, min(rows_per, kBM - dst_lo));
+        if (dst_n > 0)
+          ptx::bulk_copy_to_cluster(
+              ptx::map_to_rank(smem_base + C::kRecvOff + static_cast<uint32_t>(split * rows_per * C::kRecvPitch), tid),
+              smem_base + C::kStageOff + static_cast<uint32_t>(dst_lo * C::kRecvPitch),
+              static_cast<uint32_t>(dst_n * C::kRecvPitch), ptx::map_to_rank(bar(Bars::kRecv + mt), tid));
+      }
+      // all blocks of this CTA's rows have arrived (always waited for, so that the CTA never exits
+      // while copies into its memory are in flight)
+      if (tid == 128 && mt == 0) JET_TR(8);
+      const bool recv_ok = bounded_wait_cluster(bar(Bars::kRecv + mt), 0, abort_flag) && merge_ok;
+      if (tid == 128 && mt == 0) JET_TR(9);
+      const int items = recv_ok ? own_n * (D / 8) : 0;
+      for (int i = tid; i < items; i += C::kThreads) {
+        const int rl = i / (D / 8), c8 = i - rl * (D / 8);
+        const int R = mt * kBM + own_lo + rl;                  // row within the unit
+        const int v = node_lo + R / G, h = g * G + R % G;
+        if (v >= p.B) continue;
+        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        float lse2 = -INFINITY;
+        if (v < n) {
+          float mx = -INFINITY;
+          for (int c = 0; c < S; ++c)
+            mx = fmaxf(mx, *reinterpret_cast<const float*>(recv + (c * rows_per + rl) * C::kRecvPitch + D * 4));
+          float wsum = 0.0f;
+          if (mx > -INFINITY) {
+            for (int c = 0; c < S; ++c) {
+              const uint8_t* src = recv + (c * rows_per + rl) * C::kRecvPitch;
+              const float ls = *reinterpret_cast<const float*>(src + D * 4);
+              if (ls == -INFINITY) continue;
+              const float w = exp2f(ls - mx);
+              wsum += w;
+              const float4 x0 = *reinterpret_cast<const float4*>(src + c8 * 32);
+              const float4 x1 = *reinterpret_cast<const float4*>(src + c8 * 32 + 16);
+              acc[0] += w * x0.x; acc[1] += w * x0.y; acc[2] += w * x0.z; acc[3] += w * x0.w;
+              acc[4] += w * x1.x; acc[5] += w * x1.y; acc[6] += w * x1.z; acc[7] += w * x1.w;
+            }
+            const float inv = 1.0f / wsum;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] *= inv;
+            lse2 = mx + log2f(wsum);
+          }
+        }
+        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+            make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                       pack_bf16(acc[6], acc[7]));
+        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
       }
     }
   }
 
   // ---------------- teardown
+  if (tid == 128) JET_TR(12);
+  ptx::grid_dep_launch();
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 2) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, C::kTmemCols);
   }
-  if (tid == 0 && *abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
-}
-
-// Combines the key slices: out = sum_s exp(lse_s - lse) * O_s, lse = log sum_s exp(lse_s).
-template <int D, int MT>
-__global__ void __launch_bounds__(256)
-tree_attn_merge_kernel(const AttnParams p) {
-  constexpr int kRowsPerBlock = 256 / (D / 8);
-  const int unit = blockIdx.y;
-  const int mgroup = unit % p.n_mgroups;
-  const int bg = unit / p.n_mgroups;
-  const int g = bg % p.Hkv, b = bg / p.Hkv;
-  const int row = blockIdx.x * kRowsPerBlock + threadIdx.x / (D / 8);   // row within the MT*128 group
-  const int c8 = threadIdx.x % (D / 8);
-  const int npt = kBM / p.G;
-  const int v = mgroup * MT * npt + row / p.G;
-  const int h = g * p.G + row % p.G;
-  if (v >= p.B) return;
-  const int n = min(p.n_nodes[b], p.B);
-  __nv_bfloat16* orow = p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8;
-  float* lse_out = p.lse ? p.lse + (static_cast<size_t>(b) * p.Hq + h) * p.B + v : nullptr;
-  if (v >= n) {
-    *reinterpret_cast<uint4*>(orow) = make_uint4(0u, 0u, 0u, 0u);
-    if (lse_out && c8 == 0) *lse_out = -INFINITY;
-    return;
+  if (tid == 0) {
+    JET_TR(13);
+    if (*abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
   }
-  const size_t base = static_cast<size_t>(unit) * p.nsplit;
-  float m = -INFINITY;
-  for (int s = 0; s < p.nsplit; ++s) m = fmaxf(m, p.part_lse[(base + s) * MT * kBM + row]);
-  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  float wsum = 0.0f;
-  for (int s = 0; s < p.nsplit; ++s) {
-    const float ls = p.part_lse[(base + s) * MT * kBM + row];
-    if (ls == -INFINITY) continue;
-    const float w = __expf(ls - m);
-    wsum += w;
-    const float4* src = reinterpret_cast<const float4*>(p.part_o + ((base + s) * MT * kBM + row) * D + c8 * 8);
-    const float4 x0 = src[0], x1 = src[1];
-    acc[0] += w * x0.x; acc[1] += w * x0.y; acc[2] += w * x0.z; acc[3] += w * x0.w;
-    acc[4] += w * x1.x; acc[5] += w * x1.y; acc[6] += w * x1.z; acc[7] += w * x1.w;
-  }
-  const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
-  uint32_t w4[4];
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    __nv_bfloat162 pk = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
-    w4[k] = *reinterpret_cast<uint32_t*>(&pk);
-  }
-  *reinterpret_cast<uint4*>(orow) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-  if (lse_out && c8 == 0) *lse_out = wsum > 0.0f ? m + __logf(wsum) : -INFINITY;
 }
 
 // ------------------------------------------------------------------------------------------ host
@@ -598,29 +744,35 @@ int sm_count() {
 struct Plan {
   int mt;          // query tiles per CTA (1 or 2)
   int n_mgroups;   // groups of mt query tiles per (sequence, KV head)
-  int units;
-  int nsplit;
+  int units;       // work items before key slicing
+  int nsplit;      // key slices = cluster size
 };
 
+// Picks the query-tile grouping and the number of key slices.  Cost model: waves of CTAs x key tiles
+// per CTA x query tiles per CTA; on a tie the grouping that loads K/V fewer times wins.
 Plan make_plan(int batch, int B, int Hq, int Hkv, int max_seq_len) {
-  Plan pl;
   const int G = Hq / Hkv;
   const int rows = B * G;
-  pl.mt = rows > kBM ? 2 : 1;
-  pl.n_mgroups = (rows + pl.mt * kBM - 1) / (pl.mt * kBM);
-  pl.units = batch * Hkv * pl.n_mgroups;
   const int tiles = (max_seq_len + kBN - 1) / kBN + (B + kBN - 1) / kBN;
-  int ns = sm_count() / pl.units;
-  if (ns < 1) ns = 1;
-  if (ns > tiles) ns = tiles;
-  pl.nsplit = ns;
-  return pl;
-}
-
-size_t partial_bytes(const Plan& pl, int D) {
-  if (pl.nsplit == 1) return 0;
-  const size_t rows = static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM;
-  return round_up(rows * D * sizeof(float), 256) + round_up(rows * sizeof(float), 256);
+  const int sms = sm_count();
+  Plan best{};
+  long best_cost = -1;
+  for (int mt = (rows > kBM ? 2 : 1); mt >= 1; --mt) {
+    Plan pl;
+    pl.mt = mt;
+    pl.n_mgroups = (rows + mt * kBM - 1) / (mt * kBM);
+    pl.units = batch * Hkv * pl.n_mgroups;
+    int ns = sms / pl.units;
+    ns = ns < 1 ? 1 : ns;
+    ns = ns > kMaxSplit ? kMaxSplit : ns;
+    ns = ns > tiles ? tiles : ns;
+    pl.nsplit = ns;
+    const long ctas = static_cast<long>(pl.units) * ns;
+    const long waves = (ctas + sms - 1) / sms;
+    const long cost = waves * ((tiles + ns - 1) / ns) * mt;
+    if (best_cost < 0 || cost < best_cost) { best = pl; best_cost = cost; }
+  }
+  return best;
 }
 
 template <int D, int MT>
@@ -632,12 +784,28 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
     if (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::kSmemBytes) != cudaSuccess)
       return JET_ERR_CUDA;
+    if (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) !=
+        cudaSuccess)
+      return JET_ERR_CUDA;
     configured = true;
   }
-  tree_attn_kernel<D, MT><<<pl.units * pl.nsplit, C::kThreads, C::kSmemBytes, st>>>(tq, tk, tv, ttk, ttv, p);
-  if (pl.nsplit > 1) {
-    constexpr int kRowsPerBlock = 256 / (D / 8);
-    tree_attn_merge_kernel<D, MT><<<dim3(MT * kBM / kRowsPerBlock, pl.units), 256, 0, st>>>(p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(pl.units * pl.nsplit);
+  cfg.blockDim = dim3(C::kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attrs[2];
+  int na = 0;
+  attrs[na].id = cudaLaunchAttributeClusterDimension;
+  attrs[na].val.clusterDim.x = pl.nsplit;
+  attrs[na].val.clusterDim.y = 1;
+  attrs[na].val.clusterDim.z = 1;
+  ++na;
+  cfg.attrs = attrs;
+  cfg.numAttrs = na;
+  if (cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT>, tq, tk, tv, ttk, ttv, p) != cudaSuccess) {
+    cudaGetLastError();
+    return JET_ERR_CUDA;
   }
   return launch_status();
 }
@@ -645,11 +813,14 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
 }  // namespace
 }  // namespace jet
 
+#ifdef JET_TRACE
+extern "C" JET_API void jet_debug_set_attn_trace(void* ptr) { jet::g_trace_ptr = static_cast<long long*>(ptr); }
+#endif
+
 extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                                        int max_seq_len) {
   if (batch < 1 || B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0 || D < 1) return 0;
-  const jet::Plan pl = jet::make_plan(batch, B, Hq, Hkv, max_seq_len);
-  return jet::partial_bytes(pl, D) + 256;
+  return 256;   // key slices are merged on chip; the workspace is only a placeholder
 }
 
 extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
@@ -677,10 +848,9 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
       (k_cache && !aligned(k_cache, 16)) || (v_cache && !aligned(v_cache, 16)))
     return JET_ERR_INVALID_ARG;
   if (static_cast<int64_t>(batch) * B >= (1ll << 31)) return JET_ERR_INVALID_ARG;
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < 256) return JET_ERR_WORKSPACE;
 
   const Plan pl = make_plan(batch, B, Hq, Hkv, max_seq_len);
-  const size_t need = partial_bytes(pl, D) + 256;
-  if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
 
   // ---- tensor maps (bf16, 128-byte swizzle, 64-element inner box)
   CUtensorMap tq, tk, tv, ttk, ttv;
@@ -729,15 +899,15 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = lse;
   p.status = device_status;
-  const size_t rows = static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM;
-  p.part_o = static_cast<float*>(workspace);
-  p.part_lse = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up(rows * D * sizeof(float), 256));
   p.max_pages = max_pages_per_seq;
   p.paged = paged ? 1 : 0;
   p.batch = batch; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.words = (B + 31) / 32;
   p.nsplit = pl.nsplit;
   p.n_mgroups = pl.n_mgroups;
   p.scale_log2 = softmax_scale * 1.4426950408889634f;
+#ifdef JET_TRACE
+  p.trace = g_trace_ptr;
+#endif
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D == 128) return pl.mt == 1 ? launch<128, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
