@@ -74,12 +74,23 @@ struct Cfg {
   static constexpr int kBarBytes = 256;
   static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
   static constexpr int kThreads = 128 + 128 * MT;
-  static constexpr int kTmemCols = (MT == 1) ? 256 : 512;   // per query tile: S (128) + O (<=128)
-  // slice merge: rows arrive as [source slice][row][D fp32 + lse], padded so that the row-per-thread
-  // stores of a warp spread over all banks
+  // TMEM (512 columns): with one query tile per CTA the scores are double-buffered,
+  //   MT == 1: S0 [0,128)  S1 [128,256)  O [256,256+D)
+  //   MT == 2: tile mt owns S [mt*256, +128) and O [mt*256+128, +D)
+  static constexpr int kTmemCols = 512;
+  static constexpr int kSBufs = MT == 1 ? 2 : 1;
+  __device__ static constexpr uint32_t s_col(int mt, int t) { return MT == 1 ? (t & 1) * 128 : mt * 256; }
+  __device__ static constexpr uint32_t o_col(int mt) { return MT == 1 ? 256 : mt * 256 + 128; }
+  // Each score buffer has its own full/free barrier pair, so that neither side can run two phases
+  // ahead of the other on one barrier: buffer index and use count of tile t of query tile mt.
+  __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
+  __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
+  // Epilogue buffers (overlay the tile memory once the key loop is over): this CTA's 128 normalised
+  // rows of one query tile -- D fp32 values followed by the row's log2-sum-exp, padded so that the
+  // row-per-thread stores of a warp spread over all banks -- and the blocks received from every slice.
   static constexpr int kRecvPitch = D * 4 + 16;
-  static constexpr int kStageOff = 0;                              // this CTA's 128 normalised rows
-  static constexpr int kRecvOff = (kBM * kRecvPitch + 1023) / 1024 * 1024;   // rows received from every slice
+  static constexpr int kStageOff = 0;
+  static constexpr int kRecvOff = (kBM * kRecvPitch + 1023) / 1024 * 1024;
   static_assert(kRecvOff + (kBM + kMaxSplit) * kRecvPitch <= kTileBytes, "merge buffers must fit in the tile memory");
 };
 
@@ -92,41 +103,82 @@ struct Bars {       // offsets (in 8-byte units) inside the barrier block
 constexpr uint32_t kWaitRounds = 1u << 16;
 constexpr uint32_t kWaitHintNs = 16384;
 
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// Called by all 32 lanes of a warp; the result is warp-uniform.
+// `site` identifies the wait in the abort flag (1 + site of the first wait that gave up).
+__device__ __noinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
   bool ok = false;
   for (uint32_t i = 0; i < kWaitRounds; ++i) {
     if (ptx::mbar_try_wait(bar, parity, kWaitHintNs)) { ok = true; break; }
     if (*abort_flag) break;
   }
-  if (!ok) *abort_flag = 1u;
+  if (!ok && *abort_flag == 0u) *abort_flag = 1u + site;
   return __all_sync(0xffffffffu, ok);
 }
 
-// The same for a barrier that other CTAs of the cluster arrive on / copy into (acquire at cluster scope);
-// called by every thread of the CTA, returns a CTA-uniform result.
-__device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// The same for a barrier that other CTAs of the cluster arrive on / copy into (acquire at cluster
+// scope); called by every thread of the CTA, the result is CTA-uniform.
+__device__ __noinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint32_t* abort_flag, uint32_t site) {
   bool ok = false;
   for (uint32_t i = 0; i < kWaitRounds; ++i) {
-    if (ptx::mbar_try_wait_cluster(bar, parity, kWaitHintNs)) { ok = true; break; }
+    if (ptx::mbar_try_wait_cluster(bar, 0, kWaitHintNs)) { ok = true; break; }
     if (*abort_flag) break;
   }
-  if (!ok) *abort_flag = 1u;
+  if (!ok && *abort_flag == 0u) *abort_flag = 1u + site;
   return __syncthreads_and(ok ? 1 : 0) != 0;
 }
 
 // Cluster-wide rendezvous built from one mbarrier per CTA (count = cluster size): after a CTA-wide
 // barrier one thread arrives on the barrier of every CTA of the cluster, then everybody waits for
 // all `nsplit` arrivals on the local one.
-__device__ __forceinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag) {
+__device__ __noinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag,
+                                                uint32_t site) {
   __syncthreads();
   if (threadIdx.x == 0)
     for (int c = 0; c < nsplit; ++c) ptx::mbar_arrive_remote(ptx::map_to_rank(local_bar, c));
-  return bounded_wait_cluster(local_bar, 0, abort_flag);
+  return bounded_wait_cluster(local_bar, abort_flag, site);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 pk = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&pk);
+}
+
+__device__ __forceinline__ void max_chunk(const uint32_t (&x)[32], float (&mx)[4]) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(x[j]));
+}
+__device__ __forceinline__ void max_chunk_masked(const uint32_t (&x)[32], uint32_t bits, float (&mx)[4]) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j)
+    mx[j & 3] = fmaxf(mx[j & 3], ((bits >> j) & 1u) ? __uint_as_float(x[j]) : -INFINITY);
+}
+
+// 32 scores of one row -> probabilities (exp2 of the scaled, shifted score; masked keys exactly 0),
+// added to the row sum and written as bf16 to the row's slot of the swizzled P tile.  The stages
+// are kept apart so that the 32 independent exp2 are in flight together.
+template <bool kMasked>
+__device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
+                                          float (&sum)[4], uint8_t* p_row, int c, int r) {
+  float e[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(x[j]), sl2, -m_ref);
+#pragma unroll
+  for (int j = 0; j < 32; ++j) e[j] = exp2f(e[j]);
+  if (kMasked) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) e[j] = ((bits >> j) & 1u) ? e[j] : 0.0f;
+  }
+#pragma unroll
+  for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
+  // chunk c covers keys [32c, 32c+32): 64-key block c/2, 16-byte chunks (c%2)*4 .. +3 of the 128-byte row
+  uint8_t* dst = p_row + (c >> 1) * kHalfBytes;
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) {
+    const int ch = ((c & 1) * 4 + q4) ^ (r & 7);
+    *reinterpret_cast<uint4*>(dst + ch * 16) =
+        make_uint4(pack_bf16(e[q4 * 8], e[q4 * 8 + 1]), pack_bf16(e[q4 * 8 + 2], e[q4 * 8 + 3]),
+                   pack_bf16(e[q4 * 8 + 4], e[q4 * 8 + 5]), pack_bf16(e[q4 * 8 + 6], e[q4 * 8 + 7]));
+  }
 }
 
 template <int D, int MT>
@@ -154,8 +206,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + Bars::kCount * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   auto bar = [&](int idx) { return sBar + 8u * idx; };
+  const int S = p.nsplit;                            // key slices = cluster size
+  const int split = blockIdx.x % S;                  // = rank in the cluster
+  const int rows_per = (kBM + S - 1) / S;            // rows of a query tile that one slice combines
+  const int own_lo = split * rows_per;
+  const int own_n = max(0, min(rows_per, kBM - own_lo));
 
-  // ---------------- set-up that touches no global memory (overlaps the previous kernel's tail)
+  // ---------------- set-up that touches no global memory (may overlap the previous kernel's tail)
   if (warp == 0 && lane == 0) {
     ptx::mbar_init(bar(Bars::kQFull), 1);
     for (int s = 0; s < kStages; ++s) {
@@ -163,38 +220,43 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ptx::mbar_init(bar(Bars::kKvEmpty + s), 1);
     }
     ptx::fence_mbar_init();
-    ptx::prefetch_tmap(&tm_q);
-    ptx::prefetch_tmap(&tm_k);
-    ptx::prefetch_tmap(&tm_v);
   } else if (warp == 1 && lane == 0) {
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(bar(Bars::kSFull + i), 1);
+      ptx::mbar_init(bar(Bars::kSFree + i), 128);
+    }
     for (int mt = 0; mt < MT; ++mt) {
-      ptx::mbar_init(bar(Bars::kSFull + mt), 1);
-      ptx::mbar_init(bar(Bars::kSFree + mt), 128);
       ptx::mbar_init(bar(Bars::kPFull + mt), 128);
       ptx::mbar_init(bar(Bars::kODone + mt), 1);
-    }
-    ptx::mbar_init(bar(Bars::kClusterA), p.nsplit);
-    ptx::mbar_init(bar(Bars::kClusterC), p.nsplit);
-    for (int mt = 0; mt < MT; ++mt) {
       // slice merge: every slice sends this CTA its block of rows of query tile mt
-      const int rows_per = (kBM + p.nsplit - 1) / p.nsplit;
-      const int own_n = max(0, min(rows_per, kBM - static_cast<int>(blockIdx.x % p.nsplit) * rows_per));
       ptx::mbar_init(bar(Bars::kRecv + mt), 1);
-      if (p.nsplit > 1) ptx::mbar_arrive_expect_tx(bar(Bars::kRecv + mt), p.nsplit * own_n * C::kRecvPitch);
+      if (S > 1) ptx::mbar_arrive_expect_tx(bar(Bars::kRecv + mt), S * own_n * C::kRecvPitch);
     }
+    ptx::mbar_init(bar(Bars::kClusterA), S);
+    ptx::mbar_init(bar(Bars::kClusterC), S);
     *abort_flag = 0u;
     ptx::fence_mbar_init();
-    ptx::prefetch_tmap(&tm_tk);
-    ptx::prefetch_tmap(&tm_tv);
   } else if (warp == 2) {
     ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
     ptx::tmem_relinquish();
+  } else if (warp == 3 && lane == 0) {
+    ptx::prefetch_tmap(&tm_q);
+    ptx::prefetch_tmap(&tm_k);
+    ptx::prefetch_tmap(&tm_v);
+    ptx::prefetch_tmap(&tm_tk);
+    ptx::prefetch_tmap(&tm_tv);
   }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  // The barriers of every CTA of the cluster must exist before any CTA arrives on them remotely:
+  // arrive on the hardware cluster barrier now, wait for it only when the slices are merged.
+  if (S > 1) ptx::cluster_arrive();
+  const uint32_t tmem_base = *tmem_slot;
   ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
 
   // ---------------- work item
-  const int split = blockIdx.x % p.nsplit;     // = rank in the cluster
-  const int unit = blockIdx.x / p.nsplit;
+  const int unit = blockIdx.x / S;
   const int mgroup = unit % p.n_mgroups;
   const int bg = unit / p.n_mgroups;
   const int g = bg % p.Hkv;
@@ -210,164 +272,115 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int TP = (L + kBN - 1) / kBN;
   const int TT = (ntree + kBN - 1) / kBN;
   const int T_all = TP + TT;
-  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split) / p.nsplit);
-  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1)) / p.nsplit);
+  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split) / S);
+  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1)) / S);
   const int T = t_hi - t_lo;
+  const bool has_work = node_lo < n && T > 0;    // otherwise: no live node here, or an empty key slice
   if (tid == 0) JET_TR(1);
-  const bool dead_unit = node_lo >= n;           // no live node: uniform over the cluster
-  const bool has_work = !dead_unit && T > 0;
-
-  // Valid keys of tile t (global tile index): prefix tiles first, then tree tiles.
-  auto tile_valid = [&](int t) { return t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN); };
-
-  // One K or V tile into ring slot `item % kStages` (warp 0, all lanes).
-  auto issue_kv = [&](int item) {
-    const int t = t_lo + (item >> 1), kv = item & 1, stage = item % kStages;
-    const uint32_t dst = sKV + stage * C::kStageBytes;
-    const uint32_t full = bar(Bars::kKvFull + stage);
-    if (t < TP) {
-      if (!p.paged) {
-        if (lane == 0) {
-          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-          for (int h = 0; h < kHalves; ++h)
-            ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_v : &tm_k, full, h * 64, g, t * kBN, b);
-        }
-      } else {
-        const int npages = min(8, (L - t * kBN + 15) / 16);
-        if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
-        __syncwarp();
-        if (lane < npages) {
-          const int page = p.page_table[static_cast<size_t>(b) * p.max_pages + t * 8 + lane];
-          for (int h = 0; h < kHalves; ++h)
-            ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page * 16);
-        }
-      }
-    } else if (lane == 0) {
-      ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-      for (int h = 0; h < kHalves; ++h)
-        ptx::tma_load_4d(dst + h * kHalfBytes, kv ? &tm_tv : &tm_tk, full, h * 64, g, (t - TP) * kBN, b);
-    }
-    __syncwarp();
-  };
-
-  // The producer starts the first loads before the CTA-wide set-up barrier: its own barriers are ready.
-  int issued = 0;
-  if (warp == 0 && has_work) {
-    if (lane == 0) {
-      ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
-      for (int mt = 0; mt < n_mt; ++mt)
-        for (int h = 0; h < kHalves; ++h)
-          ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
-                           b * p.B + node_lo + mt * npt);
-    }
-    __syncwarp();
-    for (; issued < min(kStages, 2 * T); ++issued) issue_kv(issued);
-    if (lane == 0) JET_TR(14);
-  }
-  ptx::tc_fence_before();
-  if (p.nsplit > 1) {
-    // the barriers of every CTA of the cluster must exist before any CTA arrives on them remotely;
-    // this is straight-line code from the kernel entry, so the hardware cluster barrier is safe here
-    __syncwarp();
-    ptx::cluster_sync_all();
-  } else {
-    __syncthreads();
-  }
-  ptx::tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  // TMEM columns: query tile mt owns [mt*256, mt*256+128) for S and [mt*256+128, mt*256+128+D) for O.
-  if (tid == 0) JET_TR(15);
 
   // per-row state of the softmax threads, live until the epilogue
   float m_used = -INFINITY;     // running reference maximum (raw score units)
   float l = 0.0f;               // running sum of exp2((s - m_used) * sl2)
-  bool row_ok = true;           // false once a bounded wait of this warp expired
+  bool row_ok = has_work;       // false once a bounded wait of this warp expired
 
   if (has_work) {
     if (warp == 0) {
-      // =========================================================== TMA producer (remaining tiles)
+      // =========================================================== TMA producer
+      if (lane == 0) {
+        ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
+        for (int mt = 0; mt < n_mt; ++mt)
+          for (int h = 0; h < kHalves; ++h)
+            ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
+                             b * p.B + node_lo + mt * npt);
+      }
+      __syncwarp();
       bool ok = true;
-      for (; issued < 2 * T && ok; ++issued) {
-        const int stage = issued % kStages;
-        ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag);
-        if (!ok) break;
-        issue_kv(issued);
+      int issued = 0;
+#pragma unroll 1
+      for (; issued < 2 * T; ++issued) {
+        const int t = t_lo + (issued >> 1), kv = issued & 1, stage = issued % kStages;
+        if (issued >= kStages) {
+          ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
+          if (!ok) break;
+        }
+        const uint32_t dst = sKV + stage * C::kStageBytes;
+        const uint32_t full = bar(Bars::kKvFull + stage);
+        if (t < TP && p.paged) {
+          const int npages = min(8, (L - t * kBN + 15) / 16);
+          if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
+          __syncwarp();
+          if (lane < npages) {
+            const int page = p.page_table[static_cast<size_t>(b) * p.max_pages + t * 8 + lane];
+            for (int h = 0; h < kHalves; ++h)
+              ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page * 16);
+          }
+        } else if (lane == 0) {
+          const bool prefix = t < TP;
+          const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
+          const int row0 = prefix ? t * kBN : (t - TP) * kBN;
+          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+          for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
+        }
+        __syncwarp();
+        if (lane == 0 && issued == 0) JET_TR(14);
       }
       if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
         // drain: every load that was issued must land before the CTA may exit
         for (int s = 0; s < kStages; ++s) {
           if (issued > s) {
             const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
-            bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag);
+            bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
           }
         }
-        bounded_wait(bar(Bars::kQFull), 0, abort_flag);
+        bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
       }
     } else if (warp == 1) {
       // =========================================================== tcgen05 issuer
       constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
       constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
-      bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag);
+      bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
       if (lane == 0) JET_TR(2);
-
-      auto issue_qk = [&](int mt, int stage) {      // S[mt] = Q[mt] K^T
-        if (lane == 0) {
-          const uint32_t d_tmem = tmem_base + mt * 256;
-#pragma unroll
-          for (int kd = 0; kd < D / 16; ++kd) {
-            const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
-            const uint64_t a = ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0);
-            const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0);
-            ptx::umma_ss(d_tmem, a, bdesc, idesc_qk, kd > 0 ? 1u : 0u);
-          }
-        }
-      };
-      auto issue_pv = [&](int mt, int stage, bool first) {   // O[mt] (+)= P[mt] V
-        if (lane == 0) {
-          const uint32_t d_tmem = tmem_base + mt * 256 + 128;
-#pragma unroll
-          for (int kk = 0; kk < kBN / 16; ++kk) {
-            const uint64_t a =
-                ptx::smem_desc_sw128(sP + mt * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0);
-            const uint64_t bdesc = ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes);
-            ptx::umma_ss(d_tmem, a, bdesc, idesc_pv, (first && kk == 0) ? 0u : 1u);
-          }
-        }
-      };
-
-      for (int tl = 0; tl < T && ok; ++tl) {
-        if (tl == 0) {
-          ok = bounded_wait(bar(Bars::kKvFull + 0), 0, abort_flag);
-          if (!ok) break;
-          if (lane == 0) JET_TR(3);
-          ptx::tc_fence_after();
-          for (int mt = 0; mt < n_mt; ++mt) {
-            issue_qk(mt, 0);
-            if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
-          }
-          if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + 0));
-          __syncwarp();
-        }
-        if (tl + 1 < T) {        // next tile's scores as soon as the softmax groups release S
+#pragma unroll 1
+      for (int tl = -1; tl < T && ok; ++tl) {
+        if (tl + 1 < T) {
+          // ---- S = Q K^T of tile tl+1, as soon as its K tile has landed and the score buffer is free
           const int item = 2 * (tl + 1), stage = item % kStages;
-          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
+          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
+          if (lane == 0 && tl == -1) JET_TR(3);
           for (int mt = 0; mt < n_mt && ok; ++mt) {
-            ok = bounded_wait(bar(Bars::kSFree + mt), tl & 1, abort_flag);
+            const int prev = tl + 1 - C::kSBufs;            // tile that used this score buffer last
+            if (prev >= 0)
+              ok = bounded_wait(bar(Bars::kSFree + C::s_buf(mt, prev)), C::s_use(prev) & 1, abort_flag, 6);
             if (!ok) break;
             ptx::tc_fence_after();
-            issue_qk(mt, stage);
-            if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + mt));
+#ifdef JET_X_LOADONLY
+            if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + C::s_buf(mt, tl + 1)));
+            if (false) {
+#else
+            if (lane == 0) {
+#endif
+              const uint32_t d_tmem = tmem_base + C::s_col(mt, tl + 1);
+#pragma unroll
+              for (int kd = 0; kd < D / 16; ++kd) {
+                const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
+                ptx::umma_ss(d_tmem, ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0),
+                             ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0), idesc_qk, kd > 0 ? 1u : 0u);
+              }
+              ptx::umma_commit(bar(Bars::kSFull + C::s_buf(mt, tl + 1)));
+            }
             __syncwarp();
           }
           if (!ok) break;
           if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
           __syncwarp();
         }
-        {
+        if (tl >= 0) {
+          // ---- O += P V of tile tl
           const int item = 2 * tl + 1, stage = item % kStages;
-          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag);
+          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
           if (!ok) break;
-          const int valid = tile_valid(t_lo + tl);
+          const int t = t_lo + tl;
+          const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
           if (valid < kBN) {
             // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
             uint8_t* vt = gen_kv + stage * C::kStageBytes;
@@ -379,11 +392,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             __syncwarp();
           }
           for (int mt = 0; mt < n_mt && ok; ++mt) {
-            ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag);
+            ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag, 8);
             if (!ok) break;
             ptx::tc_fence_after();
-            issue_pv(mt, stage, tl == 0);
+#ifdef JET_X_LOADONLY
             if (lane == 0) ptx::umma_commit(bar(Bars::kODone + mt));
+            if (false) {
+#else
+            if (lane == 0) {
+#endif
+              const uint32_t d_tmem = tmem_base + C::o_col(mt);
+#pragma unroll
+              for (int kk = 0; kk < kBN / 16; ++kk)
+                ptx::umma_ss(d_tmem,
+                             ptx::smem_desc_sw128(sP + mt * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0),
+                             ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
+                             (tl == 0 && kk == 0) ? 0u : 1u);
+              ptx::umma_commit(bar(Bars::kODone + mt));
+            }
             __syncwarp();
           }
           if (!ok) break;
@@ -394,61 +420,65 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     } else if (warp >= 4 && ((warp - 4) >> 2) < n_mt) {
       // =========================================================== softmax warpgroups
       const int mt = (warp - 4) >> 2;
-      const int r = tid - 128 - mt * 128;                     // row of the query tile = TMEM lane
-      const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem_base + lane_base + mt * 256;
-      const uint32_t tO = tS + 128;
+      const int r = (tid - 128) & 127;                        // row of the query tile = TMEM lane
+      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+      const uint32_t tO = t_lane + C::o_col(mt);
       const int v = node_lo + mt * npt + r / G;
       const bool row_live = v < n;
       const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
-      uint8_t* my_p = gen_p + mt * 2 * kHalfBytes + r * 128;
+      uint8_t* p_row = gen_p + mt * 2 * kHalfBytes + r * 128;
       const float sl2 = p.scale_log2;
       bool ok = true;
 
+#pragma unroll 1
       for (int tl = 0; tl < T && ok; ++tl) {
         const int t = t_lo + tl;
-        // visibility bits of this row for the four 32-key chunks of the tile
-        uint32_t vis[4];
+        const uint32_t tS = t_lane + C::s_col(mt, tl);
         const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
-        if (t < TP) {
-          const int valid = L - t * kBN;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const int nv = valid - c * 32;
-            vis[c] = nv >= 32 ? 0xFFFFFFFFu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+        // visibility bits of this row for 32-key chunk c of a tile that is not full
+        auto chunk_bits = [&](int c) -> uint32_t {
+          if (t < TP) {
+            const int nv = (L - t * kBN) - c * 32;
+            return nv >= 32 ? 0xFFFFFFFFu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
           }
-        } else {
-          const int w0 = (t - TP) * 4;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) vis[c] = (row_live && w0 + c < p.words) ? __ldg(mask_row + w0 + c) : 0u;
-        }
+          const int w = (t - TP) * 4 + c;
+          return (row_live && w < p.words) ? __ldg(mask_row + w) : 0u;
+        };
 
-        ok = bounded_wait(bar(Bars::kSFull + mt), tl & 1, abort_flag);
+        ok = bounded_wait(bar(Bars::kSFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 9);
         if (!ok) break;
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
+#ifdef JET_X_LOADONLY
+        if (tl > 0) ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag, 10);
+        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));
+        ptx::mbar_arrive(bar(Bars::kPFull + mt));
+        l = 1.0f; m_used = 0.0f;
+        continue;
+#endif
 
-        // ---- scores of this row: all 128 into registers, then S is free for the next Q K^T
-        uint32_t s[4][32];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) ptx::tmem_ld32(tS + c * 32, s[c]);
-        ptx::tmem_wait_ld();
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kSFree + mt));
-
-        // ---- row maximum over visible keys
+        // ---- pass 1: row maximum over visible keys (scores are read from TMEM in 32-column chunks,
+        //      the next chunk is in flight while the current one is reduced)
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        uint32_t xa[32], xb[32];
         if (full_tile) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-#pragma unroll
-            for (int j = 0; j < 32; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[c][j]));
+          ptx::tmem_ld32(tS, xa);
+#pragma unroll 1
+          for (int c = 0; c < 4; c += 2) {
+            ptx::tmem_wait_ld();
+            ptx::tmem_ld32(tS + (c + 1) * 32, xb);
+            max_chunk(xa, mx);
+            ptx::tmem_wait_ld();
+            if (c + 2 < 4) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
+            max_chunk(xb, mx);
+          }
         } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if ((vis[c] >> j) & 1u) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[c][j]));
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            ptx::tmem_ld32(tS + c * 32, xa);
+            ptx::tmem_wait_ld();
+            max_chunk_masked(xa, chunk_bits(c), mx);
+          }
         }
         const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         if (tid == 128 && tl < 1) JET_TR(5);
@@ -463,71 +493,63 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             m_used = m_tile;
           }
         }
-        if (tid == 128 && tl < 1) JET_TR(16);
         const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
         const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
 
         // P of the previous tile must have been consumed before it is overwritten; the same
         // completion also makes O safe to rescale.
         if (tl > 0) {
-          ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag);
+          ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag, 10);
           if (!ok) break;
           ptx::tc_fence_after();
         }
+        if (tid == 128 && tl < 1) JET_TR(16);
 
-        // ---- probabilities, row sum, P -> shared memory (swizzled bf16).  Each 32-key chunk is done in
-        //      stages (scale, exp2, mask, sum, pack) so that the 32 independent exp2 are in flight together.
+        // ---- pass 2: probabilities, row sum, P -> shared memory (swizzled bf16)
         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          float e[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(s[c][j]), sl2, -m_ref);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) e[j] = exp2f(e[j]);
-          if (!full_tile) {
-            const uint32_t bits = vis[c];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) e[j] = ((bits >> j) & 1u) ? e[j] : 0.0f;
+        if (full_tile) {
+          ptx::tmem_ld32(tS, xa);
+#pragma unroll 1
+          for (int c = 0; c < 4; c += 2) {
+            ptx::tmem_wait_ld();
+            ptx::tmem_ld32(tS + (c + 1) * 32, xb);
+            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c, r);
+            ptx::tmem_wait_ld();
+            if (c + 2 < 4) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
+            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c + 1, r);
           }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
-          uint32_t packed[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) packed[j] = pack_bf16(e[2 * j], e[2 * j + 1]);
-          // chunk c covers keys [32c, 32c+32): 64-key block c/2, 16-byte chunks (c%2)*4 .. +3
-          uint8_t* dst = my_p + (c >> 1) * kHalfBytes;
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int ch = ((c & 1) * 4 + q4) ^ (r & 7);
-            *reinterpret_cast<uint4*>(dst + ch * 16) =
-                make_uint4(packed[q4 * 4], packed[q4 * 4 + 1], packed[q4 * 4 + 2], packed[q4 * 4 + 3]);
+        } else {
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            ptx::tmem_ld32(tS + c * 32, xa);
+            ptx::tmem_wait_ld();
+            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, p_row, c, r);
           }
         }
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));          // the score buffer may be overwritten
         l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
         if (tid == 128 && tl < 1) JET_TR(17);
 
         if (need_rescale && tl > 0) {
 #pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            ptx::tmem_ld32(tO + c * 32, o);
+            ptx::tmem_ld32(tO + c * 32, xa);
             ptx::tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
-            ptx::tmem_st32(tO + c * 32, o);
+            for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
+            ptx::tmem_st32(tO + c * 32, xa);
           }
           ptx::tmem_wait_st();
         }
         ptx::fence_proxy_async_smem();
-        if (tid == 128 && tl < 1) JET_TR(18);
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar(Bars::kPFull + mt));
         if (tid == 128 && tl < 1) JET_TR(6);
       }
       if (tid == 128) JET_TR(10);
-      // O complete once the last P V has been committed
-      if (ok) ok = bounded_wait(bar(Bars::kODone + mt), (T - 1) & 1, abort_flag);
+      // O is complete once the last P V has been committed
+      if (ok) ok = bounded_wait(bar(Bars::kODone + mt), (T - 1) & 1, abort_flag, 11);
       if (ok) ptx::tc_fence_after();
       row_ok = ok;
       if (tid == 128) JET_TR(11);
@@ -535,103 +557,58 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
 
   // =============================================================== epilogue
-  const bool softmax_thread = has_work && warp >= 4 && ((warp - 4) >> 2) < n_mt;
+  // One round per query tile: its softmax threads stage their normalised rows (D fp32 + log2-sum-exp)
+  // in shared memory.  With key slices every CTA then sends each owner slice its block of rows with
+  // one bulk copy credited to the owner's kRecv barrier; the owner combines the S blocks.  Without
+  // slices the CTA "combines" its own staged rows.  Either way the output rows leave as coalesced
+  // 16-byte stores, rows of padding nodes as zeros.
   const int e_mt = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
   const int e_r = (tid - 128) & 127;                           // its row within the query tile
-  const uint32_t e_tO = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + e_mt * 256 + 128;
   const float e_inv = l > 0.0f ? 1.0f / l : 0.0f;
-  const float e_lse2 = l > 0.0f ? m_used * p.scale_log2 + log2f(l) : -INFINITY;   // log2 of the row's sum
-
-  if (p.nsplit == 1) {
-    if (dead_unit || !has_work) {
-      // no live node here (or nothing to attend to): the rows of this CTA are zero
-      for (int i = tid; i < (node_hi - node_lo) * G * (D / 8); i += C::kThreads) {
-        const int row = i / (D / 8), c8 = i - row * (D / 8);
-        const int v = node_lo + row / G, h = g * G + row % G;
-        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
-            make_uint4(0u, 0u, 0u, 0u);
-        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = -INFINITY;
-      }
-    } else if (softmax_thread && row_ok) {
-      const int v = node_lo + e_mt * npt + e_r / G;
-      const int h = g * G + e_r % G;
-      const bool row_live = v < n, in_range = v < p.B;
-      __nv_bfloat16* orow = p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D;
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        ptx::tmem_ld32(e_tO + c * 32, o);
-        ptx::tmem_wait_ld();
-        if (in_range) {
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint32_t w[4];
-#pragma unroll
-            for (int k2 = 0; k2 < 4; ++k2) {
-              const float a0 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2]) * e_inv : 0.0f;
-              const float a1 = row_live ? __uint_as_float(o[q4 * 8 + k2 * 2 + 1]) * e_inv : 0.0f;
-              w[k2] = pack_bf16(a0, a1);
-            }
-            *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-      }
-      if (p.lse && in_range)
-        p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = row_live ? e_lse2 * 0.6931471805599453f : -INFINITY;
-    }
-  } else if (dead_unit) {
-    // uniform over the cluster: slice 0 clears the unit's rows, nobody takes part in a cluster barrier
-    if (split == 0) {
-      for (int i = tid; i < (node_hi - node_lo) * G * (D / 8); i += C::kThreads) {
-        const int row = i / (D / 8), c8 = i - row * (D / 8);
-        const int v = node_lo + row / G, h = g * G + row % G;
-        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
-            make_uint4(0u, 0u, 0u, 0u);
-        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = -INFINITY;
-      }
-    }
-  } else {
-    // ------------------------------------------------------------- slice merge through DSMEM
-    // One round per query tile.  The tile's 128 rows are dealt out to the slices in blocks of
-    // rows_per (row r belongs to slice r / rows_per).  Every CTA stages its normalised rows --
-    // D fp32 values followed by the row's log2-sum-exp -- in its own shared memory, then sends
-    // each owner its block with one bulk copy that is credited to the owner's kRecv barrier.
-    // Both buffers overlay the tile memory, which is idle once every CTA has left its key loop.
-    const int S = p.nsplit;
-    const int rows_per = (kBM + S - 1) / S;
-    const int own_lo = split * rows_per;
-    const int own_n = max(0, min(rows_per, kBM - own_lo));
-    uint8_t* stage = smem_gen + C::kStageOff;
-    const uint8_t* recv = smem_gen + C::kRecvOff;
-    // A: every CTA of the cluster has left its key loop, so tile memory may be overwritten
-    bool merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag);
+  const float e_lse2 = l > 0.0f ? m_used * p.scale_log2 + log2f(l) : -INFINITY;
+  uint8_t* stage = smem_gen + C::kStageOff;
+  bool merge_ok = true;
+  if (S > 1) {
+    __syncwarp();
+    ptx::cluster_wait();     // pairs with cluster_arrive above: every CTA's barriers are initialised
+    // A: every CTA of the cluster has left its key loop, so its tile memory may be overwritten
+    merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag, 12);
     if (tid == 128) JET_TR(7);
-    for (int mt = 0; mt < MT; ++mt) {
-      if (mt > 0) {
-        // C: everybody has combined the previous tile's rows, so both buffers are free again
-        merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag) && merge_ok;
-      }
-      if (warp >= 4 && ((warp - 4) >> 2) == mt) {
-        uint8_t* srow = stage + e_r * C::kRecvPitch;
-        const bool active = softmax_thread && row_ok;           // warp-uniform
-        if (active) {
+  } else {
+    __syncthreads();
+  }
 #pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            ptx::tmem_ld32(e_tO + c * 32, o);
-            ptx::tmem_wait_ld();
+  for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
+    if (mt > 0) {
+      // C: everybody has combined the previous tile's rows, so both buffers are free again
+      if (S > 1) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
+      else __syncthreads();
+    }
+    if (warp >= 4 && e_mt == mt) {
+      uint8_t* srow = stage + e_r * C::kRecvPitch;
+      const bool active = has_work && mt < n_mt && row_ok;     // warp-uniform
+      if (active) {
+        const uint32_t tO = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::o_col(mt);
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          ptx::tmem_ld32(tO + c * 32, o);
+          ptx::tmem_wait_ld();
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4)
-              *reinterpret_cast<float4*>(srow + (c * 32 + q4 * 4) * 4) =
-                  make_float4(__uint_as_float(o[q4 * 4]) * e_inv, __uint_as_float(o[q4 * 4 + 1]) * e_inv,
-                              __uint_as_float(o[q4 * 4 + 2]) * e_inv, __uint_as_float(o[q4 * 4 + 3]) * e_inv);
-          }
+          for (int q4 = 0; q4 < 8; ++q4)
+            *reinterpret_cast<float4*>(srow + (c * 32 + q4 * 4) * 4) =
+                make_float4(__uint_as_float(o[q4 * 4]) * e_inv, __uint_as_float(o[q4 * 4 + 1]) * e_inv,
+                            __uint_as_float(o[q4 * 4 + 2]) * e_inv, __uint_as_float(o[q4 * 4 + 3]) * e_inv);
         }
-        // rows this CTA computed nothing for (empty key slice, tile without nodes) are marked absent
-        *reinterpret_cast<float*>(srow + D * 4) = (active && l > 0.0f) ? e_lse2 : -INFINITY;
-        ptx::fence_proxy_async_smem();
       }
-      __syncthreads();
+      // rows this CTA computed nothing for (empty key slice, tile without nodes) are marked absent
+      *reinterpret_cast<float*>(srow + D * 4) = (active && l > 0.0f) ? e_lse2 : -INFINITY;
+      if (S > 1) ptx::fence_proxy_async_smem();
+    }
+    __syncthreads();
+    const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
+    bool rows_ok = merge_ok;
+    if (S > 1) {
       if (tid < S && merge_ok) {
         const int dst_lo = tid * rows_per;
         const int dst_n = max(0, min(rows_per, kBM - dst_lo));
@@ -641,52 +618,61 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               smem_base + C::kStageOff + static_cast<uint32_t>(dst_lo * C::kRecvPitch),
               static_cast<uint32_t>(dst_n * C::kRecvPitch), ptx::map_to_rank(bar(Bars::kRecv + mt), tid));
       }
+      if (tid == 128 && mt == 0) JET_TR(8);
       // all blocks of this CTA's rows have arrived (always waited for, so that the CTA never exits
       // while copies into its memory are in flight)
-      if (tid == 128 && mt == 0) JET_TR(8);
-      const bool recv_ok = bounded_wait_cluster(bar(Bars::kRecv + mt), 0, abort_flag) && merge_ok;
+      rows_ok = bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14) && merge_ok;
       if (tid == 128 && mt == 0) JET_TR(9);
-      const int items = recv_ok ? own_n * (D / 8) : 0;
-      for (int i = tid; i < items; i += C::kThreads) {
-        const int rl = i / (D / 8), c8 = i - rl * (D / 8);
-        const int R = mt * kBM + own_lo + rl;                  // row within the unit
-        const int v = node_lo + R / G, h = g * G + R % G;
-        if (v >= p.B) continue;
-        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        float lse2 = -INFINITY;
-        if (v < n) {
-          float mx = -INFINITY;
-          for (int c = 0; c < S; ++c)
-            mx = fmaxf(mx, *reinterpret_cast<const float*>(recv + (c * rows_per + rl) * C::kRecvPitch + D * 4));
-          float wsum = 0.0f;
-          if (mx > -INFINITY) {
-            for (int c = 0; c < S; ++c) {
-              const uint8_t* src = recv + (c * rows_per + rl) * C::kRecvPitch;
-              const float ls = *reinterpret_cast<const float*>(src + D * 4);
-              if (ls == -INFINITY) continue;
-              const float w = exp2f(ls - mx);
-              wsum += w;
-              const float4 x0 = *reinterpret_cast<const float4*>(src + c8 * 32);
-              const float4 x1 = *reinterpret_cast<const float4*>(src + c8 * 32 + 16);
-              acc[0] += w * x0.x; acc[1] += w * x0.y; acc[2] += w * x0.z; acc[3] += w * x0.w;
-              acc[4] += w * x1.x; acc[5] += w * x1.y; acc[6] += w * x1.z; acc[7] += w * x1.w;
-            }
-            const float inv = 1.0f / wsum;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) acc[k] *= inv;
-            lse2 = mx + log2f(wsum);
+      src_rows = smem_gen + C::kRecvOff;
+      // This CTA's own bulk copies read its staged rows asynchronously: it may only exit once every
+      // peer has received them.  Arrive on the hardware cluster barrier now, wait for it at the end.
+      if (mt == n_mt - 1) ptx::cluster_arrive();
+    }
+    const int items = rows_ok ? own_n * (D / 8) : 0;
+#pragma unroll 1
+    for (int i = tid; i < items; i += C::kThreads) {
+      const int rl = i / (D / 8), c8 = i - rl * (D / 8);
+      const int R = mt * kBM + own_lo + rl;                  // row within the unit
+      const int v = node_lo + R / G, h = g * G + R % G;
+      if (v >= p.B) continue;
+      float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      float lse2 = -INFINITY;
+      if (v < n) {
+        float mx = -INFINITY;
+        for (int c = 0; c < S; ++c)
+          mx = fmaxf(mx, *reinterpret_cast<const float*>(src_rows + (c * rows_per + rl) * C::kRecvPitch + D * 4));
+        float wsum = 0.0f;
+        if (mx > -INFINITY) {
+          for (int c = 0; c < S; ++c) {
+            const uint8_t* src = src_rows + (c * rows_per + rl) * C::kRecvPitch;
+            const float ls = *reinterpret_cast<const float*>(src + D * 4);
+            if (ls == -INFINITY) continue;
+            const float w = exp2f(ls - mx);
+            wsum += w;
+            const float4 x0 = *reinterpret_cast<const float4*>(src + c8 * 32);
+            const float4 x1 = *reinterpret_cast<const float4*>(src + c8 * 32 + 16);
+            acc[0] += w * x0.x; acc[1] += w * x0.y; acc[2] += w * x0.z; acc[3] += w * x0.w;
+            acc[4] += w * x1.x; acc[5] += w * x1.y; acc[6] += w * x1.z; acc[7] += w * x1.w;
           }
+          const float inv = 1.0f / wsum;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) acc[k] *= inv;
+          lse2 = mx + log2f(wsum);
         }
-        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
-            make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
-                       pack_bf16(acc[6], acc[7]));
-        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
       }
+      *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+          make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                     pack_bf16(acc[6], acc[7]));
+      if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
     }
   }
 
   // ---------------- teardown
   if (tid == 128) JET_TR(12);
+  if (S > 1) {
+    __syncwarp();
+    ptx::cluster_wait();     // every CTA of the cluster has received all of its blocks
+  }
   ptx::grid_dep_launch();
   ptx::tc_fence_before();
   __syncthreads();
@@ -697,6 +683,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (tid == 0) {
     JET_TR(13);
     if (*abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
+#ifdef JET_TRACE
+    if (*abort_flag && p.trace) p.trace[blockIdx.x * 32 + 31] = *abort_flag;
+#endif
   }
 }
 
@@ -748,13 +737,63 @@ struct Plan {
   int nsplit;      // key slices = cluster size
 };
 
-// Picks the query-tile grouping and the number of key slices.  Cost model: waves of CTAs x key tiles
-// per CTA x query tiles per CTA; on a tie the grouping that loads K/V fewer times wins.
-Plan make_plan(int batch, int B, int Hq, int Hkv, int max_seq_len) {
+template <int D, int MT>
+bool configure_kernel() {
+  static int state = 0;     // 0 = not yet, 1 = ok, -1 = failed
+  if (state == 0) {
+    state = (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  Cfg<D, MT>::kSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                 cudaSuccess)
+                ? 1
+                : -1;
+    if (state < 0) cudaGetLastError();
+  }
+  return state > 0;
+}
+
+// How many clusters of `cluster` CTAs of this kernel the device can hold at once (one CTA per SM, and a
+// cluster must fit inside one GPC).  Asked of the driver once per cluster size and cached.
+template <int D, int MT>
+int max_active_clusters(int cluster) {
+  static int cache[kMaxSplit + 1] = {};      // 0 = unknown, -1 = none
+  if (cluster < 1 || cluster > kMaxSplit) return 0;
+  if (cache[cluster] == 0) {
+    int n = 0;
+    if (configure_kernel<D, MT>()) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(cluster * 64);
+      cfg.blockDim = dim3(Cfg<D, MT>::kThreads);
+      cfg.dynamicSmemBytes = Cfg<D, MT>::kSmemBytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = cluster;
+      at[0].val.clusterDim.y = 1;
+      at[0].val.clusterDim.z = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+      if (cudaOccupancyMaxActiveClusters(&n, tree_attn_kernel<D, MT>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        n = 0;
+      }
+    }
+    cache[cluster] = n > 0 ? n : -1;
+  }
+  return cache[cluster] > 0 ? cache[cluster] : 0;
+}
+
+int max_active_clusters_for(int D, int mt, int cluster) {
+  if (D == 128) return mt == 1 ? max_active_clusters<128, 1>(cluster) : max_active_clusters<128, 2>(cluster);
+  return mt == 1 ? max_active_clusters<64, 1>(cluster) : max_active_clusters<64, 2>(cluster);
+}
+
+// Picks the query-tile grouping and the number of key slices.  Cost model: waves of clusters x key tiles
+// per CTA x query tiles per CTA; on a tie the grouping that loads K/V fewer times, then the smaller
+// cluster, wins.
+Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   const int G = Hq / Hkv;
   const int rows = B * G;
   const int tiles = (max_seq_len + kBN - 1) / kBN + (B + kBN - 1) / kBN;
-  const int sms = sm_count();
   Plan best{};
   long best_cost = -1;
   for (int mt = (rows > kBM ? 2 : 1); mt >= 1; --mt) {
@@ -762,15 +801,23 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int max_seq_len) {
     pl.mt = mt;
     pl.n_mgroups = (rows + mt * kBM - 1) / (mt * kBM);
     pl.units = batch * Hkv * pl.n_mgroups;
-    int ns = sms / pl.units;
-    ns = ns < 1 ? 1 : ns;
-    ns = ns > kMaxSplit ? kMaxSplit : ns;
-    ns = ns > tiles ? tiles : ns;
-    pl.nsplit = ns;
-    const long ctas = static_cast<long>(pl.units) * ns;
-    const long waves = (ctas + sms - 1) / sms;
-    const long cost = waves * ((tiles + ns - 1) / ns) * mt;
-    if (best_cost < 0 || cost < best_cost) { best = pl; best_cost = cost; }
+    for (int ns = 1; ns <= kMaxSplit && ns <= tiles; ++ns) {
+      const int resident = max_active_clusters_for(D, mt, ns);
+      if (resident <= 0) continue;
+      const long waves = (pl.units + resident - 1) / resident;
+      const long cost = waves * ((tiles + ns - 1) / ns) * mt;
+      if (best_cost < 0 || cost < best_cost) {
+        best = pl;
+        best.nsplit = ns;
+        best_cost = cost;
+      }
+    }
+  }
+  if (best_cost < 0) {          // the occupancy query failed: plain launch without slices
+    best.mt = rows > kBM ? 2 : 1;
+    best.n_mgroups = (rows + best.mt * kBM - 1) / (best.mt * kBM);
+    best.units = batch * Hkv * best.n_mgroups;
+    best.nsplit = 1;
   }
   return best;
 }
@@ -779,16 +826,7 @@ template <int D, int MT>
 jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& ttk,
                   const CUtensorMap& ttv, const AttnParams& p, const Plan& pl, cudaStream_t st) {
   using C = Cfg<D, MT>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             C::kSmemBytes) != cudaSuccess)
-      return JET_ERR_CUDA;
-    if (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) !=
-        cudaSuccess)
-      return JET_ERR_CUDA;
-    configured = true;
-  }
+  if (!configure_kernel<D, MT>()) return JET_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.units * pl.nsplit);
   cfg.blockDim = dim3(C::kThreads);
@@ -815,6 +853,23 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
 
 #ifdef JET_TRACE
 extern "C" JET_API void jet_debug_set_attn_trace(void* ptr) { jet::g_trace_ptr = static_cast<long long*>(ptr); }
+extern "C" JET_API int jet_debug_max_clusters(int cluster) {
+  using namespace jet;
+  using C = Cfg<128, 1>;
+  cudaFuncSetAttribute(tree_attn_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+  cudaFuncSetAttribute(tree_attn_kernel<128, 1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(cluster * 32);
+  cfg.blockDim = dim3(C::kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = -1;
+  if (cudaOccupancyMaxActiveClusters(&n, tree_attn_kernel<128, 1>, &cfg) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return n;
+}
 #endif
 
 extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
@@ -850,7 +905,7 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
   if (static_cast<int64_t>(batch) * B >= (1ll << 31)) return JET_ERR_INVALID_ARG;
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < 256) return JET_ERR_WORKSPACE;
 
-  const Plan pl = make_plan(batch, B, Hq, Hkv, max_seq_len);
+  const Plan pl = make_plan(batch, B, Hq, Hkv, D, max_seq_len);
 
   // ---- tensor maps (bf16, 128-byte swizzle, 64-element inner box)
   CUtensorMap tq, tk, tv, ttk, ttv;
