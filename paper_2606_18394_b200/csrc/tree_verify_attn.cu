@@ -71,16 +71,21 @@ struct Cfg {
   static constexpr int kStageBytes = kHalves * kHalfBytes;
   static constexpr int kStages = (D == 128) ? (MT == 1 ? 5 : 3) : 6;
   static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
+  // With one query tile per CTA two softmax warpgroups share it: each thread owns one row and half of
+  // the tile's 128 key columns, which halves the per-tile softmax latency.
+  static constexpr int kWG = MT == 1 ? 2 : 1;
   static constexpr int kBarBytes = 256;
   static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
-  static constexpr int kThreads = 128 + 128 * MT;
+  static constexpr int kThreads = 128 + 128 * MT * kWG;
   // TMEM (512 columns): with one query tile per CTA the scores are double-buffered,
-  //   MT == 1: S0 [0,128)  S1 [128,256)  O [256,256+D)
+  //   MT == 1: S0 [0,128)  S1 [128,256)  O [256,256+D)  and columns [384,392) for per-row scalars that
+  //            the two warpgroups of a row exchange (both own the row's TMEM lane)
   //   MT == 2: tile mt owns S [mt*256, +128) and O [mt*256+128, +D)
   static constexpr int kTmemCols = 512;
   static constexpr int kSBufs = MT == 1 ? 2 : 1;
   __device__ static constexpr uint32_t s_col(int mt, int t) { return MT == 1 ? (t & 1) * 128 : mt * 256; }
   __device__ static constexpr uint32_t o_col(int mt) { return MT == 1 ? 256 : mt * 256 + 128; }
+  static constexpr uint32_t kXchgCol = 384;
   // Each score buffer has its own full/free barrier pair, so that neither side can run two phases
   // ahead of the other on one barrier: buffer index and use count of tile t of query tile mt.
   __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
@@ -96,7 +101,7 @@ struct Cfg {
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
   enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
-         kClusterA = 21, kClusterC = 22, kRecv = 23, kCount = 25 };
+         kClusterA = 21, kClusterC = 22, kRecv = 23, kHalf = 25, kCount = 26 };
 };
 
 // Every wait is bounded: at most kWaitRounds suspensions of kWaitHintNs each (about a second).
@@ -223,10 +228,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else if (warp == 1 && lane == 0) {
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(bar(Bars::kSFull + i), 1);
-      ptx::mbar_init(bar(Bars::kSFree + i), 128);
+      ptx::mbar_init(bar(Bars::kSFree + i), 128 * C::kWG);
     }
+    ptx::mbar_init(bar(Bars::kHalf), 128 * C::kWG);
     for (int mt = 0; mt < MT; ++mt) {
-      ptx::mbar_init(bar(Bars::kPFull + mt), 128);
+      ptx::mbar_init(bar(Bars::kPFull + mt), 128 * C::kWG);
       ptx::mbar_init(bar(Bars::kODone + mt), 1);
       // slice merge: every slice sends this CTA its block of rows of query tile mt
       ptx::mbar_init(bar(Bars::kRecv + mt), 1);
@@ -254,6 +260,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (S > 1) ptx::cluster_arrive();
   const uint32_t tmem_base = *tmem_slot;
   ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
+  ptx::grid_dep_launch();    // the next kernel may start its own set-up as SMs become free
 
   // ---------------- work item
   const int unit = blockIdx.x / S;
@@ -353,12 +360,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               ok = bounded_wait(bar(Bars::kSFree + C::s_buf(mt, prev)), C::s_use(prev) & 1, abort_flag, 6);
             if (!ok) break;
             ptx::tc_fence_after();
-#ifdef JET_X_LOADONLY
-            if (lane == 0) ptx::umma_commit(bar(Bars::kSFull + C::s_buf(mt, tl + 1)));
-            if (false) {
-#else
             if (lane == 0) {
-#endif
               const uint32_t d_tmem = tmem_base + C::s_col(mt, tl + 1);
 #pragma unroll
               for (int kd = 0; kd < D / 16; ++kd) {
@@ -395,12 +397,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag, 8);
             if (!ok) break;
             ptx::tc_fence_after();
-#ifdef JET_X_LOADONLY
-            if (lane == 0) ptx::umma_commit(bar(Bars::kODone + mt));
-            if (false) {
-#else
             if (lane == 0) {
-#endif
               const uint32_t d_tmem = tmem_base + C::o_col(mt);
 #pragma unroll
               for (int kk = 0; kk < kBN / 16; ++kk)
@@ -417,12 +414,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           __syncwarp();
         }
       }
-    } else if (warp >= 4 && ((warp - 4) >> 2) < n_mt) {
+    } else if (warp >= 4 && (MT == 1 || ((warp - 4) >> 2) < n_mt)) {
       // =========================================================== softmax warpgroups
-      const int mt = (warp - 4) >> 2;
+      constexpr int kWG = C::kWG;
+      constexpr int kChunks = kBN / 32 / kWG;                 // 32-key chunks per thread and tile
+      const int wg = (warp - 4) >> 2;
+      const int mt = MT == 1 ? 0 : wg;                        // query tile of this warpgroup
+      const int half = MT == 1 ? wg : 0;                      // which half of the key columns it owns
+      const int c0 = half * kChunks;                          // its first 32-key chunk
       const int r = (tid - 128) & 127;                        // row of the query tile = TMEM lane
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-      const uint32_t tO = t_lane + C::o_col(mt);
+      const uint32_t tO = t_lane + C::o_col(mt) + half * (D / kWG);
       const int v = node_lo + mt * npt + r / G;
       const bool row_live = v < n;
       const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
@@ -433,7 +435,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll 1
       for (int tl = 0; tl < T && ok; ++tl) {
         const int t = t_lo + tl;
-        const uint32_t tS = t_lane + C::s_col(mt, tl);
+        const uint32_t tS = t_lane + C::s_col(mt, tl) + c0 * 32;
         const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
         // visibility bits of this row for 32-key chunk c of a tile that is not full
         auto chunk_bits = [&](int c) -> uint32_t {
@@ -449,38 +451,48 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (!ok) break;
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
-#ifdef JET_X_LOADONLY
-        if (tl > 0) ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag, 10);
-        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));
-        ptx::mbar_arrive(bar(Bars::kPFull + mt));
-        l = 1.0f; m_used = 0.0f;
-        continue;
-#endif
+        if (tid == 128 && tl < 6) JET_TR(19 + 2 * tl);
 
-        // ---- pass 1: row maximum over visible keys (scores are read from TMEM in 32-column chunks,
-        //      the next chunk is in flight while the current one is reduced)
+        // ---- pass 1: maximum over the visible keys of this thread's columns (scores are read from TMEM
+        //      in 32-column chunks, the next chunk is in flight while the current one is reduced)
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         uint32_t xa[32], xb[32];
         if (full_tile) {
           ptx::tmem_ld32(tS, xa);
 #pragma unroll 1
-          for (int c = 0; c < 4; c += 2) {
+          for (int c = 0; c < kChunks; c += 2) {
             ptx::tmem_wait_ld();
             ptx::tmem_ld32(tS + (c + 1) * 32, xb);
             max_chunk(xa, mx);
             ptx::tmem_wait_ld();
-            if (c + 2 < 4) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
+            if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
             max_chunk(xb, mx);
           }
         } else {
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < kChunks; ++c) {
             ptx::tmem_ld32(tS + c * 32, xa);
             ptx::tmem_wait_ld();
-            max_chunk_masked(xa, chunk_bits(c), mx);
+            max_chunk_masked(xa, chunk_bits(c0 + c), mx);
           }
         }
-        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        if (kWG == 2) {
+          // The two halves of a row must use one reference maximum: each writes its partial maximum to
+          // a spare TMEM column of the row's lane (double-buffered by tile parity) and reads both.
+          const uint32_t tX = t_lane + C::kXchgCol + (tl & 1) * 2;
+          ptx::tmem_st1(tX + half, __float_as_uint(m_tile));
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kHalf));
+          ok = bounded_wait(bar(Bars::kHalf), tl & 1, abort_flag, 15);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          uint32_t ma, mb;
+          ptx::tmem_ld2(tX, ma, mb);
+          ptx::tmem_wait_ld();
+          m_tile = fmaxf(__uint_as_float(ma), __uint_as_float(mb));
+        }
         if (tid == 128 && tl < 1) JET_TR(5);
 
         // ---- running maximum with lazy rescaling
@@ -510,30 +522,31 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (full_tile) {
           ptx::tmem_ld32(tS, xa);
 #pragma unroll 1
-          for (int c = 0; c < 4; c += 2) {
+          for (int c = 0; c < kChunks; c += 2) {
             ptx::tmem_wait_ld();
             ptx::tmem_ld32(tS + (c + 1) * 32, xb);
-            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c, r);
+            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c0 + c, r);
             ptx::tmem_wait_ld();
-            if (c + 2 < 4) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
-            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c + 1, r);
+            if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
+            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c0 + c + 1, r);
           }
         } else {
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < kChunks; ++c) {
             ptx::tmem_ld32(tS + c * 32, xa);
             ptx::tmem_wait_ld();
-            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, p_row, c, r);
+            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c0 + c), sum, p_row, c0 + c, r);
           }
         }
         ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));          // the score buffer may be overwritten
+        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));   // the score buffer may be overwritten
         l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
         if (tid == 128 && tl < 1) JET_TR(17);
 
         if (need_rescale && tl > 0) {
+          // each warpgroup rescales its share of the row's O columns
 #pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
+          for (int c = 0; c < D / 32 / kWG; ++c) {
             ptx::tmem_ld32(tO + c * 32, xa);
             ptx::tmem_wait_ld();
 #pragma unroll
@@ -546,6 +559,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar(Bars::kPFull + mt));
         if (tid == 128 && tl < 1) JET_TR(6);
+        if (tid == 128 && tl < 6) JET_TR(20 + 2 * tl);
       }
       if (tid == 128) JET_TR(10);
       // O is complete once the last P V has been committed
@@ -562,10 +576,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // one bulk copy credited to the owner's kRecv barrier; the owner combines the S blocks.  Without
   // slices the CTA "combines" its own staged rows.  Either way the output rows leave as coalesced
   // 16-byte stores, rows of padding nodes as zeros.
-  const int e_mt = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
+  const int e_wg = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
+  const int e_mt = MT == 1 ? 0 : e_wg;                         // its query tile
+  const int e_half = MT == 1 ? e_wg : 0;                       // its half of the row (two warpgroups per tile)
   const int e_r = (tid - 128) & 127;                           // its row within the query tile
-  const float e_inv = l > 0.0f ? 1.0f / l : 0.0f;
-  const float e_lse2 = l > 0.0f ? m_used * p.scale_log2 + log2f(l) : -INFINITY;
   uint8_t* stage = smem_gen + C::kStageOff;
   bool merge_ok = true;
   if (S > 1) {
@@ -577,6 +591,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else {
     __syncthreads();
   }
+  float l_row = l;
+  if (C::kWG == 2) {
+    // combine the row sums of the two halves through the row's spare TMEM columns
+    const uint32_t tX = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::kXchgCol + 4;
+    if (warp >= 4) {
+      ptx::tmem_st1(tX + e_half, __float_as_uint(l));
+      ptx::tmem_wait_st();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    if (warp >= 4) {
+      uint32_t la, lb;
+      ptx::tmem_ld2(tX, la, lb);
+      ptx::tmem_wait_ld();
+      l_row = __uint_as_float(la) + __uint_as_float(lb);
+    }
+  }
 #pragma unroll 1
   for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
     if (mt > 0) {
@@ -585,12 +617,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       else __syncthreads();
     }
     if (warp >= 4 && e_mt == mt) {
-      uint8_t* srow = stage + e_r * C::kRecvPitch;
+      constexpr int kColsPerWG = D / C::kWG;                   // O columns staged by this thread
+      uint8_t* srow = stage + e_r * C::kRecvPitch + e_half * kColsPerWG * 4;
       const bool active = has_work && mt < n_mt && row_ok;     // warp-uniform
+      const float e_inv = l_row > 0.0f ? 1.0f / l_row : 0.0f;
       if (active) {
-        const uint32_t tO = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::o_col(mt);
+        const uint32_t tO =
+            tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::o_col(mt) + e_half * kColsPerWG;
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < kColsPerWG / 32; ++c) {
           uint32_t o[32];
           ptx::tmem_ld32(tO + c * 32, o);
           ptx::tmem_wait_ld();
@@ -602,7 +637,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       }
       // rows this CTA computed nothing for (empty key slice, tile without nodes) are marked absent
-      *reinterpret_cast<float*>(srow + D * 4) = (active && l > 0.0f) ? e_lse2 : -INFINITY;
+      if (e_half == 0)
+        *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 4) =
+            (active && l_row > 0.0f) ? m_used * p.scale_log2 + log2f(l_row) : -INFINITY;
       if (S > 1) ptx::fence_proxy_async_smem();
     }
     __syncthreads();
@@ -673,7 +710,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     __syncwarp();
     ptx::cluster_wait();     // every CTA of the cluster has received all of its blocks
   }
-  ptx::grid_dep_launch();
   ptx::tc_fence_before();
   __syncthreads();
   if (warp == 2) {
@@ -838,6 +874,11 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   attrs[na].val.clusterDim.x = pl.nsplit;
   attrs[na].val.clusterDim.y = 1;
   attrs[na].val.clusterDim.z = 1;
+  ++na;
+  // Programmatic dependent launch: this grid may be scheduled while the previous kernel of the stream
+  // drains; the kernel touches no global memory before its griddepcontrol.wait.
+  attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[na].val.programmaticStreamSerializationAllowed = 1;
   ++na;
   cfg.attrs = attrs;
   cfg.numAttrs = na;
