@@ -123,6 +123,10 @@ JET_API jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride, 
  *                wait inside the kernel expired (outputs are then undefined).
  * Limits: D in {64,128}; Hq % Hkv == 0 and Hq/Hkv a power of two <= 16;
  * page_size == 16 when paged; all base pointers 16-byte aligned.
+ * Workspace: unlike the other calls, the first 4096 bytes of this workspace hold
+ * counters that must be ZERO when the call starts.  Zero them once after
+ * allocating the workspace; every call that completes leaves them zero again.
+ * (A call that reported JET_ERR_TIMEOUT may leave them dirty: zero them again.)
  */
 JET_API size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                             int max_seq_len);

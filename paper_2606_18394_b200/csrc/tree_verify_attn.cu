@@ -50,7 +50,10 @@ struct AttnParams {
   int32_t* status;
   int max_pages, paged;
   int batch, B, Hq, Hkv, G, words;
-  int nsplit, n_mgroups;
+  int nsplit, n_mgroups, n_units;
+  int via_global;     // key slices exchange their rows through the workspace instead of a cluster
+  int* counters;      // via_global: [2][units * MT] arrival / departure counts, zero between calls
+  uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D fp32 + log2-sum-exp]
   float scale_log2;   // softmax_scale * log2(e)
 #ifdef JET_TRACE
   long long* trace;   // 32 clock64() samples per CTA
@@ -67,9 +70,12 @@ template <int D, int MT>
 struct Cfg {
   static constexpr int kHalves = D / 64;
   static constexpr int kQBytes = MT * kHalves * kHalfBytes;
-  static constexpr int kPBytes = MT * 2 * kHalfBytes;
+  // P (probabilities, bf16): one 128x128 buffer per query tile; with a single query tile per CTA it is
+  // double-buffered so that the softmax of tile t+1 never waits for the P V product of tile t.
+  static constexpr int kPBufs = MT == 1 ? 2 : 1;
+  static constexpr int kPBytes = MT * kPBufs * 2 * kHalfBytes;
   static constexpr int kStageBytes = kHalves * kHalfBytes;
-  static constexpr int kStages = (D == 128) ? (MT == 1 ? 5 : 3) : 6;
+  static constexpr int kStages = (D == 128) ? (MT == 1 ? 4 : 3) : 6;
   static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
   // With one query tile per CTA two softmax warpgroups share it: each thread owns one row and half of
   // the tile's 128 key columns, which halves the per-tile softmax latency.
@@ -90,6 +96,9 @@ struct Cfg {
   // ahead of the other on one barrier: buffer index and use count of tile t of query tile mt.
   __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
   __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
+  // The same for the P buffers and their full / consumed (o_done) barriers.
+  __device__ static constexpr int p_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
+  __device__ static constexpr int p_use(int t) { return MT == 1 ? (t >> 1) : t; }
   // Epilogue buffers (overlay the tile memory once the key loop is over): this CTA's 128 normalised
   // rows of one query tile -- D fp32 values followed by the row's log2-sum-exp, padded so that the
   // row-per-thread stores of a warp spread over all banks -- and the blocks received from every slice.
@@ -110,7 +119,8 @@ constexpr uint32_t kWaitHintNs = 16384;
 
 // Called by all 32 lanes of a warp; the result is warp-uniform.
 // `site` identifies the wait in the abort flag (1 + site of the first wait that gave up).
-__device__ __noinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+__device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                              uint32_t site) {
   bool ok = false;
   for (uint32_t i = 0; i < kWaitRounds; ++i) {
     if (ptx::mbar_try_wait(bar, parity, kWaitHintNs)) { ok = true; break; }
@@ -118,6 +128,13 @@ __device__ __noinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatil
   }
   if (!ok && *abort_flag == 0u) *abort_flag = 1u + site;
   return __all_sync(0xffffffffu, ok);
+}
+
+// Fast path: the phase has usually completed already, which one non-blocking test shows.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                             uint32_t site) {
+  if (__all_sync(0xffffffffu, ptx::mbar_test(bar, parity))) return true;
+  return bounded_wait_slow(bar, parity, abort_flag, site);
 }
 
 // The same for a barrier that other CTAs of the cluster arrive on / copy into (acquire at cluster
@@ -231,9 +248,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ptx::mbar_init(bar(Bars::kSFree + i), 128 * C::kWG);
     }
     ptx::mbar_init(bar(Bars::kHalf), 128 * C::kWG);
+    for (int i = 0; i < 2; ++i) {
+      ptx::mbar_init(bar(Bars::kPFull + i), 128 * C::kWG);
+      ptx::mbar_init(bar(Bars::kODone + i), 1);
+    }
     for (int mt = 0; mt < MT; ++mt) {
-      ptx::mbar_init(bar(Bars::kPFull + mt), 128 * C::kWG);
-      ptx::mbar_init(bar(Bars::kODone + mt), 1);
       // slice merge: every slice sends this CTA its block of rows of query tile mt
       ptx::mbar_init(bar(Bars::kRecv + mt), 1);
       if (S > 1) ptx::mbar_arrive_expect_tx(bar(Bars::kRecv + mt), S * own_n * C::kRecvPitch);
@@ -257,7 +276,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   ptx::tc_fence_after();
   // The barriers of every CTA of the cluster must exist before any CTA arrives on them remotely:
   // arrive on the hardware cluster barrier now, wait for it only when the slices are merged.
-  if (S > 1) ptx::cluster_arrive();
+  const bool via_cluster = S > 1 && !p.via_global;
+  if (via_cluster) ptx::cluster_arrive();
   const uint32_t tmem_base = *tmem_slot;
   ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
   ptx::grid_dep_launch();    // the next kernel may start its own set-up as SMs become free
@@ -394,7 +414,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             __syncwarp();
           }
           for (int mt = 0; mt < n_mt && ok; ++mt) {
-            ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag, 8);
+            ok = bounded_wait(bar(Bars::kPFull + C::p_buf(mt, tl)), C::p_use(tl) & 1, abort_flag, 8);
             if (!ok) break;
             ptx::tc_fence_after();
             if (lane == 0) {
@@ -402,10 +422,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
               for (int kk = 0; kk < kBN / 16; ++kk)
                 ptx::umma_ss(d_tmem,
-                             ptx::smem_desc_sw128(sP + mt * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0),
+                             ptx::smem_desc_sw128(sP + C::p_buf(mt, tl) * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0),
                              ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
                              (tl == 0 && kk == 0) ? 0u : 1u);
-              ptx::umma_commit(bar(Bars::kODone + mt));
+              ptx::umma_commit(bar(Bars::kODone + C::p_buf(mt, tl)));
             }
             __syncwarp();
           }
@@ -428,7 +448,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       const int v = node_lo + mt * npt + r / G;
       const bool row_live = v < n;
       const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
-      uint8_t* p_row = gen_p + mt * 2 * kHalfBytes + r * 128;
       const float sl2 = p.scale_log2;
       bool ok = true;
 
@@ -436,6 +455,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       for (int tl = 0; tl < T && ok; ++tl) {
         const int t = t_lo + tl;
         const uint32_t tS = t_lane + C::s_col(mt, tl) + c0 * 32;
+        uint8_t* p_row = gen_p + C::p_buf(mt, tl) * 2 * kHalfBytes + r * 128;
         const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
         // visibility bits of this row for 32-key chunk c of a tile that is not full
         auto chunk_bits = [&](int c) -> uint32_t {
@@ -451,13 +471,28 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (!ok) break;
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
-        if (tid == 128 && tl < 6) JET_TR(19 + 2 * tl);
+        if (tid == 128 && tl < 4) JET_TR(19 + 2 * tl);
 
-        // ---- pass 1: maximum over the visible keys of this thread's columns (scores are read from TMEM
-        //      in 32-column chunks, the next chunk is in flight while the current one is reduced)
+        // ---- row maximum over the visible keys of this thread's columns.  With two warpgroups per tile a
+        //      thread owns 64 columns: they are read from TMEM once and kept in registers, so the score
+        //      buffer is released at once.  Otherwise (128 columns) the scores are read twice in 32-column
+        //      chunks, the next chunk in flight while the current one is reduced.
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         uint32_t xa[32], xb[32];
-        if (full_tile) {
+        if constexpr (kWG == 2) {
+          ptx::tmem_ld32(tS, xa);
+          ptx::tmem_ld32(tS + 32, xb);
+          ptx::tmem_wait_ld();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));
+          if (full_tile) {
+            max_chunk(xa, mx);
+            max_chunk(xb, mx);
+          } else {
+            max_chunk_masked(xa, chunk_bits(c0), mx);
+            max_chunk_masked(xb, chunk_bits(c0 + 1), mx);
+          }
+        } else if (full_tile) {
           ptx::tmem_ld32(tS, xa);
 #pragma unroll 1
           for (int c = 0; c < kChunks; c += 2) {
@@ -494,6 +529,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           m_tile = fmaxf(__uint_as_float(ma), __uint_as_float(mb));
         }
         if (tid == 128 && tl < 1) JET_TR(5);
+        if (tid == 128 && tl == 2) JET_TR(27);
 
         // ---- running maximum with lazy rescaling
         float factor = 1.0f;
@@ -508,40 +544,57 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
         const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
 
-        // P of the previous tile must have been consumed before it is overwritten; the same
-        // completion also makes O safe to rescale.
-        if (tl > 0) {
-          ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag, 10);
+        // The P buffer about to be overwritten must have been consumed by the P V product of the tile
+        // that used it last; a rescale of O additionally needs the previous tile's product to be complete.
+        if (tl >= C::kPBufs) {
+          const int prev = tl - C::kPBufs;
+          ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, prev)), C::p_use(prev) & 1, abort_flag, 10);
           if (!ok) break;
-          ptx::tc_fence_after();
         }
+        if (need_rescale && tl > 0 && C::kPBufs > 1) {
+          ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, tl - 1)), C::p_use(tl - 1) & 1, abort_flag, 17);
+          if (!ok) break;
+        }
+        ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(16);
+        if (tid == 128 && tl == 2) JET_TR(28);
 
-        // ---- pass 2: probabilities, row sum, P -> shared memory (swizzled bf16)
+        // ---- probabilities, row sum, P -> shared memory (swizzled bf16)
         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (full_tile) {
-          ptx::tmem_ld32(tS, xa);
-#pragma unroll 1
-          for (int c = 0; c < kChunks; c += 2) {
-            ptx::tmem_wait_ld();
-            ptx::tmem_ld32(tS + (c + 1) * 32, xb);
-            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c0 + c, r);
-            ptx::tmem_wait_ld();
-            if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
-            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c0 + c + 1, r);
+        if constexpr (kWG == 2) {
+          if (full_tile) {
+            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c0, r);
+            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c0 + 1, r);
+          } else {
+            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c0), sum, p_row, c0, r);
+            exp_chunk<true>(xb, sl2, m_ref, chunk_bits(c0 + 1), sum, p_row, c0 + 1, r);
           }
         } else {
+          if (full_tile) {
+            ptx::tmem_ld32(tS, xa);
 #pragma unroll 1
-          for (int c = 0; c < kChunks; ++c) {
-            ptx::tmem_ld32(tS + c * 32, xa);
-            ptx::tmem_wait_ld();
-            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c0 + c), sum, p_row, c0 + c, r);
+            for (int c = 0; c < kChunks; c += 2) {
+              ptx::tmem_wait_ld();
+              ptx::tmem_ld32(tS + (c + 1) * 32, xb);
+              exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c0 + c, r);
+              ptx::tmem_wait_ld();
+              if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
+              exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c0 + c + 1, r);
+            }
+          } else {
+#pragma unroll 1
+            for (int c = 0; c < kChunks; ++c) {
+              ptx::tmem_ld32(tS + c * 32, xa);
+              ptx::tmem_wait_ld();
+              exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c0 + c), sum, p_row, c0 + c, r);
+            }
           }
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));   // the score buffer may be overwritten
         }
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));   // the score buffer may be overwritten
         l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
         if (tid == 128 && tl < 1) JET_TR(17);
+        if (tid == 128 && tl == 2) JET_TR(29);
 
         if (need_rescale && tl > 0) {
           // each warpgroup rescales its share of the row's O columns
@@ -557,13 +610,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         ptx::fence_proxy_async_smem();
         ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kPFull + mt));
+        ptx::mbar_arrive(bar(Bars::kPFull + C::p_buf(mt, tl)));
         if (tid == 128 && tl < 1) JET_TR(6);
-        if (tid == 128 && tl < 6) JET_TR(20 + 2 * tl);
+        if (tid == 128 && tl < 4) JET_TR(20 + 2 * tl);
       }
       if (tid == 128) JET_TR(10);
       // O is complete once the last P V has been committed
-      if (ok) ok = bounded_wait(bar(Bars::kODone + mt), (T - 1) & 1, abort_flag, 11);
+      if (ok) ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, T - 1)), C::p_use(T - 1) & 1, abort_flag, 11);
       if (ok) ptx::tc_fence_after();
       row_ok = ok;
       if (tid == 128) JET_TR(11);
@@ -582,7 +635,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int e_r = (tid - 128) & 127;                           // its row within the query tile
   uint8_t* stage = smem_gen + C::kStageOff;
   bool merge_ok = true;
-  if (S > 1) {
+  if (via_cluster) {
     __syncwarp();
     ptx::cluster_wait();     // pairs with cluster_arrive above: every CTA's barriers are initialised
     // A: every CTA of the cluster has left its key loop, so its tile memory may be overwritten
@@ -613,7 +666,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
     if (mt > 0) {
       // C: everybody has combined the previous tile's rows, so both buffers are free again
-      if (S > 1) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
+      if (via_cluster) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
       else __syncthreads();
     }
     if (warp >= 4 && e_mt == mt) {
@@ -645,7 +698,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     __syncthreads();
     const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
     bool rows_ok = merge_ok;
-    if (S > 1) {
+    if (via_cluster) {
       if (tid < S && merge_ok) {
         const int dst_lo = tid * rows_per;
         const int dst_n = max(0, min(rows_per, kBM - dst_lo));
@@ -664,6 +717,45 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       // This CTA's own bulk copies read its staged rows asynchronously: it may only exit once every
       // peer has received them.  Arrive on the hardware cluster barrier now, wait for it at the end.
       if (mt == n_mt - 1) ptx::cluster_arrive();
+    } else if (S > 1) {
+      // Exchange through the workspace: publish this CTA's staged rows, count the slices of the unit
+      // that have published (bounded spin), then fetch this CTA's block of rows from every slice.
+      constexpr uint32_t kBlockBytes = kBM * C::kRecvPitch;
+      int* arrive = p.counters + unit * MT + mt;
+      int* depart = p.counters + p.n_units * MT + unit * MT + mt;
+      uint8_t* slots = p.partials + (static_cast<size_t>(unit) * S * MT) * kBlockBytes;
+      if (tid == 0) {
+        ptx::bulk_store_global(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes, smem_base + C::kStageOff,
+                               kBlockBytes);
+        ptx::bulk_commit_and_wait_all();
+        ptx::fence_proxy_async_all();
+        __threadfence();
+        ptx::atom_add_release_gpu(arrive, 1);
+        bool seen = false;
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+          if (ptx::ld_acquire_gpu(arrive) >= S) { seen = true; break; }
+          __nanosleep(64);
+          if (*abort_flag) break;
+        }
+        if (!seen && *abort_flag == 0u) *abort_flag = 1u + 16u;
+        ptx::fence_proxy_async_all();
+      }
+      if (tid == 128 && mt == 0) JET_TR(8);
+      const bool published = __syncthreads_and(*abort_flag == 0u ? 1 : 0) != 0;
+      if (tid < S && published && own_n > 0)
+        ptx::bulk_load_global(smem_base + C::kRecvOff + static_cast<uint32_t>(tid * rows_per * C::kRecvPitch),
+                              slots + (static_cast<size_t>(tid) * MT + mt) * kBlockBytes + own_lo * C::kRecvPitch,
+                              static_cast<uint32_t>(own_n * C::kRecvPitch), bar(Bars::kRecv + mt));
+      rows_ok = published && (own_n == 0 || bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14));
+      if (own_n == 0) __syncthreads();
+      if (tid == 128 && mt == 0) JET_TR(9);
+      src_rows = smem_gen + C::kRecvOff;
+      // the last slice to have fetched its rows leaves the counters at zero for the next call
+      if (tid == 0 && ptx::atom_add_release_gpu(depart, 1) == S - 1) {
+        *arrive = 0;
+        *depart = 0;
+        __threadfence();
+      }
     }
     const int items = rows_ok ? own_n * (D / 8) : 0;
 #pragma unroll 1
@@ -706,7 +798,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   // ---------------- teardown
   if (tid == 128) JET_TR(12);
-  if (S > 1) {
+  if (via_cluster) {
     __syncwarp();
     ptx::cluster_wait();     // every CTA of the cluster has received all of its blocks
   }
@@ -770,8 +862,11 @@ struct Plan {
   int mt;          // query tiles per CTA (1 or 2)
   int n_mgroups;   // groups of mt query tiles per (sequence, KV head)
   int units;       // work items before key slicing
-  int nsplit;      // key slices = cluster size
+  int nsplit;      // key slices
+  int via_global;  // 1: slices exchange rows through the workspace (no cluster), 0: through a cluster
 };
+
+constexpr size_t kCounterBytes = 4096;     // head of the workspace: arrival / departure counters
 
 template <int D, int MT>
 bool configure_kernel() {
@@ -838,14 +933,30 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
     pl.n_mgroups = (rows + mt * kBM - 1) / (mt * kBM);
     pl.units = batch * Hkv * pl.n_mgroups;
     for (int ns = 1; ns <= kMaxSplit && ns <= tiles; ++ns) {
+      // (a) the slices of a unit form a thread-block cluster and merge through distributed shared memory
       const int resident = max_active_clusters_for(D, mt, ns);
-      if (resident <= 0) continue;
-      const long waves = (pl.units + resident - 1) / resident;
-      const long cost = waves * ((tiles + ns - 1) / ns) * mt;
-      if (best_cost < 0 || cost < best_cost) {
-        best = pl;
-        best.nsplit = ns;
-        best_cost = cost;
+      if (resident > 0) {
+        const long waves = (pl.units + resident - 1) / resident;
+        const long cost = 2 * waves * ((tiles + ns - 1) / ns) * mt;
+        if (best_cost < 0 || cost < best_cost) {
+          best = pl;
+          best.nsplit = ns;
+          best.via_global = 0;
+          best_cost = cost;
+        }
+      }
+      // (b) independent CTAs that merge through the workspace: all of them must be resident at once
+      //     (a cluster has to fit into one GPC, which can leave a third of the SMs idle); slightly
+      //     penalised because the rows take a round trip through L2
+      if (ns > 1 && static_cast<long>(pl.units) * ns <= sm_count() &&
+          static_cast<size_t>(pl.units) * mt * 2 * sizeof(int) <= kCounterBytes) {
+        const long cost = 2 * ((tiles + ns - 1) / ns) * mt + 1;
+        if (best_cost < 0 || cost < best_cost) {
+          best = pl;
+          best.nsplit = ns;
+          best.via_global = 1;
+          best_cost = cost;
+        }
       }
     }
   }
@@ -854,8 +965,14 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
     best.n_mgroups = (rows + best.mt * kBM - 1) / (best.mt * kBM);
     best.units = batch * Hkv * best.n_mgroups;
     best.nsplit = 1;
+    best.via_global = 0;
   }
   return best;
+}
+
+size_t workspace_need(const Plan& pl, int D) {
+  if (!pl.via_global) return 256;
+  return kCounterBytes + static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM * (D * 4 + 16);
 }
 
 template <int D, int MT>
@@ -871,7 +988,7 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   cudaLaunchAttribute attrs[2];
   int na = 0;
   attrs[na].id = cudaLaunchAttributeClusterDimension;
-  attrs[na].val.clusterDim.x = pl.nsplit;
+  attrs[na].val.clusterDim.x = pl.via_global ? 1 : pl.nsplit;
   attrs[na].val.clusterDim.y = 1;
   attrs[na].val.clusterDim.z = 1;
   ++na;
@@ -915,8 +1032,8 @@ extern "C" JET_API int jet_debug_max_clusters(int cluster) {
 
 extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                                        int max_seq_len) {
-  if (batch < 1 || B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0 || D < 1) return 0;
-  return 256;   // key slices are merged on chip; the workspace is only a placeholder
+  if (batch < 1 || B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0 || (D != 64 && D != 128)) return 0;
+  return jet::workspace_need(jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len), D);
 }
 
 extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
@@ -944,9 +1061,8 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
       (k_cache && !aligned(k_cache, 16)) || (v_cache && !aligned(v_cache, 16)))
     return JET_ERR_INVALID_ARG;
   if (static_cast<int64_t>(batch) * B >= (1ll << 31)) return JET_ERR_INVALID_ARG;
-  if (!workspace || !aligned(workspace, 256) || workspace_bytes < 256) return JET_ERR_WORKSPACE;
-
   const Plan pl = make_plan(batch, B, Hq, Hkv, D, max_seq_len);
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < workspace_need(pl, D)) return JET_ERR_WORKSPACE;
 
   // ---- tensor maps (bf16, 128-byte swizzle, 64-element inner box)
   CUtensorMap tq, tk, tv, ttk, ttv;
@@ -1000,6 +1116,10 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
   p.batch = batch; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.words = (B + 31) / 32;
   p.nsplit = pl.nsplit;
   p.n_mgroups = pl.n_mgroups;
+  p.n_units = pl.units;
+  p.via_global = pl.via_global;
+  p.counters = static_cast<int*>(workspace);
+  p.partials = static_cast<uint8_t*>(workspace) + kCounterBytes;
   p.scale_log2 = softmax_scale * 1.4426950408889634f;
 #ifdef JET_TRACE
   p.trace = g_trace_ptr;

@@ -66,6 +66,7 @@ class VerifyStep:
             return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=dev)
         self.ws_build = ws(jet.jet_tree_build_workspace_bytes(batch, N, V, W))
         self.ws_attn = ws(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, self.attn_max_len))
+        self.ws_attn.zero_()         # its counters must start at zero; every call leaves them zero
         self.ws_accept = ws(jet.jet_tree_accept_workspace_bytes(batch, B, V))
         self.scale = 1.0 / math.sqrt(D)
 

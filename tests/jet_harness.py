@@ -114,6 +114,7 @@ def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_
     lse = torch.full((batch, Hq, B), float("nan"), dtype=torch.float32, device=DEV) if want_lse else None
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
+    ws.zero_()          # the attention workspace starts with counters that must be zero
     jet.jet_tree_verify_attn(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
                              d_tk, d_tv, dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
                              batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
