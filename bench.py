@@ -284,7 +284,7 @@ def bench_jet(args):
             dist.destroy_process_group()
         return
 
-    # ---------------- roofline of the dominant kernel (one attention call = attention + slice merge)
+    # ---------------- roofline of the dominant kernel (one attention call = one tree_attn_kernel launch)
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):
         peaks, peak_src = json.load(open(peaks_path)), "measured"
@@ -301,7 +301,7 @@ def bench_jet(args):
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.config)
-    roof.update(kernel="tree_attn_kernel (+ tree_attn_merge_kernel)", peak_source=peak_src, us_per_launch=attn_us,
+    roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us,
                 algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
                 roofline_us=max(t_bytes, t_flops) * 1e6)
 
@@ -320,7 +320,7 @@ def bench_jet(args):
         "attn_us_per_layer": attn_us,
         "e2e": {"value": e2e_ms_step * 1e3 / (layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step},
-        "gpu_launches": args.steps * st.launches_per_step(2),
+        "gpu_launches": args.steps * st.launches_per_step(1),
         "clocks": clocks, "roofline": roof,
     }
     if cpu is not None:

@@ -724,17 +724,26 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       int* arrive = p.counters + unit * MT + mt;
       int* depart = p.counters + p.n_units * MT + unit * MT + mt;
       uint8_t* slots = p.partials + (static_cast<size_t>(unit) * S * MT) * kBlockBytes;
-      if (tid == 0) {
-        ptx::bulk_store_global(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes, smem_base + C::kStageOff,
-                               kBlockBytes);
-        ptx::bulk_commit_and_wait_all();
+      if (tid < S) {
+        // S threads publish one row block each (the block of owner `tid`), so the copies run in parallel
+        const int blk_lo = tid * rows_per;
+        const int blk_n = max(0, min(rows_per, kBM - blk_lo));
+        if (blk_n > 0) {
+          ptx::bulk_store_global(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes + blk_lo * C::kRecvPitch,
+                                 smem_base + C::kStageOff + static_cast<uint32_t>(blk_lo * C::kRecvPitch),
+                                 static_cast<uint32_t>(blk_n * C::kRecvPitch));
+          ptx::bulk_commit_and_wait_all();
+        }
         ptx::fence_proxy_async_all();
         __threadfence();
+      }
+      __syncthreads();
+      if (tid == 0) {
         ptx::atom_add_release_gpu(arrive, 1);
         bool seen = false;
         for (uint32_t i = 0; i < (1u << 22); ++i) {
           if (ptx::ld_acquire_gpu(arrive) >= S) { seen = true; break; }
-          __nanosleep(64);
+          __nanosleep(32);
           if (*abort_flag) break;
         }
         if (!seen && *abort_flag == 0u) *abort_flag = 1u + 16u;
@@ -757,6 +766,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         __threadfence();
       }
     }
+    const uint32_t src_stride = rows_per * C::kRecvPitch;     // distance between the blocks of consecutive slices
     const int items = rows_ok ? own_n * (D / 8) : 0;
 #pragma unroll 1
     for (int i = tid; i < items; i += C::kThreads) {
@@ -767,21 +777,41 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
       float lse2 = -INFINITY;
       if (v < n) {
+        const uint8_t* row0 = src_rows + rl * C::kRecvPitch;
+        // weights first (all loads independent) ...
+        float ls[kMaxSplit];
         float mx = -INFINITY;
-        for (int c = 0; c < S; ++c)
-          mx = fmaxf(mx, *reinterpret_cast<const float*>(src_rows + (c * rows_per + rl) * C::kRecvPitch + D * 4));
+#pragma unroll
+        for (int c = 0; c < kMaxSplit; ++c) {
+          ls[c] = c < S ? *reinterpret_cast<const float*>(row0 + c * src_stride + D * 4) : -INFINITY;
+          mx = fmaxf(mx, ls[c]);
+        }
         float wsum = 0.0f;
         if (mx > -INFINITY) {
-          for (int c = 0; c < S; ++c) {
-            const uint8_t* src = src_rows + (c * rows_per + rl) * C::kRecvPitch;
-            const float ls = *reinterpret_cast<const float*>(src + D * 4);
-            if (ls == -INFINITY) continue;
-            const float w = exp2f(ls - mx);
-            wsum += w;
-            const float4 x0 = *reinterpret_cast<const float4*>(src + c8 * 32);
-            const float4 x1 = *reinterpret_cast<const float4*>(src + c8 * 32 + 16);
-            acc[0] += w * x0.x; acc[1] += w * x0.y; acc[2] += w * x0.z; acc[3] += w * x0.w;
-            acc[4] += w * x1.x; acc[5] += w * x1.y; acc[6] += w * x1.z; acc[7] += w * x1.w;
+#pragma unroll
+          for (int c = 0; c < kMaxSplit; ++c) {
+            ls[c] = ls[c] > -INFINITY ? exp2f(ls[c] - mx) : 0.0f;        // absent slices get weight 0
+            wsum += ls[c];
+          }
+          // ... then the rows, four slices at a time; a slice with weight 0 is not read (it may hold junk)
+#pragma unroll
+          for (int c0 = 0; c0 < kMaxSplit; c0 += 4) {
+            if (c0 < S) {
+              float4 x0[4], x1[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint8_t* src = row0 + (c0 + k) * src_stride;
+                const bool use = ls[c0 + k] > 0.0f;
+                x0[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32) : make_float4(0.f, 0.f, 0.f, 0.f);
+                x1[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32 + 16) : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float w = ls[c0 + k];
+                acc[0] += w * x0[k].x; acc[1] += w * x0[k].y; acc[2] += w * x0[k].z; acc[3] += w * x0[k].w;
+                acc[4] += w * x1[k].x; acc[5] += w * x1[k].y; acc[6] += w * x1[k].z; acc[7] += w * x1[k].w;
+              }
+            }
           }
           const float inv = 1.0f / wsum;
 #pragma unroll
