@@ -56,12 +56,12 @@ struct AttnParams {
   uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D fp32 + log2-sum-exp]
   float scale_log2;   // softmax_scale * log2(e)
 #ifdef JET_TRACE
-  long long* trace;   // 32 clock64() samples per CTA
+  long long* trace;   // 64 clock64() samples per CTA
 #endif
 };
 
 #ifdef JET_TRACE
-#define JET_TR(slot) do { if (p.trace) p.trace[blockIdx.x * 32 + (slot)] = clock64(); } while (0)
+#define JET_TR(slot) do { if (p.trace) p.trace[blockIdx.x * 64 + (slot)] = clock64(); } while (0)
 #else
 #define JET_TR(slot) do { } while (0)
 #endif
@@ -842,7 +842,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     JET_TR(13);
     if (*abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
 #ifdef JET_TRACE
-    if (*abort_flag && p.trace) p.trace[blockIdx.x * 32 + 31] = *abort_flag;
+    if (*abort_flag && p.trace) p.trace[blockIdx.x * 64 + 31] = *abort_flag;
 #endif
   }
 }
@@ -949,8 +949,8 @@ int max_active_clusters_for(int D, int mt, int cluster) {
 }
 
 // Picks the query-tile grouping and the number of key slices.  Cost model: waves of clusters x key tiles
-// per CTA x query tiles per CTA; on a tie the grouping that loads K/V fewer times, then the smaller
-// cluster, wins.
+// per CTA x a per-tile cost (1 for one query tile per CTA, 3 for two: the pair shares each K/V tile but
+// its shallower shared-memory ring and single-buffered P make a key tile about three times as slow).
 Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   const int G = Hq / Hkv;
   const int rows = B * G;
@@ -967,7 +967,7 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
       const int resident = max_active_clusters_for(D, mt, ns);
       if (resident > 0) {
         const long waves = (pl.units + resident - 1) / resident;
-        const long cost = 2 * waves * ((tiles + ns - 1) / ns) * mt;
+        const long cost = 4 * waves * ((tiles + ns - 1) / ns) * (mt == 2 ? 3 : 1);
         if (best_cost < 0 || cost < best_cost) {
           best = pl;
           best.nsplit = ns;
@@ -980,7 +980,7 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
       //     penalised because the rows take a round trip through L2
       if (ns > 1 && static_cast<long>(pl.units) * ns <= sm_count() &&
           static_cast<size_t>(pl.units) * mt * 2 * sizeof(int) <= kCounterBytes) {
-        const long cost = 2 * ((tiles + ns - 1) / ns) * mt + 1;
+        const long cost = 4 * ((tiles + ns - 1) / ns) * (mt == 2 ? 3 : 1) + 1;
         if (best_cost < 0 || cost < best_cost) {
           best = pl;
           best.nsplit = ns;
