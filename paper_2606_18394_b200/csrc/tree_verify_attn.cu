@@ -77,21 +77,21 @@ struct Cfg {
   static constexpr int kStageBytes = kHalves * kHalfBytes;
   static constexpr int kStages = (D == 128) ? (MT == 1 ? 4 : 3) : 6;
   static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
-  // With one query tile per CTA two softmax warpgroups share it: each thread owns one row and half of
-  // the tile's 128 key columns, which halves the per-tile softmax latency.
-  static constexpr int kWG = MT == 1 ? 2 : 1;
+  // With one query tile per CTA two softmax warpgroups work on it as two independent streams: stream 0
+  // takes the even key tiles, stream 1 the odd ones, each with its own score buffer, P buffer, O
+  // accumulator and running maximum / sum.  Their phases interleave (one computes maxima while the
+  // other exponentiates), and the two partial results are combined once, after the key loop.
+  static constexpr int kStreams = MT == 1 ? 2 : 1;
   static constexpr int kBarBytes = 256;
   static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
-  static constexpr int kThreads = 128 + 128 * MT * kWG;
-  // TMEM (512 columns): with one query tile per CTA the scores are double-buffered,
-  //   MT == 1: S0 [0,128)  S1 [128,256)  O [256,256+D)  and columns [384,392) for per-row scalars that
-  //            the two warpgroups of a row exchange (both own the row's TMEM lane)
-  //   MT == 2: tile mt owns S [mt*256, +128) and O [mt*256+128, +D)
+  static constexpr int kThreads = 128 + 128 * MT * kStreams;
+  // TMEM (512 columns):
+  //   MT == 1: stream i owns S [i*128, +128) and O [256 + i*128, +D); key tile t belongs to stream t & 1
+  //   MT == 2: query tile mt owns S [mt*256, +128) and O [mt*256+128, +D)
   static constexpr int kTmemCols = 512;
   static constexpr int kSBufs = MT == 1 ? 2 : 1;
   __device__ static constexpr uint32_t s_col(int mt, int t) { return MT == 1 ? (t & 1) * 128 : mt * 256; }
-  __device__ static constexpr uint32_t o_col(int mt) { return MT == 1 ? 256 : mt * 256 + 128; }
-  static constexpr uint32_t kXchgCol = 384;
+  __device__ static constexpr uint32_t o_col(int mt, int t) { return MT == 1 ? 256 + (t & 1) * 128 : mt * 256 + 128; }
   // Each score buffer has its own full/free barrier pair, so that neither side can run two phases
   // ahead of the other on one barrier: buffer index and use count of tile t of query tile mt.
   __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
@@ -103,14 +103,15 @@ struct Cfg {
   // rows of one query tile -- D fp32 values followed by the row's log2-sum-exp, padded so that the
   // row-per-thread stores of a warp spread over all banks -- and the blocks received from every slice.
   static constexpr int kRecvPitch = D * 4 + 16;
+  static constexpr int kBlockBytes = kBM * kRecvPitch;                   // the 128 staged rows of one stream
   static constexpr int kStageOff = 0;
-  static constexpr int kRecvOff = (kBM * kRecvPitch + 1023) / 1024 * 1024;
-  static_assert(kRecvOff + (kBM + kMaxSplit) * kRecvPitch <= kTileBytes, "merge buffers must fit in the tile memory");
+  static constexpr int kRecvOff = (kBlockBytes + 1023) / 1024 * 1024;
+  static_assert(kRecvOff + (kBM + kMaxSplit) * kRecvPitch + 2048 <= kTileBytes, "merge buffers must fit in the tile memory");
 };
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
   enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
-         kClusterA = 21, kClusterC = 22, kRecv = 23, kHalf = 25, kCount = 26 };
+         kClusterA = 21, kClusterC = 22, kRecv = 23, kCount = 25 };
 };
 
 // Every wait is bounded: at most kWaitRounds suspensions of kWaitHintNs each (about a second).
@@ -245,11 +246,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else if (warp == 1 && lane == 0) {
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(bar(Bars::kSFull + i), 1);
-      ptx::mbar_init(bar(Bars::kSFree + i), 128 * C::kWG);
+      ptx::mbar_init(bar(Bars::kSFree + i), 128);
     }
-    ptx::mbar_init(bar(Bars::kHalf), 128 * C::kWG);
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(bar(Bars::kPFull + i), 128 * C::kWG);
+      ptx::mbar_init(bar(Bars::kPFull + i), 128);
       ptx::mbar_init(bar(Bars::kODone + i), 1);
     }
     for (int mt = 0; mt < MT; ++mt) {
@@ -418,13 +418,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (!ok) break;
             ptx::tc_fence_after();
             if (lane == 0) {
-              const uint32_t d_tmem = tmem_base + C::o_col(mt);
+              const uint32_t d_tmem = tmem_base + C::o_col(mt, tl);
 #pragma unroll
               for (int kk = 0; kk < kBN / 16; ++kk)
                 ptx::umma_ss(d_tmem,
                              ptx::smem_desc_sw128(sP + C::p_buf(mt, tl) * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0),
                              ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
-                             (tl == 0 && kk == 0) ? 0u : 1u);
+                             (tl < C::kStreams && kk == 0) ? 0u : 1u);      // first product of each accumulator
               ptx::umma_commit(bar(Bars::kODone + C::p_buf(mt, tl)));
             }
             __syncwarp();
@@ -436,25 +436,25 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     } else if (warp >= 4 && (MT == 1 || ((warp - 4) >> 2) < n_mt)) {
       // =========================================================== softmax warpgroups
-      constexpr int kWG = C::kWG;
-      constexpr int kChunks = kBN / 32 / kWG;                 // 32-key chunks per thread and tile
+      constexpr int kChunks = kBN / 32;                       // 32-key chunks per row and tile
+      constexpr int kStreams = C::kStreams;
       const int wg = (warp - 4) >> 2;
       const int mt = MT == 1 ? 0 : wg;                        // query tile of this warpgroup
-      const int half = MT == 1 ? wg : 0;                      // which half of the key columns it owns
-      const int c0 = half * kChunks;                          // its first 32-key chunk
+      const int stream = MT == 1 ? wg : 0;                    // its share of the key tiles (tl % kStreams)
       const int r = (tid - 128) & 127;                        // row of the query tile = TMEM lane
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-      const uint32_t tO = t_lane + C::o_col(mt) + half * (D / kWG);
       const int v = node_lo + mt * npt + r / G;
       const bool row_live = v < n;
       const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
       const float sl2 = p.scale_log2;
       bool ok = true;
+      int last_tl = -1;
 
 #pragma unroll 1
-      for (int tl = 0; tl < T && ok; ++tl) {
+      for (int tl = stream; tl < T && ok; tl += kStreams) {
         const int t = t_lo + tl;
-        const uint32_t tS = t_lane + C::s_col(mt, tl) + c0 * 32;
+        const uint32_t tS = t_lane + C::s_col(mt, tl);
+        const uint32_t tO = t_lane + C::o_col(mt, tl);
         uint8_t* p_row = gen_p + C::p_buf(mt, tl) * 2 * kHalfBytes + r * 128;
         const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
         // visibility bits of this row for 32-key chunk c of a tile that is not full
@@ -471,28 +471,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (!ok) break;
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
-        if (tid == 128 && tl < 4) JET_TR(19 + 2 * tl);
+        if (tid == 128 && tl < 8) JET_TR(19 + tl);
 
-        // ---- row maximum over the visible keys of this thread's columns.  With two warpgroups per tile a
-        //      thread owns 64 columns: they are read from TMEM once and kept in registers, so the score
-        //      buffer is released at once.  Otherwise (128 columns) the scores are read twice in 32-column
-        //      chunks, the next chunk in flight while the current one is reduced.
+        // ---- pass 1: row maximum over the visible keys (scores are read from TMEM in 32-column chunks,
+        //      the next chunk is in flight while the current one is reduced)
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         uint32_t xa[32], xb[32];
-        if constexpr (kWG == 2) {
-          ptx::tmem_ld32(tS, xa);
-          ptx::tmem_ld32(tS + 32, xb);
-          ptx::tmem_wait_ld();
-          ptx::tc_fence_before();
-          ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));
-          if (full_tile) {
-            max_chunk(xa, mx);
-            max_chunk(xb, mx);
-          } else {
-            max_chunk_masked(xa, chunk_bits(c0), mx);
-            max_chunk_masked(xb, chunk_bits(c0 + 1), mx);
-          }
-        } else if (full_tile) {
+        if (full_tile) {
           ptx::tmem_ld32(tS, xa);
 #pragma unroll 1
           for (int c = 0; c < kChunks; c += 2) {
@@ -508,28 +493,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           for (int c = 0; c < kChunks; ++c) {
             ptx::tmem_ld32(tS + c * 32, xa);
             ptx::tmem_wait_ld();
-            max_chunk_masked(xa, chunk_bits(c0 + c), mx);
+            max_chunk_masked(xa, chunk_bits(c), mx);
           }
         }
-        float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        if (kWG == 2) {
-          // The two halves of a row must use one reference maximum: each writes its partial maximum to
-          // a spare TMEM column of the row's lane (double-buffered by tile parity) and reads both.
-          const uint32_t tX = t_lane + C::kXchgCol + (tl & 1) * 2;
-          ptx::tmem_st1(tX + half, __float_as_uint(m_tile));
-          ptx::tmem_wait_st();
-          ptx::tc_fence_before();
-          ptx::mbar_arrive(bar(Bars::kHalf));
-          ok = bounded_wait(bar(Bars::kHalf), tl & 1, abort_flag, 15);
-          if (!ok) break;
-          ptx::tc_fence_after();
-          uint32_t ma, mb;
-          ptx::tmem_ld2(tX, ma, mb);
-          ptx::tmem_wait_ld();
-          m_tile = fmaxf(__uint_as_float(ma), __uint_as_float(mb));
-        }
+        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         if (tid == 128 && tl < 1) JET_TR(5);
-        if (tid == 128 && tl == 2) JET_TR(27);
 
         // ---- running maximum with lazy rescaling
         float factor = 1.0f;
@@ -544,62 +512,45 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
         const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
 
-        // The P buffer about to be overwritten must have been consumed by the P V product of the tile
-        // that used it last; a rescale of O additionally needs the previous tile's product to be complete.
+        // The P buffer about to be overwritten must have been consumed by the P V product of the tile that
+        // used it last -- the previous tile of this accumulator, so O is then also safe to rescale.
         if (tl >= C::kPBufs) {
           const int prev = tl - C::kPBufs;
           ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, prev)), C::p_use(prev) & 1, abort_flag, 10);
           if (!ok) break;
         }
-        if (need_rescale && tl > 0 && C::kPBufs > 1) {
-          ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, tl - 1)), C::p_use(tl - 1) & 1, abort_flag, 17);
-          if (!ok) break;
-        }
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(16);
-        if (tid == 128 && tl == 2) JET_TR(28);
 
-        // ---- probabilities, row sum, P -> shared memory (swizzled bf16)
+        // ---- pass 2: probabilities, row sum, P -> shared memory (swizzled bf16)
         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if constexpr (kWG == 2) {
-          if (full_tile) {
-            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c0, r);
-            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c0 + 1, r);
-          } else {
-            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c0), sum, p_row, c0, r);
-            exp_chunk<true>(xb, sl2, m_ref, chunk_bits(c0 + 1), sum, p_row, c0 + 1, r);
+        if (full_tile) {
+          ptx::tmem_ld32(tS, xa);
+#pragma unroll 1
+          for (int c = 0; c < kChunks; c += 2) {
+            ptx::tmem_wait_ld();
+            ptx::tmem_ld32(tS + (c + 1) * 32, xb);
+            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c, r);
+            ptx::tmem_wait_ld();
+            if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
+            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c + 1, r);
           }
         } else {
-          if (full_tile) {
-            ptx::tmem_ld32(tS, xa);
 #pragma unroll 1
-            for (int c = 0; c < kChunks; c += 2) {
-              ptx::tmem_wait_ld();
-              ptx::tmem_ld32(tS + (c + 1) * 32, xb);
-              exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c0 + c, r);
-              ptx::tmem_wait_ld();
-              if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
-              exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c0 + c + 1, r);
-            }
-          } else {
-#pragma unroll 1
-            for (int c = 0; c < kChunks; ++c) {
-              ptx::tmem_ld32(tS + c * 32, xa);
-              ptx::tmem_wait_ld();
-              exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c0 + c), sum, p_row, c0 + c, r);
-            }
+          for (int c = 0; c < kChunks; ++c) {
+            ptx::tmem_ld32(tS + c * 32, xa);
+            ptx::tmem_wait_ld();
+            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, p_row, c, r);
           }
-          ptx::tc_fence_before();
-          ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));   // the score buffer may be overwritten
         }
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));   // the score buffer may be overwritten
         l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
         if (tid == 128 && tl < 1) JET_TR(17);
-        if (tid == 128 && tl == 2) JET_TR(29);
 
-        if (need_rescale && tl > 0) {
-          // each warpgroup rescales its share of the row's O columns
+        if (need_rescale && last_tl >= 0) {
 #pragma unroll 1
-          for (int c = 0; c < D / 32 / kWG; ++c) {
+          for (int c = 0; c < D / 32; ++c) {
             ptx::tmem_ld32(tO + c * 32, xa);
             ptx::tmem_wait_ld();
 #pragma unroll
@@ -612,11 +563,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar(Bars::kPFull + C::p_buf(mt, tl)));
         if (tid == 128 && tl < 1) JET_TR(6);
-        if (tid == 128 && tl < 4) JET_TR(20 + 2 * tl);
+        if (tid == 128 && tl < 8) JET_TR(20 + tl);
+        last_tl = tl;
       }
       if (tid == 128) JET_TR(10);
-      // O is complete once the last P V has been committed
-      if (ok) ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, T - 1)), C::p_use(T - 1) & 1, abort_flag, 11);
+      // O is complete once the last P V of this accumulator has been committed
+      if (ok && last_tl >= 0)
+        ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, last_tl)), C::p_use(last_tl) & 1, abort_flag, 11);
       if (ok) ptx::tc_fence_after();
       row_ok = ok;
       if (tid == 128) JET_TR(11);
@@ -630,8 +583,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // slices the CTA "combines" its own staged rows.  Either way the output rows leave as coalesced
   // 16-byte stores, rows of padding nodes as zeros.
   const int e_wg = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
-  const int e_mt = MT == 1 ? 0 : e_wg;                         // its query tile
-  const int e_half = MT == 1 ? e_wg : 0;                       // its half of the row (two warpgroups per tile)
   const int e_r = (tid - 128) & 127;                           // its row within the query tile
   uint8_t* stage = smem_gen + C::kStageOff;
   bool merge_ok = true;
@@ -644,24 +595,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else {
     __syncthreads();
   }
-  float l_row = l;
-  if (C::kWG == 2) {
-    // combine the row sums of the two halves through the row's spare TMEM columns
-    const uint32_t tX = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::kXchgCol + 4;
-    if (warp >= 4) {
-      ptx::tmem_st1(tX + e_half, __float_as_uint(l));
-      ptx::tmem_wait_st();
-    }
-    ptx::tc_fence_before();
-    __syncthreads();
-    ptx::tc_fence_after();
-    if (warp >= 4) {
-      uint32_t la, lb;
-      ptx::tmem_ld2(tX, la, lb);
-      ptx::tmem_wait_ld();
-      l_row = __uint_as_float(la) + __uint_as_float(lb);
-    }
-  }
+  // Staging of a row: normalised, D fp32 values followed by the row's log2-sum-exp.  Rows this CTA
+  // computed nothing for (empty key slice, tile without nodes) get log2-sum-exp = -inf ("absent").
+  const uint32_t e_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  const bool active = has_work && row_ok;                      // warp-uniform: TMEM loads need whole warps
+  const float own_inv = (active && l > 0.0f) ? 1.0f / l : 0.0f;
+  const float own_lse2 = (active && l > 0.0f) ? m_used * p.scale_log2 + log2f(l) : -INFINITY;
+  // MT == 1: the two streams of a row exchange (log2-sum-exp, 1/sum) through a scratch corner of the
+  // idle tile memory; afterwards both threads of a row know both weights.
+  float2* xchg = reinterpret_cast<float2*>(smem_gen + C::kTileBytes - 2048);     // [stream][row]
+  if (MT == 1 && warp >= 4) xchg[e_wg * 128 + e_r] = make_float2(own_lse2, own_inv);
 #pragma unroll 1
   for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
     if (mt > 0) {
@@ -669,32 +612,68 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (via_cluster) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
       else __syncthreads();
     }
-    if (warp >= 4 && e_mt == mt) {
-      constexpr int kColsPerWG = D / C::kWG;                   // O columns staged by this thread
-      uint8_t* srow = stage + e_r * C::kRecvPitch + e_half * kColsPerWG * 4;
-      const bool active = has_work && mt < n_mt && row_ok;     // warp-uniform
-      const float e_inv = l_row > 0.0f ? 1.0f / l_row : 0.0f;
-      if (active) {
-        const uint32_t tO =
-            tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::o_col(mt) + e_half * kColsPerWG;
+    if constexpr (MT == 1) {
+      // Both warpgroups stage half of every row (64 columns each), folding the two streams' accumulators
+      // together on the way: out = wa * O_0 / l_0 + wb * O_1 / l_1 with softmax weights of the two sums.
+      __syncthreads();
+      if (warp >= 4) {
+        const float2 s0 = xchg[e_r], s1 = xchg[128 + e_r];
+        const float mxl = fmaxf(s0.x, s1.x);
+        float a0 = 0.0f, a1 = 0.0f, lse2 = -INFINITY;
+        if (mxl > -INFINITY) {
+          const float w0 = s0.x > -INFINITY ? exp2f(s0.x - mxl) : 0.0f;
+          const float w1 = s1.x > -INFINITY ? exp2f(s1.x - mxl) : 0.0f;
+          const float inv = 1.0f / (w0 + w1);
+          a0 = w0 * inv * s0.y;
+          a1 = w1 * inv * s1.y;
+          lse2 = mxl + log2f(w0 + w1);
+        }
+        constexpr int kCols = D / 2;
+        uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 4;
 #pragma unroll 1
-        for (int c = 0; c < kColsPerWG / 32; ++c) {
-          uint32_t o[32];
-          ptx::tmem_ld32(tO + c * 32, o);
-          ptx::tmem_wait_ld();
+        for (int c = 0; c < kCols / 32; ++c) {
+          uint32_t o0[32], o1[32];
+          if (active) {
+            ptx::tmem_ld32(e_lane + C::o_col(0, 0) + e_wg * kCols + c * 32, o0);
+            ptx::tmem_ld32(e_lane + C::o_col(0, 1) + e_wg * kCols + c * 32, o1);
+            ptx::tmem_wait_ld();
+          }
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4)
-            *reinterpret_cast<float4*>(srow + (c * 32 + q4 * 4) * 4) =
-                make_float4(__uint_as_float(o[q4 * 4]) * e_inv, __uint_as_float(o[q4 * 4 + 1]) * e_inv,
-                            __uint_as_float(o[q4 * 4 + 2]) * e_inv, __uint_as_float(o[q4 * 4 + 3]) * e_inv);
+          for (int q4 = 0; q4 < 8; ++q4) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (active) {
+              // an accumulator that never received a product holds junk: its weight is exactly 0
+              x.x = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4]) : 0.0f);
+              x.y = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 1]) : 0.0f);
+              x.z = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 2]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 2]) : 0.0f);
+              x.w = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 3]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 3]) : 0.0f);
+            }
+            *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
+          }
+        }
+        if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 4) = lse2;
+      }
+    } else if (warp >= 4 && e_wg == mt) {
+      uint8_t* dst = stage + e_r * C::kRecvPitch;
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        if (active) {
+          ptx::tmem_ld32(e_lane + C::o_col(mt, 0) + c * 32, o);
+          ptx::tmem_wait_ld();
+        }
+#pragma unroll
+        for (int q4 = 0; q4 < 8; ++q4) {
+          float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (active)
+            x = make_float4(__uint_as_float(o[q4 * 4]) * own_inv, __uint_as_float(o[q4 * 4 + 1]) * own_inv,
+                            __uint_as_float(o[q4 * 4 + 2]) * own_inv, __uint_as_float(o[q4 * 4 + 3]) * own_inv);
+          *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
         }
       }
-      // rows this CTA computed nothing for (empty key slice, tile without nodes) are marked absent
-      if (e_half == 0)
-        *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 4) =
-            (active && l_row > 0.0f) ? m_used * p.scale_log2 + log2f(l_row) : -INFINITY;
-      if (S > 1) ptx::fence_proxy_async_smem();
+      *reinterpret_cast<float*>(dst + D * 4) = own_lse2;
     }
+    if (via_cluster) ptx::fence_proxy_async_smem();
     __syncthreads();
     const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
     bool rows_ok = merge_ok;
