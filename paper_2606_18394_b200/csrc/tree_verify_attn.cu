@@ -22,6 +22,7 @@
 // released and JET_ERR_TIMEOUT is reported.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cstdlib>
 
 #include "jet_common.cuh"
 #include "sm100_ptx.cuh"
@@ -70,12 +71,11 @@ template <int D, int MT>
 struct Cfg {
   static constexpr int kHalves = D / 64;
   static constexpr int kQBytes = MT * kHalves * kHalfBytes;
-  // P (probabilities, bf16): one 128x128 buffer per query tile; with a single query tile per CTA it is
-  // double-buffered so that the softmax of tile t+1 never waits for the P V product of tile t.
-  static constexpr int kPBufs = MT == 1 ? 2 : 1;
-  static constexpr int kPBytes = MT * kPBufs * 2 * kHalfBytes;
+  // P (probabilities, bf16) never touches shared memory: it is written over the first 64 columns of the
+  // score buffer it was computed from (two bf16 per 32-bit column) and read from there by the P V product.
+  static constexpr int kPBytes = 0;
   static constexpr int kStageBytes = kHalves * kHalfBytes;
-  static constexpr int kStages = (D == 128) ? (MT == 1 ? 4 : 3) : 6;
+  static constexpr int kStages = (D == 128) ? (MT == 1 ? 6 : 5) : 6;
   static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
   // With one query tile per CTA two softmax warpgroups work on it as two independent streams: stream 0
   // takes the even key tiles, stream 1 the odd ones, each with its own score buffer, P buffer, O
@@ -92,13 +92,10 @@ struct Cfg {
   static constexpr int kSBufs = MT == 1 ? 2 : 1;
   __device__ static constexpr uint32_t s_col(int mt, int t) { return MT == 1 ? (t & 1) * 128 : mt * 256; }
   __device__ static constexpr uint32_t o_col(int mt, int t) { return MT == 1 ? 256 + (t & 1) * 128 : mt * 256 + 128; }
-  // Each score buffer has its own full/free barrier pair, so that neither side can run two phases
-  // ahead of the other on one barrier: buffer index and use count of tile t of query tile mt.
+  // Each score buffer (and the P that replaces it) has its own barriers, so that neither side can run two
+  // phases ahead of the other on one barrier: buffer index and use count of key tile t of query tile mt.
   __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
   __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
-  // The same for the P buffers and their full / consumed (o_done) barriers.
-  __device__ static constexpr int p_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
-  __device__ static constexpr int p_use(int t) { return MT == 1 ? (t >> 1) : t; }
   // Epilogue buffers (overlay the tile memory once the key loop is over): this CTA's 128 normalised
   // rows of one query tile -- D fp32 values followed by the row's log2-sum-exp, padded so that the
   // row-per-thread stores of a warp spread over all banks -- and the blocks received from every slice.
@@ -177,11 +174,12 @@ __device__ __forceinline__ void max_chunk_masked(const uint32_t (&x)[32], uint32
 }
 
 // 32 scores of one row -> probabilities (exp2 of the scaled, shifted score; masked keys exactly 0),
-// added to the row sum and written as bf16 to the row's slot of the swizzled P tile.  The stages
-// are kept apart so that the 32 independent exp2 are in flight together.
+// added to the row sum and written as packed bf16 pairs to 16 TMEM columns of the row's lane (the A
+// operand of the P V product).  The stages are kept apart so that the 32 independent exp2 are in
+// flight together.
 template <bool kMasked>
 __device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
-                                          float (&sum)[4], uint8_t* p_row, int c, int r) {
+                                          float (&sum)[4], uint32_t p_tmem) {
   float e[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(x[j]), sl2, -m_ref);
@@ -193,15 +191,10 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, fl
   }
 #pragma unroll
   for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
-  // chunk c covers keys [32c, 32c+32): 64-key block c/2, 16-byte chunks (c%2)*4 .. +3 of the 128-byte row
-  uint8_t* dst = p_row + (c >> 1) * kHalfBytes;
+  uint32_t packed[16];
 #pragma unroll
-  for (int q4 = 0; q4 < 4; ++q4) {
-    const int ch = ((c & 1) * 4 + q4) ^ (r & 7);
-    *reinterpret_cast<uint4*>(dst + ch * 16) =
-        make_uint4(pack_bf16(e[q4 * 8], e[q4 * 8 + 1]), pack_bf16(e[q4 * 8 + 2], e[q4 * 8 + 3]),
-                   pack_bf16(e[q4 * 8 + 4], e[q4 * 8 + 5]), pack_bf16(e[q4 * 8 + 6], e[q4 * 8 + 7]));
-  }
+  for (int j = 0; j < 16; ++j) packed[j] = pack_bf16(e[2 * j], e[2 * j + 1]);
+  ptx::tmem_st16(p_tmem, packed);
 }
 
 template <int D, int MT>
@@ -220,11 +213,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
   const uint32_t sQ = smem_base;
-  const uint32_t sP = sQ + C::kQBytes;
-  const uint32_t sKV = sP + C::kPBytes;
+  const uint32_t sKV = sQ + C::kQBytes;
   const uint32_t sBar = sKV + kStages * C::kStageBytes;
-  uint8_t* gen_kv = smem_gen + C::kQBytes + C::kPBytes;
-  uint8_t* gen_p = smem_gen + C::kQBytes;
+  uint8_t* gen_kv = smem_gen + C::kQBytes;
   uint8_t* gen_bar = gen_kv + kStages * C::kStageBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + Bars::kCount * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -246,7 +237,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else if (warp == 1 && lane == 0) {
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(bar(Bars::kSFull + i), 1);
-      ptx::mbar_init(bar(Bars::kSFree + i), 128);
     }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(bar(Bars::kPFull + i), 128);
@@ -367,18 +357,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
       bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
       if (lane == 0) JET_TR(2);
-#pragma unroll 1
-      for (int tl = -1; tl < T && ok; ++tl) {
+      // Order of issue: with two score buffers (MT == 1) the Q K^T of tile tl+1 goes out before the P V of
+      // tile tl (it belongs to the other stream and only waits for that stream's previous product).  With one
+      // buffer per query tile (MT == 2) the Q K^T of tile tl+1 overwrites the P of tile tl, so the P V
+      // products of tile tl are issued first.
+      auto issue_qk = [&](int tl) {            // tl = tile before the one whose scores are computed
         if (tl + 1 < T) {
           // ---- S = Q K^T of tile tl+1, as soon as its K tile has landed and the score buffer is free
           const int item = 2 * (tl + 1), stage = item % kStages;
           ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
           if (lane == 0 && tl == -1) JET_TR(3);
           for (int mt = 0; mt < n_mt && ok; ++mt) {
-            const int prev = tl + 1 - C::kSBufs;            // tile that used this score buffer last
-            if (prev >= 0)
-              ok = bounded_wait(bar(Bars::kSFree + C::s_buf(mt, prev)), C::s_use(prev) & 1, abort_flag, 6);
-            if (!ok) break;
+            // The buffer still holds the P of the tile that used it last.  That tile's P V product was issued
+            // earlier by this same thread, and the tensor core executes one thread's MMAs in issue order, so
+            // this Q K^T cannot overwrite the P before it has been read: no wait is needed here.
             ptx::tc_fence_after();
             if (lane == 0) {
               const uint32_t d_tmem = tmem_base + C::s_col(mt, tl + 1);
@@ -392,15 +384,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
             __syncwarp();
           }
-          if (!ok) break;
+          if (!ok) return;
           if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
           __syncwarp();
         }
+      };
+      auto issue_pv = [&](int tl) {
         if (tl >= 0) {
           // ---- O += P V of tile tl
           const int item = 2 * tl + 1, stage = item % kStages;
           ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
-          if (!ok) break;
+          if (!ok) return;
           const int t = t_lo + tl;
           const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
           if (valid < kBN) {
@@ -414,24 +408,33 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             __syncwarp();
           }
           for (int mt = 0; mt < n_mt && ok; ++mt) {
-            ok = bounded_wait(bar(Bars::kPFull + C::p_buf(mt, tl)), C::p_use(tl) & 1, abort_flag, 8);
-            if (!ok) break;
+            ok = bounded_wait(bar(Bars::kPFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 8);
+            if (!ok) return;
             ptx::tc_fence_after();
             if (lane == 0) {
               const uint32_t d_tmem = tmem_base + C::o_col(mt, tl);
 #pragma unroll
-              for (int kk = 0; kk < kBN / 16; ++kk)
-                ptx::umma_ss(d_tmem,
-                             ptx::smem_desc_sw128(sP + C::p_buf(mt, tl) * 2 * kHalfBytes + (kk / 4) * kHalfBytes + (kk % 4) * 32, 0),
+              for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
+                ptx::umma_ts(d_tmem, tmem_base + C::s_col(mt, tl) + kk * 8,
                              ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
                              (tl < C::kStreams && kk == 0) ? 0u : 1u);      // first product of each accumulator
-              ptx::umma_commit(bar(Bars::kODone + C::p_buf(mt, tl)));
+              ptx::umma_commit(bar(Bars::kODone + C::s_buf(mt, tl)));
             }
             __syncwarp();
           }
-          if (!ok) break;
+          if (!ok) return;
           if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
           __syncwarp();
+        }
+      };
+#pragma unroll 1
+      for (int tl = -1; tl < T && ok; ++tl) {
+        if (C::kSBufs == 2) {
+          issue_qk(tl);
+          if (ok) issue_pv(tl);
+        } else {
+          issue_pv(tl);
+          if (ok) issue_qk(tl);
         }
       }
     } else if (warp >= 4 && (MT == 1 || ((warp - 4) >> 2) < n_mt)) {
@@ -455,7 +458,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int t = t_lo + tl;
         const uint32_t tS = t_lane + C::s_col(mt, tl);
         const uint32_t tO = t_lane + C::o_col(mt, tl);
-        uint8_t* p_row = gen_p + C::p_buf(mt, tl) * 2 * kHalfBytes + r * 128;
         const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
         // visibility bits of this row for 32-key chunk c of a tile that is not full
         auto chunk_bits = [&](int c) -> uint32_t {
@@ -512,17 +514,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
         const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
 
-        // The P buffer about to be overwritten must have been consumed by the P V product of the tile that
-        // used it last -- the previous tile of this accumulator, so O is then also safe to rescale.
-        if (tl >= C::kPBufs) {
-          const int prev = tl - C::kPBufs;
-          ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, prev)), C::p_use(prev) & 1, abort_flag, 10);
-          if (!ok) break;
-        }
+        // (The P V product of this accumulator's previous tile is complete: the Q K^T that produced these
+        //  scores was only issued after it.  So O may be rescaled and the score buffer overwritten with P.)
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(16);
 
-        // ---- pass 2: probabilities, row sum, P -> shared memory (swizzled bf16)
+        // ---- pass 2: probabilities, row sum; P (packed bf16) overwrites the first 64 columns of the scores
         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         if (full_tile) {
           ptx::tmem_ld32(tS, xa);
@@ -530,21 +527,19 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           for (int c = 0; c < kChunks; c += 2) {
             ptx::tmem_wait_ld();
             ptx::tmem_ld32(tS + (c + 1) * 32, xb);
-            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, p_row, c, r);
+            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS + c * 16);
             ptx::tmem_wait_ld();
             if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
-            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, p_row, c + 1, r);
+            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + (c + 1) * 16);
           }
         } else {
 #pragma unroll 1
           for (int c = 0; c < kChunks; ++c) {
             ptx::tmem_ld32(tS + c * 32, xa);
             ptx::tmem_wait_ld();
-            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, p_row, c, r);
+            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, tS + c * 16);
           }
         }
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kSFree + C::s_buf(mt, tl)));   // the score buffer may be overwritten
         l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
         if (tid == 128 && tl < 1) JET_TR(17);
 
@@ -557,11 +552,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
             ptx::tmem_st32(tO + c * 32, xa);
           }
-          ptx::tmem_wait_st();
         }
-        ptx::fence_proxy_async_smem();
+        ptx::tmem_wait_st();                     // P (and a rescaled O) are in TMEM
         ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kPFull + C::p_buf(mt, tl)));
+        ptx::mbar_arrive(bar(Bars::kPFull + C::s_buf(mt, tl)));
         if (tid == 128 && tl < 1) JET_TR(6);
         if (tid == 128 && tl < 8) JET_TR(20 + tl);
         last_tl = tl;
@@ -569,7 +563,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (tid == 128) JET_TR(10);
       // O is complete once the last P V of this accumulator has been committed
       if (ok && last_tl >= 0)
-        ok = bounded_wait(bar(Bars::kODone + C::p_buf(mt, last_tl)), C::p_use(last_tl) & 1, abort_flag, 11);
+        ok = bounded_wait(bar(Bars::kODone + C::s_buf(mt, last_tl)), C::s_use(last_tl) & 1, abort_flag, 11);
       if (ok) ptx::tc_fence_after();
       row_ok = ok;
       if (tid == 128) JET_TR(11);
@@ -936,7 +930,9 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   const int tiles = (max_seq_len + kBN - 1) / kBN + (B + kBN - 1) / kBN;
   Plan best{};
   long best_cost = -1;
+  static const int force_mt = [] { const char* e = getenv("JET_FORCE_MT"); return e ? atoi(e) : 0; }();
   for (int mt = (rows > kBM ? 2 : 1); mt >= 1; --mt) {
+    if (force_mt && mt != force_mt && !(force_mt == 2 && rows <= kBM)) continue;
     Plan pl;
     pl.mt = mt;
     pl.n_mgroups = (rows + mt * kBM - 1) / (mt * kBM);
