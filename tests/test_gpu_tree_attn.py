@@ -214,3 +214,67 @@ def test_argument_errors():
     assert jet.jet_tree_verify_attn(**{**args, "workspace": None}) == jet.JET_ERR_WORKSPACE
     assert jet.jet_tree_verify_attn(**{**args, "page_table": i32, "page_size": 32, "max_pages_per_seq": 4,
                                        "num_pages": 4}) == jet.JET_ERR_UNSUPPORTED
+
+
+def test_workspace_counters_are_left_clean_across_repeated_calls():
+    """The slice exchange through the workspace counts arrivals in the workspace head; every call must
+    leave the counters at zero so that the same workspace serves the next call (here: 5 calls, two shapes)."""
+    import torch
+    import jet_harness as H
+    import paper_2606_18394_b200 as jet
+    rng = np.random.default_rng(5)
+    B, Hq, Hkv, D, L = 64, 32, 8, 128, 2000
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = random_tree(B, rng)
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0 / np.sqrt(D)
+    ref, _ = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale)
+    nbytes = jet.jet_tree_verify_attn_workspace_bytes(1, B, Hq, Hkv, D, L)
+    assert nbytes > 4096, "this shape is expected to use the workspace exchange"
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device=H.DEV)
+    d = dict(q=H.dev_bf16(x["q"][None]), k=H.dev_bf16(x["k_prefix"][None]), v=H.dev_bf16(x["v_prefix"][None]),
+             tk=H.dev_bf16(x["tree_k"][None]), tv=H.dev_bf16(x["tree_v"][None]), anc=H.dev(anc[None].view(np.int32)),
+             n=H.dev(np.array([B], np.int32)), seq=H.dev(np.array([L], np.int32)))
+    status = torch.zeros(1, dtype=torch.int32, device=H.DEV)
+    for it in range(5):
+        out = torch.full((1, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=H.DEV)
+        jet.jet_tree_verify_attn(d["q"], d["k"], d["v"], None, 0, 0, 0, d["seq"], L, d["tk"], d["tv"], d["anc"], d["n"],
+                                 1, B, Hq, Hkv, D, L * Hkv * D, float(scale), out, None, status, ws)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        err = np.abs(H.bf16_to_f64(out)[0] - ref)
+        assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR, it
+        assert int(ws[:4096].view(torch.int32).abs().sum().item()) == 0, "counters not reset"
+
+
+def test_two_query_tiles_per_cta_variant():
+    """The kernel variant with two query tiles per CTA is not chosen by the planner's current cost model;
+    JET_FORCE_MT=2 selects it (read once per process, hence the child process)."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import sys, os
+sys.path.insert(0, os.getcwd()); sys.path.insert(0, os.path.join(os.getcwd(), "tests"))
+import numpy as np
+import jet_harness as H
+from jet_inputs import make_attn_inputs, random_tree
+from oracle import anc_from_parent, tree_attn_ref
+for B, Hq, Hkv, D, L, n in ((96, 8, 2, 128, 700, 96), (64, 8, 2, 64, 300, 50), (256, 8, 2, 128, 140, 256)):
+    rng = np.random.default_rng(B + L)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = random_tree(n, rng)
+    anc = anc_from_parent(parent, n, B)
+    scale = 1.0 / np.sqrt(D)
+    ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, n, scale)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [L], x["tree_k"][None],
+                                   x["tree_v"][None], anc[None], [n], scale)
+    err = np.abs(out[0] - ref)
+    assert st == 0 and err.max() <= 2e-2 and err.mean() <= 2e-3, (B, st, err.max(), err.mean())
+    assert (out[0][n:] == 0).all() and np.abs(lse[0][:, :n] - rlse[:, :n]).max() <= 1e-3
+print("ok")
+'''
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, JET_FORCE_MT="2")
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0 and "ok" in res.stdout, res.stdout + res.stderr
