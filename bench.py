@@ -34,7 +34,7 @@ UNIT = "us/layer"
 
 # DRAM bytes (read + write) of one tree_attn_kernel launch on the benchmark workload, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"qwen3_8b": None}
+NCU_TRAFFIC_BYTES = {"qwen3_8b": 17634560}     # profiles/tree_attn_kernel_qwen3_8b.md
 
 
 def workload(name):
