@@ -93,12 +93,24 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   for (int d = warp; d < N; d += kExpThreads / 32) {
     const unsigned long long* c = cand + (static_cast<size_t>(b) * N + d) * nchunks * Wc;
     const int total = nchunks * Wc;
+    constexpr int kHeld = 16;                 // candidates a lane can keep in registers
+    unsigned long long held[kHeld];
+    const bool in_regs = total <= 32 * kHeld; // usual case: one pass over global memory, rounds on registers
+    if (in_regs) {
+#pragma unroll
+      for (int i = 0; i < kHeld; ++i) held[i] = lane + 32 * i < total ? c[lane + 32 * i] : 0ull;
+    }
     unsigned long long prev = ~0ull;
     for (int r = 0; r < Wc; ++r) {
       unsigned long long best = 0ull;
-      for (int i = lane; i < total; i += 32) {
-        const unsigned long long k = c[i];
-        if (k < prev && k > best) best = k;
+      if (in_regs) {
+#pragma unroll
+        for (int i = 0; i < kHeld; ++i) if (held[i] < prev && held[i] > best) best = held[i];
+      } else {
+        for (int i = lane; i < total; i += 32) {
+          const unsigned long long k = c[i];
+          if (k < prev && k > best) best = k;
+        }
       }
       best = warp_max_u64(best);
       if (lane == 0) {

@@ -313,6 +313,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       __syncwarp();
       bool ok = true;
       int issued = 0;
+      // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
+      // fetched while the current tile's copies are issued, so the table look-up is off the critical path
+      auto tile_page = [&](int t) -> int {
+        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= L) return 0;
+        return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
+      };
+      int page_cur = tile_page(t_lo), page_next = tile_page(t_lo + 1);
 #pragma unroll 1
       for (; issued < 2 * T; ++issued) {
         const int t = t_lo + (issued >> 1), kv = issued & 1, stage = issued % kStages;
@@ -327,9 +334,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
           __syncwarp();
           if (lane < npages) {
-            const int page = p.page_table[static_cast<size_t>(b) * p.max_pages + t * 8 + lane];
             for (int h = 0; h < kHalves; ++h)
-              ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page * 16);
+              ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page_cur * 16);
+          }
+          if (kv) {                       // both tiles of this key range are on their way: move on
+            page_cur = page_next;
+            page_next = tile_page(t + 2);
           }
         } else if (lane == 0) {
           const bool prefix = t < TP;
