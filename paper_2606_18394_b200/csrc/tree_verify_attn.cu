@@ -112,12 +112,19 @@ struct Bars {       // offsets (in 8-byte units) inside the barrier block
 };
 
 // Every wait is bounded: at most kWaitRounds suspensions of kWaitHintNs each (about a second).
+// Register split (setmaxnreg): warps 0-3 (producer, MMA issuer, helpers) keep kRegsControl registers per
+// thread, the softmax warpgroups get kRegsSoftmax; 128 * kRegsControl + 256 * kRegsSoftmax must not exceed
+// the 384 * 168 registers the CTA is launched with.
+constexpr int kRegsControl = 104;
+constexpr int kRegsSoftmax = 200;
+static_assert(128 * kRegsControl + 256 * kRegsSoftmax <= 384 * 168, "register split exceeds the CTA's allocation");
+
 constexpr uint32_t kWaitRounds = 1u << 16;
 constexpr uint32_t kWaitHintNs = 16384;
 
 // Called by all 32 lanes of a warp; the result is warp-uniform.
 // `site` identifies the wait in the abort flag (1 + site of the first wait that gave up).
-__device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+__device__ __forceinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                               uint32_t site) {
   bool ok = false;
   for (uint32_t i = 0; i < kWaitRounds; ++i) {
@@ -137,7 +144,7 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, vola
 
 // The same for a barrier that other CTAs of the cluster arrive on / copy into (acquire at cluster
 // scope); called by every thread of the CTA, the result is CTA-uniform.
-__device__ __noinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint32_t* abort_flag, uint32_t site) {
+__device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint32_t* abort_flag, uint32_t site) {
   bool ok = false;
   for (uint32_t i = 0; i < kWaitRounds; ++i) {
     if (ptx::mbar_try_wait_cluster(bar, 0, kWaitHintNs)) { ok = true; break; }
@@ -150,7 +157,7 @@ __device__ __noinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint32_
 // Cluster-wide rendezvous built from one mbarrier per CTA (count = cluster size): after a CTA-wide
 // barrier one thread arrives on the barrier of every CTA of the cluster, then everybody waits for
 // all `nsplit` arrivals on the local one.
-__device__ __noinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag,
+__device__ __forceinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag,
                                                 uint32_t site) {
   __syncthreads();
   if (threadIdx.x == 0)
@@ -300,154 +307,409 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   float l = 0.0f;               // running sum of exp2((s - m_used) * sl2)
   bool row_ok = has_work;       // false once a bounded wait of this warp expired
 
-  if (has_work) {
-    if (warp == 0) {
-      // =========================================================== TMA producer
-      if (lane == 0) {
-        ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
-        for (int mt = 0; mt < n_mt; ++mt)
-          for (int h = 0; h < kHalves; ++h)
-            ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
-                             b * p.B + node_lo + mt * npt);
-      }
+  // The epilogue is written once and instantiated for both register classes: `sm_side` is true for the
+  // softmax warpgroups (which hold the rows, stage and combine them) and false for warps 0-3 (which take
+  // part in every CTA-wide barrier and issue the bulk copies and the counter updates).
+  auto epilogue = [&](auto sm_side) {
+    constexpr bool kSm = decltype(sm_side)::value;
+    // =============================================================== epilogue
+    // One round per query tile: its softmax threads stage their normalised rows (D fp32 + log2-sum-exp)
+    // in shared memory.  With key slices every CTA then sends each owner slice its block of rows with
+    // one bulk copy credited to the owner's kRecv barrier; the owner combines the S blocks.  Without
+    // slices the CTA "combines" its own staged rows.  Either way the output rows leave as coalesced
+    // 16-byte stores, rows of padding nodes as zeros.
+    const int e_wg = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
+    const int e_r = (tid - 128) & 127;                           // its row within the query tile
+    uint8_t* stage = smem_gen + C::kStageOff;
+    bool merge_ok = true;
+    if (via_cluster) {
       __syncwarp();
-      bool ok = true;
-      int issued = 0;
-      // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
-      // fetched while the current tile's copies are issued, so the table look-up is off the critical path
-      auto tile_page = [&](int t) -> int {
-        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= L) return 0;
-        return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
-      };
-      int page_cur = tile_page(t_lo), page_next = tile_page(t_lo + 1);
+      ptx::cluster_wait();     // pairs with cluster_arrive above: every CTA's barriers are initialised
+      // A: every CTA of the cluster has left its key loop, so its tile memory may be overwritten
+      merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag, 12);
+      if (tid == 128) JET_TR(7);
+    } else {
+      __syncthreads();
+    }
+    // Staging of a row: normalised, D fp32 values followed by the row's log2-sum-exp.  Rows this CTA
+    // computed nothing for (empty key slice, tile without nodes) get log2-sum-exp = -inf ("absent").
+    const uint32_t e_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const bool active = has_work && row_ok;                      // warp-uniform: TMEM loads need whole warps
+    const float own_inv = (active && l > 0.0f) ? 1.0f / l : 0.0f;
+    const float own_lse2 = (active && l > 0.0f) ? m_used * p.scale_log2 + log2f(l) : -INFINITY;
+    // MT == 1: the two streams of a row exchange (log2-sum-exp, 1/sum) through a scratch corner of the
+    // idle tile memory; afterwards both threads of a row know both weights.
+    float2* xchg = reinterpret_cast<float2*>(smem_gen + C::kTileBytes - 2048);     // [stream][row]
+    if constexpr (kSm && MT == 1) xchg[e_wg * 128 + e_r] = make_float2(own_lse2, own_inv);
 #pragma unroll 1
-      for (; issued < 2 * T; ++issued) {
-        const int t = t_lo + (issued >> 1), kv = issued & 1, stage = issued % kStages;
-        if (issued >= kStages) {
-          ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
-          if (!ok) break;
+    for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
+      if (mt > 0) {
+        // C: everybody has combined the previous tile's rows, so both buffers are free again
+        if (via_cluster) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
+        else __syncthreads();
+      }
+      if constexpr (MT == 1) {
+        // Both warpgroups stage half of every row (64 columns each), folding the two streams' accumulators
+        // together on the way: out = wa * O_0 / l_0 + wb * O_1 / l_1 with softmax weights of the two sums.
+        __syncthreads();
+        if constexpr (kSm) {
+          const float2 s0 = xchg[e_r], s1 = xchg[128 + e_r];
+          const float mxl = fmaxf(s0.x, s1.x);
+          float a0 = 0.0f, a1 = 0.0f, lse2 = -INFINITY;
+          if (mxl > -INFINITY) {
+            const float w0 = s0.x > -INFINITY ? exp2f(s0.x - mxl) : 0.0f;
+            const float w1 = s1.x > -INFINITY ? exp2f(s1.x - mxl) : 0.0f;
+            const float inv = 1.0f / (w0 + w1);
+            a0 = w0 * inv * s0.y;
+            a1 = w1 * inv * s1.y;
+            lse2 = mxl + log2f(w0 + w1);
+          }
+          constexpr int kCols = D / 2;
+          uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 4;
+#pragma unroll 1
+          for (int c = 0; c < kCols / 32; ++c) {
+            uint32_t o0[32], o1[32];
+            if (active) {
+              ptx::tmem_ld32(e_lane + C::o_col(0, 0) + e_wg * kCols + c * 32, o0);
+              ptx::tmem_ld32(e_lane + C::o_col(0, 1) + e_wg * kCols + c * 32, o1);
+              ptx::tmem_wait_ld();
+            }
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (active) {
+                // an accumulator that never received a product holds junk: its weight is exactly 0
+                x.x = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4]) : 0.0f);
+                x.y = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 1]) : 0.0f);
+                x.z = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 2]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 2]) : 0.0f);
+                x.w = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 3]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 3]) : 0.0f);
+              }
+              *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
+            }
+          }
+          if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 4) = lse2;
         }
-        const uint32_t dst = sKV + stage * C::kStageBytes;
-        const uint32_t full = bar(Bars::kKvFull + stage);
-        if (t < TP && p.paged) {
-          const int npages = min(8, (L - t * kBN + 15) / 16);
-          if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
-          __syncwarp();
-          if (lane < npages) {
+      } else if (kSm && e_wg == mt) {
+        uint8_t* dst = stage + e_r * C::kRecvPitch;
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          if (active) {
+            ptx::tmem_ld32(e_lane + C::o_col(mt, 0) + c * 32, o);
+            ptx::tmem_wait_ld();
+          }
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (active)
+              x = make_float4(__uint_as_float(o[q4 * 4]) * own_inv, __uint_as_float(o[q4 * 4 + 1]) * own_inv,
+                              __uint_as_float(o[q4 * 4 + 2]) * own_inv, __uint_as_float(o[q4 * 4 + 3]) * own_inv);
+            *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
+          }
+        }
+        *reinterpret_cast<float*>(dst + D * 4) = own_lse2;
+      }
+      if (via_cluster) ptx::fence_proxy_async_smem();
+      __syncthreads();
+      const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
+      bool rows_ok = merge_ok;
+      if (via_cluster) {
+        if (!kSm && tid < S && merge_ok) {
+          const int dst_lo = tid * rows_per;
+          const int dst_n = max(0, min(rows_per, kBM - dst_lo));
+          if (dst_n > 0)
+            ptx::bulk_copy_to_cluster(
+                ptx::map_to_rank(smem_base + C::kRecvOff + static_cast<uint32_t>(split * rows_per * C::kRecvPitch), tid),
+                smem_base + C::kStageOff + static_cast<uint32_t>(dst_lo * C::kRecvPitch),
+                static_cast<uint32_t>(dst_n * C::kRecvPitch), ptx::map_to_rank(bar(Bars::kRecv + mt), tid));
+        }
+        if (tid == 128 && mt == 0) JET_TR(8);
+        // all blocks of this CTA's rows have arrived (always waited for, so that the CTA never exits
+        // while copies into its memory are in flight)
+        rows_ok = bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14) && merge_ok;
+        if (tid == 128 && mt == 0) JET_TR(9);
+        src_rows = smem_gen + C::kRecvOff;
+        // This CTA's own bulk copies read its staged rows asynchronously: it may only exit once every
+        // peer has received them.  Arrive on the hardware cluster barrier now, wait for it at the end.
+        if (mt == n_mt - 1) ptx::cluster_arrive();
+      } else if (S > 1) {
+        // Exchange through the workspace: publish this CTA's staged rows, count the slices of the unit
+        // that have published (bounded spin), then fetch this CTA's block of rows from every slice.
+        constexpr uint32_t kBlockBytes = kBM * C::kRecvPitch;
+        int* arrive = p.counters + unit * MT + mt;
+        int* depart = p.counters + p.n_units * MT + unit * MT + mt;
+        uint8_t* slots = p.partials + (static_cast<size_t>(unit) * S * MT) * kBlockBytes;
+        if (!kSm && tid < S) {
+          // S threads publish one row block each (the block of owner `tid`), so the copies run in parallel
+          const int blk_lo = tid * rows_per;
+          const int blk_n = max(0, min(rows_per, kBM - blk_lo));
+          if (blk_n > 0) {
+            ptx::bulk_store_global(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes + blk_lo * C::kRecvPitch,
+                                   smem_base + C::kStageOff + static_cast<uint32_t>(blk_lo * C::kRecvPitch),
+                                   static_cast<uint32_t>(blk_n * C::kRecvPitch));
+            ptx::bulk_commit_and_wait_all();
+          }
+          ptx::fence_proxy_async_all();
+          __threadfence();
+        }
+        __syncthreads();
+        if (!kSm && tid == 0) {
+          ptx::atom_add_release_gpu(arrive, 1);
+          bool seen = false;
+          for (uint32_t i = 0; i < (1u << 22); ++i) {
+            if (ptx::ld_acquire_gpu(arrive) >= S) { seen = true; break; }
+            __nanosleep(32);
+            if (*abort_flag) break;
+          }
+          if (!seen && *abort_flag == 0u) *abort_flag = 1u + 16u;
+          ptx::fence_proxy_async_all();
+        }
+        if (tid == 128 && mt == 0) JET_TR(8);
+        const bool published = __syncthreads_and(*abort_flag == 0u ? 1 : 0) != 0;
+        if (!kSm && tid < S && published && own_n > 0)
+          ptx::bulk_load_global(smem_base + C::kRecvOff + static_cast<uint32_t>(tid * rows_per * C::kRecvPitch),
+                                slots + (static_cast<size_t>(tid) * MT + mt) * kBlockBytes + own_lo * C::kRecvPitch,
+                                static_cast<uint32_t>(own_n * C::kRecvPitch), bar(Bars::kRecv + mt));
+        rows_ok = published && (own_n == 0 || bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14));
+        if (own_n == 0) __syncthreads();
+        if (tid == 128 && mt == 0) JET_TR(9);
+        src_rows = smem_gen + C::kRecvOff;
+        // the last slice to have fetched its rows leaves the counters at zero for the next call
+        if (!kSm && tid == 0 && ptx::atom_add_release_gpu(depart, 1) == S - 1) {
+          *arrive = 0;
+          *depart = 0;
+          __threadfence();
+        }
+      }
+      const uint32_t src_stride = rows_per * C::kRecvPitch;     // distance between the blocks of consecutive slices
+      // the softmax warpgroups combine the blocks: one item = 8 output values of one row
+      const int items = rows_ok ? own_n * (D / 8) : 0;
+#pragma unroll 1
+      for (int i = kSm ? tid - 128 : items; i < items; i += C::kThreads - 128) {
+        const int rl = i / (D / 8), c8 = i - rl * (D / 8);
+        const int R = mt * kBM + own_lo + rl;                  // row within the unit
+        const int v = node_lo + R / G, h = g * G + R % G;
+        if (v >= p.B) continue;
+        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        float lse2 = -INFINITY;
+        if (v < n) {
+          const uint8_t* row0 = src_rows + rl * C::kRecvPitch;
+          // weights first (all loads independent) ...
+          float ls[kMaxSplit];
+          float mx = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < kMaxSplit; ++c) {
+            ls[c] = c < S ? *reinterpret_cast<const float*>(row0 + c * src_stride + D * 4) : -INFINITY;
+            mx = fmaxf(mx, ls[c]);
+          }
+          float wsum = 0.0f;
+          if (mx > -INFINITY) {
+#pragma unroll
+            for (int c = 0; c < kMaxSplit; ++c) {
+              ls[c] = ls[c] > -INFINITY ? exp2f(ls[c] - mx) : 0.0f;        // absent slices get weight 0
+              wsum += ls[c];
+            }
+            // ... then the rows, four slices at a time; a slice with weight 0 is not read (it may hold junk)
+#pragma unroll
+            for (int c0 = 0; c0 < kMaxSplit; c0 += 4) {
+              if (c0 < S) {
+                float4 x0[4], x1[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const uint8_t* src = row0 + (c0 + k) * src_stride;
+                  const bool use = ls[c0 + k] > 0.0f;
+                  x0[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32) : make_float4(0.f, 0.f, 0.f, 0.f);
+                  x1[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32 + 16) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const float w = ls[c0 + k];
+                  acc[0] += w * x0[k].x; acc[1] += w * x0[k].y; acc[2] += w * x0[k].z; acc[3] += w * x0[k].w;
+                  acc[4] += w * x1[k].x; acc[5] += w * x1[k].y; acc[6] += w * x1[k].z; acc[7] += w * x1[k].w;
+                }
+              }
+            }
+            const float inv = 1.0f / wsum;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc[k] *= inv;
+            lse2 = mx + log2f(wsum);
+          }
+        }
+        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+            make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                       pack_bf16(acc[6], acc[7]));
+        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
+      }
+    }
+
+  };
+
+  if (warp < 4) {
+    // Warps 0-3 need few registers; what they give up goes to the softmax warpgroups, which hold a whole
+    // score row (128 values) per thread.
+    ptx::setmaxnreg_dec<kRegsControl>();
+    if (has_work) {
+      if (warp == 0) {
+        // =========================================================== TMA producer
+        if (lane == 0) {
+          ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
+          for (int mt = 0; mt < n_mt; ++mt)
             for (int h = 0; h < kHalves; ++h)
-              ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page_cur * 16);
-          }
-          if (kv) {                       // both tiles of this key range are on their way: move on
-            page_cur = page_next;
-            page_next = tile_page(t + 2);
-          }
-        } else if (lane == 0) {
-          const bool prefix = t < TP;
-          const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
-          const int row0 = prefix ? t * kBN : (t - TP) * kBN;
-          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-          for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
+              ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
+                               b * p.B + node_lo + mt * npt);
         }
         __syncwarp();
-        if (lane == 0 && issued == 0) JET_TR(14);
-      }
-      if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
-        // drain: every load that was issued must land before the CTA may exit
-        for (int s = 0; s < kStages; ++s) {
-          if (issued > s) {
-            const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
-            bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
-          }
-        }
-        bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
-      }
-    } else if (warp == 1) {
-      // =========================================================== tcgen05 issuer
-      constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
-      constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
-      bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
-      if (lane == 0) JET_TR(2);
-      // Order of issue: with two score buffers (MT == 1) the Q K^T of tile tl+1 goes out before the P V of
-      // tile tl (it belongs to the other stream and only waits for that stream's previous product).  With one
-      // buffer per query tile (MT == 2) the Q K^T of tile tl+1 overwrites the P of tile tl, so the P V
-      // products of tile tl are issued first.
-      auto issue_qk = [&](int tl) {            // tl = tile before the one whose scores are computed
-        if (tl + 1 < T) {
-          // ---- S = Q K^T of tile tl+1, as soon as its K tile has landed and the score buffer is free
-          const int item = 2 * (tl + 1), stage = item % kStages;
-          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
-          if (lane == 0 && tl == -1) JET_TR(3);
-          for (int mt = 0; mt < n_mt && ok; ++mt) {
-            // The buffer still holds the P of the tile that used it last.  That tile's P V product was issued
-            // earlier by this same thread, and the tensor core executes one thread's MMAs in issue order, so
-            // this Q K^T cannot overwrite the P before it has been read: no wait is needed here.
-            ptx::tc_fence_after();
-            if (lane == 0) {
-              const uint32_t d_tmem = tmem_base + C::s_col(mt, tl + 1);
-#pragma unroll
-              for (int kd = 0; kd < D / 16; ++kd) {
-                const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
-                ptx::umma_ss(d_tmem, ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0),
-                             ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0), idesc_qk, kd > 0 ? 1u : 0u);
-              }
-              ptx::umma_commit(bar(Bars::kSFull + C::s_buf(mt, tl + 1)));
-            }
-            __syncwarp();
-          }
-          if (!ok) return;
-          if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-          __syncwarp();
-        }
-      };
-      auto issue_pv = [&](int tl) {
-        if (tl >= 0) {
-          // ---- O += P V of tile tl
-          const int item = 2 * tl + 1, stage = item % kStages;
-          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
-          if (!ok) return;
-          const int t = t_lo + tl;
-          const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
-          if (valid < kBN) {
-            // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
-            uint8_t* vt = gen_kv + stage * C::kStageBytes;
-            const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
-            for (int h = 0; h < kHalves; ++h)
-              for (int i = lane; i < chunks; i += 32)
-                *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-          }
-          for (int mt = 0; mt < n_mt && ok; ++mt) {
-            ok = bounded_wait(bar(Bars::kPFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 8);
-            if (!ok) return;
-            ptx::tc_fence_after();
-            if (lane == 0) {
-              const uint32_t d_tmem = tmem_base + C::o_col(mt, tl);
-#pragma unroll
-              for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
-                ptx::umma_ts(d_tmem, tmem_base + C::s_col(mt, tl) + kk * 8,
-                             ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
-                             (tl < C::kStreams && kk == 0) ? 0u : 1u);      // first product of each accumulator
-              ptx::umma_commit(bar(Bars::kODone + C::s_buf(mt, tl)));
-            }
-            __syncwarp();
-          }
-          if (!ok) return;
-          if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-          __syncwarp();
-        }
-      };
+        bool ok = true;
+        int issued = 0;
+        // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
+        // fetched while the current tile's copies are issued, so the table look-up is off the critical path
+        auto tile_page = [&](int t) -> int {
+          if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= L) return 0;
+          return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
+        };
+        int page_cur = tile_page(t_lo), page_next = tile_page(t_lo + 1);
 #pragma unroll 1
-      for (int tl = -1; tl < T && ok; ++tl) {
-        if (C::kSBufs == 2) {
-          issue_qk(tl);
-          if (ok) issue_pv(tl);
-        } else {
-          issue_pv(tl);
-          if (ok) issue_qk(tl);
+        for (; issued < 2 * T; ++issued) {
+          const int t = t_lo + (issued >> 1), kv = issued & 1, stage = issued % kStages;
+          if (issued >= kStages) {
+            ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
+            if (!ok) break;
+          }
+          const uint32_t dst = sKV + stage * C::kStageBytes;
+          const uint32_t full = bar(Bars::kKvFull + stage);
+          if (t < TP && p.paged) {
+            const int npages = min(8, (L - t * kBN + 15) / 16);
+            if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
+            __syncwarp();
+            if (lane < npages) {
+              for (int h = 0; h < kHalves; ++h)
+                ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page_cur * 16);
+            }
+            if (kv) {                       // both tiles of this key range are on their way: move on
+              page_cur = page_next;
+              page_next = tile_page(t + 2);
+            }
+          } else if (lane == 0) {
+            const bool prefix = t < TP;
+            const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
+            const int row0 = prefix ? t * kBN : (t - TP) * kBN;
+            ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+            for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
+          }
+          __syncwarp();
+          if (lane == 0 && issued == 0) JET_TR(14);
+        }
+        if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
+          // drain: every load that was issued must land before the CTA may exit
+          for (int s = 0; s < kStages; ++s) {
+            if (issued > s) {
+              const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
+              bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
+            }
+          }
+          bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
+        }
+      } else if (warp == 1) {
+        // =========================================================== tcgen05 issuer
+        constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
+        constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
+        bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
+        if (lane == 0) JET_TR(2);
+        // Order of issue: with two score buffers (MT == 1) the Q K^T of tile tl+1 goes out before the P V of
+        // tile tl (it belongs to the other stream and only waits for that stream's previous product).  With one
+        // buffer per query tile (MT == 2) the Q K^T of tile tl+1 overwrites the P of tile tl, so each query
+        // tile's P V of tile tl is issued first and its Q K^T of tile tl+1 right behind it; the two query tiles
+        // alternate, so that one tile's softmax runs while the tensor core works for the other.
+        auto issue_qk = [&](int tl, int mt_lo, int mt_hi) {   // tl = tile before the one whose scores are computed
+          if (tl + 1 < T) {
+            // ---- S = Q K^T of tile tl+1, as soon as its K tile has landed and the score buffer is free
+            const int item = 2 * (tl + 1), stage = item % kStages;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
+            if (lane == 0 && tl == -1) JET_TR(3);
+            for (int mt = mt_lo; mt < mt_hi && ok; ++mt) {
+              // The buffer still holds the P of the tile that used it last.  That tile's P V product was issued
+              // earlier by this same thread, and the tensor core executes one thread's MMAs in issue order, so
+              // this Q K^T cannot overwrite the P before it has been read: no wait is needed here.
+              ptx::tc_fence_after();
+              if (lane == 0) {
+                const uint32_t d_tmem = tmem_base + C::s_col(mt, tl + 1);
+#pragma unroll
+                for (int kd = 0; kd < D / 16; ++kd) {
+                  const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
+                  ptx::umma_ss(d_tmem, ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0),
+                               ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0), idesc_qk, kd > 0 ? 1u : 0u);
+                }
+                ptx::umma_commit(bar(Bars::kSFull + C::s_buf(mt, tl + 1)));
+                if (mt == 0 && tl >= 0 && tl < 8) JET_TR(48 + tl);
+              }
+              __syncwarp();
+            }
+            if (!ok) return;
+            if (mt_hi == n_mt) {                 // the last query tile has read this K tile
+              if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+              __syncwarp();
+            }
+          }
+        };
+        auto issue_pv = [&](int tl, int mt_lo, int mt_hi) {
+          if (tl >= 0) {
+            // ---- O += P V of tile tl
+            const int item = 2 * tl + 1, stage = item % kStages;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
+            if (!ok) return;
+            const int t = t_lo + tl;
+            const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
+            if (valid < kBN && mt_lo == 0) {
+              // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
+              uint8_t* vt = gen_kv + stage * C::kStageBytes;
+              const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
+              for (int h = 0; h < kHalves; ++h)
+                for (int i = lane; i < chunks; i += 32)
+                  *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+              ptx::fence_proxy_async_smem();
+              __syncwarp();
+            }
+            for (int mt = mt_lo; mt < mt_hi && ok; ++mt) {
+              ok = bounded_wait(bar(Bars::kPFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 8);
+              if (!ok) return;
+              ptx::tc_fence_after();
+              if (lane == 0 && mt == 0 && tl < 8) JET_TR(40 + tl);
+              if (lane == 0) {
+                const uint32_t d_tmem = tmem_base + C::o_col(mt, tl);
+#pragma unroll
+                for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
+                  ptx::umma_ts(d_tmem, tmem_base + C::s_col(mt, tl) + kk * 8,
+                               ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
+                               (tl < C::kStreams && kk == 0) ? 0u : 1u);      // first product of each accumulator
+                ptx::umma_commit(bar(Bars::kODone + C::s_buf(mt, tl)));
+              }
+              __syncwarp();
+            }
+            if (!ok) return;
+            if (mt_hi == n_mt) {                 // the last query tile has read this V tile
+              if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+              __syncwarp();
+            }
+          }
+        };
+#pragma unroll 1
+        for (int tl = -1; tl < T && ok; ++tl) {
+          if (C::kSBufs == 2) {
+            issue_qk(tl, 0, n_mt);
+            if (ok) issue_pv(tl, 0, n_mt);
+          } else {
+            for (int mt = 0; mt < n_mt && ok; ++mt) {
+              issue_pv(tl, mt, mt + 1);
+              if (ok) issue_qk(tl, mt, mt + 1);
+            }
+          }
         }
       }
-    } else if (warp >= 4 && (MT == 1 || ((warp - 4) >> 2) < n_mt)) {
+    }
+    epilogue(std::false_type{});
+  } else {
+    ptx::setmaxnreg_inc<kRegsSoftmax>();
+    if (has_work && (MT == 1 || ((warp - 4) >> 2) < n_mt)) {
       // =========================================================== softmax warpgroups
       constexpr int kChunks = kBN / 32;                       // 32-key chunks per row and tile
       constexpr int kStreams = C::kStreams;
@@ -483,23 +745,25 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (!ok) break;
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
-        if (tid == 128 && tl < 8) JET_TR(19 + tl);
+        if (tid == 128 && tl / kStreams < 4) JET_TR(19 + 2 * (tl / kStreams));
+        if (tid == 256 && tl / kStreams < 4) JET_TR(32 + 2 * (tl / kStreams));
 
-        // ---- pass 1: row maximum over the visible keys (scores are read from TMEM in 32-column chunks,
-        //      the next chunk is in flight while the current one is reduced)
+        // ---- row maximum over the visible keys.  A full tile is read from TMEM once: the thread keeps its
+        //      whole score row (128 values) in registers for both the maximum and the exponentials.  A tile
+        //      with masked keys (ragged end of the prefix, tree keys) takes two passes over TMEM, chunk by chunk.
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        uint32_t xa[32], xb[32];
+        static_assert(kChunks == 4, "the register-resident row is written out for four 32-key chunks");
+        uint32_t xa[32], xb[32], xc[32], xd[32];
         if (full_tile) {
           ptx::tmem_ld32(tS, xa);
-#pragma unroll 1
-          for (int c = 0; c < kChunks; c += 2) {
-            ptx::tmem_wait_ld();
-            ptx::tmem_ld32(tS + (c + 1) * 32, xb);
-            max_chunk(xa, mx);
-            ptx::tmem_wait_ld();
-            if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
-            max_chunk(xb, mx);
-          }
+          ptx::tmem_ld32(tS + 32, xb);
+          ptx::tmem_ld32(tS + 64, xc);
+          ptx::tmem_ld32(tS + 96, xd);
+          ptx::tmem_wait_ld();
+          max_chunk(xa, mx);
+          max_chunk(xb, mx);
+          max_chunk(xc, mx);
+          max_chunk(xd, mx);
         } else {
 #pragma unroll 1
           for (int c = 0; c < kChunks; ++c) {
@@ -532,16 +796,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // ---- pass 2: probabilities, row sum; P (packed bf16) overwrites the first 64 columns of the scores
         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         if (full_tile) {
-          ptx::tmem_ld32(tS, xa);
-#pragma unroll 1
-          for (int c = 0; c < kChunks; c += 2) {
-            ptx::tmem_wait_ld();
-            ptx::tmem_ld32(tS + (c + 1) * 32, xb);
-            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS + c * 16);
-            ptx::tmem_wait_ld();
-            if (c + 2 < kChunks) ptx::tmem_ld32(tS + (c + 2) * 32, xa);
-            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + (c + 1) * 16);
-          }
+          exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
+          exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
+          exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
+          exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
         } else {
 #pragma unroll 1
           for (int c = 0; c < kChunks; ++c) {
@@ -567,7 +825,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         ptx::tc_fence_before();
         ptx::mbar_arrive(bar(Bars::kPFull + C::s_buf(mt, tl)));
         if (tid == 128 && tl < 1) JET_TR(6);
-        if (tid == 128 && tl < 8) JET_TR(20 + tl);
+        if (tid == 128 && tl / kStreams < 4) JET_TR(20 + 2 * (tl / kStreams));
+        if (tid == 256 && tl / kStreams < 4) JET_TR(33 + 2 * (tl / kStreams));
         last_tl = tl;
       }
       if (tid == 128) JET_TR(10);
@@ -576,237 +835,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         ok = bounded_wait(bar(Bars::kODone + C::s_buf(mt, last_tl)), C::s_use(last_tl) & 1, abort_flag, 11);
       if (ok) ptx::tc_fence_after();
       row_ok = ok;
-      if (tid == 128) JET_TR(11);
     }
-  }
-
-  // =============================================================== epilogue
-  // One round per query tile: its softmax threads stage their normalised rows (D fp32 + log2-sum-exp)
-  // in shared memory.  With key slices every CTA then sends each owner slice its block of rows with
-  // one bulk copy credited to the owner's kRecv barrier; the owner combines the S blocks.  Without
-  // slices the CTA "combines" its own staged rows.  Either way the output rows leave as coalesced
-  // 16-byte stores, rows of padding nodes as zeros.
-  const int e_wg = warp >= 4 ? (warp - 4) >> 2 : 0;            // softmax warpgroup of this thread
-  const int e_r = (tid - 128) & 127;                           // its row within the query tile
-  uint8_t* stage = smem_gen + C::kStageOff;
-  bool merge_ok = true;
-  if (via_cluster) {
-    __syncwarp();
-    ptx::cluster_wait();     // pairs with cluster_arrive above: every CTA's barriers are initialised
-    // A: every CTA of the cluster has left its key loop, so its tile memory may be overwritten
-    merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag, 12);
-    if (tid == 128) JET_TR(7);
-  } else {
-    __syncthreads();
-  }
-  // Staging of a row: normalised, D fp32 values followed by the row's log2-sum-exp.  Rows this CTA
-  // computed nothing for (empty key slice, tile without nodes) get log2-sum-exp = -inf ("absent").
-  const uint32_t e_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-  const bool active = has_work && row_ok;                      // warp-uniform: TMEM loads need whole warps
-  const float own_inv = (active && l > 0.0f) ? 1.0f / l : 0.0f;
-  const float own_lse2 = (active && l > 0.0f) ? m_used * p.scale_log2 + log2f(l) : -INFINITY;
-  // MT == 1: the two streams of a row exchange (log2-sum-exp, 1/sum) through a scratch corner of the
-  // idle tile memory; afterwards both threads of a row know both weights.
-  float2* xchg = reinterpret_cast<float2*>(smem_gen + C::kTileBytes - 2048);     // [stream][row]
-  if (MT == 1 && warp >= 4) xchg[e_wg * 128 + e_r] = make_float2(own_lse2, own_inv);
-#pragma unroll 1
-  for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
-    if (mt > 0) {
-      // C: everybody has combined the previous tile's rows, so both buffers are free again
-      if (via_cluster) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
-      else __syncthreads();
-    }
-    if constexpr (MT == 1) {
-      // Both warpgroups stage half of every row (64 columns each), folding the two streams' accumulators
-      // together on the way: out = wa * O_0 / l_0 + wb * O_1 / l_1 with softmax weights of the two sums.
-      __syncthreads();
-      if (warp >= 4) {
-        const float2 s0 = xchg[e_r], s1 = xchg[128 + e_r];
-        const float mxl = fmaxf(s0.x, s1.x);
-        float a0 = 0.0f, a1 = 0.0f, lse2 = -INFINITY;
-        if (mxl > -INFINITY) {
-          const float w0 = s0.x > -INFINITY ? exp2f(s0.x - mxl) : 0.0f;
-          const float w1 = s1.x > -INFINITY ? exp2f(s1.x - mxl) : 0.0f;
-          const float inv = 1.0f / (w0 + w1);
-          a0 = w0 * inv * s0.y;
-          a1 = w1 * inv * s1.y;
-          lse2 = mxl + log2f(w0 + w1);
-        }
-        constexpr int kCols = D / 2;
-        uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 4;
-#pragma unroll 1
-        for (int c = 0; c < kCols / 32; ++c) {
-          uint32_t o0[32], o1[32];
-          if (active) {
-            ptx::tmem_ld32(e_lane + C::o_col(0, 0) + e_wg * kCols + c * 32, o0);
-            ptx::tmem_ld32(e_lane + C::o_col(0, 1) + e_wg * kCols + c * 32, o1);
-            ptx::tmem_wait_ld();
-          }
-#pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (active) {
-              // an accumulator that never received a product holds junk: its weight is exactly 0
-              x.x = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4]) : 0.0f);
-              x.y = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 1]) : 0.0f);
-              x.z = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 2]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 2]) : 0.0f);
-              x.w = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 3]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 3]) : 0.0f);
-            }
-            *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
-          }
-        }
-        if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 4) = lse2;
-      }
-    } else if (warp >= 4 && e_wg == mt) {
-      uint8_t* dst = stage + e_r * C::kRecvPitch;
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        if (active) {
-          ptx::tmem_ld32(e_lane + C::o_col(mt, 0) + c * 32, o);
-          ptx::tmem_wait_ld();
-        }
-#pragma unroll
-        for (int q4 = 0; q4 < 8; ++q4) {
-          float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (active)
-            x = make_float4(__uint_as_float(o[q4 * 4]) * own_inv, __uint_as_float(o[q4 * 4 + 1]) * own_inv,
-                            __uint_as_float(o[q4 * 4 + 2]) * own_inv, __uint_as_float(o[q4 * 4 + 3]) * own_inv);
-          *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
-        }
-      }
-      *reinterpret_cast<float*>(dst + D * 4) = own_lse2;
-    }
-    if (via_cluster) ptx::fence_proxy_async_smem();
-    __syncthreads();
-    const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
-    bool rows_ok = merge_ok;
-    if (via_cluster) {
-      if (tid < S && merge_ok) {
-        const int dst_lo = tid * rows_per;
-        const int dst_n = max(0, min(rows_per, kBM - dst_lo));
-        if (dst_n > 0)
-          ptx::bulk_copy_to_cluster(
-              ptx::map_to_rank(smem_base + C::kRecvOff + static_cast<uint32_t>(split * rows_per * C::kRecvPitch), tid),
-              smem_base + C::kStageOff + static_cast<uint32_t>(dst_lo * C::kRecvPitch),
-              static_cast<uint32_t>(dst_n * C::kRecvPitch), ptx::map_to_rank(bar(Bars::kRecv + mt), tid));
-      }
-      if (tid == 128 && mt == 0) JET_TR(8);
-      // all blocks of this CTA's rows have arrived (always waited for, so that the CTA never exits
-      // while copies into its memory are in flight)
-      rows_ok = bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14) && merge_ok;
-      if (tid == 128 && mt == 0) JET_TR(9);
-      src_rows = smem_gen + C::kRecvOff;
-      // This CTA's own bulk copies read its staged rows asynchronously: it may only exit once every
-      // peer has received them.  Arrive on the hardware cluster barrier now, wait for it at the end.
-      if (mt == n_mt - 1) ptx::cluster_arrive();
-    } else if (S > 1) {
-      // Exchange through the workspace: publish this CTA's staged rows, count the slices of the unit
-      // that have published (bounded spin), then fetch this CTA's block of rows from every slice.
-      constexpr uint32_t kBlockBytes = kBM * C::kRecvPitch;
-      int* arrive = p.counters + unit * MT + mt;
-      int* depart = p.counters + p.n_units * MT + unit * MT + mt;
-      uint8_t* slots = p.partials + (static_cast<size_t>(unit) * S * MT) * kBlockBytes;
-      if (tid < S) {
-        // S threads publish one row block each (the block of owner `tid`), so the copies run in parallel
-        const int blk_lo = tid * rows_per;
-        const int blk_n = max(0, min(rows_per, kBM - blk_lo));
-        if (blk_n > 0) {
-          ptx::bulk_store_global(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes + blk_lo * C::kRecvPitch,
-                                 smem_base + C::kStageOff + static_cast<uint32_t>(blk_lo * C::kRecvPitch),
-                                 static_cast<uint32_t>(blk_n * C::kRecvPitch));
-          ptx::bulk_commit_and_wait_all();
-        }
-        ptx::fence_proxy_async_all();
-        __threadfence();
-      }
-      __syncthreads();
-      if (tid == 0) {
-        ptx::atom_add_release_gpu(arrive, 1);
-        bool seen = false;
-        for (uint32_t i = 0; i < (1u << 22); ++i) {
-          if (ptx::ld_acquire_gpu(arrive) >= S) { seen = true; break; }
-          __nanosleep(32);
-          if (*abort_flag) break;
-        }
-        if (!seen && *abort_flag == 0u) *abort_flag = 1u + 16u;
-        ptx::fence_proxy_async_all();
-      }
-      if (tid == 128 && mt == 0) JET_TR(8);
-      const bool published = __syncthreads_and(*abort_flag == 0u ? 1 : 0) != 0;
-      if (tid < S && published && own_n > 0)
-        ptx::bulk_load_global(smem_base + C::kRecvOff + static_cast<uint32_t>(tid * rows_per * C::kRecvPitch),
-                              slots + (static_cast<size_t>(tid) * MT + mt) * kBlockBytes + own_lo * C::kRecvPitch,
-                              static_cast<uint32_t>(own_n * C::kRecvPitch), bar(Bars::kRecv + mt));
-      rows_ok = published && (own_n == 0 || bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14));
-      if (own_n == 0) __syncthreads();
-      if (tid == 128 && mt == 0) JET_TR(9);
-      src_rows = smem_gen + C::kRecvOff;
-      // the last slice to have fetched its rows leaves the counters at zero for the next call
-      if (tid == 0 && ptx::atom_add_release_gpu(depart, 1) == S - 1) {
-        *arrive = 0;
-        *depart = 0;
-        __threadfence();
-      }
-    }
-    const uint32_t src_stride = rows_per * C::kRecvPitch;     // distance between the blocks of consecutive slices
-    const int items = rows_ok ? own_n * (D / 8) : 0;
-#pragma unroll 1
-    for (int i = tid; i < items; i += C::kThreads) {
-      const int rl = i / (D / 8), c8 = i - rl * (D / 8);
-      const int R = mt * kBM + own_lo + rl;                  // row within the unit
-      const int v = node_lo + R / G, h = g * G + R % G;
-      if (v >= p.B) continue;
-      float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-      float lse2 = -INFINITY;
-      if (v < n) {
-        const uint8_t* row0 = src_rows + rl * C::kRecvPitch;
-        // weights first (all loads independent) ...
-        float ls[kMaxSplit];
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < kMaxSplit; ++c) {
-          ls[c] = c < S ? *reinterpret_cast<const float*>(row0 + c * src_stride + D * 4) : -INFINITY;
-          mx = fmaxf(mx, ls[c]);
-        }
-        float wsum = 0.0f;
-        if (mx > -INFINITY) {
-#pragma unroll
-          for (int c = 0; c < kMaxSplit; ++c) {
-            ls[c] = ls[c] > -INFINITY ? exp2f(ls[c] - mx) : 0.0f;        // absent slices get weight 0
-            wsum += ls[c];
-          }
-          // ... then the rows, four slices at a time; a slice with weight 0 is not read (it may hold junk)
-#pragma unroll
-          for (int c0 = 0; c0 < kMaxSplit; c0 += 4) {
-            if (c0 < S) {
-              float4 x0[4], x1[4];
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const uint8_t* src = row0 + (c0 + k) * src_stride;
-                const bool use = ls[c0 + k] > 0.0f;
-                x0[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32) : make_float4(0.f, 0.f, 0.f, 0.f);
-                x1[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32 + 16) : make_float4(0.f, 0.f, 0.f, 0.f);
-              }
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float w = ls[c0 + k];
-                acc[0] += w * x0[k].x; acc[1] += w * x0[k].y; acc[2] += w * x0[k].z; acc[3] += w * x0[k].w;
-                acc[4] += w * x1[k].x; acc[5] += w * x1[k].y; acc[6] += w * x1[k].z; acc[7] += w * x1[k].w;
-              }
-            }
-          }
-          const float inv = 1.0f / wsum;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) acc[k] *= inv;
-          lse2 = mx + log2f(wsum);
-        }
-      }
-      *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
-          make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
-                     pack_bf16(acc[6], acc[7]));
-      if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
-    }
+    epilogue(std::true_type{});
   }
 
   // ---------------- teardown
