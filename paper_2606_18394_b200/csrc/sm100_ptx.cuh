@@ -117,6 +117,18 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// True in exactly one lane of a converged warp.  Code under this predicate is still uniform for the
+// compiler (every operand of the tensor-core instructions can stay in uniform registers).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // Register reallocation between the warpgroups of a CTA (all four warps of a warpgroup execute it).
 template <int kRegs>
 __device__ __forceinline__ void setmaxnreg_dec() {

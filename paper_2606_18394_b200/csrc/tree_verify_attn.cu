@@ -89,7 +89,6 @@ struct Cfg {
   //   MT == 1: stream i owns S [i*128, +128) and O [256 + i*128, +D); key tile t belongs to stream t & 1
   //   MT == 2: query tile mt owns S [mt*256, +128) and O [mt*256+128, +D)
   static constexpr int kTmemCols = 512;
-  static constexpr int kSBufs = MT == 1 ? 2 : 1;
   __device__ static constexpr uint32_t s_col(int mt, int t) { return MT == 1 ? (t & 1) * 128 : mt * 256; }
   __device__ static constexpr uint32_t o_col(int mt, int t) { return MT == 1 ? 256 + (t & 1) * 128 : mt * 256 + 128; }
   // Each score buffer (and the P that replaces it) has its own barriers, so that neither side can run two
@@ -233,12 +232,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int own_lo = split * rows_per;
   const int own_n = max(0, min(rows_per, kBM - own_lo));
 
+  // ---------------- work item: what the launch parameters alone decide
+  const int unit = blockIdx.x / S;
+  const int mgroup = unit % p.n_mgroups;
+  const int bg = unit / p.n_mgroups;
+  const int g = bg % p.Hkv;
+  const int b = bg / p.Hkv;
+  const int G = p.G;
+  const int npt = kBM / G;                       // nodes per query tile
+  const int node_lo = mgroup * MT * npt;
+  const int node_hi = min(p.B, node_lo + MT * npt);
+  const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
+
   // ---------------- set-up that touches no global memory (may overlap the previous kernel's tail)
   if (warp == 0 && lane == 0) {
     ptx::mbar_init(bar(Bars::kQFull), 1);
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(bar(Bars::kKvFull + s), 1);
-      ptx::mbar_init(bar(Bars::kKvEmpty + s), 1);
+      ptx::mbar_init(bar(Bars::kKvEmpty + s), MT == 1 ? 1 : n_mt);    // one arrival per stream that reads the stage
     }
     ptx::fence_mbar_init();
   } else if (warp == 1 && lane == 0) {
@@ -279,19 +290,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
   ptx::grid_dep_launch();    // the next kernel may start its own set-up as SMs become free
 
-  // ---------------- work item
-  const int unit = blockIdx.x / S;
-  const int mgroup = unit % p.n_mgroups;
-  const int bg = unit / p.n_mgroups;
-  const int g = bg % p.Hkv;
-  const int b = bg / p.Hkv;
-  const int G = p.G;
-  const int npt = kBM / G;                       // nodes per query tile
+  // ---------------- work item, continued: what depends on device data
   const int L = p.seq_len[b];
   const int n = min(p.n_nodes[b], p.B);
-  const int node_lo = mgroup * MT * npt;
-  const int node_hi = min(p.B, node_lo + MT * npt);
-  const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
   const int ntree = min(n, node_hi);                         // tree keys any row here can see
   const int TP = (L + kBN - 1) / kBN;
   const int TT = (ntree + kBN - 1) / kBN;
@@ -611,98 +612,78 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       } else if (warp == 1) {
         // =========================================================== tcgen05 issuer
+        // A stream is a chain  S = Q K^T -> softmax -> O += P V -> next S  on its own score buffer (which the P
+        // overwrites) and accumulator: with one query tile per CTA the two streams take alternate key tiles,
+        // with two each stream is one query tile and takes every key tile.  The streams take turns: a turn
+        // issues one tile's P V and the stream's next Q K^T, so that one stream's softmax runs under the other
+        // stream's products.  Within a stream the next Q K^T overwrites the P of the tile before; it is issued
+        // after that tile's P V, and one thread's MMAs execute in issue order, so it needs no further wait.
+        // The whole warp runs the loop (uniform control flow and operands); one elected lane issues.  The
+        // tensor core queues only two or three instructions, so every instruction between two MMAs counts:
+        // descriptors are formed by adding precomputed offsets.
         constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
         constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
+        constexpr int kStep = MT == 1 ? 2 : 1;            // distance between a stream's tiles
+        const uint64_t desc_q0 = ptx::smem_desc_sw128(sQ, 0);
+        const uint64_t desc_k0 = ptx::smem_desc_sw128(sKV, 0);
+        const uint64_t desc_v0 = ptx::smem_desc_sw128(sKV, kHalfBytes);
         bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
         if (lane == 0) JET_TR(2);
-        // Order of issue: with two score buffers (MT == 1) the Q K^T of tile tl+1 goes out before the P V of
-        // tile tl (it belongs to the other stream and only waits for that stream's previous product).  With one
-        // buffer per query tile (MT == 2) the Q K^T of tile tl+1 overwrites the P of tile tl, so each query
-        // tile's P V of tile tl is issued first and its Q K^T of tile tl+1 right behind it; the two query tiles
-        // alternate, so that one tile's softmax runs while the tensor core works for the other.
-        auto issue_qk = [&](int tl, int mt_lo, int mt_hi) {   // tl = tile before the one whose scores are computed
-          if (tl + 1 < T) {
-            // ---- S = Q K^T of tile tl+1, as soon as its K tile has landed and the score buffer is free
-            const int item = 2 * (tl + 1), stage = item % kStages;
-            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
-            if (lane == 0 && tl == -1) JET_TR(3);
-            for (int mt = mt_lo; mt < mt_hi && ok; ++mt) {
-              // The buffer still holds the P of the tile that used it last.  That tile's P V product was issued
-              // earlier by this same thread, and the tensor core executes one thread's MMAs in issue order, so
-              // this Q K^T cannot overwrite the P before it has been read: no wait is needed here.
-              ptx::tc_fence_after();
-              if (lane == 0) {
-                const uint32_t d_tmem = tmem_base + C::s_col(mt, tl + 1);
+        auto issue_qk = [&](int stream, int tl) {
+          const int item = 2 * tl, stage = item % kStages;
+          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
+          if (!ok) return;
+          if (tl == 0 && stream == 0 && lane == 0) JET_TR(3);
+          ptx::tc_fence_after();
+          const int mt = MT == 1 ? 0 : stream;
+          const uint64_t desc_q = desc_q0 + static_cast<uint64_t>(mt * ((kHalves * kHalfBytes) >> 4));
+          const uint64_t desc_k = desc_k0 + static_cast<uint64_t>(stage * (C::kStageBytes >> 4));
+          const uint32_t s_tmem = tmem_base + C::s_col(mt, tl);
+          if (ptx::elect_one()) {
 #pragma unroll
-                for (int kd = 0; kd < D / 16; ++kd) {
-                  const uint32_t off = (kd / 4) * kHalfBytes + (kd % 4) * 32;
-                  ptx::umma_ss(d_tmem, ptx::smem_desc_sw128(sQ + mt * kHalves * kHalfBytes + off, 0),
-                               ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + off, 0), idesc_qk, kd > 0 ? 1u : 0u);
-                }
-                ptx::umma_commit(bar(Bars::kSFull + C::s_buf(mt, tl + 1)));
-                if (mt == 0 && tl >= 0 && tl < 8) JET_TR(48 + tl);
-              }
-              __syncwarp();
+            for (int kd = 0; kd < D / 16; ++kd) {
+              const uint64_t off = static_cast<uint64_t>(((kd / 4) * kHalfBytes + (kd % 4) * 32) >> 4);
+              ptx::umma_ss(s_tmem, desc_q + off, desc_k + off, idesc_qk, kd > 0 ? 1u : 0u);
             }
-            if (!ok) return;
-            if (mt_hi == n_mt) {                 // the last query tile has read this K tile
-              if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-              __syncwarp();
-            }
+            ptx::umma_commit(bar(Bars::kSFull + stream));
+            ptx::umma_commit(bar(Bars::kKvEmpty + stage));     // this stream has read the K tile
           }
         };
-        auto issue_pv = [&](int tl, int mt_lo, int mt_hi) {
-          if (tl >= 0) {
-            // ---- O += P V of tile tl
-            const int item = 2 * tl + 1, stage = item % kStages;
-            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
-            if (!ok) return;
-            const int t = t_lo + tl;
-            const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
-            if (valid < kBN && mt_lo == 0) {
-              // Rows of masked keys get P = 0 exactly; their V rows must be finite, so clear them.
-              uint8_t* vt = gen_kv + stage * C::kStageBytes;
-              const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
-              for (int h = 0; h < kHalves; ++h)
-                for (int i = lane; i < chunks; i += 32)
-                  *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-              ptx::fence_proxy_async_smem();
-              __syncwarp();
-            }
-            for (int mt = mt_lo; mt < mt_hi && ok; ++mt) {
-              ok = bounded_wait(bar(Bars::kPFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 8);
-              if (!ok) return;
-              ptx::tc_fence_after();
-              if (lane == 0 && mt == 0 && tl < 8) JET_TR(40 + tl);
-              if (lane == 0) {
-                const uint32_t d_tmem = tmem_base + C::o_col(mt, tl);
+        auto turn = [&](int stream, int tl) {
+          // ---- O += P V of tile tl (rows of masked keys of the V tile were cleared by the softmax threads)
+          const int item = 2 * tl + 1, stage = item % kStages;
+          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
+          if (!ok) return;
+          ok = bounded_wait(bar(Bars::kPFull + stream), C::s_use(tl) & 1, abort_flag, 8);
+          if (!ok) return;
+          ptx::tc_fence_after();
+          if (stream == 0 && tl / kStep < 8 && lane == 0) JET_TR(50 + tl / kStep);
+          const int mt = MT == 1 ? 0 : stream;
+          const uint64_t desc_v = desc_v0 + static_cast<uint64_t>(stage * (C::kStageBytes >> 4));
+          const uint32_t s_tmem = tmem_base + C::s_col(mt, tl);
+          const uint32_t o_tmem = tmem_base + C::o_col(mt, tl);
+          const bool first = tl < kStep;                       // first product of this accumulator
+          if (ptx::elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
-                  ptx::umma_ts(d_tmem, tmem_base + C::s_col(mt, tl) + kk * 8,
-                               ptx::smem_desc_sw128(sKV + stage * C::kStageBytes + kk * 2048, kHalfBytes), idesc_pv,
-                               (tl < C::kStreams && kk == 0) ? 0u : 1u);      // first product of each accumulator
-                ptx::umma_commit(bar(Bars::kODone + C::s_buf(mt, tl)));
-              }
-              __syncwarp();
-            }
-            if (!ok) return;
-            if (mt_hi == n_mt) {                 // the last query tile has read this V tile
-              if (lane == 0) ptx::umma_commit(bar(Bars::kKvEmpty + stage));
-              __syncwarp();
-            }
+            for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
+              ptx::umma_ts(o_tmem, s_tmem + kk * 8, desc_v + static_cast<uint64_t>((kk * 2048) >> 4), idesc_pv,
+                           (first && kk == 0) ? 0u : 1u);
+            ptx::umma_commit(bar(Bars::kODone + stream));
+            ptx::umma_commit(bar(Bars::kKvEmpty + stage));      // this stream has read the V tile
           }
+          // ---- S = Q K^T of the stream's next tile
+          if (tl + kStep < T) issue_qk(stream, tl + kStep);
         };
+        if constexpr (MT == 1) {
+          if (ok) issue_qk(0, 0);
+          if (ok && T > 1) issue_qk(1, 1);
 #pragma unroll 1
-        for (int tl = -1; tl < T && ok; ++tl) {
-          if (C::kSBufs == 2) {
-            issue_qk(tl, 0, n_mt);
-            if (ok) issue_pv(tl, 0, n_mt);
-          } else {
-            for (int mt = 0; mt < n_mt && ok; ++mt) {
-              issue_pv(tl, mt, mt + 1);
-              if (ok) issue_qk(tl, mt, mt + 1);
-            }
-          }
+          for (int tl = 0; tl < T && ok; ++tl) turn(tl & 1, tl);
+        } else {
+          for (int mt = 0; mt < n_mt && ok; ++mt) issue_qk(mt, 0);
+#pragma unroll 1
+          for (int tl = 0; tl < T && ok; ++tl)
+            for (int mt = 0; mt < n_mt && ok; ++mt) turn(mt, tl);
         }
       }
     }
@@ -746,6 +727,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
         if (tid == 128 && tl / kStreams < 4) JET_TR(19 + 2 * (tl / kStreams));
+        if (tid == 128 && tl / kStreams == 3) JET_TR(58);
         if (tid == 256 && tl / kStreams < 4) JET_TR(32 + 2 * (tl / kStreams));
 
         // ---- row maximum over the visible keys.  A full tile is read from TMEM once: the thread keeps its
@@ -774,6 +756,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         if (tid == 128 && tl < 1) JET_TR(5);
+        if (tid == 128 && tl / kStreams == 3) JET_TR(59);
 
         // ---- running maximum with lazy rescaling
         float factor = 1.0f;
@@ -797,8 +780,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         if (full_tile) {
           exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
+          if (tid == 128 && tl / kStreams == 3) JET_TR(61);
           exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
+          if (tid == 128 && tl / kStreams == 3) JET_TR(62);
           exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
+          if (tid == 128 && tl / kStreams == 3) JET_TR(63);
           exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
         } else {
 #pragma unroll 1
@@ -810,6 +796,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
         if (tid == 128 && tl < 1) JET_TR(17);
+        if (tid == 128 && tl / kStreams == 3) JET_TR(60);
 
         if (need_rescale && last_tl >= 0) {
 #pragma unroll 1
@@ -819,6 +806,22 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
             for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
             ptx::tmem_st32(tO + c * 32, xa);
+          }
+        }
+        if (!full_tile) {
+          // Masked keys get P = 0 exactly, but 0 * NaN is NaN: the V rows of keys beyond the valid ones
+          // (stale cache rows, rows of padding nodes) are cleared before the P V product may read them.
+          const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
+          if (valid < kBN) {
+            const int item = 2 * tl + 1, stage = item % kStages;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 10);
+            if (!ok) break;
+            uint8_t* vt = gen_kv + stage * C::kStageBytes;
+            const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
+            for (int h = 0; h < kHalves; ++h)
+              for (int i = r; i < chunks; i += 128)
+                *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+            ptx::fence_proxy_async_smem();
           }
         }
         ptx::tmem_wait_st();                     // P (and a rescaled O) are in TMEM
