@@ -40,6 +40,7 @@ constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
 constexpr int kMaxSplit = 16;          // largest cluster
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more
+constexpr float kFastSumLimit = 256.0f;    // a full tile keeps its reference maximum while its row sums stay below (so P <= 2^8)
 
 struct AttnParams {
   const int32_t* page_table;
@@ -180,12 +181,11 @@ __device__ __forceinline__ void max_chunk_masked(const uint32_t (&x)[32], uint32
 }
 
 // 32 scores of one row -> probabilities (exp2 of the scaled, shifted score; masked keys exactly 0),
-// added to the row sum and written as packed bf16 pairs to 16 TMEM columns of the row's lane (the A
-// operand of the P V product).  The stages are kept apart so that the 32 independent exp2 are in
-// flight together.
+// added to the row sum and packed as bf16 pairs (the A operand of the P V product, 16 TMEM columns of
+// the row's lane).  The stages are kept apart so that the 32 independent exp2 are in flight together.
 template <bool kMasked>
-__device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
-                                          float (&sum)[4], uint32_t p_tmem) {
+__device__ __forceinline__ void exp_chunk_to(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
+                                             float (&sum)[4], uint32_t (&packed)[16]) {
   float e[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(x[j]), sl2, -m_ref);
@@ -197,9 +197,14 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, fl
   }
 #pragma unroll
   for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
-  uint32_t packed[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) packed[j] = pack_bf16(e[2 * j], e[2 * j + 1]);
+}
+template <bool kMasked>
+__device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
+                                          float (&sum)[4], uint32_t p_tmem) {
+  uint32_t packed[16];
+  exp_chunk_to<kMasked>(x, sl2, m_ref, bits, sum, packed);
   ptx::tmem_st16(p_tmem, packed);
 }
 
@@ -730,82 +735,129 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (tid == 128 && tl / kStreams == 3) JET_TR(58);
         if (tid == 256 && tl / kStreams < 4) JET_TR(32 + 2 * (tl / kStreams));
 
-        // ---- row maximum over the visible keys.  A full tile is read from TMEM once: the thread keeps its
-        //      whole score row (128 values) in registers for both the maximum and the exponentials.  A tile
-        //      with masked keys (ragged end of the prefix, tree keys) takes two passes over TMEM, chunk by chunk.
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        // (The P V product of this accumulator's previous tile is complete: the Q K^T that produced these
+        //  scores was only issued after it.  So O may be rescaled and the score buffer overwritten with P.)
         static_assert(kChunks == 4, "the register-resident row is written out for four 32-key chunks");
         uint32_t xa[32], xb[32], xc[32], xd[32];
+        bool done = false;
         if (full_tile) {
+          // ---- fast path of a full tile: the thread reads its whole score row (128 values) from TMEM once and
+          //      exponentiates against the reference maximum it already has -- no pass for the row maximum.
+          //      Any reference is exact as long as nothing overflows; the row sum of the tile shows whether the
+          //      reference was too low (then, or if a value is not finite, the tile is redone with its true maximum).
           ptx::tmem_ld32(tS, xa);
           ptx::tmem_ld32(tS + 32, xb);
           ptx::tmem_ld32(tS + 64, xc);
           ptx::tmem_ld32(tS + 96, xd);
           ptx::tmem_wait_ld();
-          max_chunk(xa, mx);
-          max_chunk(xb, mx);
-          max_chunk(xc, mx);
-          max_chunk(xd, mx);
-        } else {
+          if (__any_sync(0xffffffffu, m_used == -INFINITY)) {
+            // first tile of the stream: the reference is the tile's own row maximum
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            max_chunk(xa, mx);
+            max_chunk(xb, mx);
+            max_chunk(xc, mx);
+            max_chunk(xd, mx);
+            if (m_used == -INFINITY) m_used = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          }
+          if (tid == 128 && tl / kStreams == 3) JET_TR(59);
+          float m_ref = m_used * sl2;
+          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          // P is stored chunk by chunk, under the arithmetic of the next chunk.  It overwrites the score columns
+          // of the first two chunks, so those two stay in registers (xa, xb) in case the tile has to be redone;
+          // the last two chunks go first, their score columns stay intact in TMEM.
+          exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
+          exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
+          exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
+          exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
+          float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          if (tid == 128 && tl / kStreams == 3) JET_TR(60);
+          float factor = 1.0f;
+          const bool redo = __any_sync(0xffffffffu, !(tile_sum <= kFastSumLimit));
+          if (redo) {
+            // The reference was too low for some row of this warp (or a value is not finite): take the tile's
+            // true row maximum as the new reference and compute the tile again.
+            ptx::tmem_ld32(tS + 64, xc);
+            ptx::tmem_ld32(tS + 96, xd);
+            ptx::tmem_wait_ld();
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            max_chunk(xa, mx);
+            max_chunk(xb, mx);
+            max_chunk(xc, mx);
+            max_chunk(xd, mx);
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            if (m_tile > m_used) {
+              factor = exp2f((m_used - m_tile) * sl2);
+              m_used = m_tile;
+            }
+            m_ref = m_used * sl2;
+            sum[0] = sum[1] = sum[2] = sum[3] = 0.0f;
+            ptx::tmem_wait_st();
+            exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
+            exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
+            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
+            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
+            tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+            if (__any_sync(0xffffffffu, factor != 1.0f) && last_tl >= 0) {
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {
+                ptx::tmem_ld32(tO + c * 32, xa);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
+                ptx::tmem_st32(tO + c * 32, xa);
+              }
+            }
+          }
+          l = l * factor + tile_sum;
+          done = true;
+        }
+        if (!done) {
+          // ---- tiles with masked keys: two passes over TMEM in 32-key chunks, row maximum first
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
           for (int c = 0; c < kChunks; ++c) {
             ptx::tmem_ld32(tS + c * 32, xa);
             ptx::tmem_wait_ld();
             max_chunk_masked(xa, chunk_bits(c), mx);
           }
-        }
-        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        if (tid == 128 && tl < 1) JET_TR(5);
-        if (tid == 128 && tl / kStreams == 3) JET_TR(59);
+          const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          if (tid == 128 && tl < 1) JET_TR(5);
 
-        // ---- running maximum with lazy rescaling
-        float factor = 1.0f;
-        if (m_tile > -INFINITY) {
-          if (m_used == -INFINITY) {
-            m_used = m_tile;                       // nothing accumulated yet for this row
-          } else if ((m_tile - m_used) * sl2 > kRescaleThreshold) {
-            factor = exp2f((m_used - m_tile) * sl2);
-            m_used = m_tile;
+          // running maximum with lazy rescaling
+          float factor = 1.0f;
+          if (m_tile > -INFINITY) {
+            if (m_used == -INFINITY) {
+              m_used = m_tile;                       // nothing accumulated yet for this row
+            } else if ((m_tile - m_used) * sl2 > kRescaleThreshold) {
+              factor = exp2f((m_used - m_tile) * sl2);
+              m_used = m_tile;
+            }
           }
-        }
-        const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
-        const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+          const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
+          const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+          ptx::tc_fence_after();
+          if (tid == 128 && tl < 1) JET_TR(16);
 
-        // (The P V product of this accumulator's previous tile is complete: the Q K^T that produced these
-        //  scores was only issued after it.  So O may be rescaled and the score buffer overwritten with P.)
-        ptx::tc_fence_after();
-        if (tid == 128 && tl < 1) JET_TR(16);
-
-        // ---- pass 2: probabilities, row sum; P (packed bf16) overwrites the first 64 columns of the scores
-        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (full_tile) {
-          exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
-          if (tid == 128 && tl / kStreams == 3) JET_TR(61);
-          exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
-          if (tid == 128 && tl / kStreams == 3) JET_TR(62);
-          exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
-          if (tid == 128 && tl / kStreams == 3) JET_TR(63);
-          exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
-        } else {
+          // probabilities, row sum; P (packed bf16) overwrites the first 64 columns of the scores
+          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll 1
           for (int c = 0; c < kChunks; ++c) {
             ptx::tmem_ld32(tS + c * 32, xa);
             ptx::tmem_wait_ld();
             exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, tS + c * 16);
           }
-        }
-        l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
-        if (tid == 128 && tl < 1) JET_TR(17);
-        if (tid == 128 && tl / kStreams == 3) JET_TR(60);
+          l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+          if (tid == 128 && tl < 1) JET_TR(17);
 
-        if (need_rescale && last_tl >= 0) {
+          if (need_rescale && last_tl >= 0) {
 #pragma unroll 1
-          for (int c = 0; c < D / 32; ++c) {
-            ptx::tmem_ld32(tO + c * 32, xa);
-            ptx::tmem_wait_ld();
+            for (int c = 0; c < D / 32; ++c) {
+              ptx::tmem_ld32(tO + c * 32, xa);
+              ptx::tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
-            ptx::tmem_st32(tO + c * 32, xa);
+              for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
+              ptx::tmem_st32(tO + c * 32, xa);
+            }
           }
         }
         if (!full_tile) {
