@@ -117,6 +117,30 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// CTA-wide barrier as an explicit instruction.  Unlike __syncthreads() the compiler can neither drop one of
+// two adjacent barriers nor merge them, so code paths that are compiled separately for different warps of
+// a CTA (and contain different work between the barriers) stay in step barrier for barrier.
+// The barrier instruction is warp-aligned: a warp must reach it converged (lanes that skipped a branch must
+// not run ahead of the lanes inside it), hence the __syncwarp() first.
+__device__ __forceinline__ void cta_sync() {
+  __syncwarp();
+  asm volatile("bar.sync 0;" ::: "memory");
+}
+// The same with an AND-reduction of a predicate over the CTA.
+__device__ __forceinline__ bool cta_sync_and(bool pred) {
+  uint32_t r;
+  __syncwarp();
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, 0, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(static_cast<uint32_t>(pred ? 1u : 0u))
+      : "memory");
+  return r != 0;
+}
+
 // True in exactly one lane of a converged warp.  Code under this predicate is still uniform for the
 // compiler (every operand of the tensor-core instructions can stay in uniform registers).
 __device__ __forceinline__ bool elect_one() {

@@ -97,9 +97,11 @@ struct Cfg {
   __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
   __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
   // Epilogue buffers (overlay the tile memory once the key loop is over): this CTA's 128 normalised
-  // rows of one query tile -- D fp32 values followed by the row's log2-sum-exp, padded so that the
-  // row-per-thread stores of a warp spread over all banks -- and the blocks received from every slice.
-  static constexpr int kRecvPitch = D * 4 + 16;
+  // rows of one query tile -- D bf16 values followed by the row's log2-sum-exp in fp32, padded so that
+  // the row-per-thread stores of a warp spread over all banks -- and the blocks received from every
+  // slice.  The partial rows travel as bf16 (every one is a normalised average of V rows, so it has the
+  // scale of the final output): the exchange is bandwidth-bound and this halves it.
+  static constexpr int kRecvPitch = D * 2 + 16;
   static constexpr int kBlockBytes = kBM * kRecvPitch;                   // the 128 staged rows of one stream
   static constexpr int kStageOff = 0;
   static constexpr int kRecvOff = (kBlockBytes + 1023) / 1024 * 1024;
@@ -151,7 +153,7 @@ __device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint
     if (*abort_flag) break;
   }
   if (!ok && *abort_flag == 0u) *abort_flag = 1u + site;
-  return __syncthreads_and(ok ? 1 : 0) != 0;
+  return ptx::cta_sync_and((ok ? 1 : 0) != 0);
 }
 
 // Cluster-wide rendezvous built from one mbarrier per CTA (count = cluster size): after a CTA-wide
@@ -159,7 +161,7 @@ __device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint
 // all `nsplit` arrivals on the local one.
 __device__ __forceinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag,
                                                 uint32_t site) {
-  __syncthreads();
+  ptx::cta_sync();
   if (threadIdx.x == 0)
     for (int c = 0; c < nsplit; ++c) ptx::mbar_arrive_remote(ptx::map_to_rank(local_bar, c));
   return bounded_wait_cluster(local_bar, abort_flag, site);
@@ -285,7 +287,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::prefetch_tmap(&tm_tv);
   }
   ptx::tc_fence_before();
-  __syncthreads();
+  ptx::cta_sync();
   ptx::tc_fence_after();
   // The barriers of every CTA of the cluster must exist before any CTA arrives on them remotely:
   // arrive on the hardware cluster barrier now, wait for it only when the slices are merged.
@@ -335,9 +337,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag, 12);
       if (tid == 128) JET_TR(7);
     } else {
-      __syncthreads();
+      ptx::cta_sync();
     }
-    // Staging of a row: normalised, D fp32 values followed by the row's log2-sum-exp.  Rows this CTA
+    // Staging of a row: normalised, D bf16 values followed by the row's log2-sum-exp (fp32).  Rows this CTA
     // computed nothing for (empty key slice, tile without nodes) get log2-sum-exp = -inf ("absent").
     const uint32_t e_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const bool active = has_work && row_ok;                      // warp-uniform: TMEM loads need whole warps
@@ -352,12 +354,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (mt > 0) {
         // C: everybody has combined the previous tile's rows, so both buffers are free again
         if (via_cluster) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
-        else __syncthreads();
+        else ptx::cta_sync();
       }
       if constexpr (MT == 1) {
         // Both warpgroups stage half of every row (64 columns each), folding the two streams' accumulators
         // together on the way: out = wa * O_0 / l_0 + wb * O_1 / l_1 with softmax weights of the two sums.
-        __syncthreads();
+        ptx::cta_sync();
         if constexpr (kSm) {
           const float2 s0 = xchg[e_r], s1 = xchg[128 + e_r];
           const float mxl = fmaxf(s0.x, s1.x);
@@ -371,7 +373,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             lse2 = mxl + log2f(w0 + w1);
           }
           constexpr int kCols = D / 2;
-          uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 4;
+          uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 2;
 #pragma unroll 1
           for (int c = 0; c < kCols / 32; ++c) {
             uint32_t o0[32], o1[32];
@@ -381,19 +383,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               ptx::tmem_wait_ld();
             }
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q8 = 0; q8 < 4; ++q8) {
+              uint32_t w[4] = {0u, 0u, 0u, 0u};
               if (active) {
-                // an accumulator that never received a product holds junk: its weight is exactly 0
-                x.x = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4]) : 0.0f);
-                x.y = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 1]) : 0.0f);
-                x.z = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 2]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 2]) : 0.0f);
-                x.w = (a0 != 0.0f ? a0 * __uint_as_float(o0[q4 * 4 + 3]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[q4 * 4 + 3]) : 0.0f);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const int j = q8 * 8 + 2 * k;
+                  const float lo = (a0 != 0.0f ? a0 * __uint_as_float(o0[j]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[j]) : 0.0f);
+                  const float hi = (a0 != 0.0f ? a0 * __uint_as_float(o0[j + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[j + 1]) : 0.0f);
+                  w[k] = pack_bf16(lo, hi);
+                }
               }
-              *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
+              *reinterpret_cast<uint4*>(dst + (c * 32 + q8 * 8) * 2) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
-          if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 4) = lse2;
+          if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 2) = lse2;
         }
       } else if (kSm && e_wg == mt) {
         uint8_t* dst = stage + e_r * C::kRecvPitch;
@@ -405,18 +409,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::tmem_wait_ld();
           }
 #pragma unroll
-          for (int q4 = 0; q4 < 8; ++q4) {
-            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (active)
-              x = make_float4(__uint_as_float(o[q4 * 4]) * own_inv, __uint_as_float(o[q4 * 4 + 1]) * own_inv,
-                              __uint_as_float(o[q4 * 4 + 2]) * own_inv, __uint_as_float(o[q4 * 4 + 3]) * own_inv);
-            *reinterpret_cast<float4*>(dst + (c * 32 + q4 * 4) * 4) = x;
+          for (int q8 = 0; q8 < 4; ++q8) {
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            if (active) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                w[k] = pack_bf16(__uint_as_float(o[q8 * 8 + 2 * k]) * own_inv, __uint_as_float(o[q8 * 8 + 2 * k + 1]) * own_inv);
+            }
+            *reinterpret_cast<uint4*>(dst + (c * 32 + q8 * 8) * 2) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
-        *reinterpret_cast<float*>(dst + D * 4) = own_lse2;
+        *reinterpret_cast<float*>(dst + D * 2) = own_lse2;
       }
       if (via_cluster) ptx::fence_proxy_async_smem();
-      __syncthreads();
+      ptx::cta_sync();
       const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
       bool rows_ok = merge_ok;
       if (via_cluster) {
@@ -458,7 +464,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ptx::fence_proxy_async_all();
           __threadfence();
         }
-        __syncthreads();
+        ptx::cta_sync();
         if (!kSm && tid == 0) {
           ptx::atom_add_release_gpu(arrive, 1);
           bool seen = false;
@@ -471,13 +477,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ptx::fence_proxy_async_all();
         }
         if (tid == 128 && mt == 0) JET_TR(8);
-        const bool published = __syncthreads_and(*abort_flag == 0u ? 1 : 0) != 0;
+        const bool published = ptx::cta_sync_and((*abort_flag == 0u ? 1 : 0) != 0);
         if (!kSm && tid < S && published && own_n > 0)
           ptx::bulk_load_global(smem_base + C::kRecvOff + static_cast<uint32_t>(tid * rows_per * C::kRecvPitch),
                                 slots + (static_cast<size_t>(tid) * MT + mt) * kBlockBytes + own_lo * C::kRecvPitch,
                                 static_cast<uint32_t>(own_n * C::kRecvPitch), bar(Bars::kRecv + mt));
         rows_ok = published && (own_n == 0 || bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14));
-        if (own_n == 0) __syncthreads();
+        if (own_n == 0) ptx::cta_sync();
         if (tid == 128 && mt == 0) JET_TR(9);
         src_rows = smem_gen + C::kRecvOff;
         // the last slice to have fetched its rows leaves the counters at zero for the next call
@@ -505,7 +511,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           float mx = -INFINITY;
 #pragma unroll
           for (int c = 0; c < kMaxSplit; ++c) {
-            ls[c] = c < S ? *reinterpret_cast<const float*>(row0 + c * src_stride + D * 4) : -INFINITY;
+            ls[c] = c < S ? *reinterpret_cast<const float*>(row0 + c * src_stride + D * 2) : -INFINITY;
             mx = fmaxf(mx, ls[c]);
           }
           float wsum = 0.0f;
@@ -519,19 +525,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
             for (int c0 = 0; c0 < kMaxSplit; c0 += 4) {
               if (c0 < S) {
-                float4 x0[4], x1[4];
+                uint4 x[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                   const uint8_t* src = row0 + (c0 + k) * src_stride;
-                  const bool use = ls[c0 + k] > 0.0f;
-                  x0[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32) : make_float4(0.f, 0.f, 0.f, 0.f);
-                  x1[k] = use ? *reinterpret_cast<const float4*>(src + c8 * 32 + 16) : make_float4(0.f, 0.f, 0.f, 0.f);
+                  x[k] = ls[c0 + k] > 0.0f ? *reinterpret_cast<const uint4*>(src + c8 * 16) : make_uint4(0u, 0u, 0u, 0u);
                 }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                   const float w = ls[c0 + k];
-                  acc[0] += w * x0[k].x; acc[1] += w * x0[k].y; acc[2] += w * x0[k].z; acc[3] += w * x0[k].w;
-                  acc[4] += w * x1[k].x; acc[5] += w * x1[k].y; acc[6] += w * x1[k].z; acc[7] += w * x1[k].w;
+                  const uint32_t v4[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
+                    acc[2 * q] += w * __uint_as_float(v4[q] << 16);
+                    acc[2 * q + 1] += w * __uint_as_float(v4[q] & 0xFFFF0000u);
+                  }
                 }
               }
             }
@@ -901,7 +909,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::cluster_wait();     // every CTA of the cluster has received all of its blocks
   }
   ptx::tc_fence_before();
-  __syncthreads();
+  ptx::cta_sync();
   if (warp == 2) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, C::kTmemCols);
@@ -1072,7 +1080,7 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
 
 size_t workspace_need(const Plan& pl, int D) {
   if (!pl.via_global) return 256;
-  return kCounterBytes + static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM * (D * 4 + 16);
+  return kCounterBytes + static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM * (D * 2 + 16);
 }
 
 template <int D, int MT>
