@@ -23,6 +23,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cstdlib>
+#include <cstring>
 
 #include "jet_common.cuh"
 #include "sm100_ptx.cuh"
@@ -39,8 +40,7 @@ constexpr int kBM = 128;               // query rows per tile
 constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
 constexpr int kMaxSplit = 16;          // largest cluster
-constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more
-constexpr float kFastSumLimit = 256.0f;    // a full tile keeps its reference maximum while its row sums stay below (so P <= 2^8)
+constexpr float kFastSumLimit = 256.0f;    // a row keeps its reference maximum while its tile sums stay below (so P <= 2^8)
 
 struct AttnParams {
   const int32_t* page_table;
@@ -176,37 +176,28 @@ __device__ __forceinline__ void max_chunk(const uint32_t (&x)[32], float (&mx)[4
 #pragma unroll
   for (int j = 0; j < 32; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(x[j]));
 }
-__device__ __forceinline__ void max_chunk_masked(const uint32_t (&x)[32], uint32_t bits, float (&mx)[4]) {
+// Scores of keys the row must not see become -inf (bit j of `bits` = key j of the chunk is visible).
+__device__ __forceinline__ void mask_chunk(uint32_t (&x)[32], uint32_t bits) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j)
-    mx[j & 3] = fmaxf(mx[j & 3], ((bits >> j) & 1u) ? __uint_as_float(x[j]) : -INFINITY);
+  for (int j = 0; j < 32; ++j) x[j] = ((bits >> j) & 1u) ? x[j] : 0xFF800000u;
 }
 
-// 32 scores of one row -> probabilities (exp2 of the scaled, shifted score; masked keys exactly 0),
-// added to the row sum and packed as bf16 pairs (the A operand of the P V product, 16 TMEM columns of
-// the row's lane).  The stages are kept apart so that the 32 independent exp2 are in flight together.
-template <bool kMasked>
-__device__ __forceinline__ void exp_chunk_to(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
-                                             float (&sum)[4], uint32_t (&packed)[16]) {
+// 32 scores of one row -> probabilities (exp2 of the scaled, shifted score; a score of -inf gives exactly
+// 0), added to the row sum and written as packed bf16 pairs to 16 TMEM columns of the row's lane (the A
+// operand of the P V product).  The stages are kept apart so that the 32 independent exp2 are in flight
+// together.
+__device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, float (&sum)[4],
+                                          uint32_t p_tmem) {
   float e[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(x[j]), sl2, -m_ref);
 #pragma unroll
   for (int j = 0; j < 32; ++j) e[j] = exp2f(e[j]);
-  if (kMasked) {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) e[j] = ((bits >> j) & 1u) ? e[j] : 0.0f;
-  }
 #pragma unroll
   for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
+  uint32_t packed[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) packed[j] = pack_bf16(e[2 * j], e[2 * j + 1]);
-}
-template <bool kMasked>
-__device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, uint32_t bits,
-                                          float (&sum)[4], uint32_t p_tmem) {
-  uint32_t packed[16];
-  exp_chunk_to<kMasked>(x, sl2, m_ref, bits, sum, packed);
   ptx::tmem_st16(p_tmem, packed);
 }
 
@@ -279,6 +270,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   } else if (warp == 2) {
     ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
     ptx::tmem_relinquish();
+    if (lane == 0) JET_TR(44);
   } else if (warp == 3 && lane == 0) {
     ptx::prefetch_tmap(&tm_q);
     ptx::prefetch_tmap(&tm_k);
@@ -286,16 +278,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::prefetch_tmap(&tm_tk);
     ptx::prefetch_tmap(&tm_tv);
   }
+  if (tid == 0) JET_TR(40);
   ptx::tc_fence_before();
   ptx::cta_sync();
   ptx::tc_fence_after();
+  if (tid == 0) JET_TR(41);
   // The barriers of every CTA of the cluster must exist before any CTA arrives on them remotely:
   // arrive on the hardware cluster barrier now, wait for it only when the slices are merged.
   const bool via_cluster = S > 1 && !p.via_global;
   if (via_cluster) ptx::cluster_arrive();
   const uint32_t tmem_base = *tmem_slot;
+  if (tid == 0) JET_TR(42);
   ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
   ptx::grid_dep_launch();    // the next kernel may start its own set-up as SMs become free
+  if (tid == 0) JET_TR(43);
 
   // ---------------- work item, continued: what depends on device data
   const int L = p.seq_len[b];
@@ -304,8 +300,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int TP = (L + kBN - 1) / kBN;
   const int TT = (ntree + kBN - 1) / kBN;
   const int T_all = TP + TT;
-  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split) / S);
-  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1)) / S);
+  // key tiles of this slice; when they do not divide evenly the first slices take the extra tile, so that
+  // the last slice, whose tree tile (masked) is the slowest kind, has the fewest
+  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split + S - 1) / S);
+  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1) + S - 1) / S);
   const int T = t_hi - t_lo;
   const bool has_work = node_lo < n && T > 0;    // otherwise: no live node here, or an empty key slice
   if (tid == 0) JET_TR(1);
@@ -571,6 +569,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             for (int h = 0; h < kHalves; ++h)
               ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
                                b * p.B + node_lo + mt * npt);
+          JET_TR(45);
         }
         __syncwarp();
         bool ok = true;
@@ -746,118 +745,81 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // (The P V product of this accumulator's previous tile is complete: the Q K^T that produced these
         //  scores was only issued after it.  So O may be rescaled and the score buffer overwritten with P.)
         static_assert(kChunks == 4, "the register-resident row is written out for four 32-key chunks");
+        // ---- The thread reads its whole score row (128 values) from TMEM once.  Keys the row must not see
+        //      (ragged end of the prefix, tree keys outside the ancestor set) are replaced by -inf right away,
+        //      so they get probability exactly 0 whatever the cache rows behind them hold.  The row is then
+        //      exponentiated against the reference maximum it already has -- no pass for the row maximum, except
+        //      in the first tile of a stream.  Any reference is exact as long as nothing overflows; the row sum
+        //      of the tile shows whether the reference was too low (then, or if a value is not finite, the tile
+        //      is redone with its true maximum).
         uint32_t xa[32], xb[32], xc[32], xd[32];
-        bool done = false;
-        if (full_tile) {
-          // ---- fast path of a full tile: the thread reads its whole score row (128 values) from TMEM once and
-          //      exponentiates against the reference maximum it already has -- no pass for the row maximum.
-          //      Any reference is exact as long as nothing overflows; the row sum of the tile shows whether the
-          //      reference was too low (then, or if a value is not finite, the tile is redone with its true maximum).
-          ptx::tmem_ld32(tS, xa);
-          ptx::tmem_ld32(tS + 32, xb);
+        uint32_t b0 = 0xFFFFFFFFu, b1 = 0xFFFFFFFFu, b2 = 0xFFFFFFFFu, b3 = 0xFFFFFFFFu;
+        if (!full_tile) { b0 = chunk_bits(0); b1 = chunk_bits(1); b2 = chunk_bits(2); b3 = chunk_bits(3); }
+        ptx::tmem_ld32(tS, xa);
+        ptx::tmem_ld32(tS + 32, xb);
+        ptx::tmem_ld32(tS + 64, xc);
+        ptx::tmem_ld32(tS + 96, xd);
+        ptx::tmem_wait_ld();
+        if (!full_tile) {
+          mask_chunk(xa, b0);
+          mask_chunk(xb, b1);
+          mask_chunk(xc, b2);
+          mask_chunk(xd, b3);
+        }
+        if (__any_sync(0xffffffffu, m_used == -INFINITY)) {
+          // nothing accumulated yet for some row: its reference is the tile's own row maximum (which stays
+          // -inf if the row sees no key of this tile)
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          max_chunk(xa, mx);
+          max_chunk(xb, mx);
+          max_chunk(xc, mx);
+          max_chunk(xd, mx);
+          if (m_used == -INFINITY) m_used = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        }
+        if (tid == 128 && tl < 1) JET_TR(5);
+        if (tid == 128 && tl / kStreams == 3) JET_TR(59);
+        float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        // P is stored chunk by chunk, under the arithmetic of the next chunk.  It overwrites the score columns
+        // of the first two chunks, so those two stay in registers (xa, xb) in case the tile has to be redone;
+        // the last two chunks go first, their score columns stay intact in TMEM.
+        exp_chunk(xc, sl2, m_ref, sum, tS + 32);
+        exp_chunk(xd, sl2, m_ref, sum, tS + 48);
+        exp_chunk(xa, sl2, m_ref, sum, tS);
+        exp_chunk(xb, sl2, m_ref, sum, tS + 16);
+        float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        if (tid == 128 && tl < 1) JET_TR(17);
+        if (tid == 128 && tl / kStreams == 3) JET_TR(60);
+        float factor = 1.0f;
+        if (__any_sync(0xffffffffu, !(tile_sum <= kFastSumLimit))) {
+          // The reference was too low for some row of this warp (or a value is not finite): take the tile's
+          // true row maximum as the new reference and compute the tile again.
           ptx::tmem_ld32(tS + 64, xc);
           ptx::tmem_ld32(tS + 96, xd);
           ptx::tmem_wait_ld();
-          if (__any_sync(0xffffffffu, m_used == -INFINITY)) {
-            // first tile of the stream: the reference is the tile's own row maximum
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            max_chunk(xa, mx);
-            max_chunk(xb, mx);
-            max_chunk(xc, mx);
-            max_chunk(xd, mx);
-            if (m_used == -INFINITY) m_used = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          if (!full_tile) {
+            mask_chunk(xc, b2);
+            mask_chunk(xd, b3);
           }
-          if (tid == 128 && tl / kStreams == 3) JET_TR(59);
-          float m_ref = m_used * sl2;
-          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-          // P is stored chunk by chunk, under the arithmetic of the next chunk.  It overwrites the score columns
-          // of the first two chunks, so those two stay in registers (xa, xb) in case the tile has to be redone;
-          // the last two chunks go first, their score columns stay intact in TMEM.
-          exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
-          exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
-          exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
-          exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
-          float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-          if (tid == 128 && tl / kStreams == 3) JET_TR(60);
-          float factor = 1.0f;
-          const bool redo = __any_sync(0xffffffffu, !(tile_sum <= kFastSumLimit));
-          if (redo) {
-            // The reference was too low for some row of this warp (or a value is not finite): take the tile's
-            // true row maximum as the new reference and compute the tile again.
-            ptx::tmem_ld32(tS + 64, xc);
-            ptx::tmem_ld32(tS + 96, xd);
-            ptx::tmem_wait_ld();
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            max_chunk(xa, mx);
-            max_chunk(xb, mx);
-            max_chunk(xc, mx);
-            max_chunk(xd, mx);
-            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            if (m_tile > m_used) {
-              factor = exp2f((m_used - m_tile) * sl2);
-              m_used = m_tile;
-            }
-            m_ref = m_used * sl2;
-            sum[0] = sum[1] = sum[2] = sum[3] = 0.0f;
-            ptx::tmem_wait_st();
-            exp_chunk<false>(xc, sl2, m_ref, 0u, sum, tS + 32);
-            exp_chunk<false>(xd, sl2, m_ref, 0u, sum, tS + 48);
-            exp_chunk<false>(xa, sl2, m_ref, 0u, sum, tS);
-            exp_chunk<false>(xb, sl2, m_ref, 0u, sum, tS + 16);
-            tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-            if (__any_sync(0xffffffffu, factor != 1.0f) && last_tl >= 0) {
-#pragma unroll 1
-              for (int c = 0; c < D / 32; ++c) {
-                ptx::tmem_ld32(tO + c * 32, xa);
-                ptx::tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
-                ptx::tmem_st32(tO + c * 32, xa);
-              }
-            }
-          }
-          l = l * factor + tile_sum;
-          done = true;
-        }
-        if (!done) {
-          // ---- tiles with masked keys: two passes over TMEM in 32-key chunks, row maximum first
           float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-          for (int c = 0; c < kChunks; ++c) {
-            ptx::tmem_ld32(tS + c * 32, xa);
-            ptx::tmem_wait_ld();
-            max_chunk_masked(xa, chunk_bits(c), mx);
-          }
+          max_chunk(xa, mx);
+          max_chunk(xb, mx);
+          max_chunk(xc, mx);
+          max_chunk(xd, mx);
           const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-          if (tid == 128 && tl < 1) JET_TR(5);
-
-          // running maximum with lazy rescaling
-          float factor = 1.0f;
-          if (m_tile > -INFINITY) {
-            if (m_used == -INFINITY) {
-              m_used = m_tile;                       // nothing accumulated yet for this row
-            } else if ((m_tile - m_used) * sl2 > kRescaleThreshold) {
-              factor = exp2f((m_used - m_tile) * sl2);
-              m_used = m_tile;
-            }
+          if (m_tile > m_used) {
+            if (m_used > -INFINITY) factor = exp2f((m_used - m_tile) * sl2);
+            m_used = m_tile;
           }
-          const bool need_rescale = __any_sync(0xffffffffu, factor != 1.0f);
-          const float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
-          ptx::tc_fence_after();
-          if (tid == 128 && tl < 1) JET_TR(16);
-
-          // probabilities, row sum; P (packed bf16) overwrites the first 64 columns of the scores
-          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll 1
-          for (int c = 0; c < kChunks; ++c) {
-            ptx::tmem_ld32(tS + c * 32, xa);
-            ptx::tmem_wait_ld();
-            exp_chunk<true>(xa, sl2, m_ref, chunk_bits(c), sum, tS + c * 16);
-          }
-          l = l * factor + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
-          if (tid == 128 && tl < 1) JET_TR(17);
-
-          if (need_rescale && last_tl >= 0) {
+          m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+          sum[0] = sum[1] = sum[2] = sum[3] = 0.0f;
+          ptx::tmem_wait_st();
+          exp_chunk(xc, sl2, m_ref, sum, tS + 32);
+          exp_chunk(xd, sl2, m_ref, sum, tS + 48);
+          exp_chunk(xa, sl2, m_ref, sum, tS);
+          exp_chunk(xb, sl2, m_ref, sum, tS + 16);
+          tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          if (__any_sync(0xffffffffu, factor != 1.0f) && last_tl >= 0) {
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
               ptx::tmem_ld32(tO + c * 32, xa);
@@ -868,6 +830,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
           }
         }
+        l = l * factor + tile_sum;
         if (!full_tile) {
           // Masked keys get P = 0 exactly, but 0 * NaN is NaN: the V rows of keys beyond the valid ones
           // (stale cache rows, rows of padding nodes) are cleared before the P V product may read them.
@@ -1024,51 +987,57 @@ int max_active_clusters_for(int D, int mt, int cluster) {
   return mt == 1 ? max_active_clusters<64, 1>(cluster) : max_active_clusters<64, 2>(cluster);
 }
 
-// Picks the query-tile grouping and the number of key slices.  Cost model: waves of clusters x key tiles
-// per CTA x a per-tile cost (1 for one query tile per CTA, 3 for two: the pair shares each K/V tile but
-// its shallower shared-memory ring and single-buffered P make a key tile about three times as slow).
+// Picks the query-tile grouping and the number of key slices with a cost model fitted to measurements, in
+// units of one key tile of a one-query-tile CTA whose K/V comes out of L2 (about 1900 cycles):
+//   key tile, one query tile per CTA   1 + 0.75 / g    g = CTAs that read the same K/V tile side by side
+//                                                      (the first one fetches it from HBM, the others hit L2)
+//   key tile, two query tiles per CTA  max(2.2, 1 + 0.75 / g)   two softmax chains share the tensor core,
+//                                                      but the K/V tile is loaded once for both
+//   fixed cost of a CTA                6 (no slices), 8 (slices merged inside a cluster), 10 (through the
+//                                      workspace); 1.6 times that with two query tiles (two merge rounds)
+// and the CTAs run in waves of what the device holds at once.
 Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   const int G = Hq / Hkv;
   const int rows = B * G;
   const int tiles = (max_seq_len + kBN - 1) / kBN + (B + kBN - 1) / kBN;
   Plan best{};
-  long best_cost = -1;
+  double best_cost = -1.0;
+  // Test hooks (read once per process): JET_FORCE_MT = query tiles per CTA, JET_FORCE_SPLIT = "slices" or
+  // "slices,g" (g = merge through the workspace); a forced choice the device cannot hold is ignored.
   static const int force_mt = [] { const char* e = getenv("JET_FORCE_MT"); return e ? atoi(e) : 0; }();
-  for (int mt = (rows > kBM ? 2 : 1); mt >= 1; --mt) {
+  static const int force_ns = [] { const char* e = getenv("JET_FORCE_SPLIT"); return e ? atoi(e) : 0; }();
+  static const int force_via = [] { const char* e = getenv("JET_FORCE_SPLIT"); return (e && strstr(e, ",g")) ? 1 : 0; }();
+  for (int mt = 1; mt <= (rows > kBM ? 2 : 1); ++mt) {
     if (force_mt && mt != force_mt && !(force_mt == 2 && rows <= kBM)) continue;
     Plan pl;
     pl.mt = mt;
     pl.n_mgroups = (rows + mt * kBM - 1) / (mt * kBM);
     pl.units = batch * Hkv * pl.n_mgroups;
+    const double shared = 1.0 + 0.75 / pl.n_mgroups;
+    const double tile_cost = mt == 1 ? shared : (shared > 2.2 ? shared : 2.2);
+    const double fixed_scale = mt == 1 ? 1.0 : 1.6;
+    auto consider = [&](int ns, int via_global, double waves, double fixed) {
+      if (force_ns && (ns != force_ns || (ns > 1 && via_global != force_via))) return;
+      const double cost = waves * (((tiles + ns - 1) / ns) * tile_cost + fixed * fixed_scale);
+      if (best_cost < 0.0 || cost < best_cost) {
+        best = pl;
+        best.nsplit = ns;
+        best.via_global = via_global;
+        best_cost = cost;
+      }
+    };
     for (int ns = 1; ns <= kMaxSplit && ns <= tiles; ++ns) {
       // (a) the slices of a unit form a thread-block cluster and merge through distributed shared memory
       const int resident = max_active_clusters_for(D, mt, ns);
-      if (resident > 0) {
-        const long waves = (pl.units + resident - 1) / resident;
-        const long cost = 4 * waves * ((tiles + ns - 1) / ns) * (mt == 2 ? 3 : 1);
-        if (best_cost < 0 || cost < best_cost) {
-          best = pl;
-          best.nsplit = ns;
-          best.via_global = 0;
-          best_cost = cost;
-        }
-      }
+      if (resident > 0) consider(ns, 0, static_cast<double>((pl.units + resident - 1) / resident), ns == 1 ? 6.0 : 8.0);
       // (b) independent CTAs that merge through the workspace: all of them must be resident at once
-      //     (a cluster has to fit into one GPC, which can leave a third of the SMs idle); slightly
-      //     penalised because the rows take a round trip through L2
+      //     (a cluster has to fit into one GPC, which can leave a third of the SMs idle)
       if (ns > 1 && static_cast<long>(pl.units) * ns <= sm_count() &&
-          static_cast<size_t>(pl.units) * mt * 2 * sizeof(int) <= kCounterBytes) {
-        const long cost = 4 * ((tiles + ns - 1) / ns) * (mt == 2 ? 3 : 1) + 1;
-        if (best_cost < 0 || cost < best_cost) {
-          best = pl;
-          best.nsplit = ns;
-          best.via_global = 1;
-          best_cost = cost;
-        }
-      }
+          static_cast<size_t>(pl.units) * mt * 2 * sizeof(int) <= kCounterBytes)
+        consider(ns, 1, 1.0, 10.0);
     }
   }
-  if (best_cost < 0) {          // the occupancy query failed: plain launch without slices
+  if (best_cost < 0.0) {        // the occupancy query failed: plain launch without slices
     best.mt = rows > kBM ? 2 : 1;
     best.n_mgroups = (rows + best.mt * kBM - 1) / (best.mt * kBM);
     best.units = batch * Hkv * best.n_mgroups;

@@ -223,7 +223,7 @@ def test_workspace_counters_are_left_clean_across_repeated_calls():
     import jet_harness as H
     import paper_2606_18394_b200 as jet
     rng = np.random.default_rng(5)
-    B, Hq, Hkv, D, L = 64, 32, 8, 128, 2000
+    B, Hq, Hkv, D, L = 64, 32, 8, 128, 4096
     x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
     parent, _, _ = random_tree(B, rng)
     anc = anc_from_parent(parent, B, B)
@@ -248,8 +248,9 @@ def test_workspace_counters_are_left_clean_across_repeated_calls():
 
 
 def test_two_query_tiles_per_cta_variant():
-    """The kernel variant with two query tiles per CTA is not chosen by the planner's current cost model;
-    JET_FORCE_MT=2 selects it (read once per process, hence the child process)."""
+    """The planner picks the kernel variant with two query tiles per CTA for batched shapes only;
+    JET_FORCE_MT=2 selects it for these single-sequence shapes too (read once per process, hence the
+    child process)."""
     import os
     import subprocess
     import sys
