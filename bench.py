@@ -34,7 +34,7 @@ UNIT = "us/layer"
 
 # DRAM bytes (read + write) of one tree_attn_kernel launch on the benchmark workload, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"qwen3_8b": 17634560}     # profiles/tree_attn_kernel_qwen3_8b.md
+NCU_TRAFFIC_BYTES = {"qwen3_8b": 17659392}     # profiles/tree_attn_kernel_qwen3_8b.md
 
 
 def workload(name):
@@ -63,15 +63,47 @@ def attn_algorithmic_flops(c, seq_lens, depths):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    """Samples SM clock and throttle reasons while the timed region runs.
+
+    Reads NVML directly from a thread (every 2 ms, so that a timed region of a few milliseconds still gets
+    samples); falls back to polling nvidia-smi where the NVML binding is missing.  Read-only: no setting of
+    the GPU is touched."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    REASON_BITS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
+                   ("sw_power_cap", 0x4))
 
-    def __init__(self, index):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index, uuid=None):
+        self.index, self.uuid = index, uuid
+        self.rows, self.proc, self.thread = [], None, None
+        self.sm, self.reason_mask, self.sm_max = [], 0, None
+        self.stop_flag = threading.Event()
+        self.nvml = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            handle = None
+            if self.uuid:
+                for cand in (f"GPU-{self.uuid}", str(self.uuid)):
+                    try:
+                        handle = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if hasattr(cand, "encode") else cand)
+                        break
+                    except Exception:
+                        handle = None
+            if handle is None:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(pynvml, "nvmlDeviceGetCurrentClocksThrottleReasons")
+            self.nvml = (pynvml, handle, reasons_fn)
+            self.thread = threading.Thread(target=self._poll_nvml, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
@@ -81,11 +113,27 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
+    def _poll_nvml(self):
+        pynvml, handle, reasons_fn = self.nvml
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)))
+                self.reason_mask |= int(reasons_fn(handle))
+            except Exception:
+                break
+            time.sleep(0.002)
+
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
     def stop(self):
+        if self.nvml is not None:
+            self.stop_flag.set()
+            self.thread.join(timeout=2)
+            reasons = [n for n, bit in self.REASON_BITS if self.reason_mask & bit]
+            return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.sm_max,
+                    "reasons": reasons, "samples": len(self.sm), "source": "nvml"}
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -95,7 +143,7 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for i, n in enumerate(names) if any(len(r) >= 6 and r[2 + i].lower() == "active" for r in self.rows)]
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+                "reasons": reasons, "samples": len(sm), "source": "nvidia-smi"}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -209,7 +257,11 @@ def bench_jet(args):
         torch.cuda.synchronize()
 
     # ---------------- device-resident timing of K whole steps
-    sampler = ClockSampler(local_rank)
+    try:
+        gpu_uuid = str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        gpu_uuid = None
+    sampler = ClockSampler(local_rank, gpu_uuid)
     if rank == 0:
         sampler.start()
     barrier()
@@ -231,22 +283,46 @@ def bench_jet(args):
     acc = st.accept_len.cpu().numpy().tolist()
     assert acc == info["planted"], (acc, info["planted"])
 
-    # ---------------- per-call timing of the attention layer (events around every call; cold KV)
+    # ---------------- the attention launches alone (the dominant kernel): `layers` launches per repetition, each
+    #                  on its own KV buffers (cold), replayed as a graph like the step itself; CUDA events on the
+    #                  launching stream around `steps` repetitions.  Without a graph: events around every call.
     with torch.cuda.stream(stream):
         st.seq_len.copy_(st.seq_len0)
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-               for _ in range(layers * args.steps)]
-        for rep in range(2):                       # first repetition warms up
-            i = 0
-            for _ in range(args.steps):
-                for layer in range(layers):
-                    a, b_ = evs[i]
-                    a.record(stream)
-                    st.verify_attn(layer)
-                    b_.record(stream)
-                    i += 1
+        if not args.no_graph:
+            attn_graph = torch.cuda.CUDAGraph()
+            for layer in range(layers):
+                st.verify_attn(layer)
             stream.synchronize()
-    attn_us = statistics.mean(a.elapsed_time(b_) for a, b_ in evs) * 1e3
+            with torch.cuda.graph(attn_graph, stream=stream):
+                for layer in range(layers):
+                    st.verify_attn(layer)
+            for _ in range(3):
+                attn_graph.replay()
+            stream.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(args.steps):
+                attn_graph.replay()
+            a1.record(stream)
+            stream.synchronize()
+            attn_us = a0.elapsed_time(a1) * 1e3 / (args.steps * layers)
+            attn_timing = f"CUDA events around {args.steps} replays of a graph of the {layers} attention launches"
+        else:
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(layers * args.steps)]
+            for rep in range(2):                       # first repetition warms up
+                i = 0
+                for _ in range(args.steps):
+                    for layer in range(layers):
+                        a, b_ = evs[i]
+                        a.record(stream)
+                        st.verify_attn(layer)
+                        b_.record(stream)
+                        i += 1
+                stream.synchronize()
+            attn_us = statistics.mean(a.elapsed_time(b_) for a, b_ in evs) * 1e3
+            attn_timing = "CUDA events around every attention call"
+    assert int(st.status.item()) == 0, "a bounded device wait expired"
 
     # ---------------- end to end: host buffers in, result out, every step
     pinned = {k: getattr(st, k).cpu().pin_memory() for k in ("logp", "root_token", "logits", "q", "tree_k", "tree_v")}
@@ -301,7 +377,7 @@ def bench_jet(args):
                 "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.config)
-    roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us,
+    roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us, timing=attn_timing,
                 algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
                 roofline_us=max(t_bytes, t_flops) * 1e6)
 
@@ -438,7 +514,7 @@ def bench_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["jet", "reference"], default="jet")
     ap.add_argument("--config", default="qwen3_8b", choices=[k for k, v in CONFIGS.items() if "B" in v])
