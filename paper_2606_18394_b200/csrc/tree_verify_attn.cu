@@ -223,7 +223,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   uint8_t* gen_bar = gen_kv + kStages * C::kStageBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + Bars::kCount * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  volatile int* len_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);     // [0] prefix length, [1] node count
   auto bar = [&](int idx) { return sBar + 8u * idx; };
   const int S = p.nsplit;                            // key slices = cluster size
   const int split = blockIdx.x % S;                  // = rank in the cluster
@@ -278,11 +277,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::prefetch_tmap(&tm_v);
     ptx::prefetch_tmap(&tm_tk);
     ptx::prefetch_tmap(&tm_tv);
-    // this thread alone fetches the sequence's prefix length and node count, while the others set up
-    ptx::grid_dep_wait();
-    const int len = p.seq_len[b], cnt = p.n_nodes[b];
-    len_slot[0] = len;
-    len_slot[1] = cnt;
   }
   if (tid == 0) JET_TR(40);
   ptx::tc_fence_before();
@@ -300,8 +294,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (tid == 0) JET_TR(43);
 
   // ---------------- work item, continued: what depends on device data
-  const int L = len_slot[0];
-  const int n = min(len_slot[1], p.B);
+  const int L = p.seq_len[b];
+  const int n = min(p.n_nodes[b], p.B);
   const int ntree = min(n, node_hi);                         // tree keys any row here can see
   const int TP = (L + kBN - 1) / kBN;
   const int TT = (ntree + kBN - 1) / kBN;
@@ -377,29 +371,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             lse2 = mxl + log2f(w0 + w1);
           }
           constexpr int kCols = D / 2;
-          constexpr int kIter = kCols / 32;
           uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 2;
-          uint32_t o0[kIter][32], o1[kIter][32];
-          if (active) {
-#pragma unroll
-            for (int c = 0; c < kIter; ++c) {
-              ptx::tmem_ld32(e_lane + C::o_col(0, 0) + e_wg * kCols + c * 32, o0[c]);
-              ptx::tmem_ld32(e_lane + C::o_col(0, 1) + e_wg * kCols + c * 32, o1[c]);
+#pragma unroll 1
+          for (int c = 0; c < kCols / 32; ++c) {
+            uint32_t o0[32], o1[32];
+            if (active) {
+              ptx::tmem_ld32(e_lane + C::o_col(0, 0) + e_wg * kCols + c * 32, o0);
+              ptx::tmem_ld32(e_lane + C::o_col(0, 1) + e_wg * kCols + c * 32, o1);
+              ptx::tmem_wait_ld();
             }
-            ptx::tmem_wait_ld();
-          }
-#pragma unroll
-          for (int c = 0; c < kIter; ++c) {
 #pragma unroll
             for (int q8 = 0; q8 < 4; ++q8) {
               uint32_t w[4] = {0u, 0u, 0u, 0u};
               if (active) {
-                // an accumulator that never received a product holds junk: its weight is exactly 0
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                   const int j = q8 * 8 + 2 * k;
-                  const float lo = (a0 != 0.0f ? a0 * __uint_as_float(o0[c][j]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[c][j]) : 0.0f);
-                  const float hi = (a0 != 0.0f ? a0 * __uint_as_float(o0[c][j + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[c][j + 1]) : 0.0f);
+                  const float lo = (a0 != 0.0f ? a0 * __uint_as_float(o0[j]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[j]) : 0.0f);
+                  const float hi = (a0 != 0.0f ? a0 * __uint_as_float(o0[j + 1]) : 0.0f) + (a1 != 0.0f ? a1 * __uint_as_float(o1[j + 1]) : 0.0f);
                   w[k] = pack_bf16(lo, hi);
                 }
               }
@@ -575,9 +564,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (warp == 0) {
         // =========================================================== TMA producer
         if (lane == 0) {
-          JET_TR(46);
           ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
-          JET_TR(47);
           for (int mt = 0; mt < n_mt; ++mt)
             for (int h = 0; h < kHalves; ++h)
               ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
@@ -619,9 +606,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const bool prefix = t < TP;
             const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
             const int row0 = prefix ? t * kBN : (t - TP) * kBN;
-            if (issued == 0) JET_TR(48);
             ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-            if (issued == 0) JET_TR(49);
             for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
           }
           __syncwarp();
