@@ -40,6 +40,7 @@ constexpr int kBM = 128;               // query rows per tile
 constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
 constexpr int kMaxSplit = 16;          // largest cluster
+constexpr int kMaxSorted = 128;          // batches up to this size are launched longest prefix first
 constexpr float kFastSumLimit = 256.0f;    // a row keeps its reference maximum while its tile sums stay below (so P <= 2^8)
 
 struct AttnParams {
@@ -201,7 +202,8 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, fl
   ptx::tmem_st16(p_tmem, packed);
 }
 
-template <int D, int MT>
+// kSorted: the sequences of a batch are launched longest prefix first (see the set-up of warp 3).
+template <int D, int MT, bool kSorted = false>
 __global__ void __launch_bounds__(Cfg<D, MT>::kThreads, 1)
 tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tk,
@@ -223,6 +225,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   uint8_t* gen_bar = gen_kv + kStages * C::kStageBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + Bars::kCount * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile int* seq_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);     // sequence of this CTA when launch order is sorted
   auto bar = [&](int idx) { return sBar + 8u * idx; };
   const int S = p.nsplit;                            // key slices = cluster size
   const int split = blockIdx.x % S;                  // = rank in the cluster
@@ -235,7 +238,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int mgroup = unit % p.n_mgroups;
   const int bg = unit / p.n_mgroups;
   const int g = bg % p.Hkv;
-  const int b = bg / p.Hkv;
+  const int b_rank = bg / p.Hkv;                 // position of the sequence in launch order
+  constexpr bool sorted_launch = kSorted;
   const int G = p.G;
   const int npt = kBM / G;                       // nodes per query tile
   const int node_lo = mgroup * MT * npt;
@@ -271,12 +275,46 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
     ptx::tmem_relinquish();
     if (lane == 0) JET_TR(44);
-  } else if (warp == 3 && lane == 0) {
-    ptx::prefetch_tmap(&tm_q);
-    ptx::prefetch_tmap(&tm_k);
-    ptx::prefetch_tmap(&tm_v);
-    ptx::prefetch_tmap(&tm_tk);
-    ptx::prefetch_tmap(&tm_tv);
+  } else if (warp == 3) {
+    if (lane == 0) {
+      ptx::prefetch_tmap(&tm_q);
+      ptx::prefetch_tmap(&tm_k);
+      ptx::prefetch_tmap(&tm_v);
+      ptx::prefetch_tmap(&tm_tk);
+      ptx::prefetch_tmap(&tm_tv);
+    }
+    __syncwarp();
+    if (sorted_launch) {
+      // Launch order = longest prefix first (CTAs are dispatched in index order, so with more work items than
+      // SMs the long sequences start early and the short ones fill the tail): this warp finds the sequence of
+      // rank b_rank by counting and leaves it in shared memory.  Beyond kMaxSorted sequences the order stays
+      // as given (many small items balance by themselves, and the count is quadratic).
+      ptx::grid_dep_wait();
+      int len[kMaxSorted / 32];
+#pragma unroll
+      for (int c = 0; c < kMaxSorted / 32; ++c) len[c] = c * 32 + lane < p.batch ? __ldg(p.seq_len + c * 32 + lane) : -1;
+      int found = -1;
+#pragma unroll
+      for (int c = 0; c < kMaxSorted / 32; ++c) {
+        if (c * 32 < p.batch) {
+          const int mine = len[c], me = c * 32 + lane;
+          int before = 0;                                // sequences that come before `me` in launch order
+#pragma unroll
+          for (int c2 = 0; c2 < kMaxSorted / 32; ++c2) {
+            if (c2 * 32 < p.batch) {
+              for (int j = 0; j < 32; ++j) {
+                const int other = __shfl_sync(0xffffffffu, len[c2], j), ob = c2 * 32 + j;
+                before += (ob < p.batch && (other > mine || (other == mine && ob < me))) ? 1 : 0;
+              }
+            }
+          }
+          if (me < p.batch && before == b_rank) found = me;
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) found = max(found, __shfl_xor_sync(0xffffffffu, found, o));
+      if (lane == 0) *seq_slot = found;
+    }
   }
   if (tid == 0) JET_TR(40);
   ptx::tc_fence_before();
@@ -294,6 +332,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (tid == 0) JET_TR(43);
 
   // ---------------- work item, continued: what depends on device data
+  const int b = sorted_launch ? *seq_slot : b_rank;
   const int L = p.seq_len[b];
   const int n = min(p.n_nodes[b], p.B);
   const int ntree = min(n, node_hi);                         // tree keys any row here can see
@@ -941,10 +980,12 @@ template <int D, int MT>
 bool configure_kernel() {
   static int state = 0;     // 0 = not yet, 1 = ok, -1 = failed
   if (state == 0) {
-    state = (cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  Cfg<D, MT>::kSmemBytes) == cudaSuccess &&
-             cudaFuncSetAttribute(tree_attn_kernel<D, MT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
-                 cudaSuccess)
+    auto set = [](auto kernel) {
+      return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D, MT>::kSmemBytes) ==
+                 cudaSuccess &&
+             cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    };
+    state = (set(tree_attn_kernel<D, MT, false>) && set(tree_attn_kernel<D, MT, true>))
                 ? 1
                 : -1;
     if (state < 0) cudaGetLastError();
@@ -1076,7 +1117,10 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   ++na;
   cfg.attrs = attrs;
   cfg.numAttrs = na;
-  if (cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT>, tq, tk, tv, ttk, ttv, p) != cudaSuccess) {
+  const bool sorted = p.batch > 1 && p.batch <= kMaxSorted;
+  const cudaError_t err = sorted ? cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, true>, tq, tk, tv, ttk, ttv, p)
+                                 : cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, false>, tq, tk, tv, ttk, ttv, p);
+  if (err != cudaSuccess) {
     cudaGetLastError();
     return JET_ERR_CUDA;
   }
