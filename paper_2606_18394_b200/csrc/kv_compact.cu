@@ -14,6 +14,7 @@ kv_compact_kernel(const uint4* __restrict__ tree_k, const uint4* __restrict__ tr
                   const int32_t* __restrict__ page_table, int max_pages, int page_size,
                   const int32_t* __restrict__ path, const int32_t* __restrict__ accept_len,
                   const int32_t* __restrict__ seq_len, int batch, int B, int row16, int N) {
+  grid_dependency_wait();
   const int i = blockIdx.x, b = blockIdx.y, layer = blockIdx.z;
   if (i > accept_len[b]) return;
   const int node = path[static_cast<size_t>(b) * (N + 1) + i];
@@ -36,6 +37,7 @@ kv_compact_kernel(const uint4* __restrict__ tree_k, const uint4* __restrict__ tr
 
 __global__ void advance_seq_len_kernel(const int32_t* __restrict__ accept_len,
                                        int32_t* __restrict__ seq_len, int batch) {
+  grid_dependency_wait();
   for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < batch; b += gridDim.x * blockDim.x)
     seq_len[b] += accept_len[b] + 1;
 }
@@ -66,11 +68,11 @@ extern "C" jet_status jet_kv_compact(const void* tree_k, const void* tree_v, voi
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int row16 = static_cast<int>(row_elems / 8);
-  kv_compact_kernel<<<dim3(N + 1, batch, layers), 256, 0, st>>>(
+  launch_dependent(kv_compact_kernel, dim3(N + 1, batch, layers), dim3(256), st,
       static_cast<const uint4*>(tree_k), static_cast<const uint4*>(tree_v),
       static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), cache_layer_stride / 8,
       kv_batch_stride / 8, page_table, max_pages_per_seq, page_size, path, accept_len, seq_len,
       batch, B, row16, N);
-  advance_seq_len_kernel<<<1, 256, 0, st>>>(accept_len, seq_len, batch);
+  launch_dependent(advance_seq_len_kernel, dim3(1), dim3(256), st, accept_len, seq_len, batch);
   return launch_status();
 }

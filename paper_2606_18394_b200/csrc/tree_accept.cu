@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kArgThreads)
 argmax_partial_kernel(const float* __restrict__ logits, int64_t row_stride, int V, int B,
                       const int32_t* __restrict__ n_nodes, int nchunks, bool vec_ok,
                       unsigned long long* __restrict__ partial) {
+  grid_dependency_wait();
   const int chunk = blockIdx.x;
   const int row = blockIdx.y;
   const int b = row / B, v = row - b * B;
@@ -74,6 +75,7 @@ accept_path_kernel(const unsigned long long* __restrict__ partial, int nchunks,
                    const int32_t* __restrict__ n_nodes, int B, int N,
                    int32_t* __restrict__ tgt_out, int32_t* __restrict__ accept_len,
                    int32_t* __restrict__ path, int32_t* __restrict__ out_tokens) {
+  grid_dependency_wait();
   __shared__ int32_t s_tgt[JET_MAX_NODES];
   __shared__ uint32_t s_match[JET_MAX_NODES / 32];
   __shared__ uint32_t s_best[JET_MAX_NODES / 32];
@@ -176,10 +178,10 @@ extern "C" jet_status jet_tree_accept(const float* logits, int64_t logits_row_st
   const bool vec_ok = aligned(logits, 16) && logits_row_stride % 4 == 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto* partial = static_cast<unsigned long long*>(workspace);
-  argmax_partial_kernel<<<dim3(nchunks, batch * B), kArgThreads, 0, st>>>(
+  launch_dependent(argmax_partial_kernel, dim3(nchunks, batch * B), dim3(kArgThreads), st,
       logits, logits_row_stride, V, B, n_nodes, nchunks, vec_ok, partial);
   const int threads = (B + 31) / 32 * 32;
-  accept_path_kernel<<<batch, threads, 0, st>>>(partial, nchunks, token, parent, depth, anc_mask,
+  launch_dependent(accept_path_kernel, dim3(batch), dim3(threads), st, partial, nchunks, token, parent, depth, anc_mask,
                                                  n_nodes, B, N, tgt_argmax, accept_len, path,
                                                  out_tokens);
   return launch_status();

@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kTopThreads)
 topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
                     int V, int Wc, int nchunks, bool vec_ok,
                     unsigned long long* __restrict__ cand) {
+  grid_dependency_wait();
   const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x;
   const float* row = logp + b * batch_stride + d * depth_stride;
@@ -47,25 +48,35 @@ topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_
     }
   }
 
-  __shared__ unsigned long long warp_best[kTopThreads / 32];
-  __shared__ unsigned long long winner;
-  unsigned long long* out = cand + ((static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk) * Wc;
+  // Every warp first selects the W best of its own 512 elements with warp shuffles alone; one block-wide
+  // barrier later warp 0 selects the block's W best among the warps' candidates.
+  __shared__ unsigned long long warp_cand[kTopThreads / 32][JET_MAX_WIDTH];
+  const int lane = tid & 31, warp = tid >> 5;
   for (int r = 0; r < Wc; ++r) {
     unsigned long long best = 0ull;
 #pragma unroll
     for (int i = 0; i < kTopElems; ++i) best = keys[i] > best ? keys[i] : best;
     best = warp_max_u64(best);
-    if ((tid & 31) == 0) warp_best[tid >> 5] = best;
-    __syncthreads();
-    if (tid < 32) {
-      unsigned long long w = tid < kTopThreads / 32 ? warp_best[tid] : 0ull;
-      w = warp_max_u64(w);
-      if (tid == 0) { winner = w; out[r] = w; }
-    }
-    __syncthreads();
-    const unsigned long long w = winner;
+    if (lane == 0) warp_cand[warp][r] = best;
 #pragma unroll
-    for (int i = 0; i < kTopElems; ++i) if (keys[i] == w) keys[i] = 0ull;   // keys are unique
+    for (int i = 0; i < kTopElems; ++i) if (keys[i] == best) keys[i] = 0ull;   // keys are unique
+  }
+  __syncthreads();
+  if (warp == 0) {
+    constexpr int kWarps = kTopThreads / 32;
+    unsigned long long c[kWarps];           // lane holds candidate `lane` of every warp (lane < Wc)
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) c[w] = lane < Wc ? warp_cand[w][lane] : 0ull;
+    unsigned long long* out = cand + ((static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk) * Wc;
+    for (int r = 0; r < Wc; ++r) {
+      unsigned long long best = 0ull;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) best = c[w] > best ? c[w] : best;
+      best = warp_max_u64(best);
+      if (lane == 0) out[r] = best;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) if (c[w] == best) c[w] = 0ull;
+    }
   }
 }
 
@@ -78,6 +89,7 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
                    int32_t* __restrict__ parent_out, int32_t* __restrict__ depth_out,
                    int32_t* __restrict__ token_out, float* __restrict__ score_out,
                    uint32_t* __restrict__ anc_out, int32_t* __restrict__ n_nodes_out) {
+  grid_dependency_wait();
   __shared__ int32_t s_top_tok[JET_MAX_DEPTH][JET_MAX_WIDTH];
   __shared__ float s_top_lp[JET_MAX_DEPTH][JET_MAX_WIDTH];
   __shared__ int32_t s_parent[JET_MAX_NODES], s_depth[JET_MAX_NODES], s_token[JET_MAX_NODES];
@@ -86,7 +98,6 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   __shared__ int s_n;
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* lp = logp + b * batch_stride;
 
   // ---- merge the per-slice candidates: depth d's W best of nchunks*Wc keys (keys are unique,
   //      so "largest key below the previous winner" walks them in rank order)
@@ -116,7 +127,7 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
       if (lane == 0) {
         const uint32_t t = key_index(best);
         s_top_tok[d][r] = static_cast<int32_t>(t);
-        s_top_lp[d][r] = lp[d * depth_stride + t];   // the stored bits, not the canonicalised key
+        s_top_lp[d][r] = key_value(best);            // the key holds the value itself: no second look-up
       }
       prev = best;
     }
@@ -212,9 +223,9 @@ extern "C" jet_status jet_tree_build(const float* logp, int64_t logp_batch_strid
   const bool vec_ok = aligned(logp, 16) && logp_batch_stride % 4 == 0 && logp_depth_stride % 4 == 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto* cand = static_cast<unsigned long long*>(workspace);
-  topw_partial_kernel<<<dim3(nchunks, N, batch), kTopThreads, 0, st>>>(
+  launch_dependent(topw_partial_kernel, dim3(nchunks, N, batch), dim3(kTopThreads), st,
       logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand);
-  tree_expand_kernel<<<batch, kExpThreads, 0, st>>>(logp, logp_batch_stride, logp_depth_stride,
+  launch_dependent(tree_expand_kernel, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
                                                      root_token, N, Wc, B, nchunks, cand, parent,
                                                      depth, token, score, anc_mask, n_nodes);
   return launch_status();
