@@ -230,6 +230,21 @@ def time_step(st, steps, warmup, use_graph):
     return stream, run
 
 
+def max_over_ranks(value, device, world):
+    """A per-rank duration -> the slowest rank's (what a multi-GPU number is reported as)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_seed(base, rank):
+    """Every rank verifies its own sequence(s): inputs are seeded per rank."""
+    return 1000 * base + rank
+
+
 def bench_jet(args):
     import torch
     import torch.distributed as dist
@@ -246,7 +261,7 @@ def bench_jet(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
     c = workload(args.config)
-    st, info = build_inputs(c, args.config, 1000 * 2 + rank, device)
+    st, info = build_inputs(c, args.config, rank_seed(2, rank), device)
     layers = c["layers"]
 
     stream, run = time_step(st, args.steps, max(args.warmup, 3), not args.no_graph)
@@ -275,10 +290,7 @@ def bench_jet(args):
     barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    t = torch.tensor([ms_total], device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, device, world) / args.steps
     assert int(st.status.item()) == 0, "a bounded device wait expired"
     acc = st.accept_len.cpu().numpy().tolist()
     assert acc == info["planted"], (acc, info["planted"])
@@ -349,10 +361,7 @@ def bench_jet(args):
         e1.record(stream)
         stream.synchronize()
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms_step = float(t.item()) / args.steps
+    e2e_ms_step = max_over_ranks(e0.elapsed_time(e1), device, world) / args.steps
     assert host_out["accept_len"].numpy().tolist() == info["planted"]
 
     if rank != 0:
