@@ -136,6 +136,64 @@ def test_sweep_16k_sampled_rows():
     assert np.abs(np.array([lse[0, h, v] for v, h in rows]) - rlse).max() <= LSE_ERR
 
 
+def test_moe_30b_full_size_sampled_rows():
+    """Largest single-sequence shape (8 query heads per KV head, prefix 32768, 512-node tree, depth 12): the
+    launch configuration the planner picks at full size; the oracle checks a seeded sample of rows."""
+    import jet_harness as H
+    c = CONFIGS["moe_30b"]
+    B, Hq, Hkv, D, L = 512, c["Hq"], c["Hkv"], c["D"], c["L"]
+    rng = np.random.default_rng(5000)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = random_tree(B, rng, max_depth=c["N"])
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0 / np.sqrt(D)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [L],
+                                   x["tree_k"][None], x["tree_v"][None], anc[None], [B], scale)
+    assert st == 0 and not np.isnan(out).any()
+    rows = [(int(rng.integers(0, B)), int(rng.integers(0, Hq))) for _ in range(64)] + [(0, 0), (B - 1, Hq - 1)]
+    ref, rlse = tree_attn_rows_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale,
+                                   rows)
+    got = np.stack([out[0, v, h] for v, h in rows])
+    err = np.abs(got - ref)
+    assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR
+    assert np.abs(np.array([lse[0, h, v] for v, h in rows]) - rlse).max() <= LSE_ERR
+
+
+def test_batched_paged_full_size_sampled_rows():
+    """The serving shape at full size (32 sequences, prefixes 1024..8192, paged, shuffled page table): the
+    configuration in which sequences are launched longest first and CTAs take two query tiles; the oracle
+    checks a seeded sample of rows of the shortest, the longest and one more sequence."""
+    import jet_harness as H
+    c = CONFIGS["batched_paged"]
+    batch, B, Hq, Hkv, D = c["batch"], c["B"], c["Hq"], c["Hkv"], c["D"]
+    rng = np.random.default_rng(4500)
+    seq = rng.integers(c["L_range"][0], c["L_range"][1] + 1, size=batch).astype(np.int32)
+    kp, vp, table = make_paged_cache(rng, seq, 16, Hkv, D, reserve=9)
+    n_nodes = np.full(batch, B, np.int32)
+    n_nodes[3] = 17
+    qs, tks, tvs, ancs = [], [], [], []
+    for b in range(batch):
+        x = make_attn_inputs(rng, B, Hq, Hkv, D, 0)
+        parent, _, _ = random_tree(int(n_nodes[b]), rng, max_depth=c["N"])
+        qs.append(x["q"]); tks.append(x["tree_k"]); tvs.append(x["tree_v"])
+        ancs.append(anc_from_parent(parent, int(n_nodes[b]), B))
+    scale = 1.0 / np.sqrt(D)
+    out, lse, st = H.run_tree_attn(np.stack(qs), kp, vp, table, seq, np.stack(tks), np.stack(tvs), np.stack(ancs),
+                                   n_nodes, scale)
+    assert st == 0 and not np.isnan(out).any()
+    for b in sorted({int(np.argmin(seq)), int(np.argmax(seq)), 3}):
+        n = int(n_nodes[b])
+        kpre = gather_paged_prefix(kp, table[b], int(seq[b]))
+        vpre = gather_paged_prefix(vp, table[b], int(seq[b]))
+        rows = [(int(rng.integers(0, n)), int(rng.integers(0, Hq))) for _ in range(24)] + [(0, 0), (n - 1, Hq - 1)]
+        ref, rlse = tree_attn_rows_ref(qs[b], kpre, vpre, tks[b], tvs[b], ancs[b], n, scale, rows)
+        got = np.stack([out[b, v, h] for v, h in rows])
+        err = np.abs(got - ref)
+        assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR, b
+        assert np.abs(np.array([lse[b, h, v] for v, h in rows]) - rlse).max() <= LSE_ERR
+        assert (out[b, n:] == 0).all()
+
+
 @pytest.mark.parametrize("batch,B,Hq,Hkv,D", [(3, 16, 8, 2, 64), (5, 64, 8, 2, 128), (32, 64, 32, 8, 128)])
 def test_batched_paged_ragged(batch, B, Hq, Hkv, D):
     import jet_harness as H
