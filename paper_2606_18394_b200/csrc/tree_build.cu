@@ -18,65 +18,105 @@ constexpr int kTopThreads = 256;
 constexpr int kTopElems = 16;                        // elements per thread
 constexpr int kTopChunk = kTopThreads * kTopElems;   // vocabulary slice per block
 
+// One block scans a 4096-element slice of one vocabulary row and leaves its W best keys.  Almost every
+// element is dismissed with one compare: an element among a warp's W best is at least as large as the W-th
+// largest of the 32 per-lane maxima (tau), so only elements >= tau become candidates (as ordered 64-bit keys
+// in shared memory); the block then selects its W best among the few candidates.  Exact for any input: with
+// many equal values all of them become candidates and the key order (value, then lowest index) decides.
 __global__ void __launch_bounds__(kTopThreads)
 topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
                     int V, int Wc, int nchunks, bool vec_ok,
                     unsigned long long* __restrict__ cand) {
   grid_dependency_wait();
   const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
   const float* row = logp + b * batch_stride + d * depth_stride;
   const int base = chunk * kTopChunk;
 
-  unsigned long long keys[kTopElems];
-  if (vec_ok && base + kTopChunk <= V) {
+  // element e of this thread has vocabulary index idx_of(e); out-of-range elements are -inf and never candidates
+  float v[kTopElems];
+  const bool vec = vec_ok && base + kTopChunk <= V;
+  auto idx_of = [&](int e) -> int {
+    return vec ? base + ((e >> 2) * kTopThreads + tid) * 4 + (e & 3) : base + e * kTopThreads + tid;
+  };
+  if (vec) {
     const float4* row4 = reinterpret_cast<const float4*>(row + base);
 #pragma unroll
     for (int i = 0; i < kTopElems / 4; ++i) {
-      float4 x = __ldg(row4 + i * kTopThreads + tid);
-      const uint32_t idx = base + (i * kTopThreads + tid) * 4;
-      keys[i * 4 + 0] = make_key(x.x, idx + 0);
-      keys[i * 4 + 1] = make_key(x.y, idx + 1);
-      keys[i * 4 + 2] = make_key(x.z, idx + 2);
-      keys[i * 4 + 3] = make_key(x.w, idx + 3);
+      const float4 x = __ldg(row4 + i * kTopThreads + tid);
+      v[i * 4 + 0] = x.x; v[i * 4 + 1] = x.y; v[i * 4 + 2] = x.z; v[i * 4 + 3] = x.w;
     }
   } else {
 #pragma unroll
     for (int i = 0; i < kTopElems; ++i) {
       const int idx = base + i * kTopThreads + tid;
-      keys[i] = idx < V ? make_key(__ldg(row + idx), idx) : 0ull;
+      v[i] = idx < V ? __ldg(row + idx) : -INFINITY;
     }
   }
 
-  // Every warp first selects the W best of its own 512 elements with warp shuffles alone; one block-wide
-  // barrier later warp 0 selects the block's W best among the warps' candidates.
-  __shared__ unsigned long long warp_cand[kTopThreads / 32][JET_MAX_WIDTH];
-  const int lane = tid & 31, warp = tid >> 5;
-  for (int r = 0; r < Wc; ++r) {
-    unsigned long long best = 0ull;
+  // tau = Wc-th largest of the warp's 32 lane maxima: every lane ranks its maximum (ties by lane) against
+  // the others' with 32 independent shuffles; the lane of rank Wc-1 holds tau
+  float lane_max = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < kTopElems; ++i) best = keys[i] > best ? keys[i] : best;
-    best = warp_max_u64(best);
-    if (lane == 0) warp_cand[warp][r] = best;
+  for (int i = 0; i < kTopElems; ++i) lane_max = fmaxf(lane_max, v[i]);
+  int rank = 0;
 #pragma unroll
-    for (int i = 0; i < kTopElems; ++i) if (keys[i] == best) keys[i] = 0ull;   // keys are unique
+  for (int j = 0; j < 32; ++j) {
+    const float other = __shfl_sync(0xffffffffu, lane_max, j);
+    rank += (other > lane_max || (other == lane_max && j < lane)) ? 1 : 0;
+  }
+  const unsigned holder = __ballot_sync(0xffffffffu, rank == Wc - 1);
+  const float tau = __shfl_sync(0xffffffffu, lane_max, __ffs(holder) - 1);
+
+  __shared__ unsigned long long s_cand[kTopChunk];      // worst case: every element of the slice
+  __shared__ int s_count;
+  if (tid == 0) s_count = 0;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < kTopElems; ++i) {
+    const int idx = idx_of(i);
+    if (v[i] >= tau && idx < V) s_cand[atomicAdd(&s_count, 1)] = make_key(v[i], static_cast<uint32_t>(idx));
   }
   __syncthreads();
-  if (warp == 0) {
-    constexpr int kWarps = kTopThreads / 32;
-    unsigned long long c[kWarps];           // lane holds candidate `lane` of every warp (lane < Wc)
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) c[w] = lane < Wc ? warp_cand[w][lane] : 0ull;
-    unsigned long long* out = cand + ((static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk) * Wc;
-    for (int r = 0; r < Wc; ++r) {
-      unsigned long long best = 0ull;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) best = c[w] > best ? c[w] : best;
-      best = warp_max_u64(best);
-      if (lane == 0) out[r] = best;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) if (c[w] == best) c[w] = 0ull;
+  const int count = s_count;
+
+  // the block's Wc best candidates, in rank order (keys are unique)
+  unsigned long long* out = cand + ((static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk) * Wc;
+  if (count <= kTopThreads) {
+    // usual case: one candidate per thread, ranked against all others (broadcast reads, no serial rounds)
+    if (tid < count) {
+      const unsigned long long mine = s_cand[tid];
+      int rank = 0;
+      for (int j = 0; j < count; ++j) rank += s_cand[j] > mine ? 1 : 0;
+      if (rank < Wc) out[rank] = mine;
     }
+    if (tid >= count && tid < Wc) out[tid] = 0ull;          // fewer candidates than Wc: no key
+    return;
+  }
+  // many equal values: warp 0 alone walks the candidates in rank order
+  if (tid >= 32) return;
+  constexpr int kHeld = 8;                       // candidates a lane keeps in registers (usual case)
+  unsigned long long held[kHeld];
+  const bool in_regs = count <= 32 * kHeld;
+  if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < kHeld; ++i) held[i] = lane + 32 * i < count ? s_cand[lane + 32 * i] : 0ull;
+  }
+  unsigned long long prev = ~0ull;
+  for (int r = 0; r < Wc; ++r) {
+    unsigned long long best = 0ull;
+    if (in_regs) {
+#pragma unroll
+      for (int i = 0; i < kHeld; ++i) if (held[i] < prev && held[i] > best) best = held[i];
+    } else {
+      for (int i = lane; i < count; i += 32) {
+        const unsigned long long k = s_cand[i];
+        if (k < prev && k > best) best = k;
+      }
+    }
+    best = warp_max_u64(best);
+    if (lane == 0) out[r] = best;
+    prev = best;
   }
 }
 
