@@ -120,6 +120,55 @@ topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_
   }
 }
 
+// Algorithm 1 in one warp.  The pending queue lives in registers: node u is kept by lane u % 32 in register
+// u / 32 as a key (score, lowest index first, depth in the low byte), so a pop is a register maximum plus one
+// warp reduction, and the popped node's score and depth come out of the key itself.  kSlots = registers per
+// lane (32 * kSlots >= B); the instruction count of a pop grows with it, hence the template.
+template <int kSlots>
+__device__ __forceinline__ int expand_tree(int lane, int N, int Wc, int B, int root, const float (*top_lp)[JET_MAX_WIDTH],
+                                           const int32_t (*top_tok)[JET_MAX_WIDTH], int32_t* s_parent,
+                                           int32_t* s_depth, int32_t* s_token, float* s_score) {
+  unsigned long long q[kSlots];
+#pragma unroll
+  for (int i = 0; i < kSlots; ++i) q[i] = 0ull;
+  auto queue_key = [](float score, int node, int dep) -> unsigned long long {
+    return (static_cast<unsigned long long>(f32_order(score)) << 32) |
+           (static_cast<unsigned long long>(0xFFFFFFu - static_cast<uint32_t>(node)) << 8) |
+           static_cast<unsigned long long>(dep);
+  };
+  if (lane == 0) {
+    s_parent[0] = -1; s_depth[0] = 0; s_token[0] = root; s_score[0] = 0.0f;
+    q[0] = queue_key(0.0f, 0, 0);
+  }
+  int n = 1;
+  while (n < B) {
+    unsigned long long best = 0ull;
+#pragma unroll
+    for (int i = 0; i < kSlots; ++i) best = q[i] > best ? q[i] : best;
+    best = warp_max_u64(best);
+    if (best == 0ull) break;                        // nothing pending
+    const int v = static_cast<int>(0xFFFFFFu - (static_cast<uint32_t>(best >> 8) & 0xFFFFFFu));
+    const int d = static_cast<int>(best & 0xFFull);
+    const float sv = key_value(best);
+#pragma unroll
+    for (int i = 0; i < kSlots; ++i) if (q[i] == best) q[i] = 0ull;      // popped (only its keeper matches)
+    if (d < N) {
+      const int cnt = min(Wc, B - n);
+      const int j = (lane - n) & 31;                // child rank whose node n + j this lane keeps
+      if (j < cnt) {
+        const int u = n + j;
+        const float s = __fadd_rn(sv, top_lp[d][j]);
+        s_parent[u] = v; s_depth[u] = d + 1; s_token[u] = top_tok[d][j]; s_score[u] = s;
+        const unsigned long long key = queue_key(s, u, d + 1);
+#pragma unroll
+        for (int i = 0; i < kSlots; ++i) if (i == (u >> 5)) q[i] = key;
+      }
+      n += cnt;
+    }
+  }
+  return n;
+}
+
 constexpr int kExpThreads = 256;
 
 __global__ void __launch_bounds__(kExpThreads)
@@ -134,7 +183,6 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   __shared__ float s_top_lp[JET_MAX_DEPTH][JET_MAX_WIDTH];
   __shared__ int32_t s_parent[JET_MAX_NODES], s_depth[JET_MAX_NODES], s_token[JET_MAX_NODES];
   __shared__ float s_score[JET_MAX_NODES];
-  __shared__ unsigned long long s_qkey[JET_MAX_NODES];
   __shared__ int s_n;
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -174,36 +222,15 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   }
   __syncthreads();
 
-  // ---- Algorithm 1: one warp, pending queue = keys (score, lowest index first) in shared memory
+  // ---- Algorithm 1: one warp, queue in registers (as many per lane as the budget needs)
   if (warp == 0) {
-    if (lane == 0) {
-      s_parent[0] = -1; s_depth[0] = 0; s_token[0] = root_token[b]; s_score[0] = 0.0f;
-      s_qkey[0] = make_key(0.0f, 0);
-    }
-    __syncwarp();
-    int n = 1;
-    while (n < B) {
-      unsigned long long best = 0ull;
-      for (int i = lane; i < n; i += 32) { const unsigned long long k = s_qkey[i]; best = k > best ? k : best; }
-      best = warp_max_u64(best);
-      if (best == 0ull) break;                        // nothing pending
-      const int v = static_cast<int>(key_index(best));
-      const int d = s_depth[v];
-      const float sv = s_score[v];
-      __syncwarp();
-      if (lane == 0) s_qkey[v] = 0ull;                // popped
-      if (d < N) {
-        const int cnt = min(Wc, B - n);
-        if (lane < cnt) {
-          const int u = n + lane;
-          const float s = __fadd_rn(sv, s_top_lp[d][lane]);
-          s_parent[u] = v; s_depth[u] = d + 1; s_token[u] = s_top_tok[d][lane]; s_score[u] = s;
-          s_qkey[u] = make_key(s, u);
-        }
-        n += cnt;
-      }
-      __syncwarp();
-    }
+    const int root = root_token[b];
+    int n;
+    if (B <= 32) n = expand_tree<1>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
+    else if (B <= 64) n = expand_tree<2>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
+    else if (B <= 128) n = expand_tree<4>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
+    else if (B <= 256) n = expand_tree<8>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
+    else n = expand_tree<JET_MAX_NODES / 32>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
     if (lane == 0) s_n = n;
   }
   __syncthreads();
