@@ -114,6 +114,7 @@ JET_API jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride, 
  *                when contiguous.
  *   max_seq_len  host value, >= every seq_len[b]; sizes the grid and, when
  *                contiguous, bounds the rows per sequence.
+ *   softmax_scale  positive and finite (1/sqrt(D) in the paper), else JET_ERR_INVALID_ARG
  *   seq_len      i32 [batch] prefix lengths (0 allowed)
  *   tree_k, tree_v  bf16 [batch, B, Hkv, D]
  *   out          bf16 [batch, B, Hq, D]

@@ -11,7 +11,9 @@ from .jet_oracle import (  # noqa: F401
     bf16_bits_to_f64,
     gather_paged_prefix,
     kv_compact_ref,
+    target_probs_ref,
     tree_accept_ref,
+    tree_accept_sample_ref,
     tree_attn_ref,
     tree_attn_rows_ref,
     tree_build_ref,

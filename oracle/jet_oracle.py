@@ -15,6 +15,10 @@ Each function follows one passage of the paper:
   and the target prediction at its last node is the correction token.
 * ``kv_compact_ref``   -- "the accepted path is committed" (Appendix E): the
   K/V rows of the accepted path are copied behind the prefix.
+* ``tree_accept_sample_ref`` -- the non-greedy acceptance rule of Section 3.3
+  (Eq. nongreedy_specdec): along every branch a draft token is accepted with
+  probability min(1, p/q); a correction token is sampled from the target where
+  the accepted prefix ends.
 
 Nothing here is blocked, fused or reordered; loops are literal so the code can
 be checked against the paper by eye.  Readings taken where the paper is silent
@@ -31,7 +35,13 @@ chains, the ancestor-bitmask formulation and planted paths for
 ``tree_accept_ref``; attention-after-commit round trip for ``kv_compact_ref``.
 The tie-break conventions themselves have no counterpart to be checked
 against (the authors' code is not available): parity unpinned for tie-breaks
-only.
+only.  ``tree_accept_sample_ref`` is pinned by the defining property of
+speculative sampling (on a chain whose tokens are drawn from the draft
+distribution the emitted token is distributed exactly as the target's), the
+closed-form expected accepted length, and the q == p / disjoint-support
+special cases; its reading of the rule for several rejected siblings (the
+single-draft residual max(0, p - q)) has no counterpart to be checked against:
+parity unpinned for that reading only.
 """
 from __future__ import annotations
 
@@ -296,6 +306,98 @@ def tree_accept_ref(logits, token, parent, depth, n_nodes, N) -> dict:
         out_tokens[t - 1] = token[chain[t]]
     out_tokens[best_len] = tgt[best_end]
     return dict(tgt=tgt, accept_len=best_len, end_node=best_end, path=path, out_tokens=out_tokens)
+
+
+# --------------------------------------------------------------------------
+# O3b  non-greedy acceptance (Section 3.3, Eq. nongreedy_specdec)
+# --------------------------------------------------------------------------
+def target_probs_ref(logits_row, temperature: float) -> np.ndarray:
+    """softmax(logits / temperature) of one row in fp64."""
+    z = np.asarray(logits_row, dtype=np.float64) / float(temperature)
+    z = z - z.max()
+    e = np.exp(z)
+    return e / e.sum()
+
+
+def tree_accept_sample_ref(logits, temperature, draft_logp, token, parent, depth, n_nodes, N,
+                           u_accept, u_sample) -> dict:
+    """Non-greedy tree acceptance for one sequence.
+
+    ``logits`` [B,V] fp32: row v is the target's next-token logits after node
+    v; p_v = softmax(row / temperature).  ``draft_logp`` [N,V]: row d is the
+    draft's log-distribution for the children of depth-d nodes; q_d = exp(row).
+    ``u_accept`` [B] and ``u_sample`` (scalar) are uniform numbers in [0,1)
+    supplied by the caller (the method's randomness is an input).
+
+    For every node v >= 1 with parent w and token y:
+        alpha_v = min(1, p_w(y) / q_{depth(w)}(y)),   A_v = [u_accept[v] < alpha_v]
+    (alpha_v = 1 where q is 0).  A node is accepted iff A holds for it and all
+    its ancestors below the root; the deepest accepted node v* ends the prefix
+    (several at that depth: smallest index), accept_len = depth[v*].
+
+    Correction token at v* (depth d): if v* has children in the tree (all of
+    them were rejected) it is drawn from the residual max(0, p_{v*} - q_d)
+    normalised -- the single-draft rule; a residual without mass falls back to
+    p_{v*} -- and from p_{v*} itself if v* is a leaf.  Drawing = inverse CDF in
+    vocabulary order: the first token whose cumulative mass exceeds
+    u_sample * total.
+    """
+    logits = np.asarray(logits)
+    draft_logp = np.asarray(draft_logp, dtype=np.float64)
+    B = len(token)
+    alpha = np.ones(B, dtype=np.float64)
+    ok = np.zeros(B, dtype=bool)
+    ok[0] = True
+    probs = {}
+
+    def p_of(v):
+        if v not in probs:
+            probs[v] = target_probs_ref(logits[v], temperature)
+        return probs[v]
+
+    for v in range(1, n_nodes):
+        w = int(parent[v])
+        y = int(token[v])
+        q = float(np.exp(draft_logp[int(depth[w]), y]))
+        pw = float(p_of(w)[y])
+        alpha[v] = 1.0 if q == 0.0 else min(1.0, pw / q)
+        ok[v] = bool(u_accept[v] < alpha[v])
+
+    accepted = np.zeros(B, dtype=bool)
+    accepted[0] = True
+    for v in range(1, n_nodes):                      # parent[v] < v: parents come first
+        accepted[v] = ok[v] and accepted[int(parent[v])]
+    best_end, best_len = 0, 0
+    for v in range(n_nodes):
+        if accepted[v] and int(depth[v]) > best_len:
+            best_end, best_len = v, int(depth[v])
+
+    has_child = any(int(parent[v]) == best_end for v in range(1, n_nodes))
+    p_end = p_of(best_end)
+    dist = p_end
+    if has_child:
+        resid = np.maximum(0.0, p_end - np.exp(draft_logp[int(depth[best_end])]))
+        if resid.sum() > 0.0:
+            dist = resid
+    cdf = np.cumsum(dist)
+    target = float(u_sample) * float(cdf[-1])
+    corr = int(np.searchsorted(cdf, target, side="right"))       # first index with cdf > target
+    corr = min(corr, len(dist) - 1)
+
+    chain = []
+    v = best_end
+    while v != -1:
+        chain.append(v)
+        v = int(parent[v])
+    chain.reverse()
+    path = np.full(N + 1, -1, dtype=np.int32)
+    out_tokens = np.full(N + 1, -1, dtype=np.int32)
+    path[: len(chain)] = chain
+    for t in range(1, len(chain)):
+        out_tokens[t - 1] = token[chain[t]]
+    out_tokens[best_len] = corr
+    return dict(alpha=alpha, ok=ok, accept_len=best_len, end_node=best_end, path=path, out_tokens=out_tokens,
+                correction=corr, dist=dist, cdf=cdf, residual_used=bool(has_child and dist is not p_end))
 
 
 # --------------------------------------------------------------------------

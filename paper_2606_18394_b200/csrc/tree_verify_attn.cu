@@ -56,7 +56,7 @@ struct AttnParams {
   int nsplit, n_mgroups, n_units;
   int via_global;     // key slices exchange their rows through the workspace instead of a cluster
   int* counters;      // via_global: [2][units * MT] arrival / departure counts, zero between calls
-  uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D fp32 + log2-sum-exp]
+  uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D bf16 + log2-sum-exp (fp32) + pad]
   float scale_log2;   // softmax_scale * log2(e)
 #ifdef JET_TRACE
   long long* trace;   // 64 clock64() samples per CTA
@@ -358,7 +358,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   auto epilogue = [&](auto sm_side) {
     constexpr bool kSm = decltype(sm_side)::value;
     // =============================================================== epilogue
-    // One round per query tile: its softmax threads stage their normalised rows (D fp32 + log2-sum-exp)
+    // One round per query tile: its softmax threads stage their normalised rows (D bf16 + log2-sum-exp)
     // in shared memory.  With key slices every CTA then sends each owner slice its block of rows with
     // one bulk copy credited to the owner's kRecv barrier; the owner combines the S blocks.  Without
     // slices the CTA "combines" its own staged rows.  Either way the output rows leave as coalesced
@@ -1171,6 +1171,8 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
     return JET_ERR_INVALID_ARG;
   if (max_seq_len > 0 && (!k_cache || !v_cache)) return JET_ERR_INVALID_ARG;
   const int G = Hq / Hkv;
+  // the running reference maximum is kept in raw score units, which needs a positive, finite scale
+  if (!(softmax_scale > 0.0f) || !(softmax_scale < INFINITY)) return JET_ERR_INVALID_ARG;
   if (D != 64 && D != 128) return JET_ERR_UNSUPPORTED;
   if (G > 16 || (G & (G - 1)) != 0) return JET_ERR_UNSUPPORTED;
   const bool paged = page_table != nullptr;

@@ -270,6 +270,8 @@ def test_argument_errors():
     assert jet.jet_tree_verify_attn(**{**args, "B": 513}) == jet.JET_ERR_INVALID_ARG
     assert jet.jet_tree_verify_attn(**{**args, "q": None}) == jet.JET_ERR_INVALID_ARG
     assert jet.jet_tree_verify_attn(**{**args, "workspace": None}) == jet.JET_ERR_WORKSPACE
+    assert jet.jet_tree_verify_attn(**{**args, "softmax_scale": -0.1}) == jet.JET_ERR_INVALID_ARG
+    assert jet.jet_tree_verify_attn(**{**args, "softmax_scale": float("nan")}) == jet.JET_ERR_INVALID_ARG
     assert jet.jet_tree_verify_attn(**{**args, "page_table": i32, "page_size": 32, "max_pages_per_seq": 4,
                                        "num_pages": 4}) == jet.JET_ERR_UNSUPPORTED
 
