@@ -201,6 +201,44 @@ JET_API jet_status jet_tree_accept_static(const float* logits, int64_t logits_ro
                                   int32_t* out_tokens, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * jet_tree_accept_sample -- non-greedy tree acceptance (Section 3.3, the
+ * rejection-sampling rule of Eq. nongreedy_specdec applied along every branch).
+ *
+ * Target distribution of row v: p_v = softmax(logits[v,:] / temperature).
+ * Draft distribution for the children of a depth-d node: q_d = exp(draft_logp[b,d,:]).
+ * For every node v >= 1 with parent w and token y:
+ *     alpha_v = min(1, p_w(y) / q_depth(w)(y))   (1 where q is 0),
+ *     the node passes iff u_accept[b,v] < alpha_v.
+ * The accepted prefix ends at the deepest node all of whose branch passes (several
+ * at that depth: lowest index); accept_len = its depth, path / out_tokens as in
+ * jet_tree_accept.  The correction token (out_tokens[accept_len]) is drawn by
+ * inverse CDF in vocabulary order with u_sample[b] -- the first token whose
+ * cumulative mass exceeds u_sample * total -- from max(0, p - q) at the end node if
+ * that node has children in the tree (all rejected; a residual without mass falls
+ * back to p), and from p itself if it is a leaf.  The random numbers are inputs:
+ * uniform in [0,1), one per node and one per sequence.
+ *
+ *   logits       fp32 [batch*B rows, V], row stride in elements
+ *   draft_logp   fp32 [batch, N, V] log-probabilities (strides in elements)
+ *   u_accept     fp32 [batch, B]; u_sample fp32 [batch]
+ *   alpha        optional out fp32 [batch, B] (0 for padding rows, 1 for the root)
+ *   accept_len   i32 [batch]; path, out_tokens i32 [batch, N+1], -1 padded
+ * Precision: fp32 throughout, cumulative masses in fp64; a draw or a test that
+ * falls within rounding of its threshold may differ from an fp64 evaluation.
+ * temperature must be positive and finite.
+ */
+JET_API size_t jet_tree_accept_sample_workspace_bytes(int batch, int B, int V);
+
+JET_API jet_status jet_tree_accept_sample(const float* logits, int64_t logits_row_stride, float temperature,
+                                  const float* draft_logp, int64_t logp_batch_stride,
+                                  int64_t logp_depth_stride, const int32_t* token, const int32_t* parent,
+                                  const int32_t* depth, const uint32_t* anc_mask, const int32_t* n_nodes,
+                                  const float* u_accept, const float* u_sample, int batch, int B, int V,
+                                  int N, float* alpha, int32_t* accept_len, int32_t* path,
+                                  int32_t* out_tokens, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
+/* ---------------------------------------------------------------------------
  * jet_kv_compact -- commit of the accepted path (Appendix E: "the accepted path
  * is committed"): for every layer l, sequence b and i in [0, accept_len[b]] the
  * K and V rows of tree node path[b,i] are copied to cache position

@@ -15,6 +15,8 @@ from .binding import (  # noqa: F401
     exported_symbols,
     jet_kv_compact,
     jet_tree_accept,
+    jet_tree_accept_sample,
+    jet_tree_accept_sample_workspace_bytes,
     jet_tree_accept_static,
     jet_tree_accept_workspace_bytes,
     jet_tree_build,

@@ -37,6 +37,9 @@ _SIGNATURES = {
                                      _vp, _vp, _sz, _vp]),
     "jet_tree_accept_static": (_c.c_int32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp,
                                             _vp, _vp]),
+    "jet_tree_accept_sample_workspace_bytes": (_sz, [_i, _i, _i]),
+    "jet_tree_accept_sample": (_c.c_int32, [_vp, _i64, _f, _vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                            _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_kv_compact": (_c.c_int32, [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _i, _i, _vp, _vp, _vp, _i, _i,
                                     _i, _i, _i, _i, _vp]),
 }
@@ -160,6 +163,26 @@ def jet_tree_accept_static(logits, logits_row_stride, token, parent, depth, anc_
                                        _p(accept_len), _p(path), _p(out_tokens), _stream(stream))
     if check:
         _check(st, "jet_tree_accept_static")
+    return st
+
+
+def jet_tree_accept_sample_workspace_bytes(batch, B, V) -> int:
+    return load().jet_tree_accept_sample_workspace_bytes(batch, B, V)
+
+
+def jet_tree_accept_sample(logits, logits_row_stride, temperature, draft_logp, logp_batch_stride,
+                           logp_depth_stride, token, parent, depth, anc_mask, n_nodes, u_accept, u_sample,
+                           batch, B, V, N, alpha, accept_len, path, out_tokens, workspace, workspace_bytes=None,
+                           stream=None, check=True):
+    wb = workspace_bytes if workspace_bytes is not None else (workspace.numel() * workspace.element_size()
+                                                              if workspace is not None else 0)
+    st = load().jet_tree_accept_sample(_p(logits), logits_row_stride, temperature, _p(draft_logp),
+                                       logp_batch_stride, logp_depth_stride, _p(token), _p(parent), _p(depth),
+                                       _p(anc_mask), _p(n_nodes), _p(u_accept), _p(u_sample), batch, B, V, N,
+                                       _p(alpha), _p(accept_len), _p(path), _p(out_tokens), _p(workspace), wb,
+                                       _stream(stream))
+    if check:
+        _check(st, "jet_tree_accept_sample")
     return st
 
 

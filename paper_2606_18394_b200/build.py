@@ -9,7 +9,8 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libjet.so")
-SOURCES = ["jet_api.cu", "tree_build.cu", "tree_verify_attn.cu", "tree_accept.cu", "kv_compact.cu"]
+SOURCES = ["jet_api.cu", "tree_build.cu", "tree_verify_attn.cu", "tree_accept.cu", "tree_accept_sample.cu",
+           "kv_compact.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

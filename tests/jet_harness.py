@@ -66,6 +66,26 @@ def run_tree_accept(logits, token, parent, depth, anc_mask, n_nodes, N):
                 out_tokens=toks.cpu().numpy())
 
 
+def run_tree_accept_sample(logits, temperature, draft_logp, token, parent, depth, anc_mask, n_nodes, N, u_accept,
+                           u_sample):
+    """logits [batch,B,V], draft_logp [batch,N,V], u_accept [batch,B], u_sample [batch]; returns numpy arrays."""
+    batch, B, V = logits.shape
+    alpha = torch.full((batch, B), -7.0, dtype=torch.float32, device=DEV)
+    acc = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
+    path = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
+    toks = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
+    ws = workspace(jet.jet_tree_accept_sample_workspace_bytes(batch, B, V))
+    jet.jet_tree_accept_sample(dev(logits), V, float(temperature), dev(draft_logp.astype(np.float32)), N * V, V,
+                               dev(token.astype(np.int32)), dev(parent.astype(np.int32)),
+                               dev(depth.astype(np.int32)), dev(anc_mask.view(np.int32)),
+                               dev(np.asarray(n_nodes, dtype=np.int32)), dev(u_accept.astype(np.float32)),
+                               dev(np.asarray(u_sample, dtype=np.float32)), batch, B, V, N, alpha, acc, path,
+                               toks, ws)
+    torch.cuda.synchronize()
+    return dict(alpha=alpha.cpu().numpy(), accept_len=acc.cpu().numpy(), path=path.cpu().numpy(),
+                out_tokens=toks.cpu().numpy())
+
+
 def run_kv_compact(tree_k, tree_v, k_cache, v_cache, page_table, path, accept_len, seq_len, N):
     """bf16-bit numpy arrays laid out as the oracle's kv_compact_ref takes them."""
     layers, batch, B, Hkv, D = tree_k.shape
