@@ -4,12 +4,17 @@
 //   row_lse_partial_kernel  grid (slices, batch*B): one pass over the target logits; every block
 //                           leaves the maximum and the sum of exp((x - max) / T) of one 8192-entry
 //                           slice of one row in the workspace.  Padding rows are not read.
-//   accept_sample_kernel    grid (batch), 512 threads: finishes the rows' log-sum-exp, computes
+//   accept_sample_kernel    one cluster of 8 CTAs per sequence, 1024 threads each: finishes the rows' log-sum-exp, computes
 //                           alpha_v = min(1, p_parent(token_v) / q_depth(token_v)) and the accept
 //                           bit u_v < alpha_v for every node, picks the deepest node whose whole
 //                           branch is accepted, then draws the correction token at that node by
 //                           inverse CDF in vocabulary order (residual max(0, p - q) if the node has
-//                           rejected children, p itself if it is a leaf).
+//                           rejected children, p itself if it is a leaf).  Every CTA of the cluster
+//                           repeats the (small) per-node part; the pass over the vocabulary that sums
+//                           the masses is split between the CTAs, which leave their sums in the shared
+//                           memory of CTA 0; CTA 0 locates the token.
+#include <cooperative_groups.h>
+
 #include "jet_common.cuh"
 
 namespace jet {
@@ -18,7 +23,10 @@ namespace {
 constexpr int kLseThreads = 256;
 constexpr int kLseElems = 32;
 constexpr int kLseChunk = kLseThreads * kLseElems;
-constexpr int kSampleThreads = 512;
+constexpr int kSampleThreads = 1024;
+constexpr int kSampleStep = 128;          // vocabulary entries a warp handles per step (4 per lane)
+constexpr int kSampleCluster = 8;         // CTAs per sequence
+constexpr int kMaxStepsTotal = 4096;      // 128-entry steps per row: vocabularies up to 524288 entries
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float warp_max_f(float x) {
@@ -99,16 +107,19 @@ accept_sample_kernel(const float2* __restrict__ partial, int nchunks, const floa
                      const int32_t* __restrict__ token, const int32_t* __restrict__ parent,
                      const int32_t* __restrict__ depth, const uint32_t* __restrict__ anc_mask,
                      const int32_t* __restrict__ n_nodes, const float* __restrict__ u_accept,
-                     const float* __restrict__ u_sample, int B, int V, int N, float* __restrict__ alpha_out,
+                     const float* __restrict__ u_sample, int B, int V, int N, bool vec_rows, float* __restrict__ alpha_out,
                      int32_t* __restrict__ accept_len, int32_t* __restrict__ path,
                      int32_t* __restrict__ out_tokens) {
   grid_dependency_wait();
   __shared__ float s_max[JET_MAX_NODES], s_lnsum[JET_MAX_NODES];      // per row: max, ln sum exp((x - max) / T)
   __shared__ uint32_t s_ok[JET_MAX_NODES / 32], s_best[kSampleThreads / 32], s_end_row[JET_MAX_NODES / 32];
-  __shared__ int s_end, s_has_child, s_pick_warp, s_token;
-  __shared__ double s_wsum[kSampleThreads / 32], s_before;
+  __shared__ int s_end, s_has_child, s_pick_warp, s_pick_step, s_token;
+  __shared__ double s_step[kMaxStepsTotal], s_before, s_target;      // CTA 0: mass of every 128-entry step, vocabulary order
 
-  const int b = blockIdx.x, v = threadIdx.x, lane = v & 31, warp = v >> 5;
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = static_cast<int>(cluster.block_rank());
+  const int b = blockIdx.x / kSampleCluster, v = threadIdx.x, lane = v & 31, warp = v >> 5;
   const int n = min(n_nodes[b], B);
   const int words = (B + 31) / 32;
   const size_t o = static_cast<size_t>(b) * B;
@@ -147,7 +158,7 @@ accept_sample_kernel(const float2* __restrict__ partial, int nchunks, const floa
   }
   if (alpha_out && v < B) alpha_out[o + v] = live ? alpha : 0.0f;
   const uint32_t okbits = __ballot_sync(0xffffffffu, ok);
-  if (lane == 0 && warp < JET_MAX_NODES / 32) s_ok[warp] = okbits;
+  if (lane == 0 && warp < JET_MAX_NODES / 32) s_ok[warp] = okbits;      // threads beyond the budget hold no node
   __syncthreads();
 
   // ---- deepest node whose branch is accepted throughout (ties -> lowest index)
@@ -174,85 +185,147 @@ accept_sample_kernel(const float2* __restrict__ partial, int nchunks, const floa
   const bool residual = s_has_child != 0;
 
   // ---- correction token: inverse CDF over the vocabulary of r(x) = max(0, p(x) - q(x)) (or p(x)).
-  //      Every warp owns a contiguous range of the vocabulary; pass 1 sums the ranges, pass 2 walks the range
-  //      that contains the target mass.  If the residual has no mass the draw falls back to p.
+  //      Every warp owns a contiguous range of the vocabulary and walks it in steps of 128 entries (4 per
+  //      lane), keeping the mass of every step (fp64) in shared memory; one thread then finds the warp and
+  //      the step that contain the target mass, and that warp recomputes the one step to locate the token.
+  //      If the residual has no mass the draw falls back to p.
   const float* xrow = logits + static_cast<int64_t>(o + end) * row_stride;
   const float* qrow = lp + static_cast<int64_t>(a) * logp_depth_stride;      // only read when the node has children (a < N)
   const float m_e = s_max[end], ln_e = s_lnsum[end];
   constexpr int kWarps = kSampleThreads / 32;
-  const int per_warp = ((V + kWarps - 1) / kWarps + 31) / 32 * 32;
-  const int lo = warp * per_warp, hi = min(V, lo + per_warp);
-  auto mass = [&](int idx, bool use_residual) -> float {
-    const float pe = expf((xrow[idx] - m_e) * inv_t - ln_e);
-    if (!use_residual) return pe;
-    return fmaxf(0.0f, pe - expf(qrow[idx]));
-  };
-  bool use_residual = residual;
-  int picked = -1;
-  for (int attempt = 0; attempt < 2 && picked < 0; ++attempt) {
-    double part = 0.0;
-    for (int idx = lo + lane; idx < hi; idx += 32) part += static_cast<double>(mass(idx, use_residual));
-    part = warp_sum_d(part);
-    if (lane == 0) s_wsum[warp] = part;
-    __syncthreads();
-    if (v == 0) {
-      double total = 0.0;
-      for (int w = 0; w < kWarps; ++w) total += s_wsum[w];
-      s_pick_warp = -1;
-      s_token = -1;
-      if (total > 0.0) {
-        const double target = static_cast<double>(u_sample[b]) * total;
-        double cum = 0.0;
-        int pick = -1;
-        for (int w = 0; w < kWarps; ++w) {
-          if (s_wsum[w] > 0.0) {
-            pick = w;                                  // last range with mass, unless an earlier one exceeds the target
-            if (cum + s_wsum[w] > target) break;
-          }
-          cum += s_wsum[w];
-        }
-        // cum = mass before range `pick` (ranges after the break are not added)
-        double before = 0.0;
-        for (int w = 0; w < pick; ++w) before += s_wsum[w];
-        s_before = before;
-        s_pick_warp = pick;
-        s_wsum[0] = target;                            // reuse: the target mass for pass 2
+  const int total_steps = (V + kSampleStep - 1) / kSampleStep;              // host checks <= kMaxStepsTotal
+  const int steps = (total_steps + kWarps * kSampleCluster - 1) / (kWarps * kSampleCluster);      // per warp
+  const int first_step = (rank * kWarps + warp) * steps;                    // this warp's steps, vocabulary order
+  const bool vec = vec_rows;
+  // masses of the 4 entries of this lane in step `g` (global step index)
+  auto masses = [&](int g, bool use_residual, float (&mval)[4]) {
+    const int idx = g * kSampleStep + lane * 4;
+    float x4[4], q4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (vec && idx + 3 < V) {
+      const float4 t = *reinterpret_cast<const float4*>(xrow + idx);
+      x4[0] = t.x; x4[1] = t.y; x4[2] = t.z; x4[3] = t.w;
+      if (use_residual) {
+        const float4 u4 = *reinterpret_cast<const float4*>(qrow + idx);
+        q4[0] = u4.x; q4[1] = u4.y; q4[2] = u4.z; q4[3] = u4.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        x4[j] = idx + j < V ? xrow[idx + j] : -INFINITY;
+        if (use_residual) q4[j] = idx + j < V ? qrow[idx + j] : -INFINITY;
       }
     }
-    __syncthreads();
-    if (s_pick_warp < 0) {                             // no mass: fall back to the target distribution itself
-      use_residual = false;
-      __syncthreads();
-      continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float pe = expf((x4[j] - m_e) * inv_t - ln_e);
+      mval[j] = use_residual ? fmaxf(0.0f, pe - expf(q4[j])) : pe;
     }
-    if (warp == s_pick_warp) {
-      const double target = s_wsum[0];
-      double run = s_before;
-      int found = -1, last_pos = -1;
-      for (int start = lo; start < hi && found < 0; start += 32) {
-        const int idx = start + lane;
-        const float mval = idx < hi ? mass(idx, use_residual) : 0.0f;
-        // inclusive prefix sum over the warp
-        double pre = static_cast<double>(mval);
+  };
+  double* step0 = cluster.map_shared_rank(&s_step[0], 0);      // the step table lives in CTA 0
+  cluster.sync();                                              // every CTA of the cluster is running
+  bool use_residual = residual;
+  int picked = -1;
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    for (int st = 0; st < steps; ++st) {
+      const int g = first_step + st;
+      if (g < total_steps) {
+        float mval[4];
+        masses(g, use_residual, mval);
+        const double part = warp_sum_d(static_cast<double>(mval[0]) + mval[1] + mval[2] + mval[3]);
+        if (lane == 0) step0[g] = part;
+      }
+    }
+    cluster.sync();                                            // the table is complete
+    bool retry = false;
+    if (rank == 0) {
+      if (warp == 0) {
+        // lane i: mass of a contiguous run of steps; inclusive scan over the lanes = cumulative mass
+        const int per_lane = (total_steps + 31) / 32;
+        const int s_lo = lane * per_lane, s_hi = min(total_steps, s_lo + per_lane);
+        double tot_l = 0.0;
+        for (int g = s_lo; g < s_hi; ++g) tot_l += s_step[g];
+        double cum_l = tot_l;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, cum_l, off);
+          if (lane >= off) cum_l += up;
+        }
+        const double total = __shfl_sync(0xffffffffu, cum_l, 31);
+        const double target = static_cast<double>(u_sample[b]) * total;
+        // the run that holds the target: first with mass whose cumulative mass exceeds it, else the last with mass
+        const unsigned has = __ballot_sync(0xffffffffu, tot_l > 0.0);
+        const unsigned over = __ballot_sync(0xffffffffu, tot_l > 0.0 && cum_l > target);
+        const int pl = over ? __ffs(over) - 1 : (has ? 31 - __clz(has) : -1);
+        int ps = -1;
+        double before = 0.0;
+        if (lane == pl) {                                      // walk that run step by step
+          double run = cum_l - tot_l;
+          int last_step = -1;
+          double last_before = 0.0;
+          for (int g = s_lo; g < s_hi; ++g) {
+            const double m = s_step[g];
+            if (m > 0.0) {
+              last_step = g; last_before = run;
+              if (run + m > target) { ps = g; before = run; break; }
+            }
+            run += m;
+          }
+          if (ps < 0) { ps = last_step; before = last_before; }
+          s_pick_step = ps;
+          s_before = before;
+          s_target = target;
+        }
+        if (lane == 0) { s_token = -1; if (pl < 0) s_pick_step = -1; }
+      }
+      __syncthreads();
+      if (s_pick_step < 0) {
+        retry = true;                                          // no mass: fall back to the target distribution itself
+      } else if (warp == 0) {
+        float mval[4];
+        masses(s_pick_step, use_residual, mval);
+        const double mine = static_cast<double>(mval[0]) + mval[1] + mval[2] + mval[3];
+        double pre = mine;                                     // inclusive prefix sum over the lanes
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
           const double up = __shfl_up_sync(0xffffffffu, pre, off);
           if (lane >= off) pre += up;
         }
-        const bool hit = mval > 0.0f && run + pre > target;
-        const unsigned hits = __ballot_sync(0xffffffffu, hit);
-        const unsigned pos = __ballot_sync(0xffffffffu, mval > 0.0f);
-        if (pos) last_pos = start + 31 - __clz(pos);
-        if (hits) found = start + __ffs(hits) - 1;
-        run += __shfl_sync(0xffffffffu, pre, 31);
+        double run = s_before + pre - mine;                    // mass before this lane's entries
+        int found = -1, last_pos = -1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          run += static_cast<double>(mval[j]);
+          if (mval[j] > 0.0f) {
+            last_pos = j;
+            if (found < 0 && run > s_target) found = j;
+          }
+        }
+        const unsigned hits = __ballot_sync(0xffffffffu, found >= 0);
+        const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
+        const int base_idx = s_pick_step * kSampleStep;
+        if (hits) {
+          const int src = __ffs(hits) - 1;
+          const int j = __shfl_sync(0xffffffffu, found, src);
+          if (lane == 0) s_token = base_idx + src * 4 + j;
+        } else if (pos) {                                      // rounding left the target just above the step's mass
+          const int src = 31 - __clz(pos);
+          const int j = __shfl_sync(0xffffffffu, last_pos, src);
+          if (lane == 0) s_token = base_idx + src * 4 + j;
+        }
       }
-      if (found < 0) found = last_pos;                 // rounding left the target just above the range's mass
-      if (lane == 0) s_token = found;
+      __syncthreads();
+      picked = s_token;
     }
-    __syncthreads();
-    picked = s_token;
-    __syncthreads();
+    // the whole cluster learns whether the pass has to be repeated with p itself (only when the residual is empty)
+    int* retry_flag = cluster.map_shared_rank(&s_pick_warp, 0);
+    if (rank == 0 && v == 0) s_pick_warp = retry ? 1 : 0;
+    cluster.sync();
+    const bool again = *retry_flag != 0 && use_residual;
+    cluster.sync();                                            // everybody has read the flag before it changes again
+    if (!again) break;
+    use_residual = false;
   }
+  if (rank != 0) return;                                       // CTA 0 alone writes the results
 
   // ---- outputs
   int32_t* my_path = path + static_cast<size_t>(b) * (N + 1);
@@ -297,16 +370,38 @@ extern "C" jet_status jet_tree_accept_sample(const float* logits, int64_t logits
   const size_t need = jet_tree_accept_sample_workspace_bytes(batch, B, V);
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
 
+  if (V > kMaxStepsTotal * kSampleStep) return JET_ERR_UNSUPPORTED;
   const int nchunks = lse_chunks_for(V);
+  const bool vec_rows = aligned(logits, 16) && aligned(draft_logp, 16) && logits_row_stride % 4 == 0 &&
+                        logp_depth_stride % 4 == 0 && logp_batch_stride % 4 == 0;
   const bool vec_ok = aligned(logits, 16) && logits_row_stride % 4 == 0;
   const float inv_t = 1.0f / temperature;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto* partial = static_cast<float2*>(workspace);
   launch_dependent(row_lse_partial_kernel, dim3(nchunks, batch * B), dim3(kLseThreads), st, logits,
                    logits_row_stride, V, B, n_nodes, nchunks, vec_ok, inv_t * kLog2e, partial);
-  launch_dependent(accept_sample_kernel, dim3(batch), dim3(kSampleThreads), st,
-                   static_cast<const float2*>(partial), nchunks, logits, logits_row_stride, inv_t, draft_logp,
-                   logp_batch_stride, logp_depth_stride, token, parent, depth, anc_mask, n_nodes, u_accept,
-                   u_sample, B, V, N, alpha, accept_len, path, out_tokens);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(batch * kSampleCluster);
+    cfg.blockDim = dim3(kSampleThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kSampleCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, accept_sample_kernel, static_cast<const float2*>(partial), nchunks, logits,
+                           logits_row_stride, inv_t, draft_logp, logp_batch_stride, logp_depth_stride, token, parent,
+                           depth, anc_mask, n_nodes, u_accept, u_sample, B, V, N, vec_rows, alpha, accept_len, path,
+                           out_tokens) != cudaSuccess) {
+      cudaGetLastError();
+      return JET_ERR_CUDA;
+    }
+  }
   return launch_status();
 }

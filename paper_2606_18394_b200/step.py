@@ -67,7 +67,14 @@ class VerifyStep:
         self.ws_build = ws(jet.jet_tree_build_workspace_bytes(batch, N, V, W))
         self.ws_attn = ws(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, self.attn_max_len))
         self.ws_attn.zero_()         # its counters must start at zero; every call leaves them zero
-        self.ws_accept = ws(jet.jet_tree_accept_workspace_bytes(batch, B, V))
+        self.ws_accept = ws(max(jet.jet_tree_accept_workspace_bytes(batch, B, V),
+                                jet.jet_tree_accept_sample_workspace_bytes(batch, B, V)))
+        # non-greedy acceptance: the caller's random numbers (uniform in [0,1)) and the acceptance ratios
+        self.temperature = 1.0
+        self.u_accept = torch.zeros((batch, B), dtype=torch.float32, device=dev)
+        self.u_sample = torch.zeros((batch,), dtype=torch.float32, device=dev)
+        self.alpha = torch.zeros((batch, B), dtype=torch.float32, device=dev)
+        self.accept_mode = "greedy"
         self.scale = 1.0 / math.sqrt(D)
 
     @property
@@ -99,6 +106,12 @@ class VerifyStep:
                             self.batch, self.B, self.V, self.N, self.tgt, self.accept_len, self.path,
                             self.out_tokens, self.ws_accept)
 
+    def tree_accept_sample(self):
+        jet.jet_tree_accept_sample(self.logits, self.V, self.temperature, self.logp, self.N * self.V, self.V,
+                                   self.token, self.parent, self.depth, self.anc_mask, self.n_nodes, self.u_accept,
+                                   self.u_sample, self.batch, self.B, self.V, self.N, self.alpha, self.accept_len,
+                                   self.path, self.out_tokens, self.ws_accept)
+
     def kv_compact(self):
         jet.jet_kv_compact(self.tree_k, self.tree_v, self.k_cache, self.v_cache,
                            self.cache_layer_stride, self.kv_batch_stride,
@@ -112,7 +125,10 @@ class VerifyStep:
         self.tree_build()
         for layer in range(self.layers):
             self.verify_attn(layer)
-        self.tree_accept()
+        if self.accept_mode == "sample":
+            self.tree_accept_sample()
+        else:
+            self.tree_accept()
         self.kv_compact()
 
     LAUNCHES_PER_STEP_FIXED = 6      # tree_build 2, tree_accept 2, kv_compact 2
