@@ -126,6 +126,11 @@ __device__ __forceinline__ void cta_sync() {
   __syncwarp();
   asm volatile("bar.sync 0;" ::: "memory");
 }
+// Barrier `id` (1..15) among `count` threads (a multiple of 32: whole warps).
+__device__ __forceinline__ void named_sync(uint32_t id, uint32_t count) {
+  __syncwarp();
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 // The same with an AND-reduction of a predicate over the CTA.
 __device__ __forceinline__ bool cta_sync_and(bool pred) {
   uint32_t r;

@@ -41,6 +41,7 @@ constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
 constexpr int kMaxSplit = 16;          // largest cluster
 constexpr int kMaxSorted = 128;          // batches up to this size are launched longest prefix first
+constexpr float kSharedSumLimit = 1.2089258e24f;   // 2^80: tile sums a fixed reference may reach before the CTA falls back
 constexpr float kFastSumLimit = 256.0f;    // a row keeps its reference maximum while its tile sums stay below (so P <= 2^8)
 
 struct AttnParams {
@@ -84,7 +85,7 @@ struct Cfg {
   // accumulator and running maximum / sum.  Their phases interleave (one computes maxima while the
   // other exponentiates), and the two partial results are combined once, after the key loop.
   static constexpr int kStreams = MT == 1 ? 2 : 1;
-  static constexpr int kBarBytes = 256;
+  static constexpr int kBarBytes = 1024;
   static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
   static constexpr int kThreads = 128 + 128 * MT * kStreams;
   // TMEM (512 columns):
@@ -97,6 +98,11 @@ struct Cfg {
   // phases ahead of the other on one barrier: buffer index and use count of key tile t of query tile mt.
   __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
   __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
+  // MT == 1, shared-accumulator pass (see the kernel): one accumulator for both warpgroups, a score buffer
+  // and a separate P buffer (64 columns of packed bf16 pairs) per warpgroup.
+  __device__ static constexpr uint32_t shared_o() { return 0; }
+  __device__ static constexpr uint32_t shared_s(int w) { return 128 + 128 * w; }
+  __device__ static constexpr uint32_t shared_p(int w) { return 384 + 64 * w; }
   // Epilogue buffers (overlay the tile memory once the key loop is over): this CTA's 128 normalised
   // rows of one query tile -- D bf16 values followed by the row's log2-sum-exp in fp32, padded so that
   // the row-per-thread stores of a warp spread over all banks -- and the blocks received from every
@@ -111,7 +117,8 @@ struct Cfg {
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
   enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
-         kClusterA = 21, kClusterC = 22, kRecv = 23, kCount = 25 };
+         kClusterA = 21, kClusterC = 22, kRecv = 23, kOFinal = 25, kCount = 26,
+         kLoopFirst = kKvFull, kLoopEnd = kClusterA };    // the key loop's barriers exist twice (one set per pass)
 };
 
 // Every wait is bounded: at most kWaitRounds suspensions of kWaitHintNs each (about a second).
@@ -223,10 +230,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t sBar = sKV + kStages * C::kStageBytes;
   uint8_t* gen_kv = smem_gen + C::kQBytes;
   uint8_t* gen_bar = gen_kv + kStages * C::kStageBytes;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + Bars::kCount * 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + 2 * Bars::kCount * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   volatile int* seq_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);     // sequence of this CTA when launch order is sorted
+  volatile uint32_t* redo_flag = tmem_slot + 3;          // the shared-accumulator pass met a row it cannot hold
+  float* ref_s = reinterpret_cast<float*>(gen_bar + 512);  // [128] the rows' common reference (shared-accumulator pass)
+  static_assert(2 * Bars::kCount * 8 + 16 <= 512 && 512 + 128 * 4 <= C::kBarBytes, "barrier block layout");
   auto bar = [&](int idx) { return sBar + 8u * idx; };
+  uint32_t sBarLoop = sBar;        // base of the key loop's barrier set in use
+  auto lbar = [&](int idx) { return sBarLoop + 8u * idx; };
   const int S = p.nsplit;                            // key slices = cluster size
   const int split = blockIdx.x % S;                  // = rank in the cluster
   const int rows_per = (kBM + S - 1) / S;            // rows of a query tile that one slice combines
@@ -261,7 +273,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(bar(Bars::kPFull + i), 128);
       ptx::mbar_init(bar(Bars::kODone + i), 1);
+      ptx::mbar_init(bar(Bars::kSFree + i), 128);
     }
+    ptx::mbar_init(bar(Bars::kOFinal), 1);
+    *redo_flag = 0u;
     for (int mt = 0; mt < MT; ++mt) {
       // slice merge: every slice sends this CTA its block of rows of query tile mt
       ptx::mbar_init(bar(Bars::kRecv + mt), 1);
@@ -351,6 +366,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   float m_used = -INFINITY;     // running reference maximum (raw score units)
   float l = 0.0f;               // running sum of exp2((s - m_used) * sl2)
   bool row_ok = has_work;       // false once a bounded wait of this warp expired
+  bool classic = true;                      // the classic key loop has to run
+  bool shared_result = false;               // the rows come out of the shared-accumulator pass
+  float m_ref_common = 0.0f;                // softmax threads: the row's fixed reference (log2 units)
+  constexpr int kAhead = 3;     // shared-accumulator form of the key loop: Q K^T runs this many key tiles ahead of P V
 
   // The epilogue is written once and instantiated for both register classes: `sm_side` is true for the
   // softmax warpgroups (which hold the rows, stage and combine them) and false for warps 0-3 (which take
@@ -385,7 +404,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // MT == 1: the two streams of a row exchange (log2-sum-exp, 1/sum) through a scratch corner of the
     // idle tile memory; afterwards both threads of a row know both weights.
     float2* xchg = reinterpret_cast<float2*>(smem_gen + C::kTileBytes - 2048);     // [stream][row]
-    if constexpr (kSm && MT == 1) xchg[e_wg * 128 + e_r] = make_float2(own_lse2, own_inv);
+    // (after a shared-accumulator pass: the warpgroup's part of the row sum and the row's reference)
+    if constexpr (kSm && MT == 1)
+      xchg[e_wg * 128 + e_r] = shared_result ? make_float2(active ? l : 0.0f, m_ref_common) : make_float2(own_lse2, own_inv);
 #pragma unroll 1
     for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
       if (mt > 0) {
@@ -398,6 +419,34 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // together on the way: out = wa * O_0 / l_0 + wb * O_1 / l_1 with softmax weights of the two sums.
         ptx::cta_sync();
         if constexpr (kSm) {
+         if (shared_result) {
+          // one accumulator, one reference: the row sum is the sum of the warpgroups' parts
+          const float2 s0 = xchg[e_r], s1 = xchg[128 + e_r];
+          const float lt = s0.x + s1.x;
+          const bool any = lt > 0.0f && lt < INFINITY;
+          const float inv = any ? 1.0f / lt : 0.0f;
+          constexpr int kCols = D / 2;
+          uint8_t* dst = stage + e_r * C::kRecvPitch + e_wg * kCols * 2;
+#pragma unroll 1
+          for (int c = 0; c < kCols / 32; ++c) {
+            uint32_t o[32];
+            if (active) {
+              ptx::tmem_ld32(e_lane + C::shared_o() + e_wg * kCols + c * 32, o);
+              ptx::tmem_wait_ld();
+            }
+#pragma unroll
+            for (int q8 = 0; q8 < 4; ++q8) {
+              uint32_t w[4] = {0u, 0u, 0u, 0u};
+              if (active && any) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  w[k] = pack_bf16(__uint_as_float(o[q8 * 8 + 2 * k]) * inv, __uint_as_float(o[q8 * 8 + 2 * k + 1]) * inv);
+              }
+              *reinterpret_cast<uint4*>(dst + (c * 32 + q8 * 8) * 2) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+          if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 2) = any ? s0.y + log2f(lt) : -INFINITY;
+         } else {
           const float2 s0 = xchg[e_r], s1 = xchg[128 + e_r];
           const float mxl = fmaxf(s0.x, s1.x);
           float a0 = 0.0f, a1 = 0.0f, lse2 = -INFINITY;
@@ -435,6 +484,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
           }
           if (e_wg == 0) *reinterpret_cast<float*>(stage + e_r * C::kRecvPitch + D * 2) = lse2;
+         }
         }
       } else if (kSm && e_wg == mt) {
         uint8_t* dst = stage + e_r * C::kRecvPitch;
@@ -595,94 +645,227 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   };
 
+  // ---------------- the key loop
+  // Two forms.  The classic form gives every stream its own accumulator and reference maximum, which may rise
+  // at any tile (the accumulator is rescaled); it is exact for any input.  With one query tile per CTA the
+  // loop first runs in the shared-accumulator form: both warpgroups add into ONE accumulator against a per-row
+  // reference that is fixed after the first key tile, which frees the TMEM columns for P buffers apart from
+  // the score buffers -- so a warpgroup's next Q K^T runs while it still exponentiates the tile before, and
+  // the chain  softmax -> P V -> Q K^T -> softmax  of the classic form becomes  softmax -> softmax.  A fixed
+  // reference is exact as long as no probability overflows; a row whose tile sum passes kSharedSumLimit (or is
+  // not finite) raises redo_flag, and the CTA then runs the whole key range again in the classic form (on a
+  // second set of barriers; the first pass has drained by then).
+
+  // Position in the ring of the V tile of key tile tl when K runs `ahead` tiles in front of V
+  // (ring order: K_0 .. K_ahead, then V_t, K_{t+ahead+1} alternating, then the remaining V).
+  auto v_item = [&](int tl, int ahead) {
+    const int lead = min(ahead + 1, T);
+    return lead + tl + min(tl, T - lead);
+  };
+  // The barriers of the classic pass when it follows a shared-accumulator pass: a fresh set.
+  auto second_barrier_set = [&]() {
+    sBarLoop = sBar + 8u * Bars::kCount;
+    if (tid == 0) {
+      for (int s = 0; s < kStages; ++s) {
+        ptx::mbar_init(lbar(Bars::kKvFull + s), 1);
+        ptx::mbar_init(lbar(Bars::kKvEmpty + s), 1);
+      }
+      for (int i = 0; i < 2; ++i) {
+        ptx::mbar_init(lbar(Bars::kSFull + i), 1);
+        ptx::mbar_init(lbar(Bars::kPFull + i), 128);
+        ptx::mbar_init(lbar(Bars::kODone + i), 1);
+      }
+      ptx::fence_mbar_init();
+    }
+    ptx::cta_sync();
+  };
+
   if (warp < 4) {
     // Warps 0-3 need few registers; what they give up goes to the softmax warpgroups, which hold a whole
     // score row (128 values) per thread.
     ptx::setmaxnreg_dec<kRegsControl>();
-    if (has_work) {
-      if (warp == 0) {
-        // =========================================================== TMA producer
-        if (lane == 0) {
-          ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
-          for (int mt = 0; mt < n_mt; ++mt)
+
+    // =========================================================== TMA producer (warp 0)
+    // K runs `ahead` key tiles in front of V in the ring (0: K_t, V_t alternate).
+    auto produce = [&](const int ahead, const bool load_q) {
+      if (load_q && lane == 0) {
+        ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
+        for (int mt = 0; mt < n_mt; ++mt)
+          for (int h = 0; h < kHalves; ++h)
+            ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
+                             b * p.B + node_lo + mt * npt);
+        JET_TR(45);
+      }
+      __syncwarp();
+      bool ok = true;
+      int issued = 0;
+      // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
+      // fetched while the current tile's copies are issued, so the table look-up is off the critical path
+      auto tile_page = [&](int t) -> int {
+        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= L) return 0;
+        return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
+      };
+      int kt = 0, vt = 0;                       // next K tile, next V tile
+      int pk_cur = tile_page(t_lo), pk_next = tile_page(t_lo + 1);
+      int pv_cur = pk_cur, pv_next = pk_next;
+#pragma unroll 1
+      for (; issued < 2 * T; ++issued) {
+        const bool take_k = kt < T && kt <= vt + ahead;
+        const int t = t_lo + (take_k ? kt : vt), kv = take_k ? 0 : 1, stage = issued % kStages;
+        if (issued >= kStages) {
+          ok = bounded_wait(lbar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
+          if (!ok) break;
+        }
+        const uint32_t dst = sKV + stage * C::kStageBytes;
+        const uint32_t full = lbar(Bars::kKvFull + stage);
+        if (t < TP && p.paged) {
+          const int npages = min(8, (L - t * kBN + 15) / 16);
+          const int page = take_k ? pk_cur : pv_cur;
+          if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
+          __syncwarp();
+          if (lane < npages) {
             for (int h = 0; h < kHalves; ++h)
-              ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
-                               b * p.B + node_lo + mt * npt);
-          JET_TR(45);
+              ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page * 16);
+          }
+        } else if (lane == 0) {
+          const bool prefix = t < TP;
+          const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
+          const int row0 = prefix ? t * kBN : (t - TP) * kBN;
+          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+          for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
+        }
+        if (take_k) {
+          ++kt;
+          pk_cur = pk_next;
+          pk_next = tile_page(t + 2);
+        } else {
+          ++vt;
+          pv_cur = pv_next;
+          pv_next = tile_page(t + 2);
         }
         __syncwarp();
-        bool ok = true;
-        int issued = 0;
-        // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
-        // fetched while the current tile's copies are issued, so the table look-up is off the critical path
-        auto tile_page = [&](int t) -> int {
-          if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= L) return 0;
-          return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
-        };
-        int page_cur = tile_page(t_lo), page_next = tile_page(t_lo + 1);
+        if (lane == 0 && issued == 0) JET_TR(14);
+      }
+      if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
+        // drain: every load that was issued must land before the CTA may exit
+        for (int s = 0; s < kStages; ++s) {
+          if (issued > s) {
+            const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
+            bounded_wait(lbar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
+          }
+        }
+        bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
+      }
+    };
+
+    // The tensor core queues only two or three instructions, so every instruction between two MMAs counts:
+    // the whole warp runs the issue loops (uniform control flow and operands), one elected lane issues, and
+    // descriptors are formed by adding precomputed offsets.
+    constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
+    constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
+    const uint64_t desc_q0 = ptx::smem_desc_sw128(sQ, 0);
+    const uint64_t desc_k0 = ptx::smem_desc_sw128(sKV, 0);
+    const uint64_t desc_v0 = ptx::smem_desc_sw128(sKV, kHalfBytes);
+
+    if constexpr (MT == 1) {
+      if (has_work) {
+        if (warp == 0) {
+          produce(kAhead, true);
+        } else if (warp == 1) {
+          // =========================================================== tcgen05 issuers, shared-accumulator form
+          // Key tile tl belongs to warpgroup tl & 1 (score buffer and P buffer of that warpgroup).  Warp 1
+          // issues every Q K^T, warp 3 every P V: the two chains depend on each other only through the softmax
+          // warpgroups' barriers, and while one warp sits in the (blocking) issue of its eight instructions the
+          // other gets through its waits.  A Q K^T may overwrite a score buffer once its warpgroup has read the
+          // scores before (kSFree); a warpgroup may overwrite its P buffer once the P V that read it is
+          // complete (kODone).  Ring positions: K_0 .. K_kAhead, then V_t, K_{t+kAhead+1} alternating.
+          bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
+          if (lane == 0) JET_TR(2);
+          const int lead = min(kAhead + 1, T);
 #pragma unroll 1
-        for (; issued < 2 * T; ++issued) {
-          const int t = t_lo + (issued >> 1), kv = issued & 1, stage = issued % kStages;
-          if (issued >= kStages) {
-            ok = bounded_wait(bar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
+          for (int tl = 0; tl < T && ok; ++tl) {
+            const int w = tl & 1, j = tl >> 1;
+            const int item = tl < lead ? tl : 2 * tl - lead + 1;
+            const int stage = item % kStages;
+            const uint32_t par = (item / kStages) & 1;
+            if (tl == 12 && lane == 0) JET_TR(61);
+            if (j > 0) {
+              ok = bounded_wait(bar(Bars::kSFree + w), (j - 1) & 1, abort_flag, 20);
+              if (!ok) break;
+            }
+            if (tl == 12 && lane == 0) JET_TR(62);
+            ok = bounded_wait(bar(Bars::kKvFull + stage), par, abort_flag, 5);
             if (!ok) break;
-          }
-          const uint32_t dst = sKV + stage * C::kStageBytes;
-          const uint32_t full = bar(Bars::kKvFull + stage);
-          if (t < TP && p.paged) {
-            const int npages = min(8, (L - t * kBN + 15) / 16);
-            if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
-            __syncwarp();
-            if (lane < npages) {
-              for (int h = 0; h < kHalves; ++h)
-                ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page_cur * 16);
+            if (tl == 12 && lane == 0) JET_TR(63);
+            if (tl == 0 && lane == 0) JET_TR(3);
+            ptx::tc_fence_after();
+            const uint64_t desc_k = desc_k0 + static_cast<uint64_t>(stage * (C::kStageBytes >> 4));
+            const uint32_t s_tmem = tmem_base + C::shared_s(w);
+            if (ptx::elect_one()) {
+#pragma unroll
+              for (int kd = 0; kd < D / 16; ++kd) {
+                const uint64_t off = static_cast<uint64_t>(((kd / 4) * kHalfBytes + (kd % 4) * 32) >> 4);
+                ptx::umma_ss(s_tmem, desc_q0 + off, desc_k + off, idesc_qk, kd > 0 ? 1u : 0u);
+              }
+              ptx::umma_commit(bar(Bars::kSFull + w));
+              ptx::umma_commit(bar(Bars::kKvEmpty + stage));
             }
-            if (kv) {                       // both tiles of this key range are on their way: move on
-              page_cur = page_next;
-              page_next = tile_page(t + 2);
-            }
-          } else if (lane == 0) {
-            const bool prefix = t < TP;
-            const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
-            const int row0 = prefix ? t * kBN : (t - TP) * kBN;
-            ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-            for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
           }
-          __syncwarp();
-          if (lane == 0 && issued == 0) JET_TR(14);
+        } else if (warp == 3) {
+          bool ok = true;
+#pragma unroll 1
+          for (int tl = 0; tl < T && ok; ++tl) {
+            const int w = tl & 1, j = tl >> 1;
+            const int item = v_item(tl, kAhead);
+            const int stage = item % kStages;
+            const uint32_t par = (item / kStages) & 1;
+            if (tl == 8 && lane == 0) JET_TR(58);
+            ok = bounded_wait(bar(Bars::kKvFull + stage), par, abort_flag, 7);
+            if (!ok) break;
+            if (tl == 8 && lane == 0) JET_TR(59);
+            ok = bounded_wait(bar(Bars::kPFull + w), j & 1, abort_flag, 8);
+            if (!ok) break;
+            if (tl == 8 && lane == 0) JET_TR(60);
+            ptx::tc_fence_after();
+            if (w == 0 && j < 8 && lane == 0) JET_TR(50 + j);
+            const uint64_t desc_v = desc_v0 + static_cast<uint64_t>(stage * (C::kStageBytes >> 4));
+            const uint32_t p_tmem = tmem_base + C::shared_p(w);
+            const uint32_t o_tmem = tmem_base + C::shared_o();
+            if (ptx::elect_one()) {
+#pragma unroll
+              for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
+                ptx::umma_ts(o_tmem, p_tmem + kk * 8, desc_v + static_cast<uint64_t>((kk * 2048) >> 4), idesc_pv,
+                             (tl == 0 && kk == 0) ? 0u : 1u);
+              ptx::umma_commit(bar(Bars::kODone + w));
+              ptx::umma_commit(bar(Bars::kKvEmpty + stage));
+              if (tl == T - 1) ptx::umma_commit(bar(Bars::kOFinal));
+            }
+          }
         }
-        if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
-          // drain: every load that was issued must land before the CTA may exit
-          for (int s = 0; s < kStages; ++s) {
-            if (issued > s) {
-              const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
-              bounded_wait(bar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
-            }
-          }
-          bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
-        }
+      }
+      ptx::cta_sync();                                  // every role has left the shared-accumulator pass
+      classic = *redo_flag != 0u && *abort_flag == 0u;
+      shared_result = !classic;
+      if (classic) second_barrier_set();
+    }
+
+    if (classic && has_work) {
+      if (warp == 0) {
+        produce(0, MT == 2);
       } else if (warp == 1) {
-        // =========================================================== tcgen05 issuer
+        // =========================================================== tcgen05 issuer, classic form
         // A stream is a chain  S = Q K^T -> softmax -> O += P V -> next S  on its own score buffer (which the P
         // overwrites) and accumulator: with one query tile per CTA the two streams take alternate key tiles,
         // with two each stream is one query tile and takes every key tile.  The streams take turns: a turn
         // issues one tile's P V and the stream's next Q K^T, so that one stream's softmax runs under the other
         // stream's products.  Within a stream the next Q K^T overwrites the P of the tile before; it is issued
         // after that tile's P V, and one thread's MMAs execute in issue order, so it needs no further wait.
-        // The whole warp runs the loop (uniform control flow and operands); one elected lane issues.  The
-        // tensor core queues only two or three instructions, so every instruction between two MMAs counts:
-        // descriptors are formed by adding precomputed offsets.
-        constexpr uint32_t idesc_qk = ptx::umma_idesc_bf16(kBM, kBN, false);
-        constexpr uint32_t idesc_pv = ptx::umma_idesc_bf16(kBM, D, true);
         constexpr int kStep = MT == 1 ? 2 : 1;            // distance between a stream's tiles
-        const uint64_t desc_q0 = ptx::smem_desc_sw128(sQ, 0);
-        const uint64_t desc_k0 = ptx::smem_desc_sw128(sKV, 0);
-        const uint64_t desc_v0 = ptx::smem_desc_sw128(sKV, kHalfBytes);
         bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
         if (lane == 0) JET_TR(2);
         auto issue_qk = [&](int stream, int tl) {
           const int item = 2 * tl, stage = item % kStages;
-          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
+          ok = bounded_wait(lbar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
           if (!ok) return;
           if (tl == 0 && stream == 0 && lane == 0) JET_TR(3);
           ptx::tc_fence_after();
@@ -696,16 +879,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               const uint64_t off = static_cast<uint64_t>(((kd / 4) * kHalfBytes + (kd % 4) * 32) >> 4);
               ptx::umma_ss(s_tmem, desc_q + off, desc_k + off, idesc_qk, kd > 0 ? 1u : 0u);
             }
-            ptx::umma_commit(bar(Bars::kSFull + stream));
-            ptx::umma_commit(bar(Bars::kKvEmpty + stage));     // this stream has read the K tile
+            ptx::umma_commit(lbar(Bars::kSFull + stream));
+            ptx::umma_commit(lbar(Bars::kKvEmpty + stage));     // this stream has read the K tile
           }
         };
         auto turn = [&](int stream, int tl) {
           // ---- O += P V of tile tl (rows of masked keys of the V tile were cleared by the softmax threads)
           const int item = 2 * tl + 1, stage = item % kStages;
-          ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
+          ok = bounded_wait(lbar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
           if (!ok) return;
-          ok = bounded_wait(bar(Bars::kPFull + stream), C::s_use(tl) & 1, abort_flag, 8);
+          ok = bounded_wait(lbar(Bars::kPFull + stream), C::s_use(tl) & 1, abort_flag, 8);
           if (!ok) return;
           ptx::tc_fence_after();
           if (stream == 0 && tl / kStep < 8 && lane == 0) JET_TR(50 + tl / kStep);
@@ -719,8 +902,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             for (int kk = 0; kk < kBN / 16; ++kk)      // 16 keys = 8 TMEM columns of packed bf16 pairs
               ptx::umma_ts(o_tmem, s_tmem + kk * 8, desc_v + static_cast<uint64_t>((kk * 2048) >> 4), idesc_pv,
                            (first && kk == 0) ? 0u : 1u);
-            ptx::umma_commit(bar(Bars::kODone + stream));
-            ptx::umma_commit(bar(Bars::kKvEmpty + stage));      // this stream has read the V tile
+            ptx::umma_commit(lbar(Bars::kODone + stream));
+            ptx::umma_commit(lbar(Bars::kKvEmpty + stage));      // this stream has read the V tile
           }
           // ---- S = Q K^T of the stream's next tile
           if (tl + kStep < T) issue_qk(stream, tl + kStep);
@@ -741,19 +924,149 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     epilogue(std::false_type{});
   } else {
     ptx::setmaxnreg_inc<kRegsSoftmax>();
-    if (has_work && (MT == 1 || ((warp - 4) >> 2) < n_mt)) {
-      // =========================================================== softmax warpgroups
-      constexpr int kChunks = kBN / 32;                       // 32-key chunks per row and tile
-      constexpr int kStreams = C::kStreams;
-      const int wg = (warp - 4) >> 2;
-      const int mt = MT == 1 ? 0 : wg;                        // query tile of this warpgroup
-      const int stream = MT == 1 ? wg : 0;                    // its share of the key tiles (tl % kStreams)
-      const int r = (tid - 128) & 127;                        // row of the query tile = TMEM lane
-      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-      const int v = node_lo + mt * npt + r / G;
-      const bool row_live = v < n;
-      const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
-      const float sl2 = p.scale_log2;
+    constexpr int kChunks = kBN / 32;                       // 32-key chunks per row and tile
+    static_assert(kChunks == 4, "the register-resident row is written out for four 32-key chunks");
+    constexpr int kStreams = C::kStreams;
+    const int wg = (warp - 4) >> 2;
+    const int mt = MT == 1 ? 0 : wg;                        // query tile of this warpgroup
+    const int stream = MT == 1 ? wg : 0;                    // its share of the key tiles (tl % kStreams)
+    const int r = (tid - 128) & 127;                        // row of the query tile = TMEM lane
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const int v = node_lo + mt * npt + r / G;
+    const bool row_live = v < n;
+    const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
+    const float sl2 = p.scale_log2;
+    // visibility bits of this row for 32-key chunk c of key tile t (a tile that is not full)
+    auto chunk_bits = [&](int t, int c) -> uint32_t {
+      if (t < TP) {
+        const int nv = (L - t * kBN) - c * 32;
+        return nv >= 32 ? 0xFFFFFFFFu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+      }
+      const int w = (t - TP) * 4 + c;
+      return (row_live && w < p.words) ? __ldg(mask_row + w) : 0u;
+    };
+    // Masked keys get P = 0 exactly, but 0 * NaN is NaN: the V rows of keys beyond the valid ones (stale
+    // cache rows, rows of padding nodes) are cleared before the P V product may read them.  `item` = the V
+    // tile's position in the ring.  Returns false if the wait for the tile gave up.
+    auto clear_v_tail = [&](int t, int item) -> bool {
+      const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
+      if (valid >= kBN) return true;
+      const int stage = item % kStages;
+      if (!bounded_wait(lbar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 10)) return false;
+      uint8_t* vt = gen_kv + stage * C::kStageBytes;
+      const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
+      for (int h = 0; h < kHalves; ++h)
+        for (int i = r; i < chunks; i += 128)
+          *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+      ptx::fence_proxy_async_smem();
+      return true;
+    };
+
+    if constexpr (MT == 1) {
+      if (has_work) {
+        // =========================================================== softmax, shared-accumulator form
+        // Warpgroup wg takes key tiles wg, wg + 2, ...  A thread reads its whole score row from TMEM, hands
+        // the score buffer back at once (the tile after next can be computed into it), exponentiates against
+        // the row's fixed reference and writes P to the warpgroup's P buffer.
+        bool ok = true;
+        bool synced = false;                 // the two warpgroups have met at the reference hand-over
+        float m_ref = 0.0f;
+        const uint32_t tS = t_lane + C::shared_s(wg);
+        const uint32_t tP = t_lane + C::shared_p(wg);
+#pragma unroll 1
+        for (int tl = wg; tl < T && ok; tl += 2) {
+          const int t = t_lo + tl, j = tl >> 1;
+          const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
+          ok = bounded_wait(bar(Bars::kSFull + wg), j & 1, abort_flag, 9);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          if (tid == 128 && j == 4) JET_TR(4);
+          if (tid == 128 && j < 4) JET_TR(19 + 2 * j);
+          if (tid == 256 && j < 4) JET_TR(32 + 2 * j);
+          uint32_t xa[32], xb[32], xc[32], xd[32];
+          uint32_t b0 = 0xFFFFFFFFu, b1 = 0xFFFFFFFFu, b2 = 0xFFFFFFFFu, b3 = 0xFFFFFFFFu;
+          if (!full_tile) { b0 = chunk_bits(t, 0); b1 = chunk_bits(t, 1); b2 = chunk_bits(t, 2); b3 = chunk_bits(t, 3); }
+          ptx::tmem_ld32(tS, xa);
+          ptx::tmem_ld32(tS + 32, xb);
+          ptx::tmem_ld32(tS + 64, xc);
+          ptx::tmem_ld32(tS + 96, xd);
+          ptx::tmem_wait_ld();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kSFree + wg));          // the scores are in registers
+          if (!full_tile) {
+            mask_chunk(xa, b0);
+            mask_chunk(xb, b1);
+            mask_chunk(xc, b2);
+            mask_chunk(xd, b3);
+          }
+          if (j == 0) {
+            // The reference of a row: its maximum over the first key tile (0 if it sees no key there), found
+            // by warpgroup 0 and handed to warpgroup 1 through shared memory.
+            if (wg == 0) {
+              float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+              max_chunk(xa, mx);
+              max_chunk(xb, mx);
+              max_chunk(xc, mx);
+              max_chunk(xd, mx);
+              const float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+              m_ref = (m == -INFINITY) ? 0.0f : m * sl2;
+              if (T > 1) {
+                ref_s[r] = m_ref;
+                ptx::named_sync(1, 256);
+              }
+            } else {
+              ptx::named_sync(1, 256);
+              m_ref = ref_s[r];
+            }
+            synced = true;
+          }
+          if (tid == 128 && j == 4) JET_TR(5);
+          if (j > 0) {
+            // the P V product of this warpgroup's tile before has read the P buffer
+            ok = bounded_wait(bar(Bars::kODone + wg), (j - 1) & 1, abort_flag, 21);
+            if (!ok) break;
+          }
+          if (tid == 128 && j == 4) JET_TR(16);
+          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          exp_chunk(xa, sl2, m_ref, sum, tP);
+          exp_chunk(xb, sl2, m_ref, sum, tP + 16);
+          exp_chunk(xc, sl2, m_ref, sum, tP + 32);
+          exp_chunk(xd, sl2, m_ref, sum, tP + 48);
+          const float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          if (row_live && !(tile_sum <= kSharedSumLimit)) *redo_flag = 1u;
+          l += tile_sum;
+          if (tid == 128 && j == 4) JET_TR(17);
+          if (!full_tile) {
+            ok = clear_v_tail(t, v_item(tl, kAhead));
+            if (!ok) break;
+          }
+          ptx::tmem_wait_st();                     // P is in TMEM
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kPFull + wg));
+          if (tid == 128 && j == 4) JET_TR(6);
+          if (tid == 128 && j < 4) JET_TR(20 + 2 * j);
+          if (tid == 256 && j < 4) JET_TR(33 + 2 * j);
+        }
+        if (T > 1 && !synced) ptx::named_sync(1, 256);       // a warpgroup that gave up early still meets the other
+        if (tid == 128) JET_TR(10);
+        if (ok) ok = bounded_wait(bar(Bars::kOFinal), 0, abort_flag, 11);      // the last P V is complete
+        if (ok) ptx::tc_fence_after();
+        row_ok = ok;
+        m_ref_common = m_ref;
+      }
+      ptx::cta_sync();                                  // every role has left the shared-accumulator pass
+      classic = *redo_flag != 0u && *abort_flag == 0u;
+      shared_result = !classic;
+      if (classic) {
+        second_barrier_set();
+        m_used = -INFINITY;
+        l = 0.0f;
+        row_ok = has_work;
+      }
+    }
+
+    if (classic && has_work && (MT == 1 || wg < n_mt)) {
+      // =========================================================== softmax, classic form
       bool ok = true;
       int last_tl = -1;
 
@@ -763,17 +1076,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint32_t tS = t_lane + C::s_col(mt, tl);
         const uint32_t tO = t_lane + C::o_col(mt, tl);
         const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
-        // visibility bits of this row for 32-key chunk c of a tile that is not full
-        auto chunk_bits = [&](int c) -> uint32_t {
-          if (t < TP) {
-            const int nv = (L - t * kBN) - c * 32;
-            return nv >= 32 ? 0xFFFFFFFFu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
-          }
-          const int w = (t - TP) * 4 + c;
-          return (row_live && w < p.words) ? __ldg(mask_row + w) : 0u;
-        };
 
-        ok = bounded_wait(bar(Bars::kSFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 9);
+        ok = bounded_wait(lbar(Bars::kSFull + C::s_buf(mt, tl)), C::s_use(tl) & 1, abort_flag, 9);
         if (!ok) break;
         ptx::tc_fence_after();
         if (tid == 128 && tl < 1) JET_TR(4);
@@ -783,7 +1087,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
         // (The P V product of this accumulator's previous tile is complete: the Q K^T that produced these
         //  scores was only issued after it.  So O may be rescaled and the score buffer overwritten with P.)
-        static_assert(kChunks == 4, "the register-resident row is written out for four 32-key chunks");
         // ---- The thread reads its whole score row (128 values) from TMEM once.  Keys the row must not see
         //      (ragged end of the prefix, tree keys outside the ancestor set) are replaced by -inf right away,
         //      so they get probability exactly 0 whatever the cache rows behind them hold.  The row is then
@@ -793,7 +1096,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         //      is redone with its true maximum).
         uint32_t xa[32], xb[32], xc[32], xd[32];
         uint32_t b0 = 0xFFFFFFFFu, b1 = 0xFFFFFFFFu, b2 = 0xFFFFFFFFu, b3 = 0xFFFFFFFFu;
-        if (!full_tile) { b0 = chunk_bits(0); b1 = chunk_bits(1); b2 = chunk_bits(2); b3 = chunk_bits(3); }
+        if (!full_tile) { b0 = chunk_bits(t, 0); b1 = chunk_bits(t, 1); b2 = chunk_bits(t, 2); b3 = chunk_bits(t, 3); }
         ptx::tmem_ld32(tS, xa);
         ptx::tmem_ld32(tS + 32, xb);
         ptx::tmem_ld32(tS + 64, xc);
@@ -871,24 +1174,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         l = l * factor + tile_sum;
         if (!full_tile) {
-          // Masked keys get P = 0 exactly, but 0 * NaN is NaN: the V rows of keys beyond the valid ones
-          // (stale cache rows, rows of padding nodes) are cleared before the P V product may read them.
-          const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
-          if (valid < kBN) {
-            const int item = 2 * tl + 1, stage = item % kStages;
-            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 10);
-            if (!ok) break;
-            uint8_t* vt = gen_kv + stage * C::kStageBytes;
-            const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
-            for (int h = 0; h < kHalves; ++h)
-              for (int i = r; i < chunks; i += 128)
-                *reinterpret_cast<uint4*>(vt + h * kHalfBytes + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-            ptx::fence_proxy_async_smem();
-          }
+          ok = clear_v_tail(t, 2 * tl + 1);
+          if (!ok) break;
         }
         ptx::tmem_wait_st();                     // P (and a rescaled O) are in TMEM
         ptx::tc_fence_before();
-        ptx::mbar_arrive(bar(Bars::kPFull + C::s_buf(mt, tl)));
+        ptx::mbar_arrive(lbar(Bars::kPFull + C::s_buf(mt, tl)));
         if (tid == 128 && tl < 1) JET_TR(6);
         if (tid == 128 && tl / kStreams < 4) JET_TR(20 + 2 * (tl / kStreams));
         if (tid == 256 && tl / kStreams < 4) JET_TR(33 + 2 * (tl / kStreams));
@@ -897,7 +1188,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (tid == 128) JET_TR(10);
       // O is complete once the last P V of this accumulator has been committed
       if (ok && last_tl >= 0)
-        ok = bounded_wait(bar(Bars::kODone + C::s_buf(mt, last_tl)), C::s_use(last_tl) & 1, abort_flag, 11);
+        ok = bounded_wait(lbar(Bars::kODone + C::s_buf(mt, last_tl)), C::s_use(last_tl) & 1, abort_flag, 11);
       if (ok) ptx::tc_fence_after();
       row_ok = ok;
     }

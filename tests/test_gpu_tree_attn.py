@@ -114,6 +114,39 @@ def test_large_scores_stay_finite():
     _run_contiguous(64, 8, 2, 128, 900, 3, scale=1.0)
 
 
+@pytest.mark.parametrize("jump", [12.0, 40.0])
+@pytest.mark.parametrize("where", ["prefix", "tree"])
+def test_scores_far_above_the_first_tile(jump, where):
+    """One query tile per CTA keeps the row reference of the first key tile for the whole key range; keys whose
+    scores lie far above it (here by about 2^110 and by more than the fp32 range, in the later prefix tiles or only
+    in the tree) must send the CTA through its exact two-accumulator pass.  Rows stay within tolerance."""
+    import jet_harness as H
+    from jet_inputs import bf16_bits_to_f32, f32_to_bf16_bits
+    B, Hq, Hkv, D, L = 32, 8, 2, 128, 700
+    rng = np.random.default_rng(77)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    q = np.abs(bf16_bits_to_f32(x["q"])) * 0.25                  # every score against an all-positive key is positive
+    x["q"] = f32_to_bf16_bits(q)
+    k = bf16_bits_to_f32(x["k_prefix"]) * 0.05
+    tk = bf16_bits_to_f32(x["tree_k"]) * 0.05
+    if where == "prefix":
+        k[300:520] = jump * 0.25                                 # keys 300..519: scores of about 25 * jump * 0.25 * 0.8
+    else:
+        tk[:] = jump * 0.25                                      # the tree's own keys only
+    x["k_prefix"], x["tree_k"] = f32_to_bf16_bits(k), f32_to_bf16_bits(tk)
+    parent, _, _ = random_tree(B, rng)
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0
+    s_big = (bf16_bits_to_f32(x["q"])[0, 0] * jump * 0.25).sum() * scale * 1.4427
+    assert s_big > (100 if jump == 12.0 else 130)                 # log2 units above the first tile's scores
+    ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [L],
+                                   x["tree_k"][None], x["tree_v"][None], anc[None], [B], scale)
+    assert st == 0
+    _check(out[0], None, ref, rlse, B)
+    assert np.abs(lse[0] - rlse).max() <= 1e-3 * max(1.0, np.abs(rlse).max())
+
+
 def test_sweep_16k_sampled_rows():
     """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
     import jet_harness as H
