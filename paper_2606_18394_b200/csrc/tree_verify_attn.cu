@@ -6,20 +6,26 @@
 //                 so all G heads of a KV group share every K/V tile that is loaded.
 //   warp 0      = TMA producer: Q tiles once, then K and V tiles (128 keys) through a ring of
 //                 shared-memory stages; paged caches are fetched one 16-row page per TMA box.
-//   warp 1      = tcgen05 issuer: S = Q K^T into TMEM, later O += P V into TMEM.
+//   warp 1      = tcgen05 issuer: S = Q K^T into TMEM, O += P V into TMEM (in the shared-accumulator
+//                 form of the key loop warp 1 issues the Q K^T and warp 3 the P V products).
 //   warp 2      = TMEM allocation / release.
-//   warps 4..   = one softmax warpgroup per query tile, one thread per row: reads S from TMEM,
-//                 applies the key-validity / ancestor-bit mask, keeps the running maximum and sum
-//                 (online softmax with lazy rescaling of O), writes P (bf16) to shared memory in
-//                 the swizzled operand layout, and finally normalises O.
+//   warps 4..11 = two softmax warpgroups, one thread per row: the thread reads its 128 scores of a key
+//                 tile from TMEM, replaces the scores of keys the row must not see (key validity,
+//                 ancestor bits) by -inf, exponentiates against the row's reference maximum, adds
+//                 to the row sum and writes P (bf16) back to TMEM, where the P V product reads it.
+//   key loop    = with one query tile per CTA: both warpgroups (alternate key tiles) add into one
+//                 accumulator against a reference fixed after the first tile; if a row overflows that
+//                 reference the CTA repeats the key range in the classic form (own accumulator and
+//                 running maximum per stream, accumulator rescaled when the maximum rises), which is
+//                 also the form used with two query tiles per CTA.  See "the key loop" below.
 //   key slices  = when there are fewer work items than SMs the key range is cut into `nsplit`
-//                 slices that run as one thread-block cluster.  After the key loop every CTA
-//                 sends its normalised rows and their log-sum-exp to the row's owner CTA through
-//                 distributed shared memory; the owners combine the slices and write the output.
-//                 Nothing goes through global memory and there is no second launch.
+//                 slices.  After the key loop every CTA hands the normalised rows (bf16) and their
+//                 log-sum-exp to the rows' owner CTAs -- through distributed shared memory when the
+//                 slices form a thread-block cluster, else through the workspace -- and the owners
+//                 combine the slices and write the output.  There is no second launch.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
-// loops (still taking part in the cluster barriers), outstanding TMA loads are drained, TMEM is
-// released and JET_ERR_TIMEOUT is reported.
+// loops (still taking part in the CTA-wide and cluster barriers), outstanding TMA loads are drained,
+// TMEM is released and JET_ERR_TIMEOUT is reported.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cstdlib>
