@@ -354,6 +354,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   // ---------------- work item, continued: what depends on device data
   const int b = sorted_launch ? *seq_slot : b_rank;
+  // The query rows depend on nothing but the work item: warp 2 (idle after the TMEM allocation) requests them
+  // now, under the look-up of the sequence's lengths.
+  if (warp == 2 && lane == 0) {
+    JET_TR(46);
+    ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
+    for (int mt = 0; mt < n_mt; ++mt)
+      for (int h = 0; h < kHalves; ++h)
+        ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
+                         b * p.B + node_lo + mt * npt);
+    JET_TR(45);
+  }
   const int L = p.seq_len[b];
   const int n = min(p.n_nodes[b], p.B);
   const int ntree = min(n, node_hi);                         // tree keys any row here can see
@@ -362,10 +373,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int T_all = TP + TT;
   // key tiles of this slice; when they do not divide evenly the first slices take the extra tile, so that
   // the last slice, whose tree tile (masked) is the slowest kind, has the fewest
-  const int t_lo = static_cast<int>((static_cast<int64_t>(T_all) * split + S - 1) / S);
-  const int t_hi = static_cast<int>((static_cast<int64_t>(T_all) * (split + 1) + S - 1) / S);
+  const int t_lo = static_cast<int>((static_cast<uint32_t>(T_all) * split + S - 1) / static_cast<uint32_t>(S));
+  const int t_hi = static_cast<int>((static_cast<uint32_t>(T_all) * (split + 1) + S - 1) / static_cast<uint32_t>(S));
   const int T = t_hi - t_lo;
   const bool has_work = node_lo < n && T > 0;    // otherwise: no live node here, or an empty key slice
+  // A CTA without work never looks at its query rows, but they must have landed before the epilogue reuses
+  // their memory (and before the CTA exits).
+  if (!has_work && warp == 2) bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
   if (tid == 0) JET_TR(1);
 
   // per-row state of the softmax threads, live until the epilogue
@@ -689,20 +703,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (warp < 4) {
     // Warps 0-3 need few registers; what they give up goes to the softmax warpgroups, which hold a whole
     // score row (128 values) per thread.
+    if (tid == 0) JET_TR(15);
     ptx::setmaxnreg_dec<kRegsControl>();
+    if (tid == 0) JET_TR(18);
 
     // =========================================================== TMA producer (warp 0)
     // K runs `ahead` key tiles in front of V in the ring (0: K_t, V_t alternate).
-    auto produce = [&](const int ahead, const bool load_q) {
-      if (load_q && lane == 0) {
-        ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
-        for (int mt = 0; mt < n_mt; ++mt)
-          for (int h = 0; h < kHalves; ++h)
-            ptx::tma_load_4d(sQ + (mt * kHalves + h) * kHalfBytes, &tm_q, bar(Bars::kQFull), h * 64, 0, g,
-                             b * p.B + node_lo + mt * npt);
-        JET_TR(45);
-      }
-      __syncwarp();
+    auto produce = [&](const int ahead) {
+      if (tid == 0) JET_TR(27);
       bool ok = true;
       int issued = 0;
       // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
@@ -714,6 +722,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       int kt = 0, vt = 0;                       // next K tile, next V tile
       int pk_cur = tile_page(t_lo), pk_next = tile_page(t_lo + 1);
       int pv_cur = pk_cur, pv_next = pk_next;
+      if (tid == 0) JET_TR(28);
 #pragma unroll 1
       for (; issued < 2 * T; ++issued) {
         const bool take_k = kt < T && kt <= vt + ahead;
@@ -733,12 +742,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             for (int h = 0; h < kHalves; ++h)
               ptx::tma_load_3d(dst + h * kHalfBytes + lane * 2048, kv ? &tm_v : &tm_k, full, h * 64, g, page * 16);
           }
-        } else if (lane == 0) {
+        } else {
           const bool prefix = t < TP;
           const CUtensorMap* map = prefix ? (kv ? &tm_v : &tm_k) : (kv ? &tm_tv : &tm_tk);
           const int row0 = prefix ? t * kBN : (t - TP) * kBN;
-          ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
-          for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
+          if (issued == 0 && lane == 0) JET_TR(48);
+          if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+            for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(dst + h * kHalfBytes, map, full, h * 64, g, row0, b);
+          }
+          if (issued == 0 && lane == 0) JET_TR(49);
         }
         if (take_k) {
           ++kt;
@@ -776,7 +789,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if constexpr (MT == 1) {
       if (has_work) {
         if (warp == 0) {
-          produce(kAhead, true);
+          produce(kAhead);
         } else if (warp == 1) {
           // =========================================================== tcgen05 issuers, shared-accumulator form
           // Key tile tl belongs to warpgroup tl & 1 (score buffer and P buffer of that warpgroup).  Warp 1
@@ -857,7 +870,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
     if (classic && has_work) {
       if (warp == 0) {
-        produce(0, MT == 2);
+        produce(0);
       } else if (warp == 1) {
         // =========================================================== tcgen05 issuer, classic form
         // A stream is a chain  S = Q K^T -> softmax -> O += P V -> next S  on its own score buffer (which the P
