@@ -131,6 +131,13 @@ __device__ __forceinline__ void named_sync(uint32_t id, uint32_t count) {
   __syncwarp();
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
+// Producer side of barrier `id`: counts this warp's threads as arrived without waiting (the consumers use
+// named_sync with the same count).  Writes before it are visible to the consumers after their barrier.
+__device__ __forceinline__ void named_arrive(uint32_t id, uint32_t count) {
+  __threadfence_block();
+  __syncwarp();
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 // The same with an AND-reduction of a predicate over the CTA.
 __device__ __forceinline__ bool cta_sync_and(bool pred) {
   uint32_t r;

@@ -1031,7 +1031,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               m_ref = (m == -INFINITY) ? 0.0f : m * sl2;
               if (T > 1) {
                 ref_s[r] = m_ref;
-                ptx::named_sync(1, 256);
+                ptx::named_arrive(1, 256);          // warpgroup 1 waits for this, warpgroup 0 goes on
               }
             } else {
               ptx::named_sync(1, 256);
@@ -1066,7 +1066,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           if (tid == 128 && j < 4) JET_TR(20 + 2 * j);
           if (tid == 256 && j < 4) JET_TR(33 + 2 * j);
         }
-        if (T > 1 && !synced) ptx::named_sync(1, 256);       // a warpgroup that gave up early still meets the other
+        if (T > 1 && !synced) {                   // a warpgroup that gave up early still takes part in the hand-over
+          if (wg == 0) ptx::named_arrive(1, 256);
+          else ptx::named_sync(1, 256);
+        }
         if (tid == 128) JET_TR(10);
         if (ok) ok = bounded_wait(bar(Bars::kOFinal), 0, abort_flag, 11);      // the last P V is complete
         if (ok) ptx::tc_fence_after();
