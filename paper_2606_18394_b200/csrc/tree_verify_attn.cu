@@ -558,24 +558,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         int* arrive = p.counters + unit * MT + mt;
         int* depart = p.counters + p.n_units * MT + unit * MT + mt;
         uint8_t* slots = p.partials + (static_cast<size_t>(unit) * S * MT) * kBlockBytes;
-        if (!kSm && tid < S) {
-          // S threads publish one row block each (the block of owner `tid`), so the copies run in parallel
-          const int blk_lo = tid * rows_per;
-          const int blk_n = max(0, min(rows_per, kBM - blk_lo));
-          if (blk_n > 0) {
-            ptx::bulk_store_global(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes + blk_lo * C::kRecvPitch,
-                                   smem_base + C::kStageOff + static_cast<uint32_t>(blk_lo * C::kRecvPitch),
-                                   static_cast<uint32_t>(blk_n * C::kRecvPitch));
-            ptx::bulk_commit_and_wait_all();
-          }
-          ptx::fence_proxy_async_all();
-          __threadfence();
+        if (!kSm && tid == 0) JET_TR(63);
+        {
+          // every thread of the CTA copies its share of the staged block (consecutive threads, consecutive
+          // 16 bytes); the release of the arrival count below, behind the CTA-wide barrier, publishes all of it
+          const uint4* src4 = reinterpret_cast<const uint4*>(stage);
+          uint4* dst4 = reinterpret_cast<uint4*>(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes);
+          for (int i = tid; i < static_cast<int>(kBlockBytes / 16); i += C::kThreads) __stcg(dst4 + i, src4[i]);
         }
         ptx::cta_sync();
         if (!kSm && tid == 0) {
-          ptx::atom_add_release_gpu(arrive, 1);
-          bool seen = false;
-          for (uint32_t i = 0; i < (1u << 22); ++i) {
+          // the last slice to arrive knows from its own count that everybody has published
+          JET_TR(29);
+          bool seen = ptx::atom_add_acq_rel_gpu(arrive, 1) + 1 >= S;
+          JET_TR(30);
+          for (uint32_t i = 0; i < (1u << 22) && !seen; ++i) {
             if (ptx::ld_acquire_gpu(arrive) >= S) { seen = true; break; }
             __nanosleep(32);
             if (*abort_flag) break;
