@@ -265,33 +265,23 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
 
   // ---------------- set-up that touches no global memory (may overlap the previous kernel's tail)
-  if (warp == 0 && lane == 0) {
-    ptx::mbar_init(bar(Bars::kQFull), 1);
-    for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(bar(Bars::kKvFull + s), 1);
-      ptx::mbar_init(bar(Bars::kKvEmpty + s), MT == 1 ? 1 : n_mt);    // one arrival per stream that reads the stage
+  if (warp == 0) {
+    // one lane per barrier of the block
+    if (lane < Bars::kCount) {
+      uint32_t count = 1;
+      if (lane >= Bars::kKvEmpty && lane < Bars::kSFull) count = MT == 1 ? 1 : n_mt;     // one arrival per stream that reads the stage
+      else if (lane >= Bars::kSFree && lane < Bars::kODone) count = 128;                // kSFree, kPFull: a softmax warpgroup
+      else if (lane == Bars::kClusterA || lane == Bars::kClusterC) count = S;
+      ptx::mbar_init(bar(lane), count);
+      // slice merge: every slice sends this CTA its block of rows of query tile (lane - kRecv)
+      if (S > 1 && lane >= Bars::kRecv && lane < Bars::kRecv + MT)
+        ptx::mbar_arrive_expect_tx(bar(lane), S * own_n * C::kRecvPitch);
+      ptx::fence_mbar_init();
     }
-    ptx::fence_mbar_init();
-  } else if (warp == 1 && lane == 0) {
-    for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(bar(Bars::kSFull + i), 1);
+    if (lane == 31) {
+      *redo_flag = 0u;
+      *abort_flag = 0u;
     }
-    for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(bar(Bars::kPFull + i), 128);
-      ptx::mbar_init(bar(Bars::kODone + i), 1);
-      ptx::mbar_init(bar(Bars::kSFree + i), 128);
-    }
-    ptx::mbar_init(bar(Bars::kOFinal), 1);
-    *redo_flag = 0u;
-    for (int mt = 0; mt < MT; ++mt) {
-      // slice merge: every slice sends this CTA its block of rows of query tile mt
-      ptx::mbar_init(bar(Bars::kRecv + mt), 1);
-      if (S > 1) ptx::mbar_arrive_expect_tx(bar(Bars::kRecv + mt), S * own_n * C::kRecvPitch);
-    }
-    ptx::mbar_init(bar(Bars::kClusterA), S);
-    ptx::mbar_init(bar(Bars::kClusterC), S);
-    *abort_flag = 0u;
-    ptx::fence_mbar_init();
   } else if (warp == 2) {
     ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
     ptx::tmem_relinquish();
