@@ -9,6 +9,7 @@ may call it.
 from .jet_oracle import (  # noqa: F401
     anc_from_parent,
     bf16_bits_to_f64,
+    depth_entropy_ref,
     gather_paged_prefix,
     kv_compact_ref,
     target_probs_ref,

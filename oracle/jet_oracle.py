@@ -6,7 +6,10 @@ Each function follows one passage of the paper:
 
 * ``tree_build_ref``   -- Algorithm 1 (Parallel Tree Drafting) with the
   accumulated draft log-probability score of Eq. (accum_logp) in Section 3.3,
-  fed by the per-depth top-W extraction described in Section 3.3 / Appendix E.
+  fed by the per-depth top-W extraction described in Section 3.3 / Appendix E;
+  its ``score_mode`` argument selects the alternative expansion scores of
+  Appendix C (per-depth entropy alone, accumulated log-probability plus alpha
+  times the per-depth entropy), with ``depth_entropy_ref`` as the entropy.
 * ``tree_attn_ref``    -- the tree-causal mask and masked attention equations
   of Section 3.2 (prefix visible to every node, a node sees Anc(v) + {v}).
 * ``tree_accept_ref``  -- the greedy acceptance rule of Section 3.3 and
@@ -41,7 +44,13 @@ distribution the emitted token is distributed exactly as the target's), the
 closed-form expected accepted length, and the q == p / disjoint-support
 special cases; its reading of the rule for several rejected siblings (the
 single-draft residual max(0, p - q)) has no counterpart to be checked against:
-parity unpinned for that reading only.
+parity unpinned for that reading only.  The expansion scores of Appendix C are
+pinned by the limits the appendix states (alpha = 0 gives the default tree, a
+large alpha the entropy-only tree), closed-form entropies (uniform, two-point),
+closed-form trees for monotone entropies (level order / comb) and by replaying
+the pop order against priorities recomputed from the paths; whether the entropy
+term is that of the node's own depth or a sum along the branch is a reading
+with no counterpart to check against: parity unpinned for that reading only.
 """
 from __future__ import annotations
 
@@ -76,7 +85,19 @@ def gather_paged_prefix(cache: np.ndarray, page_table_row: np.ndarray, L: int) -
 # --------------------------------------------------------------------------
 # O1  tree_build  -- Algorithm 1 + Eq. (accum_logp)
 # --------------------------------------------------------------------------
-def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int) -> dict:
+def depth_entropy_ref(logp: np.ndarray, N: int) -> np.ndarray:
+    """Per-depth entropy of the draft distributions (Appendix C): H[d] = -sum_v exp(l_v) * l_v over row d of
+    the log-probabilities, summed in float64 (entries of -inf contribute 0) and rounded once to float32."""
+    H = np.zeros(N, dtype=np.float32)
+    for d in range(N):
+        l = np.asarray(logp[d], dtype=np.float64)
+        fin = np.isfinite(l)
+        H[d] = np.float32(-np.sum(np.exp(l[fin]) * l[fin]))
+    return H
+
+
+def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int,
+                   score_mode: str = "accum_logp", alpha: float = 0.0) -> dict:
     """Algorithm 1 for one sequence.
 
     ``logp`` is [N, V] float32: row d is the draft log-distribution that the
@@ -89,7 +110,20 @@ def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int) ->
     one float32 add ``score[parent] + logp[depth[parent], token]``; a popped
     node at depth N is discarded (stays in the tree as a leaf); all of a
     node's children are appended at once, cut short only by the budget.
+
+    Expansion scores (Appendix C).  ``score_mode`` selects the queue's priority; the
+    ``score`` output is the accumulated log-probability in every mode:
+      "accum_logp"  priority = score (Eq. accum_logp, the default);
+      "entropy"     priority = H of the node's depth alone;
+      "hybrid"      priority = score + alpha * H of the node's depth.
+    H of depth d >= 1 is the entropy of the distribution the depth-d tokens were
+    drawn from (row d-1 of ``logp``), see depth_entropy_ref; the root's H is 0.
+    Readings: the entropy term is the one of the node's own depth, not a sum along
+    the branch (so that alpha -> infinity is the entropy-only rule, as the appendix
+    states); it enters with a plus sign; the priority is formed in float32 as
+    fl(score + fl(alpha * H)), two roundings, no fused multiply-add.
     """
+    assert score_mode in ("accum_logp", "entropy", "hybrid")
     logp = np.asarray(logp)
     assert logp.dtype == np.float32 and logp.ndim == 2 and logp.shape[0] >= N
     V = logp.shape[1]
@@ -109,15 +143,28 @@ def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int) ->
     score = np.zeros(B, dtype=np.float32)
     score64 = np.zeros(B, dtype=np.float64)
 
+    H = depth_entropy_ref(logp, N)                     # H[d-1] belongs to the nodes of depth d
+    prio = np.zeros(B, dtype=np.float32)
+    alpha32 = np.float32(alpha)
+
+    def priority(u):
+        h = np.float32(0.0) if depth[u] == 0 else H[depth[u] - 1]
+        if score_mode == "accum_logp":
+            return score[u]
+        if score_mode == "entropy":
+            return h
+        return np.float32(score[u] + np.float32(alpha32 * h))
+
     parent[0], depth[0], token[0] = -1, 0, int(root_token)
     score[0] = np.float32(0.0)
+    prio[0] = priority(0)
     n = 1
     queue = [0]
     pops = []
     while n < B and queue:
         best = queue[0]
         for v in queue[1:]:
-            if score[v] > score[best] or (score[v] == score[best] and v < best):
+            if prio[v] > prio[best] or (prio[v] == prio[best] and v < best):
                 best = v
         queue.remove(best)
         v = best
@@ -134,6 +181,7 @@ def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int) ->
             parent[u], depth[u], token[u] = v, d + 1, y
             score[u] = np.float32(score[v]) + np.float32(logp[d, y])
             score64[u] = score64[v] + float(logp[d, y])
+            prio[u] = priority(u)
             queue.append(u)
 
     anc = np.zeros((B, words), dtype=np.uint32)
@@ -143,7 +191,7 @@ def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int) ->
         anc[u, u // 32] |= np.uint32(1) << np.uint32(u % 32)
 
     return dict(parent=parent, depth=depth, token=token, score=score, score64=score64,
-                anc_mask=anc, n_nodes=n, pops=pops,
+                anc_mask=anc, n_nodes=n, pops=pops, priority=prio, depth_entropy=H,
                 top_tok=np.stack(top).astype(np.int32) if N > 0 else np.zeros((0, Wc), np.int32))
 
 
