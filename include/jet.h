@@ -5,6 +5,7 @@
  * Four operations, in the order one verification step runs them:
  *
  *   jet_tree_build        per-depth draft log-probs -> budgeted candidate tree
+ *   jet_tree_build_scored the same with the entropy / hybrid expansion scores
  *   jet_tree_verify_attn  attention of all tree nodes over prefix KV + tree KV
  *                         under the ancestor mask (once per layer)
  *   jet_tree_accept       greedy acceptance of the deepest matching path
@@ -92,6 +93,40 @@ JET_API jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride, 
                           int32_t* parent, int32_t* depth, int32_t* token, float* score,
                           uint32_t* anc_mask, int32_t* n_nodes, void* workspace,
                           size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * jet_tree_build_scored -- jet_tree_build with the alternative expansion scores
+ * of Appendix C (tree-drafting ablation).  Everything is as for jet_tree_build,
+ * except the priority by which the pending node is taken:
+ *   JET_SCORE_ACCUM_LOGP  the accumulated log-probability (= jet_tree_build);
+ *   JET_SCORE_ENTROPY     H of the node's depth alone;
+ *   JET_SCORE_HYBRID      fl32(score + fl32(alpha * H of the node's depth)).
+ * H of depth d >= 1 is the entropy of the distribution the depth-d tokens were
+ * drawn from, H = -sum_t exp(l_t) * l_t over logp[b, d-1, :], summed in fp64
+ * (entries of -inf contribute 0) and rounded once to fp32; the root's H is 0.
+ * (The appendix gives the formula "sum log r + alpha * H" only; taken here: the
+ * entropy of the node's own depth, so that a large alpha gives the entropy-only
+ * rule as the appendix states.)  Ties -> lowest node index; `score` is the
+ * accumulated log-probability in every mode.
+ *
+ *   score_mode    one of JET_SCORE_*
+ *   alpha         finite; used by JET_SCORE_HYBRID only
+ *   depth_entropy fp32 [batch, N] out, may be NULL: H of logp[b, d, :]
+ *                 (not written with JET_SCORE_ACCUM_LOGP)
+ * Workspace: jet_tree_build_scored_workspace_bytes (larger than jet_tree_build's).
+ */
+#define JET_SCORE_ACCUM_LOGP 0
+#define JET_SCORE_ENTROPY 1
+#define JET_SCORE_HYBRID 2
+
+JET_API size_t jet_tree_build_scored_workspace_bytes(int batch, int N, int V, int W);
+
+JET_API jet_status jet_tree_build_scored(const float* logp, int64_t logp_batch_stride, int64_t logp_depth_stride,
+                                 const int32_t* root_token, int batch, int N, int V, int W, int B,
+                                 int score_mode, float alpha, int32_t* parent, int32_t* depth,
+                                 int32_t* token, float* score, uint32_t* anc_mask, int32_t* n_nodes,
+                                 float* depth_entropy, void* workspace, size_t workspace_bytes,
+                                 void* stream);
 
 /* ---------------------------------------------------------------------------
  * jet_tree_verify_attn -- the masked tree attention of Section 3.2 (tree-causal

@@ -1,5 +1,9 @@
 // jet_tree_build: per-depth top-W extraction followed by Algorithm 1 (best-first
 // budgeted tree construction with the accumulated log-probability score).
+// jet_tree_build_scored: the same with the expansion scores of Appendix C (per-depth
+// entropy alone; accumulated log-probability + alpha * per-depth entropy): the scan
+// also leaves per-slice sums of p * log p (fp64), the expansion kernel adds them up
+// per depth and uses the entropy in the queue's priority.
 //
 // Two launches:
 //   topw_partial_kernel  grid (chunks, N, batch): every block scans one slice of one
@@ -23,10 +27,13 @@ constexpr int kTopChunk = kTopThreads * kTopElems;   // vocabulary slice per blo
 // largest of the 32 per-lane maxima (tau), so only elements >= tau become candidates (as ordered 64-bit keys
 // in shared memory); the block then selects its W best among the few candidates.  Exact for any input: with
 // many equal values all of them become candidates and the key order (value, then lowest index) decides.
+// kEntropy: the block also leaves sum(exp(l) * l) over its slice (fp64; entries of -inf contribute 0) for the
+// per-depth entropy; the reduction order is fixed, so the value does not change from run to run.
+template <bool kEntropy>
 __global__ void __launch_bounds__(kTopThreads)
 topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
                     int V, int Wc, int nchunks, bool vec_ok,
-                    unsigned long long* __restrict__ cand) {
+                    unsigned long long* __restrict__ cand, double* __restrict__ plogp_partial) {
   grid_dependency_wait();
   const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31;
@@ -51,6 +58,23 @@ topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_
     for (int i = 0; i < kTopElems; ++i) {
       const int idx = base + i * kTopThreads + tid;
       v[i] = idx < V ? __ldg(row + idx) : -INFINITY;
+    }
+  }
+
+  if constexpr (kEntropy) {
+    double acc = 0.0;
+#pragma unroll
+    for (int i = 0; i < kTopElems; ++i)
+      if (v[i] > -INFINITY) acc += exp(static_cast<double>(v[i])) * static_cast<double>(v[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    __shared__ double s_acc[kTopThreads / 32];
+    if (lane == 0) s_acc[tid >> 5] = acc;
+    __syncthreads();
+    if (tid == 0) {
+      double total = 0.0;
+      for (int w = 0; w < kTopThreads / 32; ++w) total += s_acc[w];
+      plogp_partial[(static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk] = total;
     }
   }
 
@@ -124,10 +148,15 @@ topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_
 // u / 32 as a key (score, lowest index first, depth in the low byte), so a pop is a register maximum plus one
 // warp reduction, and the popped node's score and depth come out of the key itself.  kSlots = registers per
 // lane (32 * kSlots >= B); the instruction count of a pop grows with it, hence the template.
-template <int kSlots>
+// kMode: 0 = priority is the accumulated log-probability (the key's value is the node's score); 1 = priority
+// is the entropy of the node's depth; 2 = score + alpha * that entropy, formed as two rounded float operations.
+// depth_h[d] = entropy of the distribution the tokens of depth d + 1 were drawn from.  In modes 1 and 2 the
+// popped node's score is read back from shared memory.
+template <int kSlots, int kMode>
 __device__ __forceinline__ int expand_tree(int lane, int N, int Wc, int B, int root, const float (*top_lp)[JET_MAX_WIDTH],
                                            const int32_t (*top_tok)[JET_MAX_WIDTH], int32_t* s_parent,
-                                           int32_t* s_depth, int32_t* s_token, float* s_score) {
+                                           int32_t* s_depth, int32_t* s_token, float* s_score,
+                                           const float* depth_h, float alpha) {
   unsigned long long q[kSlots];
 #pragma unroll
   for (int i = 0; i < kSlots; ++i) q[i] = 0ull;
@@ -149,7 +178,9 @@ __device__ __forceinline__ int expand_tree(int lane, int N, int Wc, int B, int r
     if (best == 0ull) break;                        // nothing pending
     const int v = static_cast<int>(0xFFFFFFu - (static_cast<uint32_t>(best >> 8) & 0xFFFFFFu));
     const int d = static_cast<int>(best & 0xFFull);
-    const float sv = key_value(best);
+    float sv;
+    if constexpr (kMode == 0) sv = key_value(best);
+    else sv = s_score[v];
 #pragma unroll
     for (int i = 0; i < kSlots; ++i) if (q[i] == best) q[i] = 0ull;      // popped (only its keeper matches)
     if (d < N) {
@@ -159,11 +190,15 @@ __device__ __forceinline__ int expand_tree(int lane, int N, int Wc, int B, int r
         const int u = n + j;
         const float s = __fadd_rn(sv, top_lp[d][j]);
         s_parent[u] = v; s_depth[u] = d + 1; s_token[u] = top_tok[d][j]; s_score[u] = s;
-        const unsigned long long key = queue_key(s, u, d + 1);
+        float prio = s;
+        if constexpr (kMode == 1) prio = depth_h[d];
+        if constexpr (kMode == 2) prio = __fadd_rn(s, __fmul_rn(alpha, depth_h[d]));
+        const unsigned long long key = queue_key(prio, u, d + 1);
 #pragma unroll
         for (int i = 0; i < kSlots; ++i) if (i == (u >> 5)) q[i] = key;
       }
       n += cnt;
+      if constexpr (kMode != 0) __syncwarp();          // the children's scores are read back when they are popped
     }
   }
   return n;
@@ -171,18 +206,21 @@ __device__ __forceinline__ int expand_tree(int lane, int N, int Wc, int B, int r
 
 constexpr int kExpThreads = 256;
 
+template <int kMode>
 __global__ void __launch_bounds__(kExpThreads)
 tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
                    const int32_t* __restrict__ root_token, int N, int Wc, int B, int nchunks,
                    const unsigned long long* __restrict__ cand,
                    int32_t* __restrict__ parent_out, int32_t* __restrict__ depth_out,
                    int32_t* __restrict__ token_out, float* __restrict__ score_out,
-                   uint32_t* __restrict__ anc_out, int32_t* __restrict__ n_nodes_out) {
+                   uint32_t* __restrict__ anc_out, int32_t* __restrict__ n_nodes_out,
+                   const double* __restrict__ plogp_partial, float alpha, float* __restrict__ depth_entropy_out) {
   grid_dependency_wait();
   __shared__ int32_t s_top_tok[JET_MAX_DEPTH][JET_MAX_WIDTH];
   __shared__ float s_top_lp[JET_MAX_DEPTH][JET_MAX_WIDTH];
   __shared__ int32_t s_parent[JET_MAX_NODES], s_depth[JET_MAX_NODES], s_token[JET_MAX_NODES];
   __shared__ float s_score[JET_MAX_NODES];
+  __shared__ float s_depth_h[JET_MAX_DEPTH];
   __shared__ int s_n;
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -190,6 +228,19 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   // ---- merge the per-slice candidates: depth d's W best of nchunks*Wc keys (keys are unique,
   //      so "largest key below the previous winner" walks them in rank order)
   for (int d = warp; d < N; d += kExpThreads / 32) {
+    if constexpr (kMode != 0) {
+      // entropy of row d: minus the sum of the slices' partial sums (fp64, fixed order), rounded once
+      const double* part = plogp_partial + (static_cast<size_t>(b) * N + d) * nchunks;
+      double acc = 0.0;
+      for (int i = lane; i < nchunks; i += 32) acc += part[i];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) {
+        const float h = static_cast<float>(-acc);
+        s_depth_h[d] = h;
+        if (depth_entropy_out) depth_entropy_out[static_cast<size_t>(b) * N + d] = h;
+      }
+    }
     const unsigned long long* c = cand + (static_cast<size_t>(b) * N + d) * nchunks * Wc;
     const int total = nchunks * Wc;
     constexpr int kHeld = 16;                 // candidates a lane can keep in registers
@@ -226,11 +277,11 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   if (warp == 0) {
     const int root = root_token[b];
     int n;
-    if (B <= 32) n = expand_tree<1>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
-    else if (B <= 64) n = expand_tree<2>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
-    else if (B <= 128) n = expand_tree<4>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
-    else if (B <= 256) n = expand_tree<8>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
-    else n = expand_tree<JET_MAX_NODES / 32>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score);
+    if (B <= 32) n = expand_tree<1, kMode>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score, s_depth_h, alpha);
+    else if (B <= 64) n = expand_tree<2, kMode>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score, s_depth_h, alpha);
+    else if (B <= 128) n = expand_tree<4, kMode>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score, s_depth_h, alpha);
+    else if (B <= 256) n = expand_tree<8, kMode>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score, s_depth_h, alpha);
+    else n = expand_tree<JET_MAX_NODES / 32, kMode>(lane, N, Wc, B, root, s_top_lp, s_top_tok, s_parent, s_depth, s_token, s_score, s_depth_h, alpha);
     if (lane == 0) s_n = n;
   }
   __syncthreads();
@@ -260,13 +311,60 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
 
 int chunks_for(int V) { return (V + kTopChunk - 1) / kTopChunk; }
 
+size_t cand_bytes(int batch, int N, int V, int W) {
+  const size_t Wc = static_cast<size_t>(W < V ? W : V);
+  return round_up(static_cast<size_t>(batch) * N * chunks_for(V) * Wc * sizeof(unsigned long long), 256);
+}
+
+// Checks and launches shared by the two entry points (score_mode: JET_SCORE_*).
+jet_status tree_build_launch(const float* logp, int64_t logp_batch_stride, int64_t logp_depth_stride,
+                             const int32_t* root_token, int batch, int N, int V, int W, int B, int score_mode,
+                             float alpha, int32_t* parent, int32_t* depth, int32_t* token, float* score,
+                             uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy, void* workspace,
+                             size_t workspace_bytes, size_t need, void* stream) {
+  if (!logp || !root_token || !parent || !depth || !token || !anc_mask || !n_nodes)
+    return JET_ERR_INVALID_ARG;
+  if (batch < 1 || batch > 65535 || N < 1 || N > JET_MAX_DEPTH || W < 1 || W > JET_MAX_WIDTH || V < 1 ||
+      B < 1 || B > JET_MAX_NODES || logp_depth_stride < V || logp_batch_stride < 0)
+    return JET_ERR_INVALID_ARG;
+  if (score_mode < JET_SCORE_ACCUM_LOGP || score_mode > JET_SCORE_HYBRID) return JET_ERR_INVALID_ARG;
+  if (score_mode == JET_SCORE_HYBRID && !(alpha == alpha && alpha > -INFINITY && alpha < INFINITY)) return JET_ERR_INVALID_ARG;
+  if (!aligned(logp, 4)) return JET_ERR_INVALID_ARG;
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
+
+  const int Wc = W < V ? W : V;
+  const int nchunks = chunks_for(V);
+  const bool vec_ok = aligned(logp, 16) && logp_batch_stride % 4 == 0 && logp_depth_stride % 4 == 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  auto* cand = static_cast<unsigned long long*>(workspace);
+  auto* plogp = reinterpret_cast<double*>(static_cast<uint8_t*>(workspace) + cand_bytes(batch, N, V, W));
+  if (score_mode == JET_SCORE_ACCUM_LOGP) {
+    launch_dependent(topw_partial_kernel<false>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+        logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, static_cast<double*>(nullptr));
+    launch_dependent(tree_expand_kernel<0>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
+        root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
+        static_cast<const double*>(nullptr), 0.0f, static_cast<float*>(nullptr));
+    return launch_status();
+  }
+  launch_dependent(topw_partial_kernel<true>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+      logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, plogp);
+  if (score_mode == JET_SCORE_ENTROPY)
+    launch_dependent(tree_expand_kernel<1>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
+        root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
+        static_cast<const double*>(plogp), 0.0f, depth_entropy);
+  else
+    launch_dependent(tree_expand_kernel<2>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
+        root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
+        static_cast<const double*>(plogp), alpha, depth_entropy);
+  return launch_status();
+}
+
 }  // namespace
 }  // namespace jet
 
 extern "C" size_t jet_tree_build_workspace_bytes(int batch, int N, int V, int W) {
   if (batch < 1 || N < 1 || V < 1 || W < 1) return 0;
-  const size_t Wc = static_cast<size_t>(W < V ? W : V);
-  return jet::round_up(static_cast<size_t>(batch) * N * jet::chunks_for(V) * Wc * sizeof(unsigned long long), 256);
+  return jet::cand_bytes(batch, N, V, W);
 }
 
 extern "C" jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride,
@@ -275,25 +373,26 @@ extern "C" jet_status jet_tree_build(const float* logp, int64_t logp_batch_strid
                                      int32_t* depth, int32_t* token, float* score,
                                      uint32_t* anc_mask, int32_t* n_nodes, void* workspace,
                                      size_t workspace_bytes, void* stream) {
-  using namespace jet;
-  if (!logp || !root_token || !parent || !depth || !token || !anc_mask || !n_nodes)
-    return JET_ERR_INVALID_ARG;
-  if (batch < 1 || batch > 65535 || N < 1 || N > JET_MAX_DEPTH || W < 1 || W > JET_MAX_WIDTH || V < 1 ||
-      B < 1 || B > JET_MAX_NODES || logp_depth_stride < V || logp_batch_stride < 0)
-    return JET_ERR_INVALID_ARG;
-  if (!aligned(logp, 4)) return JET_ERR_INVALID_ARG;
-  const size_t need = jet_tree_build_workspace_bytes(batch, N, V, W);
-  if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return JET_ERR_WORKSPACE;
+  const size_t need = (batch >= 1 && N >= 1 && V >= 1 && W >= 1) ? jet::cand_bytes(batch, N, V, W) : 0;
+  return jet::tree_build_launch(logp, logp_batch_stride, logp_depth_stride, root_token, batch, N, V, W, B,
+                                JET_SCORE_ACCUM_LOGP, 0.0f, parent, depth, token, score, anc_mask, n_nodes, nullptr,
+                                workspace, workspace_bytes, need, stream);
+}
 
-  const int Wc = W < V ? W : V;
-  const int nchunks = chunks_for(V);
-  const bool vec_ok = aligned(logp, 16) && logp_batch_stride % 4 == 0 && logp_depth_stride % 4 == 0;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  auto* cand = static_cast<unsigned long long*>(workspace);
-  launch_dependent(topw_partial_kernel, dim3(nchunks, N, batch), dim3(kTopThreads), st,
-      logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand);
-  launch_dependent(tree_expand_kernel, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
-                                                     root_token, N, Wc, B, nchunks, cand, parent,
-                                                     depth, token, score, anc_mask, n_nodes);
-  return launch_status();
+extern "C" size_t jet_tree_build_scored_workspace_bytes(int batch, int N, int V, int W) {
+  if (batch < 1 || N < 1 || V < 1 || W < 1) return 0;
+  return jet::cand_bytes(batch, N, V, W) +
+         jet::round_up(static_cast<size_t>(batch) * N * jet::chunks_for(V) * sizeof(double), 256);
+}
+
+extern "C" jet_status jet_tree_build_scored(const float* logp, int64_t logp_batch_stride,
+                                            int64_t logp_depth_stride, const int32_t* root_token,
+                                            int batch, int N, int V, int W, int B, int score_mode, float alpha,
+                                            int32_t* parent, int32_t* depth, int32_t* token, float* score,
+                                            uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy,
+                                            void* workspace, size_t workspace_bytes, void* stream) {
+  const size_t need = jet_tree_build_scored_workspace_bytes(batch, N, V, W);
+  return jet::tree_build_launch(logp, logp_batch_stride, logp_depth_stride, root_token, batch, N, V, W, B, score_mode,
+                                alpha, parent, depth, token, score, anc_mask, n_nodes, depth_entropy, workspace,
+                                workspace_bytes, need, stream);
 }

@@ -49,6 +49,28 @@ def run_tree_build(logp, root_token, N, W, B, with_score=True):
                 anc_mask=anc.cpu().numpy().view(np.uint32), n_nodes=n_nodes.cpu().numpy())
 
 
+def run_tree_build_scored(logp, root_token, N, W, B, score_mode, alpha):
+    """As run_tree_build, through jet_tree_build_scored; also returns depth_entropy [batch,N]."""
+    batch, _, V = logp.shape
+    d_logp = dev(logp)
+    d_root = dev(np.asarray(root_token, dtype=np.int32))
+    words = (B + 31) // 32
+    parent = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
+    depth = torch.full_like(parent, -7)
+    token = torch.full_like(parent, -7)
+    score = torch.full((batch, B), 123.0, dtype=torch.float32, device=DEV)
+    anc = torch.full((batch, B, words), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
+    n_nodes = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
+    ent = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
+    ws = workspace(jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W))
+    jet.jet_tree_build_scored(d_logp, d_root, batch, N, V, W, B, score_mode, alpha, parent, depth, token, score,
+                              anc, n_nodes, ent, ws)
+    torch.cuda.synchronize()
+    return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
+                score=score.cpu().numpy(), anc_mask=anc.cpu().numpy().view(np.uint32),
+                n_nodes=n_nodes.cpu().numpy(), depth_entropy=ent.cpu().numpy())
+
+
 def run_tree_accept(logits, token, parent, depth, anc_mask, n_nodes, N):
     """logits [batch,B,V]; tree arrays [batch,B]; returns dict of numpy arrays."""
     batch, B, V = logits.shape
