@@ -147,7 +147,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-def build_inputs(c, name, seed, device):
+def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0):
     """Seeded synthetic step inputs on the device.  Returns (VerifyStep, info dict)."""
     import torch
     from paper_2606_18394_b200.step import VerifyStep
@@ -195,6 +195,7 @@ def build_inputs(c, name, seed, device):
     st.root_token.copy_(torch.arange(batch, device=device, dtype=torch.int32) + 1)
     st.logits.copy_(torch.randn(st.logits.shape, generator=gen, device=device, dtype=torch.float32) * c["sigma_target"])
     # plant the target arg-max along one random path of the tree that jet_tree_build produces
+    st.score_mode, st.score_alpha = score_mode, score_alpha
     st.seq_len.copy_(st.seq_len0)
     st.tree_build()
     torch.cuda.synchronize()
@@ -261,7 +262,7 @@ def bench_jet(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
     c = workload(args.config)
-    st, info = build_inputs(c, args.config, rank_seed(2, rank), device)
+    st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha)
     layers = c["layers"]
     if args.accept == "sample":
         st.accept_mode = "sample"
@@ -409,7 +410,8 @@ def bench_jet(args):
                    "tree_nodes": c["B"], "max_depth": c["N"], "width": c["W"], "vocab": c["V"],
                    "paged": bool(c.get("paged")), "cuda_graph": not args.no_graph,
                    "l2": "every layer streams its own KV buffers; one step reads far more than the 126 MB L2",
-                   "accepted_len": acc, "accept": args.accept},
+                   "accepted_len": acc, "accept": args.accept,
+                   "score": args.score if args.score != "hybrid" else f"hybrid(alpha={args.score_alpha})"},
         "attn_us_per_layer": attn_us,
         "e2e": {"value": e2e_ms_step * 1e3 / (layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step},
@@ -537,6 +539,9 @@ def main():
     ap.add_argument("--config", default="qwen3_8b", choices=[k for k, v in CONFIGS.items() if "B" in v])
     ap.add_argument("--no-graph", action="store_true", help="issue the calls directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--score", choices=["accum_logp", "entropy", "hybrid"], default="accum_logp",
+                    help="expansion score of the tree construction (hybrid: --score-alpha)")
+    ap.add_argument("--score-alpha", type=float, default=1.0)
     ap.add_argument("--accept", choices=["greedy", "sample"], default="greedy",
                     help="acceptance rule of the step: greedy (the headline) or the non-greedy rule at temperature 1")
     args = ap.parse_args()

@@ -64,7 +64,12 @@ class VerifyStep:
         # ---- workspaces
         def ws(nbytes):
             return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=dev)
-        self.ws_build = ws(jet.jet_tree_build_workspace_bytes(batch, N, V, W))
+        self.ws_build = ws(max(jet.jet_tree_build_workspace_bytes(batch, N, V, W),
+                               jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W)))
+        # expansion score of the tree construction: "accum_logp" (default), "entropy" or "hybrid" (+ score_alpha)
+        self.score_mode = "accum_logp"
+        self.score_alpha = 0.0
+        self.depth_entropy = torch.zeros((batch, N), dtype=torch.float32, device=dev)
         self.ws_attn = ws(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, self.attn_max_len))
         self.ws_attn.zero_()         # its counters must start at zero; every call leaves them zero
         self.ws_accept = ws(max(jet.jet_tree_accept_workspace_bytes(batch, B, V),
@@ -91,8 +96,14 @@ class VerifyStep:
 
     # ------------------------------------------------------------------ the four calls
     def tree_build(self):
-        jet.jet_tree_build(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, self.parent,
-                           self.depth, self.token, self.score, self.anc_mask, self.n_nodes, self.ws_build)
+        if self.score_mode == "accum_logp":
+            jet.jet_tree_build(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, self.parent,
+                               self.depth, self.token, self.score, self.anc_mask, self.n_nodes, self.ws_build)
+        else:
+            mode = {"entropy": 1, "hybrid": 2}[self.score_mode]
+            jet.jet_tree_build_scored(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, mode,
+                                      self.score_alpha, self.parent, self.depth, self.token, self.score,
+                                      self.anc_mask, self.n_nodes, self.depth_entropy, self.ws_build)
 
     def verify_attn(self, layer):
         jet.jet_tree_verify_attn(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
