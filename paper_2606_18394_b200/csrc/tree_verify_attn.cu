@@ -199,16 +199,32 @@ __device__ __forceinline__ void mask_chunk(uint32_t (&x)[32], uint32_t bits) {
 // 32 scores of one row -> probabilities (exp2 of the scaled, shifted score; a score of -inf gives exactly
 // 0), added to the row sum and written as packed bf16 pairs to 16 TMEM columns of the row's lane (the A
 // operand of the P V product).  The stages are kept apart so that the 32 independent exp2 are in flight
-// together.
+// together.  The scale-and-shift and the row sum take two values per instruction (fma.rn.f32x2 /
+// add.rn.f32x2: the same roundings as the scalar forms, half the issue slots); sum[j & 3] collects column j.
 __device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, float m_ref, float (&sum)[4],
                                           uint32_t p_tmem) {
+  using u64 = unsigned long long;
+  auto pk2 = [](uint32_t lo, uint32_t hi) { u64 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi)); return r; };
+  const u64 s2 = pk2(__float_as_uint(sl2), __float_as_uint(sl2));
+  const u64 m2 = pk2(__float_as_uint(-m_ref), __float_as_uint(-m_ref));
   float e[32];
 #pragma unroll
-  for (int j = 0; j < 32; ++j) e[j] = fmaf(__uint_as_float(x[j]), sl2, -m_ref);
+  for (int j = 0; j < 32; j += 2) {
+    u64 t;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(t) : "l"(pk2(x[j], x[j + 1])), "l"(s2), "l"(m2));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(e[j]), "=f"(e[j + 1]) : "l"(t));
+  }
 #pragma unroll
   for (int j = 0; j < 32; ++j) e[j] = exp2f(e[j]);
+  u64 acc0 = pk2(__float_as_uint(sum[0]), __float_as_uint(sum[1]));
+  u64 acc1 = pk2(__float_as_uint(sum[2]), __float_as_uint(sum[3]));
 #pragma unroll
-  for (int j = 0; j < 32; ++j) sum[j & 3] += e[j];
+  for (int j = 0; j < 32; j += 4) {
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc0) : "l"(pk2(__float_as_uint(e[j]), __float_as_uint(e[j + 1]))));
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(acc1) : "l"(pk2(__float_as_uint(e[j + 2]), __float_as_uint(e[j + 3]))));
+  }
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(sum[0]), "=f"(sum[1]) : "l"(acc0));
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(sum[2]), "=f"(sum[3]) : "l"(acc1));
   uint32_t packed[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) packed[j] = pack_bf16(e[2 * j], e[2 * j + 1]);
