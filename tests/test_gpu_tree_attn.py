@@ -147,6 +147,35 @@ def test_scores_far_above_the_first_tile(jump, where):
     assert np.abs(lse[0] - rlse).max() <= 1e-3 * max(1.0, np.abs(rlse).max())
 
 
+def test_scores_far_above_the_first_tile_headline_shape():
+    """The same at the benchmark's shape (16 work items x 9 key slices that merge through the workspace): only
+    some slices contain the overflowing keys, so CTAs that kept the fixed reference and CTAs that fell back to
+    the exact pass are merged with each other."""
+    import jet_harness as H
+    from jet_inputs import bf16_bits_to_f32, f32_to_bf16_bits
+    B, Hq, Hkv, D, L = 64, 32, 8, 128, 4096
+    rng = np.random.default_rng(78)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    x["q"] = f32_to_bf16_bits(np.abs(bf16_bits_to_f32(x["q"])) * 0.25)
+    k = bf16_bits_to_f32(x["k_prefix"]) * 0.05
+    k[1500:1700] = 10.0                                         # inside the 4th of the 9 slices, not at its start
+    x["k_prefix"] = f32_to_bf16_bits(k)
+    parent, _, _ = random_tree(B, rng)
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0
+    rows = [(int(rng.integers(0, B)), int(rng.integers(0, Hq))) for _ in range(64)] + [(0, 0), (B - 1, Hq - 1)]
+    ref, rlse = tree_attn_rows_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale,
+                                   rows)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [L],
+                                   x["tree_k"][None], x["tree_v"][None], anc[None], [B], scale)
+    assert st == 0 and not np.isnan(out).any()
+    got = np.stack([out[0, v, h] for v, h in rows])
+    err = np.abs(got - ref)
+    assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR
+    got_lse = np.array([lse[0, h, v] for v, h in rows])
+    assert np.abs(got_lse - rlse).max() <= 1e-3 * max(1.0, np.abs(rlse).max())
+
+
 def test_sweep_16k_sampled_rows():
     """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
     import jet_harness as H
