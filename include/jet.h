@@ -176,6 +176,24 @@ JET_API jet_status jet_tree_verify_attn(const void* q, const void* k_cache, cons
                                 int32_t* device_status, void* workspace, size_t workspace_bytes,
                                 void* stream);
 
+/* jet_tree_verify_attn_tail -- the same attention for a cache that already holds
+ * the tree's K/V rows behind the prefix (the serving layout of Appendix E: the
+ * tree lives in the tail of the paged cache): node v of sequence b is the cache
+ * row at position seq_len[b] + v (contiguous or through the page table), there are
+ * no tree_k / tree_v buffers.  The key tiles then run over positions
+ * 0 .. seq_len[b] + n_nodes[b] - 1 without a break between prefix and tree.
+ * max_seq_len bounds seq_len[b] + n_nodes[b] (and is the row extent of a
+ * contiguous cache); rows of padding nodes may hold anything.  Everything else as
+ * for jet_tree_verify_attn; same workspace query.
+ */
+JET_API jet_status jet_tree_verify_attn_tail(const void* q, const void* k_cache, const void* v_cache,
+                                     const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                     int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                     const uint32_t* anc_mask, const int32_t* n_nodes, int batch, int B,
+                                     int Hq, int Hkv, int D, int64_t kv_batch_stride, float softmax_scale,
+                                     void* out, float* lse, int32_t* device_status, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------
  * jet_tree_accept -- greedy acceptance (Section 3.3, Appendix E): a node is
  * accepted iff its token equals the target's arg-max prediction at its parent;
@@ -296,6 +314,18 @@ JET_API jet_status jet_kv_compact(const void* tree_k, const void* tree_v, void* 
                           const int32_t* page_table, int max_pages_per_seq, int page_size,
                           const int32_t* path, const int32_t* accept_len, int32_t* seq_len,
                           int layers, int batch, int B, int Hkv, int D, int N, void* stream);
+
+/* jet_kv_compact_tail -- the commit for the layout of jet_tree_verify_attn_tail:
+ * for every layer, sequence b and i in [1, accept_len[b]] the K and V rows at
+ * position seq_len[b] + path[b,i] move to position seq_len[b] + i (the root's row
+ * is already in place; all rows are read before any is written); afterwards
+ * seq_len[b] += accept_len[b] + 1.  Rows behind the new length keep what they held.
+ */
+JET_API jet_status jet_kv_compact_tail(void* k_cache, void* v_cache, int64_t cache_layer_stride,
+                               int64_t kv_batch_stride, const int32_t* page_table, int max_pages_per_seq,
+                               int page_size, const int32_t* path, const int32_t* accept_len,
+                               int32_t* seq_len, int layers, int batch, int B, int Hkv, int D, int N,
+                               void* stream);
 
 #ifdef __cplusplus
 }

@@ -12,6 +12,7 @@ from .jet_oracle import (  # noqa: F401
     depth_entropy_ref,
     gather_paged_prefix,
     kv_compact_ref,
+    kv_compact_tail_ref,
     target_probs_ref,
     tree_accept_ref,
     tree_accept_sample_ref,

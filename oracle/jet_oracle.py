@@ -17,7 +17,9 @@ Each function follows one passage of the paper:
   prediction at its parent; the deepest fully accepted root-to-node path wins
   and the target prediction at its last node is the correction token.
 * ``kv_compact_ref``   -- "the accepted path is committed" (Appendix E): the
-  K/V rows of the accepted path are copied behind the prefix.
+  K/V rows of the accepted path are copied behind the prefix;
+  ``kv_compact_tail_ref`` is the same commit for a cache that already holds the
+  tree's rows behind the prefix (the serving layout of Appendix E).
 * ``tree_accept_sample_ref`` -- the non-greedy acceptance rule of Section 3.3
   (Eq. nongreedy_specdec): along every branch a draft token is accepted with
   probability min(1, p/q); a correction token is sampled from the target where
@@ -35,7 +37,8 @@ Pins (tests marked "not gpu"): brute-force full-tree enumeration, closed forms
 torch's CPU scaled_dot_product_attention, zero influence of masked nodes and
 uniform-V for ``tree_attn_ref``; the expected-token closed form of Eq. (1) on
 chains, the ancestor-bitmask formulation and planted paths for
-``tree_accept_ref``; attention-after-commit round trip for ``kv_compact_ref``.
+``tree_accept_ref``; attention-after-commit round trip for ``kv_compact_ref``,
+and agreement of ``kv_compact_tail_ref`` with it on a cache whose tail holds the tree.
 The tie-break conventions themselves have no counterpart to be checked
 against (the authors' code is not available): parity unpinned for tie-breaks
 only.  ``tree_accept_sample_ref`` is pinned by the defining property of
@@ -479,6 +482,38 @@ def kv_compact_ref(tree_k, tree_v, k_cache, v_cache, page_table, path, accept_le
                     page = int(page_table[b, pos // page_size])
                     k_out[layer, page, pos % page_size] = tree_k[layer, b, node]
                     v_out[layer, page, pos % page_size] = tree_v[layer, b, node]
+    for b in range(batch):
+        new_len[b] = seq_len[b] + accept_len[b] + 1
+    return k_out, v_out, new_len
+
+
+def kv_compact_tail_ref(k_cache, v_cache, page_table, path, accept_len, seq_len):
+    """The commit when the tree's K/V rows already sit in the cache behind the prefix (node v of
+    sequence b at position ``seq_len[b] + v``; layouts as in kv_compact_ref): for i = 1..accept_len[b]
+    the row at position ``seq_len[b] + path[b,i]`` moves to position ``seq_len[b] + i`` (the root's row
+    stays), every row is read before any is written, and the new length is ``seq_len[b] +
+    accept_len[b] + 1``.  Rows beyond the new length keep whatever they held.  Returns new
+    (k_cache, v_cache, seq_len)."""
+    k_out = np.array(k_cache, copy=True)
+    v_out = np.array(v_cache, copy=True)
+    new_len = np.array(seq_len, copy=True)
+    layers = k_cache.shape[0]
+    batch = len(seq_len)
+
+    def slot(b, pos):
+        if page_table is None:
+            return (b, pos)
+        page_size = k_cache.shape[2]
+        return (int(page_table[b, pos // page_size]), pos % page_size)
+
+    for layer in range(layers):
+        for b in range(batch):
+            L = int(seq_len[b])
+            for i in range(1, int(accept_len[b]) + 1):
+                src = slot(b, L + int(path[b, i]))
+                dst = slot(b, L + i)
+                k_out[(layer,) + dst] = k_cache[(layer,) + src]        # sources are read from the old cache
+                v_out[(layer,) + dst] = v_cache[(layer,) + src]
     for b in range(batch):
         new_len[b] = seq_len[b] + accept_len[b] + 1
     return k_out, v_out, new_len

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     JetError,
     exported_symbols,
     jet_kv_compact,
+    jet_kv_compact_tail,
     jet_tree_accept,
     jet_tree_accept_sample,
     jet_tree_accept_sample_workspace_bytes,
@@ -24,6 +25,7 @@ from .binding import (  # noqa: F401
     jet_tree_build_scored_workspace_bytes,
     jet_tree_build_workspace_bytes,
     jet_tree_verify_attn,
+    jet_tree_verify_attn_tail,
     jet_tree_verify_attn_workspace_bytes,
     load,
     status_string,

@@ -35,6 +35,10 @@ _SIGNATURES = {
     "jet_tree_verify_attn_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "jet_tree_verify_attn": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp,
                                           _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "jet_tree_verify_attn_tail": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp,
+                                               _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "jet_kv_compact_tail": (_c.c_int32, [_vp, _vp, _i64, _i64, _vp, _i, _i, _vp, _vp, _vp, _i, _i, _i, _i,
+                                         _i, _i, _vp]),
     "jet_tree_accept_workspace_bytes": (_sz, [_i, _i, _i]),
     "jet_tree_accept": (_c.c_int32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp,
                                      _vp, _vp, _sz, _vp]),
@@ -157,6 +161,32 @@ def jet_tree_verify_attn(q, k_cache, v_cache, page_table, max_pages_per_seq, pag
                                      _stream(stream))
     if check:
         _check(st, "jet_tree_verify_attn")
+    return st
+
+
+def jet_tree_verify_attn_tail(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len,
+                              max_seq_len, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride,
+                              softmax_scale, out, lse, device_status, workspace, workspace_bytes=None, stream=None,
+                              check=True):
+    wb = workspace_bytes if workspace_bytes is not None else (workspace.numel() * workspace.element_size()
+                                                              if workspace is not None else 0)
+    st = load().jet_tree_verify_attn_tail(_p(q), _p(k_cache), _p(v_cache), _p(page_table), max_pages_per_seq,
+                                          page_size, num_pages, _p(seq_len), max_seq_len, _p(anc_mask),
+                                          _p(n_nodes), batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
+                                          _p(out), _p(lse), _p(device_status), _p(workspace), wb, _stream(stream))
+    if check:
+        _check(st, "jet_tree_verify_attn_tail")
+    return st
+
+
+def jet_kv_compact_tail(k_cache, v_cache, cache_layer_stride, kv_batch_stride, page_table, max_pages_per_seq,
+                        page_size, path, accept_len, seq_len, layers, batch, B, Hkv, D, N, stream=None,
+                        check=True):
+    st = load().jet_kv_compact_tail(_p(k_cache), _p(v_cache), cache_layer_stride, kv_batch_stride, _p(page_table),
+                                    max_pages_per_seq, page_size, _p(path), _p(accept_len), _p(seq_len), layers,
+                                    batch, B, Hkv, D, N, _stream(stream))
+    if check:
+        _check(st, "jet_kv_compact_tail")
     return st
 
 

@@ -59,6 +59,7 @@ struct AttnParams {
   float* lse;
   int32_t* status;
   int max_pages, paged;
+  int tail;           // the tree's K/V rows sit in the cache behind the prefix (rows seq_len .. seq_len + n - 1)
   int batch, B, Hq, Hkv, G, words;
   int nsplit, n_mgroups, n_units;
   int via_global;     // key slices exchange their rows through the workspace instead of a cluster
@@ -374,8 +375,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int L = p.seq_len[b];
   const int n = min(p.n_nodes[b], p.B);
   const int ntree = min(n, node_hi);                         // tree keys any row here can see
-  const int TP = (L + kBN - 1) / kBN;
-  const int TT = (ntree + kBN - 1) / kBN;
+  // Keys that come out of the cache: the prefix, and with p.tail also the tree's own rows behind it (then
+  // there are no separate tree tiles: key j >= L is tree node j - L).
+  const int Lc = p.tail ? L + ntree : L;
+  const int TP = (Lc + kBN - 1) / kBN;
+  const int TT = p.tail ? 0 : (ntree + kBN - 1) / kBN;
   const int T_all = TP + TT;
   // key tiles of this slice; when they do not divide evenly the first slices take the extra tile, so that
   // the last slice, whose tree tile (masked) is the slowest kind, has the fewest
@@ -719,7 +723,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
       // fetched while the current tile's copies are issued, so the table look-up is off the critical path
       auto tile_page = [&](int t) -> int {
-        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= L) return 0;
+        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= Lc) return 0;
         return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
       };
       int kt = 0, vt = 0;                       // next K tile, next V tile
@@ -737,7 +741,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint32_t dst = sKV + stage * C::kStageBytes;
         const uint32_t full = lbar(Bars::kKvFull + stage);
         if (t < TP && p.paged) {
-          const int npages = min(8, (L - t * kBN + 15) / 16);
+          const int npages = min(8, (Lc - t * kBN + 15) / 16);
           const int page = take_k ? pk_cur : pv_cur;
           if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * kHalves * 2048);
           __syncwarp();
@@ -961,8 +965,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // visibility bits of this row for 32-key chunk c of key tile t (a tile that is not full)
     auto chunk_bits = [&](int t, int c) -> uint32_t {
       if (t < TP) {
-        const int nv = (L - t * kBN) - c * 32;
-        return nv >= 32 ? 0xFFFFFFFFu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+        const int nv = (L - t * kBN) - c * 32;              // prefix keys in this chunk (all of them visible)
+        if (nv >= 32) return 0xFFFFFFFFu;
+        const uint32_t prefix_bits = nv <= 0 ? 0u : ((1u << nv) - 1u);
+        if (!p.tail) return prefix_bits;
+        // the rest of the chunk are tree nodes s, s + 1, ... (s = -nv; negative: the chunk starts in the prefix)
+        auto word = [&](int i) -> uint32_t { return (row_live && i >= 0 && i < p.words) ? __ldg(mask_row + i) : 0u; };
+        if (nv > 0) return prefix_bits | (word(0) << nv);
+        const int s = -nv, w = s >> 5, sh = s & 31;
+        return sh ? ((word(w) >> sh) | (word(w + 1) << (32 - sh))) : word(w);
       }
       const int w = (t - TP) * 4 + c;
       return (row_live && w < p.words) ? __ldg(mask_row + w) : 0u;
@@ -971,7 +982,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // cache rows, rows of padding nodes) are cleared before the P V product may read them.  `item` = the V
     // tile's position in the ring.  Returns false if the wait for the tile gave up.
     auto clear_v_tail = [&](int t, int item) -> bool {
-      const int valid = t < TP ? min(kBN, L - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
+      const int valid = t < TP ? min(kBN, Lc - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
       if (valid >= kBN) return true;
       const int stage = item % kStages;
       if (!bounded_wait(lbar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 10)) return false;
@@ -1473,16 +1484,19 @@ extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq,
   return jet::workspace_need(jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len), D);
 }
 
-extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
-                                           const int32_t* page_table, int max_pages_per_seq, int page_size,
-                                           int64_t num_pages, const int32_t* seq_len, int max_seq_len,
-                                           const void* tree_k, const void* tree_v, const uint32_t* anc_mask,
-                                           const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D,
-                                           int64_t kv_batch_stride, float softmax_scale, void* out, float* lse,
-                                           int32_t* device_status, void* workspace, size_t workspace_bytes,
-                                           void* stream) {
-  using namespace jet;
-  if (!q || !seq_len || !tree_k || !tree_v || !anc_mask || !n_nodes || !out) return JET_ERR_INVALID_ARG;
+namespace jet {
+namespace {
+
+// Checks, tensor maps and launch shared by the two entry points.  tail: the tree's K/V rows are in the cache
+// behind the prefix (tree_k / tree_v unused), and max_seq_len bounds seq_len + n_nodes.
+jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, const int32_t* page_table,
+                     int max_pages_per_seq, int page_size, int64_t num_pages, const int32_t* seq_len,
+                     int max_seq_len, const void* tree_k, const void* tree_v, bool tail, const uint32_t* anc_mask,
+                     const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D, int64_t kv_batch_stride,
+                     float softmax_scale, void* out, float* lse, int32_t* device_status, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+  if (!q || !seq_len || !anc_mask || !n_nodes || !out) return JET_ERR_INVALID_ARG;
+  if (tail ? (!k_cache || !v_cache || max_seq_len < 1) : (!tree_k || !tree_v)) return JET_ERR_INVALID_ARG;
   if (batch < 1 || B < 1 || B > JET_MAX_NODES || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0)
     return JET_ERR_INVALID_ARG;
   if (max_seq_len > 0 && (!k_cache || !v_cache)) return JET_ERR_INVALID_ARG;
@@ -1496,7 +1510,7 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
   if (paged && static_cast<int64_t>(max_pages_per_seq) * 16 < max_seq_len) return JET_ERR_INVALID_ARG;
   if (!paged && batch > 1 && (kv_batch_stride < static_cast<int64_t>(max_seq_len) * Hkv * D || kv_batch_stride % 8 != 0))
     return JET_ERR_INVALID_ARG;
-  if (!aligned(q, 16) || !aligned(tree_k, 16) || !aligned(tree_v, 16) || !aligned(out, 16) ||
+  if (!aligned(q, 16) || (!tail && (!aligned(tree_k, 16) || !aligned(tree_v, 16))) || !aligned(out, 16) ||
       (k_cache && !aligned(k_cache, 16)) || (v_cache && !aligned(v_cache, 16)))
     return JET_ERR_INVALID_ARG;
   if (static_cast<int64_t>(batch) * B >= (1ll << 31)) return JET_ERR_INVALID_ARG;
@@ -1513,7 +1527,7 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
     const uint32_t box[4] = {64, static_cast<uint32_t>(G), 1, static_cast<uint32_t>(kBM / G)};
     if (!make_map(&tq, q, 4, dims, str, box)) return JET_ERR_CUDA;
   }
-  {
+  if (!tail) {
     const uint64_t dims[4] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Hkv), static_cast<uint64_t>(B),
                               static_cast<uint64_t>(batch)};
     const uint64_t str[3] = {D * eb, static_cast<uint64_t>(Hkv) * D * eb, static_cast<uint64_t>(B) * Hkv * D * eb};
@@ -1552,6 +1566,7 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
   p.status = device_status;
   p.max_pages = max_pages_per_seq;
   p.paged = paged ? 1 : 0;
+  p.tail = tail ? 1 : 0;
   p.batch = batch; p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.words = (B + 31) / 32;
   p.nsplit = pl.nsplit;
   p.n_mgroups = pl.n_mgroups;
@@ -1564,9 +1579,41 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
   p.trace = g_trace_ptr;
 #endif
 
+  if (tail) {       // no separate tree tiles: the maps are never used
+    ttk = tk;
+    ttv = tv;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D == 128) return pl.mt == 1 ? launch<128, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
                                   : launch<128, 2>(tq, tk, tv, ttk, ttv, p, pl, st);
   return pl.mt == 1 ? launch<64, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
                     : launch<64, 2>(tq, tk, tv, ttk, ttv, p, pl, st);
+}
+
+}  // namespace
+}  // namespace jet
+
+extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
+                                           const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                           int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                           const void* tree_k, const void* tree_v, const uint32_t* anc_mask,
+                                           const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D,
+                                           int64_t kv_batch_stride, float softmax_scale, void* out, float* lse,
+                                           int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                           void* stream) {
+  return jet::attn_call(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len, max_seq_len,
+                        tree_k, tree_v, false, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
+                        out, lse, device_status, workspace, workspace_bytes, stream);
+}
+
+extern "C" jet_status jet_tree_verify_attn_tail(const void* q, const void* k_cache, const void* v_cache,
+                                                const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                                int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                                const uint32_t* anc_mask, const int32_t* n_nodes, int batch, int B,
+                                                int Hq, int Hkv, int D, int64_t kv_batch_stride,
+                                                float softmax_scale, void* out, float* lse, int32_t* device_status,
+                                                void* workspace, size_t workspace_bytes, void* stream) {
+  return jet::attn_call(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len, max_seq_len,
+                        nullptr, nullptr, true, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
+                        out, lse, device_status, workspace, workspace_bytes, stream);
 }

@@ -163,3 +163,50 @@ def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_
     torch.cuda.synchronize()
     return (bf16_to_f64(out), lse.cpu().numpy().astype(np.float64) if want_lse else None,
             int(status.cpu()[0]))
+
+
+def run_tree_attn_tail(q, k_cache, v_cache, page_table, seq_len, anc_mask, n_nodes, scale, max_seq_len, Hkv):
+    """As run_tree_attn for a cache that already holds the tree rows behind each prefix."""
+    batch, B, Hq, D = q.shape
+    seq_len = np.asarray(seq_len, dtype=np.int32)
+    d_q, d_k, d_v = dev_bf16(q), dev_bf16(k_cache), dev_bf16(v_cache)
+    if page_table is None:
+        pt, max_pages, page_size, num_pages = None, 0, 0, 0
+        kv_batch_stride = int(k_cache.shape[1] * Hkv * D)
+    else:
+        pt = dev(page_table.astype(np.int32))
+        max_pages, page_size, num_pages = page_table.shape[1], k_cache.shape[1], k_cache.shape[0]
+        kv_batch_stride = 0
+    out = torch.full((batch, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((batch, Hq, B), float("nan"), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
+    ws.zero_()
+    jet.jet_tree_verify_attn_tail(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
+                                  dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
+                                  batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
+    torch.cuda.synchronize()
+    return bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), int(status.cpu()[0])
+
+
+def run_kv_compact_tail(k_cache, v_cache, page_table, path, accept_len, seq_len, B):
+    """k_cache/v_cache [layers, ...] bf16 bits (contiguous [layers,batch,Lmax,Hkv,D] or paged
+    [layers,num_pages,page,Hkv,D]); returns new (k, v, seq_len) as numpy."""
+    layers = k_cache.shape[0]
+    Hkv, D = k_cache.shape[-2], k_cache.shape[-1]
+    batch, N = path.shape[0], path.shape[1] - 1
+    d_k, d_v = dev(k_cache.view(np.int16)), dev(v_cache.view(np.int16))
+    layer_stride = int(np.prod(k_cache.shape[1:]))
+    if page_table is None:
+        pt, max_pages, page_size = None, 0, 0
+        kv_batch_stride = int(np.prod(k_cache.shape[2:]))
+    else:
+        pt = dev(page_table.astype(np.int32))
+        max_pages, page_size = page_table.shape[1], k_cache.shape[2]
+        kv_batch_stride = 0
+    d_seq = dev(np.asarray(seq_len, dtype=np.int32))
+    jet.jet_kv_compact_tail(d_k, d_v, layer_stride, kv_batch_stride, pt, max_pages, page_size,
+                            dev(path.astype(np.int32)), dev(np.asarray(accept_len, dtype=np.int32)), d_seq,
+                            layers, batch, B, Hkv, D, N)
+    torch.cuda.synchronize()
+    return (d_k.cpu().numpy().view(np.uint16), d_v.cpu().numpy().view(np.uint16), d_seq.cpu().numpy())

@@ -2,7 +2,7 @@
 import numpy as np
 
 from jet_inputs import make_attn_inputs, make_paged_cache, random_tree
-from oracle import (anc_from_parent, gather_paged_prefix, kv_compact_ref, tree_attn_ref)
+from oracle import (anc_from_parent, gather_paged_prefix, kv_compact_ref, kv_compact_tail_ref, tree_attn_ref)
 
 
 def _setup(rng, layers, batch, B, Hkv, D, Lmax):
@@ -87,3 +87,57 @@ def test_chain_commit_equals_extending_the_chain():
     o, _ = tree_attn_ref(x["q"][5:6], k2[0, 0, : seq2[0]], v2[0, 0, : seq2[0]],
                          x["tree_k"][5:6], x["tree_v"][5:6], one, 1, 0.3)
     np.testing.assert_allclose(o[0], full[5], rtol=1e-12, atol=1e-14)
+
+
+def test_tail_commit_agrees_with_the_copying_commit():
+    """A cache whose rows seq_len .. seq_len + B - 1 hold the tree: committing in place must leave the new
+    prefix (positions < new length) exactly as the copying commit from separate tree buffers does; both
+    contiguous and paged."""
+    rng = np.random.default_rng(9)
+    layers, batch, B, Hkv, D, N, page = 2, 3, 12, 2, 8, 5, 4
+    seq = np.array([5, 9, 2], dtype=np.int32)
+    path = np.array([[0, 2, 5, 11, -1, -1], [0, -1, -1, -1, -1, -1], [0, 1, 2, 3, 4, 5]], dtype=np.int32)
+    acc = np.array([3, 0, 5], dtype=np.int32)
+    tk = rng.integers(0, 1 << 16, size=(layers, batch, B, Hkv, D)).astype(np.uint16)
+    tv = rng.integers(0, 1 << 16, size=(layers, batch, B, Hkv, D)).astype(np.uint16)
+    # contiguous
+    Lmax = 24
+    kc = rng.integers(0, 1 << 16, size=(layers, batch, Lmax, Hkv, D)).astype(np.uint16)
+    vc = rng.integers(0, 1 << 16, size=(layers, batch, Lmax, Hkv, D)).astype(np.uint16)
+    kt, vt = kc.copy(), vc.copy()
+    for b in range(batch):
+        kt[:, b, seq[b]:seq[b] + B] = tk[:, b]
+        vt[:, b, seq[b]:seq[b] + B] = tv[:, b]
+    k_ref, v_ref, len_ref = kv_compact_ref(tk, tv, kc, vc, None, path, acc, seq)
+    k_new, v_new, len_new = kv_compact_tail_ref(kt, vt, None, path, acc, seq)
+    assert len_new.tolist() == len_ref.tolist()
+    for b in range(batch):
+        n = int(len_new[b])
+        assert np.array_equal(k_new[:, b, :n], k_ref[:, b, :n]) and np.array_equal(v_new[:, b, :n], v_ref[:, b, :n])
+        assert np.array_equal(k_new[:, b, seq[b] + B:], kt[:, b, seq[b] + B:])        # nothing behind the tail is touched
+    # paged
+    need = [(int(L) + B + page - 1) // page for L in seq]
+    num_pages = sum(need) + 2
+    perm = rng.permutation(num_pages)
+    table = np.zeros((batch, max(need)), np.int32)
+    pos = 0
+    for b, cnt in enumerate(need):
+        table[b, :cnt] = perm[pos:pos + cnt]
+        pos += cnt
+    kp = rng.integers(0, 1 << 16, size=(layers, num_pages, page, Hkv, D)).astype(np.uint16)
+    vp = rng.integers(0, 1 << 16, size=(layers, num_pages, page, Hkv, D)).astype(np.uint16)
+    kpt, vpt = kp.copy(), vp.copy()
+    for b in range(batch):
+        for v in range(B):
+            j = int(seq[b]) + v
+            kpt[:, table[b, j // page], j % page] = tk[:, b, v]
+            vpt[:, table[b, j // page], j % page] = tv[:, b, v]
+    k_ref, v_ref, _ = kv_compact_ref(tk, tv, kp, vp, table, path, acc, seq)
+    k_new, v_new, len_new = kv_compact_tail_ref(kpt, vpt, table, path, acc, seq)
+    for b in range(batch):
+        for layer in range(layers):
+            got = gather_paged_prefix(k_new[layer], table[b], int(len_new[b]))
+            ref = gather_paged_prefix(k_ref[layer], table[b], int(len_new[b]))
+            assert np.array_equal(got, ref)
+            assert np.array_equal(gather_paged_prefix(v_new[layer], table[b], int(len_new[b])),
+                                  gather_paged_prefix(v_ref[layer], table[b], int(len_new[b])))
