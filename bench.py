@@ -153,7 +153,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0):
+def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0, tail=False):
     """Seeded synthetic step inputs on the device.  Returns (VerifyStep, info dict)."""
     import torch
     from paper_2606_18394_b200.step import VerifyStep
@@ -166,7 +166,7 @@ def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0
         rng = np.random.default_rng(seed)
         lo, hi = c["L_range"]
         seq = rng.integers(lo, hi + 1, size=batch).astype(np.int32)
-        need = [(int(L) + N + 1 + 15) // 16 for L in seq]
+        need = [(int(L) + (max(N + 1, B) if tail else N + 1) + 15) // 16 for L in seq]
         num_pages = sum(need) + 3
         perm = rng.permutation(num_pages)
         max_pages = max(need)
@@ -177,18 +177,20 @@ def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0
             pos += cnt
         st = VerifyStep(batch=batch, layers=layers, Hq=Hq, Hkv=Hkv, D=D, B=B, N=N, W=W, V=V,
                         max_seq_len=int(seq.max()), page_size=16, num_pages=num_pages, max_pages=max_pages,
-                        device=device)
+                        device=device, tail=tail)
         st.page_table.copy_(torch.from_numpy(table))
     else:
         seq = np.full(batch, c["L"], dtype=np.int32)
         st = VerifyStep(batch=batch, layers=layers, Hq=Hq, Hkv=Hkv, D=D, B=B, N=N, W=W, V=V,
-                        max_seq_len=int(c["L"]), device=device)
+                        max_seq_len=int(c["L"]), device=device, tail=tail)
     st.seq_len0.copy_(torch.from_numpy(seq))
     for t in (st.q, st.tree_k, st.tree_v):
         t.copy_(torch.randn(t.shape, generator=gen, device=device, dtype=torch.float32))
     for layer in range(layers):      # layer by layer: bounded temporaries
         st.k_cache[layer].copy_(torch.randn(st.k_cache[layer].shape, generator=gen, device=device, dtype=torch.float32))
         st.v_cache[layer].copy_(torch.randn(st.v_cache[layer].shape, generator=gen, device=device, dtype=torch.float32))
+    if tail:
+        st.place_tree()
     # draft log-probs: log_softmax of N(0, sigma) logits with one confident token per depth (p = 0.7),
     # evaluated in fp64 and rounded to fp32
     for b in range(batch):
@@ -268,7 +270,7 @@ def bench_jet(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
     c = workload(args.config, args.budget, args.batch)
-    st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha)
+    st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha, args.layout == "tail")
     layers = c["layers"]
     if args.accept == "sample":
         st.accept_mode = "sample"
@@ -361,6 +363,9 @@ def bench_jet(args):
     def e2e_step():
         for k, v in pinned.items():
             getattr(st, k).copy_(v, non_blocking=True)
+        if st.tail:
+            st.seq_len.copy_(st.seq_len0)
+            st.place_tree()                # the tree's K/V arrive in staging buffers and are put behind the prefixes
         run()
         for k, v in host_out.items():
             v.copy_(getattr(st, k), non_blocking=True)
@@ -424,7 +429,7 @@ def bench_jet(args):
                    "tree_nodes": c["B"], "max_depth": c["N"], "width": c["W"], "vocab": c["V"],
                    "paged": bool(c.get("paged")), "cuda_graph": not args.no_graph,
                    "l2": "every layer streams its own KV buffers; one step reads far more than the 126 MB L2",
-                   "accepted_len": acc, "accept": args.accept,
+                   "accepted_len": acc, "accept": args.accept, "tree_kv": args.layout,
                    "score": args.score if args.score != "hybrid" else f"hybrid(alpha={args.score_alpha})"},
         "attn_us_per_layer": attn_us,
         "e2e": {"value": e2e_ms_step * 1e3 / (layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -555,6 +560,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="batch, for configurations that list several")
     ap.add_argument("--no-graph", action="store_true", help="issue the calls directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layout", choices=["separate", "tail"], default="separate",
+                    help="tree K/V in their own buffers, or in the cache behind each prefix")
     ap.add_argument("--score", choices=["accum_logp", "entropy", "hybrid"], default="accum_logp",
                     help="expansion score of the tree construction (hybrid: --score-alpha)")
     ap.add_argument("--score-alpha", type=float, default=1.0)

@@ -15,11 +15,14 @@ from . import binding as jet
 
 class VerifyStep:
     def __init__(self, *, batch, layers, Hq, Hkv, D, B, N, W, V, max_seq_len, page_size=0, num_pages=0,
-                 max_pages=0, device="cuda:0"):
+                 max_pages=0, device="cuda:0", tail=False):
         self.batch, self.layers, self.Hq, self.Hkv, self.D = batch, layers, Hq, Hkv, D
         self.B, self.N, self.W, self.V = B, N, W, V
         self.max_seq_len = max_seq_len
         self.paged = page_size > 0
+        # tail: the tree's K/V rows live in the cache behind each prefix (jet_tree_verify_attn_tail /
+        # jet_kv_compact_tail); tree_k / tree_v are then only the staging buffers place_tree() copies from
+        self.tail = bool(tail)
         self.page_size, self.num_pages, self.max_pages = page_size, num_pages, max_pages
         self.device = torch.device(device)
         dev = self.device
@@ -41,7 +44,7 @@ class VerifyStep:
             self.rows_per_seq = 0
         else:
             # room for the committed path behind the longest prefix
-            self.rows_per_seq = max_seq_len + N + 1
+            self.rows_per_seq = max_seq_len + (max(N + 1, B) if self.tail else N + 1)
             self.k_cache = torch.zeros((kv_layers, batch, self.rows_per_seq, Hkv, D), dtype=torch.bfloat16,
                                        device=dev)
             self.page_table = None
@@ -84,7 +87,28 @@ class VerifyStep:
 
     @property
     def attn_max_len(self):
-        return self.max_seq_len if self.paged else self.rows_per_seq
+        if self.paged:
+            return self.max_seq_len + (self.B if self.tail else 0)
+        return self.rows_per_seq
+
+    def place_tree(self):
+        """Tail layout: writes tree_k / tree_v to the cache rows seq_len0[b] + v (what the model's K/V
+        projection does in a serving stack; plain torch copies, not part of the timed path's kernels)."""
+        assert self.tail
+        L = self.seq_len0.to(torch.int64)
+        v = torch.arange(self.B, device=self.device, dtype=torch.int64)
+        pos = L[:, None] + v[None, :]                                     # [batch, B]
+        if self.paged:
+            page = torch.gather(self.page_table.to(torch.int64), 1, pos // self.page_size)
+            rows = (page * self.page_size + pos % self.page_size).reshape(-1)
+            for cache, tree in ((self.k_cache, self.tree_k), (self.v_cache, self.tree_v)):
+                flat = cache.view(self.layers, self.num_pages * self.page_size, self.Hkv, self.D)
+                flat[:, rows] = tree.reshape(self.layers, -1, self.Hkv, self.D)
+        else:
+            rows = (torch.arange(self.batch, device=self.device)[:, None] * self.rows_per_seq + pos).reshape(-1)
+            for cache, tree in ((self.k_cache, self.tree_k), (self.v_cache, self.tree_v)):
+                flat = cache.view(self.layers, self.batch * self.rows_per_seq, self.Hkv, self.D)
+                flat[:, rows] = tree.reshape(self.layers, -1, self.Hkv, self.D)
 
     @property
     def kv_batch_stride(self):
@@ -106,6 +130,13 @@ class VerifyStep:
                                       self.anc_mask, self.n_nodes, self.depth_entropy, self.ws_build)
 
     def verify_attn(self, layer):
+        if self.tail:
+            jet.jet_tree_verify_attn_tail(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
+                                          self.max_pages, self.page_size, self.num_pages, self.seq_len,
+                                          self.attn_max_len, self.anc_mask, self.n_nodes, self.batch, self.B,
+                                          self.Hq, self.Hkv, self.D, self.kv_batch_stride, self.scale,
+                                          self.out[layer], None, self.status, self.ws_attn)
+            return
         jet.jet_tree_verify_attn(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
                                  self.max_pages, self.page_size, self.num_pages, self.seq_len, self.attn_max_len,
                                  self.tree_k[layer], self.tree_v[layer], self.anc_mask, self.n_nodes, self.batch,
@@ -124,6 +155,11 @@ class VerifyStep:
                                    self.path, self.out_tokens, self.ws_accept)
 
     def kv_compact(self):
+        if self.tail:
+            jet.jet_kv_compact_tail(self.k_cache, self.v_cache, self.cache_layer_stride, self.kv_batch_stride,
+                                    self.page_table, self.max_pages, self.page_size, self.path, self.accept_len,
+                                    self.seq_len, self.layers, self.batch, self.B, self.Hkv, self.D, self.N)
+            return
         jet.jet_kv_compact(self.tree_k, self.tree_v, self.k_cache, self.v_cache,
                            self.cache_layer_stride, self.kv_batch_stride,
                            self.page_table, self.max_pages, self.page_size, self.path, self.accept_len,
