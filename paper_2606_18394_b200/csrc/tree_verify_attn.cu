@@ -47,6 +47,7 @@ constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
 constexpr int kMaxSplit = 16;          // largest cluster
 constexpr int kMaxSorted = 128;          // batches up to this size are launched longest prefix first
+constexpr float kSharedSumFloor = 8.6736174e-19f;  // 2^-60: a row that saw keys but summed to less has lost them to underflow
 constexpr float kSharedSumLimit = 1.2089258e24f;   // 2^80: tile sums a fixed reference may reach before the CTA falls back
 constexpr float kFastSumLimit = 256.0f;    // a row keeps its reference maximum while its tile sums stay below (so P <= 2^8)
 
@@ -1003,6 +1004,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // the row's fixed reference and writes P to the warpgroup's P buffer.
         bool ok = true;
         bool synced = false;                 // the two warpgroups have met at the reference hand-over
+        bool saw_key = false;                // some key of this warpgroup's tiles is visible to the row
         float m_ref = 0.0f;
         const uint32_t tS = t_lane + C::shared_s(wg);
         const uint32_t tP = t_lane + C::shared_p(wg);
@@ -1019,6 +1021,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           uint32_t xa[32], xb[32], xc[32], xd[32];
           uint32_t b0 = 0xFFFFFFFFu, b1 = 0xFFFFFFFFu, b2 = 0xFFFFFFFFu, b3 = 0xFFFFFFFFu;
           if (!full_tile) { b0 = chunk_bits(t, 0); b1 = chunk_bits(t, 1); b2 = chunk_bits(t, 2); b3 = chunk_bits(t, 3); }
+          saw_key = saw_key || (b0 | b1 | b2 | b3) != 0u;
           ptx::tmem_ld32(tS, xa);
           ptx::tmem_ld32(tS + 32, xb);
           ptx::tmem_ld32(tS + 64, xc);
@@ -1042,7 +1045,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               max_chunk(xc, mx);
               max_chunk(xd, mx);
               const float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-              m_ref = (m == -INFINITY) ? 0.0f : m * sl2;
+              m_ref = (m == -INFINITY) ? -0.0f : m * sl2;     // -0.0 marks "no reference of its own" (same arithmetic as 0)
               if (T > 1) {
                 ref_s[r] = m_ref;
                 ptx::named_arrive(1, 256);          // warpgroup 1 waits for this, warpgroup 0 goes on
@@ -1080,6 +1083,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           if (tid == 128 && j < 4) JET_TR(20 + 2 * j);
           if (tid == 256 && j < 4) JET_TR(33 + 2 * j);
         }
+        // A row whose reference was not taken from scores of its own (no key of the first tile was visible to it:
+        // reference 0) may have lost its keys to underflow; such a row sums to (almost) nothing although it saw
+        // keys, and the CTA repeats the key range in the classic form.  (A row with a reference of its own sums
+        // to at least 1 in warpgroup 0.  The test is per warpgroup and errs on the safe side.)
+        if (row_live && saw_key && __float_as_uint(m_ref) == 0x80000000u && !(l >= kSharedSumFloor)) *redo_flag = 1u;
         if (T > 1 && !synced) {                   // a warpgroup that gave up early still takes part in the hand-over
           if (wg == 0) ptx::named_arrive(1, 256);
           else ptx::named_sync(1, 256);

@@ -176,6 +176,55 @@ def test_scores_far_above_the_first_tile_headline_shape():
     assert np.abs(got_lse - rlse).max() <= 1e-3 * max(1.0, np.abs(rlse).max())
 
 
+def test_rows_without_a_key_in_their_first_tile_and_very_negative_scores():
+    """512-node tree, no prefix: the rows of the later query tiles see no key in the first key tiles of
+    their slices (their ancestors lie elsewhere), so those rows start without a reference of their own; all
+    scores are about -300 (far below what exp2 can represent against a reference of 0).  The result must still
+    be the softmax over the visible keys."""
+    import jet_harness as H
+    from jet_inputs import bf16_bits_to_f32, f32_to_bf16_bits
+    B, Hq, Hkv, D, L = 512, 4, 1, 128, 0
+    rng = np.random.default_rng(91)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    x["q"] = f32_to_bf16_bits(np.abs(bf16_bits_to_f32(x["q"])) * 0.5 + 0.5)
+    x["tree_k"] = f32_to_bf16_bits(-(np.abs(bf16_bits_to_f32(x["tree_k"])) * 0.5 + 2.0))
+    parent = np.zeros(B, dtype=np.int32)                     # a star: every node hangs off the root ...
+    parent[0] = -1
+    parent[300:384] = np.arange(299, 383)                    # ... except a chain 299 -> 300 -> ... -> 383
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0
+    rows = [(v, h) for v in (0, 1, 127, 128, 200, 255, 256, 299, 300, 383, 384, 400, 415, 416, 500, 511) for h in (0, 3)]
+    ref, rlse = tree_attn_rows_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale,
+                                   rows)
+    assert rlse.max() < -150                                 # every visible score is far below zero
+    out, lse, st = H.run_tree_attn(x["q"][None], None, None, None, [L], x["tree_k"][None], x["tree_v"][None],
+                                   anc[None], [B], scale, max_seq_len=0)
+    assert st == 0 and not np.isnan(out).any()
+    got = np.stack([out[0, v, h] for v, h in rows])
+    err = np.abs(got - ref)
+    assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR, (err.max(), err.mean())
+    got_lse = np.array([lse[0, h, v] for v, h in rows])
+    assert np.abs(got_lse - rlse).max() <= 1e-3 * np.abs(rlse).max()
+
+
+@pytest.mark.parametrize("force", ["2", "2,g", "4"])
+def test_adversarial_scores_under_forced_slicings(force):
+    """The launch plan decides where the key slices begin, and with it which rows meet an empty first tile.  The
+    library reads JET_FORCE_MT / JET_FORCE_SPLIT once per process, so the adversarial-score tests run again in
+    a child process under one query tile per CTA and 2 or 4 key slices (merged in a cluster or through the
+    workspace)."""
+    import os
+    import subprocess
+    import sys
+    if os.environ.get("JET_FORCE_SPLIT"):
+        pytest.skip("already inside a forced run")
+    env = dict(os.environ, JET_FORCE_MT="1", JET_FORCE_SPLIT=force)
+    r = subprocess.run([sys.executable, "-m", "pytest", __file__, "-m", "gpu", "-x", "-q", "-k",
+                        "very_negative or far_above"], env=env, capture_output=True, text=True,
+                       cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))), timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_sweep_16k_sampled_rows():
     """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
     import jet_harness as H
