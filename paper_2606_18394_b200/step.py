@@ -165,18 +165,26 @@ class VerifyStep:
                            self.page_table, self.max_pages, self.page_size, self.path, self.accept_len,
                            self.seq_len, self.layers, self.batch, self.B, self.Hkv, self.D, self.N)
 
-    def run(self):
-        """The whole hot path once, on the current stream.  seq_len restarts from seq_len0 so that
-        repeated steps (and graph replays) see the same prefix lengths."""
+    def run_front(self):
+        """Everything that does not need the target logits: tree construction and the attention of all layers.
+        seq_len restarts from seq_len0 so that repeated steps (and graph replays) see the same prefix lengths."""
         self.seq_len.copy_(self.seq_len0)
         self.tree_build()
         for layer in range(self.layers):
             self.verify_attn(layer)
+
+    def run_back(self):
+        """Acceptance against the target logits and the commit."""
         if self.accept_mode == "sample":
             self.tree_accept_sample()
         else:
             self.tree_accept()
         self.kv_compact()
+
+    def run(self):
+        """The whole hot path once, on the current stream."""
+        self.run_front()
+        self.run_back()
 
     LAUNCHES_PER_STEP_FIXED = 6      # tree_build 2, tree_accept 2, kv_compact 2
 
