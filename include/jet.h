@@ -109,6 +109,10 @@ JET_API jet_status jet_tree_build(const float* logp, int64_t logp_batch_stride, 
  * rule as the appendix states.)  Ties -> lowest node index; `score` is the
  * accumulated log-probability in every mode.
  *
+ *   node_budget   i32 [batch] or NULL: sequence b's own budget min(B, max(1,
+ *                 node_budget[b])) (load-dependent budgets, which Section 5 leaves
+ *                 to future work); every array keeps its [batch, B] shape, rows
+ *                 past n_nodes[b] are padding as usual
  *   score_mode    one of JET_SCORE_*
  *   alpha         finite; used by JET_SCORE_HYBRID only
  *   depth_entropy fp32 [batch, N] out, may be NULL: H of logp[b, d, :]
@@ -123,7 +127,8 @@ JET_API size_t jet_tree_build_scored_workspace_bytes(int batch, int N, int V, in
 
 JET_API jet_status jet_tree_build_scored(const float* logp, int64_t logp_batch_stride, int64_t logp_depth_stride,
                                  const int32_t* root_token, int batch, int N, int V, int W, int B,
-                                 int score_mode, float alpha, int32_t* parent, int32_t* depth,
+                                 const int32_t* node_budget, int score_mode, float alpha, int32_t* parent,
+                                 int32_t* depth,
                                  int32_t* token, float* score, uint32_t* anc_mask, int32_t* n_nodes,
                                  float* depth_entropy, void* workspace, size_t workspace_bytes,
                                  void* stream);

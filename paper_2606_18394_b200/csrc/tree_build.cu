@@ -214,7 +214,8 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
                    int32_t* __restrict__ parent_out, int32_t* __restrict__ depth_out,
                    int32_t* __restrict__ token_out, float* __restrict__ score_out,
                    uint32_t* __restrict__ anc_out, int32_t* __restrict__ n_nodes_out,
-                   const double* __restrict__ plogp_partial, float alpha, float* __restrict__ depth_entropy_out) {
+                   const double* __restrict__ plogp_partial, float alpha, float* __restrict__ depth_entropy_out,
+                   const int32_t* __restrict__ node_budget) {
   grid_dependency_wait();
   __shared__ int32_t s_top_tok[JET_MAX_DEPTH][JET_MAX_WIDTH];
   __shared__ float s_top_lp[JET_MAX_DEPTH][JET_MAX_WIDTH];
@@ -274,6 +275,9 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
   __syncthreads();
 
   // ---- Algorithm 1: one warp, queue in registers (as many per lane as the budget needs)
+  // this sequence's budget: B, or its own smaller one (the arrays are padded to B either way)
+  const int Bmax = B;
+  if (node_budget) B = max(1, min(B, node_budget[b]));
   if (warp == 0) {
     const int root = root_token[b];
     int n;
@@ -288,6 +292,7 @@ tree_expand_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t
 
   // ---- emit
   const int n = s_n;
+  B = Bmax;
   const size_t o = static_cast<size_t>(b) * B;
   for (int v = tid; v < B; v += kExpThreads) {
     const bool live = v < n;
@@ -320,8 +325,9 @@ size_t cand_bytes(int batch, int N, int V, int W) {
 jet_status tree_build_launch(const float* logp, int64_t logp_batch_stride, int64_t logp_depth_stride,
                              const int32_t* root_token, int batch, int N, int V, int W, int B, int score_mode,
                              float alpha, int32_t* parent, int32_t* depth, int32_t* token, float* score,
-                             uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy, void* workspace,
-                             size_t workspace_bytes, size_t need, void* stream) {
+                             uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy,
+                             const int32_t* node_budget, void* workspace, size_t workspace_bytes, size_t need,
+                             void* stream) {
   if (!logp || !root_token || !parent || !depth || !token || !anc_mask || !n_nodes)
     return JET_ERR_INVALID_ARG;
   if (batch < 1 || batch > 65535 || N < 1 || N > JET_MAX_DEPTH || W < 1 || W > JET_MAX_WIDTH || V < 1 ||
@@ -343,7 +349,7 @@ jet_status tree_build_launch(const float* logp, int64_t logp_batch_stride, int64
         logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, static_cast<double*>(nullptr));
     launch_dependent(tree_expand_kernel<0>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
         root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
-        static_cast<const double*>(nullptr), 0.0f, static_cast<float*>(nullptr));
+        static_cast<const double*>(nullptr), 0.0f, static_cast<float*>(nullptr), node_budget);
     return launch_status();
   }
   launch_dependent(topw_partial_kernel<true>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
@@ -351,11 +357,11 @@ jet_status tree_build_launch(const float* logp, int64_t logp_batch_stride, int64
   if (score_mode == JET_SCORE_ENTROPY)
     launch_dependent(tree_expand_kernel<1>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
         root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
-        static_cast<const double*>(plogp), 0.0f, depth_entropy);
+        static_cast<const double*>(plogp), 0.0f, depth_entropy, node_budget);
   else
     launch_dependent(tree_expand_kernel<2>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
         root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
-        static_cast<const double*>(plogp), alpha, depth_entropy);
+        static_cast<const double*>(plogp), alpha, depth_entropy, node_budget);
   return launch_status();
 }
 
@@ -376,7 +382,7 @@ extern "C" jet_status jet_tree_build(const float* logp, int64_t logp_batch_strid
   const size_t need = (batch >= 1 && N >= 1 && V >= 1 && W >= 1) ? jet::cand_bytes(batch, N, V, W) : 0;
   return jet::tree_build_launch(logp, logp_batch_stride, logp_depth_stride, root_token, batch, N, V, W, B,
                                 JET_SCORE_ACCUM_LOGP, 0.0f, parent, depth, token, score, anc_mask, n_nodes, nullptr,
-                                workspace, workspace_bytes, need, stream);
+                                nullptr, workspace, workspace_bytes, need, stream);
 }
 
 extern "C" size_t jet_tree_build_scored_workspace_bytes(int batch, int N, int V, int W) {
@@ -387,12 +393,13 @@ extern "C" size_t jet_tree_build_scored_workspace_bytes(int batch, int N, int V,
 
 extern "C" jet_status jet_tree_build_scored(const float* logp, int64_t logp_batch_stride,
                                             int64_t logp_depth_stride, const int32_t* root_token,
-                                            int batch, int N, int V, int W, int B, int score_mode, float alpha,
-                                            int32_t* parent, int32_t* depth, int32_t* token, float* score,
-                                            uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy,
-                                            void* workspace, size_t workspace_bytes, void* stream) {
+                                            int batch, int N, int V, int W, int B, const int32_t* node_budget,
+                                            int score_mode, float alpha, int32_t* parent, int32_t* depth,
+                                            int32_t* token, float* score, uint32_t* anc_mask, int32_t* n_nodes,
+                                            float* depth_entropy, void* workspace, size_t workspace_bytes,
+                                            void* stream) {
   const size_t need = jet_tree_build_scored_workspace_bytes(batch, N, V, W);
   return jet::tree_build_launch(logp, logp_batch_stride, logp_depth_stride, root_token, batch, N, V, W, B, score_mode,
-                                alpha, parent, depth, token, score, anc_mask, n_nodes, depth_entropy, workspace,
-                                workspace_bytes, need, stream);
+                                alpha, parent, depth, token, score, anc_mask, n_nodes, depth_entropy, node_budget,
+                                workspace, workspace_bytes, need, stream);
 }

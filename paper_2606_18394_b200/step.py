@@ -71,6 +71,7 @@ class VerifyStep:
                                jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W)))
         # expansion score of the tree construction: "accum_logp" (default), "entropy" or "hybrid" (+ score_alpha)
         self.score_mode = "accum_logp"
+        self.node_budget = None        # optional i32 [batch]: per-sequence budgets <= B
         self.score_alpha = 0.0
         self.depth_entropy = torch.zeros((batch, N), dtype=torch.float32, device=dev)
         self.ws_attn = ws(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, self.attn_max_len))
@@ -120,14 +121,15 @@ class VerifyStep:
 
     # ------------------------------------------------------------------ the four calls
     def tree_build(self):
-        if self.score_mode == "accum_logp":
+        if self.score_mode == "accum_logp" and self.node_budget is None:
             jet.jet_tree_build(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, self.parent,
                                self.depth, self.token, self.score, self.anc_mask, self.n_nodes, self.ws_build)
         else:
-            mode = {"entropy": 1, "hybrid": 2}[self.score_mode]
+            mode = {"accum_logp": 0, "entropy": 1, "hybrid": 2}[self.score_mode]
             jet.jet_tree_build_scored(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, mode,
                                       self.score_alpha, self.parent, self.depth, self.token, self.score,
-                                      self.anc_mask, self.n_nodes, self.depth_entropy, self.ws_build)
+                                      self.anc_mask, self.n_nodes, self.depth_entropy, self.ws_build,
+                                      node_budget=self.node_budget)
 
     def verify_attn(self, layer):
         if self.tail:

@@ -49,7 +49,7 @@ def run_tree_build(logp, root_token, N, W, B, with_score=True):
                 anc_mask=anc.cpu().numpy().view(np.uint32), n_nodes=n_nodes.cpu().numpy())
 
 
-def run_tree_build_scored(logp, root_token, N, W, B, score_mode, alpha):
+def run_tree_build_scored(logp, root_token, N, W, B, score_mode, alpha, node_budget=None):
     """As run_tree_build, through jet_tree_build_scored; also returns depth_entropy [batch,N]."""
     batch, _, V = logp.shape
     d_logp = dev(logp)
@@ -64,7 +64,8 @@ def run_tree_build_scored(logp, root_token, N, W, B, score_mode, alpha):
     ent = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
     ws = workspace(jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W))
     jet.jet_tree_build_scored(d_logp, d_root, batch, N, V, W, B, score_mode, alpha, parent, depth, token, score,
-                              anc, n_nodes, ent, ws)
+                              anc, n_nodes, ent, ws,
+                              node_budget=dev(np.asarray(node_budget, dtype=np.int32)) if node_budget is not None else None)
     torch.cuda.synchronize()
     return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
                 score=score.cpu().numpy(), anc_mask=anc.cpu().numpy().view(np.uint32),

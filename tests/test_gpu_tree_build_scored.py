@@ -122,3 +122,27 @@ def test_argument_errors():
     if small.numel() < ws.numel():
         assert jet.jet_tree_build_scored(*args(1, 0.0, small), check=False) == jet.JET_ERR_WORKSPACE
     assert jet.jet_tree_build_scored(*args(1, 0.0, ws), check=False) == jet.JET_OK
+
+
+@pytest.mark.parametrize("mode,alpha", [("accum_logp", 0.0), ("hybrid", 1.0)])
+def test_per_sequence_budgets(mode, alpha):
+    """Each sequence of a batch with its own budget: the tree equals the oracle's tree for that budget, padded
+    to B like any shorter tree (a budget above B counts as B, below 1 as 1)."""
+    import jet_harness as H
+    rng = np.random.default_rng(4100)
+    batch, N, V, W, B = 6, 8, 20000, 7, 128
+    budgets = [128, 64, 17, 1, 500, 0]
+    logp = np.stack([make_logp(rng, N, V, 3.0, peaked_p=0.7) for _ in range(batch)])
+    got = H.run_tree_build_scored(logp, np.arange(batch), N, W, B, MODES[mode], alpha, node_budget=budgets)
+    words = (B + 31) // 32
+    for b in range(batch):
+        Bb = max(1, min(B, budgets[b]))
+        ref = tree_build_ref(logp[b], b, N, W, Bb, score_mode=mode, alpha=alpha)
+        n = ref["n_nodes"]
+        assert got["n_nodes"][b] == n
+        for k in ("parent", "depth", "token"):
+            assert np.array_equal(got[k][b][:Bb], ref[k]) and (got[k][b][Bb:] == -1).all(), (b, k)
+        assert np.array_equal(got["score"][b][:n].view(np.uint32), ref["score"][:n].view(np.uint32))
+        anc = np.zeros((B, words), np.uint32)
+        anc[:Bb, :ref["anc_mask"].shape[1]] = ref["anc_mask"]
+        assert np.array_equal(got["anc_mask"][b], anc), b
