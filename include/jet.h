@@ -5,11 +5,18 @@
  * Four operations, in the order one verification step runs them:
  *
  *   jet_tree_build        per-depth draft log-probs -> budgeted candidate tree
- *   jet_tree_build_scored the same with the entropy / hybrid expansion scores
  *   jet_tree_verify_attn  attention of all tree nodes over prefix KV + tree KV
  *                         under the ancestor mask (once per layer)
  *   jet_tree_accept       greedy acceptance of the deepest matching path
  *   jet_kv_compact        commit of the accepted path's K/V into the cache
+ *
+ * and their variants:
+ *
+ *   jet_tree_build_scored      entropy / hybrid expansion scores, per-sequence budgets
+ *   jet_tree_verify_attn_tail  the tree's K/V rows live in the cache behind the prefix
+ *   jet_kv_compact_tail        in-place commit for that layout
+ *   jet_tree_accept_static     greedy acceptance on scratch built into the library
+ *   jet_tree_accept_sample     non-greedy (min(1, p/q)) acceptance with a correction draw
  *
  * Conventions shared by every call
  *   - Every pointer is a DEVICE pointer owned by the caller unless a comment
