@@ -45,7 +45,7 @@ namespace {
 constexpr int kBM = 128;               // query rows per tile
 constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
-constexpr int kMaxSplit = 16;          // largest cluster
+constexpr int kMaxSplit = 20;          // most key slices (a cluster holds at most 16; more only through the workspace)
 constexpr int kMaxSorted = 128;          // batches up to this size are launched longest prefix first
 constexpr float kSharedSumFloor = 8.6736174e-19f;  // 2^-60: a row that saw keys but summed to less has lost them to underflow
 constexpr float kSharedSumLimit = 1.2089258e24f;   // 2^80: tile sums a fixed reference may reach before the CTA falls back

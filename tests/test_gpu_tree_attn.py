@@ -225,6 +225,25 @@ def test_adversarial_scores_under_forced_slicings(force):
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
 
+@pytest.mark.parametrize("B", [16, 32])
+def test_small_budgets_at_the_full_prefix(B):
+    """Few query rows per KV head (one query tile per KV head): the key range is cut into as many slices as
+    the device has room for (more than a cluster can hold, merged through the workspace; the last slices own
+    no rows to combine)."""
+    import jet_harness as H
+    Hq, Hkv, D, L = 32, 8, 128, 4096
+    rng = np.random.default_rng(600 + B)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = random_tree(B, rng)
+    anc = anc_from_parent(parent, B, B)
+    scale = 1.0 / np.sqrt(D)
+    ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale)
+    out, lse, st = H.run_tree_attn(x["q"][None], x["k_prefix"][None], x["v_prefix"][None], None, [L],
+                                   x["tree_k"][None], x["tree_v"][None], anc[None], [B], scale)
+    assert st == 0
+    _check(out[0], lse[0], ref, rlse, B)
+
+
 def test_sweep_16k_sampled_rows():
     """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
     import jet_harness as H
