@@ -35,6 +35,9 @@ UNIT = "us/layer"
 # DRAM bytes (read + write) of one tree_attn_kernel launch on the benchmark workload, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the workload).
 NCU_TRAFFIC_BYTES = {"qwen3_8b": 17659392}     # profiles/tree_attn_kernel_qwen3_8b.md
+# Workloads too large to capture whole: DRAM traffic of a smaller capture of the same kernel as a fraction of
+# that capture's algorithmic bytes (the traffic is the K/V stream and grows in proportion).
+NCU_TRAFFIC_RATIO = {"batched_paged": 0.997}     # profiles/tree_attn_kernel_batched_paged.md
 
 
 def workload(name, budget=None, batch=None):
@@ -445,6 +448,9 @@ def bench_jet(args):
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"]}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.config)
+    if roof["traffic"] is None and args.config in NCU_TRAFFIC_RATIO:
+        roof["traffic"] = int(NCU_TRAFFIC_RATIO[args.config] * bytes_alg)
+        roof["traffic_note"] = "scaled from a smaller ncu capture of the same kernel by the algorithmic bytes"
     roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us, timing=attn_timing,
                 algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
                 roofline_us=max(t_bytes, t_flops) * 1e6)

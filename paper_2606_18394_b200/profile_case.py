@@ -1,21 +1,37 @@
-"""One attention-heavy case for profiling: `python -m paper_2606_18394_b200.profile_case B L [layers]`
-runs `layers` attention calls (own KV buffers per layer) of a single sequence at the Qwen3-8B head shape,
-twice (warm-up and measured), and prints the time per call.  Meant to be run under ncu with -k / -c."""
+"""One attention-heavy case for profiling:
+
+    python -m paper_2606_18394_b200.profile_case B L [layers [batch [paged]]]
+
+runs `layers` attention calls (own KV buffers per layer) at the Qwen3-8B head shape, twice (warm-up and
+measured), and prints the time per call.  batch > 1 gives every sequence the prefix length L; paged = 1 puts
+the prefixes into a paged cache (page size 16) behind a shuffled page table.  Meant to be run under ncu with
+-k / -c on a case of a few GB at most."""
 import sys
 
+import numpy as np
 import torch
 
 from .step import VerifyStep
 
 
 def main():
-    B = int(sys.argv[1]) if len(sys.argv) > 1 else 256
-    L = int(sys.argv[2]) if len(sys.argv) > 2 else 16384
-    layers = int(sys.argv[3]) if len(sys.argv) > 3 else 6
-    st = VerifyStep(batch=1, layers=layers, Hq=32, Hkv=8, D=128, B=B, N=12, W=7, V=4096, max_seq_len=L)
+    arg = lambda i, d: int(sys.argv[i]) if len(sys.argv) > i else d
+    B, L, layers, batch, paged = arg(1, 256), arg(2, 16384), arg(3, 6), arg(4, 1), arg(5, 0)
+    kw = {}
+    if paged:
+        per = (L + 16 + 15) // 16
+        kw = dict(page_size=16, num_pages=batch * per + 8, max_pages=per)
+    st = VerifyStep(batch=batch, layers=layers, Hq=32, Hkv=8, D=128, B=B, N=12, W=7, V=4096, max_seq_len=L, **kw)
     gen = torch.Generator(device="cuda").manual_seed(1)
-    for t in (st.q, st.tree_k, st.tree_v, st.k_cache, st.v_cache):
+    for t in (st.q, st.tree_k, st.tree_v):
         t.copy_(torch.randn(t.shape, generator=gen, device="cuda", dtype=torch.float32))
+    for layer in range(layers):
+        st.k_cache[layer].copy_(torch.randn(st.k_cache[layer].shape, generator=gen, device="cuda", dtype=torch.float32))
+        st.v_cache[layer].copy_(torch.randn(st.v_cache[layer].shape, generator=gen, device="cuda", dtype=torch.float32))
+    if paged:
+        ids = np.random.default_rng(0).permutation(kw["num_pages"]).astype(np.int32)
+        table = ids[:batch * kw["max_pages"]].reshape(batch, kw["max_pages"])
+        st.page_table.copy_(torch.from_numpy(table).cuda())
     st.seq_len0.fill_(L)
     st.seq_len.fill_(L)
     st.logp.copy_(torch.log_softmax(torch.randn(st.logp.shape, generator=gen, device="cuda") * 3, -1))
@@ -29,7 +45,8 @@ def main():
         e1.record()
         torch.cuda.synchronize()
     assert int(st.status.item()) == 0
-    print(f"B={B} L={L}: {e0.elapsed_time(e1) * 1e3 / layers:.2f} us per attention call, {layers} layers")
+    print(f"B={B} L={L} batch={batch} paged={paged}: {e0.elapsed_time(e1) * 1e3 / layers:.2f} us per attention call, "
+          f"{layers} layers")
 
 
 if __name__ == "__main__":
