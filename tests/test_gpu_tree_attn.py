@@ -437,6 +437,45 @@ def test_workspace_counters_are_left_clean_across_repeated_calls():
         assert int(ws[:4096].view(torch.int32).abs().sum().item()) == 0, "counters not reset"
 
 
+def test_two_streams_with_their_own_workspaces():
+    """Calls that may overlap on the device are allowed as long as each has its own workspace: two streams
+    run the benchmark shape back to back, interleaved, and every result matches the oracle."""
+    import torch
+    import jet_harness as H
+    import paper_2606_18394_b200 as jet
+    rng = np.random.default_rng(8)
+    B, Hq, Hkv, D, L = 64, 32, 8, 128, 4096
+    scale = 1.0 / np.sqrt(D)
+    cases = []
+    for _ in range(2):
+        x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+        parent, _, _ = random_tree(B, rng)
+        anc = anc_from_parent(parent, B, B)
+        ref, _ = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale)
+        d = dict(q=H.dev_bf16(x["q"][None]), k=H.dev_bf16(x["k_prefix"][None]), v=H.dev_bf16(x["v_prefix"][None]),
+                 tk=H.dev_bf16(x["tree_k"][None]), tv=H.dev_bf16(x["tree_v"][None]),
+                 anc=H.dev(anc[None].view(np.int32)), n=H.dev(np.array([B], np.int32)),
+                 seq=H.dev(np.array([L], np.int32)),
+                 ws=torch.zeros(jet.jet_tree_verify_attn_workspace_bytes(1, B, Hq, Hkv, D, L), dtype=torch.uint8,
+                                device=H.DEV),
+                 status=torch.zeros(1, dtype=torch.int32, device=H.DEV),
+                 outs=[torch.full((1, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=H.DEV) for _ in range(6)],
+                 stream=torch.cuda.Stream())
+        cases.append((d, ref))
+    torch.cuda.synchronize()
+    for it in range(6):
+        for d, _ in cases:
+            jet.jet_tree_verify_attn(d["q"], d["k"], d["v"], None, 0, 0, 0, d["seq"], L, d["tk"], d["tv"], d["anc"],
+                                     d["n"], 1, B, Hq, Hkv, D, L * Hkv * D, float(scale), d["outs"][it], None,
+                                     d["status"], d["ws"], stream=d["stream"])
+    torch.cuda.synchronize()
+    for d, ref in cases:
+        assert int(d["status"].item()) == 0
+        for out in d["outs"]:
+            err = np.abs(H.bf16_to_f64(out)[0] - ref)
+            assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR
+
+
 def test_two_query_tiles_per_cta_variant():
     """The planner picks the kernel variant with two query tiles per CTA for batched shapes only;
     JET_FORCE_MT=2 selects it for these single-sequence shapes too (read once per process, hence the
