@@ -244,6 +244,26 @@ def test_small_budgets_at_the_full_prefix(B):
     _check(out[0], lse[0], ref, rlse, B)
 
 
+@pytest.mark.parametrize("mt,split", [("1", "1"), ("1", "3"), ("1", "6"), ("1", "9,g"), ("1", "16,g"), ("1", "18,g"),
+                                      ("2", "1"), ("2", "2"), ("2", "4,g")])
+def test_every_kind_of_launch_plan(mt, split):
+    """The planner picks one plan per shape; the others (query tiles per CTA, number of key slices, merge through
+    a cluster or through the workspace) must compute the same thing.  Runs the benchmark-shape test, the tile
+    boundary tests and the tree-shape tests in a child process under a forced plan (a forced plan the device
+    cannot hold is ignored by the library, i.e. falls back to the planner's)."""
+    import os
+    import subprocess
+    import sys
+    if os.environ.get("JET_FORCE_SPLIT") or os.environ.get("JET_FORCE_MT"):
+        pytest.skip("already inside a forced run")
+    env = dict(os.environ, JET_FORCE_MT=mt, JET_FORCE_SPLIT=split)
+    r = subprocess.run([sys.executable, "-m", "pytest", __file__, "-m", "gpu", "-x", "-q", "-k",
+                        "qwen3_8b_config or tile_boundaries or tree_shapes or padding_nodes or small_budgets"],
+                       env=env, capture_output=True, text=True,
+                       cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))), timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_sweep_16k_sampled_rows():
     """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
     import jet_harness as H
