@@ -108,6 +108,12 @@ struct Cfg {
   __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
   // MT == 1, shared-accumulator pass (see the kernel): one accumulator for both warpgroups, a score buffer
   // and a separate P buffer (64 columns of packed bf16 pairs) per warpgroup.
+  // MT == 2, shared-score-buffer form (see the kernel): accumulators [mt*128, +D), ONE 128-column score buffer
+  // that the two query tiles use in turn, one P buffer (64 columns of packed bf16 pairs) per query tile.
+  static constexpr bool kHalfTiles = MT == 2;
+  __device__ static constexpr uint32_t half_o(int mt) { return mt * 128; }
+  __device__ static constexpr uint32_t half_s() { return 256; }
+  __device__ static constexpr uint32_t half_p(int mt) { return 384 + mt * 64; }
   __device__ static constexpr uint32_t shared_o() { return 0; }
   __device__ static constexpr uint32_t shared_s(int w) { return 128 + 128 * w; }
   __device__ static constexpr uint32_t shared_p(int w) { return 384 + 64 * w; }
@@ -125,7 +131,7 @@ struct Cfg {
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
   enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
-         kClusterA = 21, kClusterC = 22, kRecv = 23, kOFinal = 25, kCount = 26,
+         kClusterA = 21, kClusterC = 22, kRecv = 23, kOFinal = 25, kPFullB = 26, kODoneB = 28, kCount = 30,
          kLoopFirst = kKvFull, kLoopEnd = kClusterA };    // the key loop's barriers exist twice (one set per pass)
 };
 
@@ -287,8 +293,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // one lane per barrier of the block
     if (lane < Bars::kCount) {
       uint32_t count = 1;
-      if (lane >= Bars::kKvEmpty && lane < Bars::kSFull) count = MT == 1 ? 1 : n_mt;     // one arrival per stream that reads the stage
-      else if (lane >= Bars::kSFree && lane < Bars::kODone) count = 128;                // kSFree, kPFull: a softmax warpgroup
+      if (lane >= Bars::kKvEmpty && lane < Bars::kSFull) count = (MT == 1 || C::kHalfTiles) ? 1 : n_mt;   // arrivals per stage
+      else if ((lane >= Bars::kSFree && lane < Bars::kODone) || (lane >= Bars::kPFullB && lane < Bars::kODoneB))
+        count = 128;                                                                    // kSFree, kPFull: a softmax warpgroup
       else if (lane == Bars::kClusterA || lane == Bars::kClusterC) count = S;
       ptx::mbar_init(bar(lane), count);
       // slice merge: every slice sends this CTA its block of rows of query tile (lane - kRecv)
@@ -523,7 +530,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
           if (active) {
-            ptx::tmem_ld32(e_lane + C::o_col(mt, 0) + c * 32, o);
+            ptx::tmem_ld32(e_lane + (C::kHalfTiles ? C::half_o(mt) : C::o_col(mt, 0)) + c * 32, o);
             ptx::tmem_wait_ld();
           }
 #pragma unroll
@@ -717,7 +724,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
     // =========================================================== TMA producer (warp 0)
     // K runs `ahead` key tiles in front of V in the ring (0: K_t, V_t alternate).
-    auto produce = [&](const int ahead) {
+    // only: -1 = this warp requests every tile, 0 = the K tiles only, 1 = the V tiles only (two producer warps).
+    auto produce = [&](const int ahead, const int only = -1) {
       if (tid == 0) JET_TR(27);
       bool ok = true;
       int issued = 0;
@@ -735,6 +743,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       for (; issued < 2 * T; ++issued) {
         const bool take_k = kt < T && kt <= vt + ahead;
         const int t = t_lo + (take_k ? kt : vt), kv = take_k ? 0 : 1, stage = issued % kStages;
+        if (only >= 0 && kv != only) {          // the other producer warp's tile
+          if (take_k) ++kt; else ++vt;
+          continue;
+        }
         if (issued >= kStages) {
           ok = bounded_wait(lbar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
           if (!ok) break;
@@ -876,7 +888,78 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (classic) second_barrier_set();
     }
 
-    if (classic && has_work) {
+    if constexpr (C::kHalfTiles) {
+      // =========================================================== two query tiles per CTA
+      // Each query tile (stream) keeps the classic bookkeeping -- own accumulator, running reference, rescale
+      // when it rises -- but the two tiles take turns on ONE score buffer, which leaves TMEM columns for a P
+      // buffer per tile: a thread releases the score buffer as soon as it has read its row, the other tile's
+      // Q K^T (warp 1) follows at once, and the P V products (warp 3) read P from buffers of their own.  The
+      // chain softmax -> P V -> Q K^T -> softmax of the classic form is gone.
+      classic = false;
+      if (has_work) {
+        if (warp == 0) {
+          produce(0, 0);                     // K tiles
+        } else if (warp == 2) {
+          produce(0, 1);                     // V tiles (a paged tile is 16 small copies: two warps request them)
+        } else if (warp == 1) {
+          bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
+          int prev_mt = -1, prev_tl = 0;
+#pragma unroll 1
+          for (int tl = 0; tl < T && ok; ++tl) {
+            const int item = 2 * tl, stage = item % kStages;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
+            if (!ok) break;
+            const uint64_t desc_k = desc_k0 + static_cast<uint64_t>((stage * C::kStageBytes) >> 4);
+            for (int mt = 0; mt < n_mt && ok; ++mt) {
+              if (prev_mt >= 0) {       // the warpgroup that used the score buffer before has read its scores
+                ok = bounded_wait(bar(Bars::kSFree + prev_mt), prev_tl & 1, abort_flag, 20);
+                if (!ok) break;
+              }
+              ptx::tc_fence_after();
+              const uint64_t desc_q = desc_q0 + static_cast<uint64_t>(mt * ((kHalves * kHalfBytes) >> 4));
+              const uint32_t s_tmem = tmem_base + C::half_s();
+              if (ptx::elect_one()) {
+#pragma unroll
+                for (int kd = 0; kd < D / 16; ++kd) {
+                  const uint64_t off = static_cast<uint64_t>(((kd / 4) * kHalfBytes + (kd % 4) * 32) >> 4);
+                  ptx::umma_ss(s_tmem, desc_q + off, desc_k + off, idesc_qk, kd > 0 ? 1u : 0u);
+                }
+                ptx::umma_commit(bar(Bars::kSFull + mt));
+                if (mt == n_mt - 1) ptx::umma_commit(bar(Bars::kKvEmpty + stage));    // K tile read
+              }
+              prev_mt = mt;
+              prev_tl = tl;
+            }
+          }
+        } else if (warp == 3) {
+          bool ok = true;
+#pragma unroll 1
+          for (int tl = 0; tl < T && ok; ++tl) {
+            const int item = 2 * tl + 1, stage = item % kStages;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
+            if (!ok) break;
+            const uint64_t desc_v = desc_v0 + static_cast<uint64_t>((stage * C::kStageBytes) >> 4);
+            for (int mt = 0; mt < n_mt && ok; ++mt) {
+              ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag, 8);
+              if (!ok) break;
+              ptx::tc_fence_after();
+              const uint32_t p_tmem = tmem_base + C::half_p(mt);
+              const uint32_t o_tmem = tmem_base + C::half_o(mt);
+              if (ptx::elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < kBN / 16; ++kk)
+                  ptx::umma_ts(o_tmem, p_tmem + kk * 8, desc_v + static_cast<uint64_t>((kk * 2048) >> 4), idesc_pv,
+                               (tl == 0 && kk == 0) ? 0u : 1u);
+                ptx::umma_commit(bar(Bars::kODone + mt));
+                if (mt == n_mt - 1) ptx::umma_commit(bar(Bars::kKvEmpty + stage));    // V tile read
+              }
+            }
+          }
+        }
+      }
+    }
+
+    if (!C::kHalfTiles && classic && has_work) {
       if (warp == 0) {
         produce(0);
       } else if (warp == 1) {
@@ -1109,7 +1192,111 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
 
-    if (classic && has_work && (MT == 1 || wg < n_mt)) {
+    if constexpr (C::kHalfTiles) {
+      classic = false;
+      if (has_work && wg < n_mt) {
+        // =========================================================== softmax, one query tile of two
+        bool ok = true;
+        const uint32_t tS = t_lane + C::half_s();
+        const uint32_t tO = t_lane + C::half_o(mt);
+        const uint32_t tP = t_lane + C::half_p(mt);
+        int last_tl = -1;
+#pragma unroll 1
+        for (int tl = 0; tl < T && ok; ++tl) {
+          const int t = t_lo + tl;
+          const bool full_tile = t < TP && (L - t * kBN) >= kBN;      // uniform: every key visible to every row
+          ok = bounded_wait(bar(Bars::kSFull + mt), tl & 1, abort_flag, 9);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          uint32_t xa[32], xb[32], xc[32], xd[32];
+          uint32_t b0 = 0xFFFFFFFFu, b1 = 0xFFFFFFFFu, b2 = 0xFFFFFFFFu, b3 = 0xFFFFFFFFu;
+          if (!full_tile) { b0 = chunk_bits(t, 0); b1 = chunk_bits(t, 1); b2 = chunk_bits(t, 2); b3 = chunk_bits(t, 3); }
+          ptx::tmem_ld32(tS, xa);
+          ptx::tmem_ld32(tS + 32, xb);
+          ptx::tmem_ld32(tS + 64, xc);
+          ptx::tmem_ld32(tS + 96, xd);
+          ptx::tmem_wait_ld();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kSFree + mt));            // the scores are in registers: the other tile's turn
+          if (!full_tile) {
+            mask_chunk(xa, b0);
+            mask_chunk(xb, b1);
+            mask_chunk(xc, b2);
+            mask_chunk(xd, b3);
+          }
+          if (__any_sync(0xffffffffu, m_used == -INFINITY)) {
+            // nothing accumulated yet for some row: its reference is this tile's own row maximum
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            max_chunk(xa, mx);
+            max_chunk(xb, mx);
+            max_chunk(xc, mx);
+            max_chunk(xd, mx);
+            if (m_used == -INFINITY) m_used = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          }
+          float m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          if (tl >= 1) {
+            // the P V product of the tile before is complete: the P buffer is free and O may be rescaled
+            ok = bounded_wait(bar(Bars::kODone + mt), (tl - 1) & 1, abort_flag, 21);
+            if (!ok) break;
+            ptx::tc_fence_after();
+          }
+          exp_chunk(xa, sl2, m_ref, sum, tP);
+          exp_chunk(xb, sl2, m_ref, sum, tP + 16);
+          exp_chunk(xc, sl2, m_ref, sum, tP + 32);
+          exp_chunk(xd, sl2, m_ref, sum, tP + 48);
+          float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          float factor = 1.0f;
+          if (__any_sync(0xffffffffu, !(tile_sum <= kFastSumLimit))) {
+            // The reference was too low for some row of this warp (or a value is not finite): take the tile's
+            // true row maximum as the new reference and compute the tile again (the scores are in registers).
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            max_chunk(xa, mx);
+            max_chunk(xb, mx);
+            max_chunk(xc, mx);
+            max_chunk(xd, mx);
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            if (m_tile > m_used) {
+              if (m_used > -INFINITY) factor = exp2f((m_used - m_tile) * sl2);
+              m_used = m_tile;
+            }
+            m_ref = (m_used == -INFINITY) ? 0.0f : m_used * sl2;
+            sum[0] = sum[1] = sum[2] = sum[3] = 0.0f;
+            ptx::tmem_wait_st();
+            exp_chunk(xa, sl2, m_ref, sum, tP);
+            exp_chunk(xb, sl2, m_ref, sum, tP + 16);
+            exp_chunk(xc, sl2, m_ref, sum, tP + 32);
+            exp_chunk(xd, sl2, m_ref, sum, tP + 48);
+            tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+            if (__any_sync(0xffffffffu, factor != 1.0f) && tl > 0) {
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {
+                ptx::tmem_ld32(tO + c * 32, xa);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xa[j] = __float_as_uint(__uint_as_float(xa[j]) * factor);
+                ptx::tmem_st32(tO + c * 32, xa);
+              }
+            }
+          }
+          l = l * factor + tile_sum;
+          if (!full_tile) {
+            ok = clear_v_tail(t, 2 * tl + 1);
+            if (!ok) break;
+          }
+          ptx::tmem_wait_st();                     // P (and a rescaled O) are in TMEM
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(bar(Bars::kPFull + mt));
+          last_tl = tl;
+        }
+        // O is complete once the last P V of this accumulator has been committed
+        if (ok && last_tl >= 0) ok = bounded_wait(bar(Bars::kODone + mt), last_tl & 1, abort_flag, 11);
+        if (ok) ptx::tc_fence_after();
+        row_ok = ok;
+      }
+    }
+
+    if (!C::kHalfTiles && classic && has_work && (MT == 1 || wg < n_mt)) {
       // =========================================================== softmax, classic form
       bool ok = true;
       int last_tl = -1;

@@ -207,18 +207,18 @@ def test_rows_without_a_key_in_their_first_tile_and_very_negative_scores():
     assert np.abs(got_lse - rlse).max() <= 1e-3 * np.abs(rlse).max()
 
 
-@pytest.mark.parametrize("force", ["2", "2,g", "4"])
-def test_adversarial_scores_under_forced_slicings(force):
+@pytest.mark.parametrize("mt,force", [("1", "2"), ("1", "2,g"), ("1", "4"), ("2", "1"), ("2", "2"), ("2", "4,g")])
+def test_adversarial_scores_under_forced_slicings(mt, force):
     """The launch plan decides where the key slices begin, and with it which rows meet an empty first tile.  The
     library reads JET_FORCE_MT / JET_FORCE_SPLIT once per process, so the adversarial-score tests run again in
-    a child process under one query tile per CTA and 2 or 4 key slices (merged in a cluster or through the
-    workspace)."""
+    a child process under one or two query tiles per CTA and 1, 2 or 4 key slices (merged in a cluster or through
+    the workspace)."""
     import os
     import subprocess
     import sys
     if os.environ.get("JET_FORCE_SPLIT"):
         pytest.skip("already inside a forced run")
-    env = dict(os.environ, JET_FORCE_MT="1", JET_FORCE_SPLIT=force)
+    env = dict(os.environ, JET_FORCE_MT=mt, JET_FORCE_SPLIT=force)
     r = subprocess.run([sys.executable, "-m", "pytest", __file__, "-m", "gpu", "-x", "-q", "-k",
                         "very_negative or far_above"], env=env, capture_output=True, text=True,
                        cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))), timeout=600)
