@@ -110,10 +110,10 @@ struct Cfg {
   // and a separate P buffer (64 columns of packed bf16 pairs) per warpgroup.
   // MT == 2, shared-score-buffer form (see the kernel): accumulators [mt*128, +D), ONE 128-column score buffer
   // that the two query tiles use in turn, one P buffer (64 columns of packed bf16 pairs) per query tile.
-  static constexpr bool kHalfTiles = MT == 2;
-  __device__ static constexpr uint32_t half_o(int mt) { return mt * 128; }
-  __device__ static constexpr uint32_t half_s() { return 256; }
-  __device__ static constexpr uint32_t half_p(int mt) { return 384 + mt * 64; }
+  static constexpr bool kTurns = MT == 2;
+  __device__ static constexpr uint32_t turn_o(int mt) { return mt * 128; }
+  __device__ static constexpr uint32_t turn_s() { return 256; }
+  __device__ static constexpr uint32_t turn_p(int mt) { return 384 + mt * 64; }
   __device__ static constexpr uint32_t shared_o() { return 0; }
   __device__ static constexpr uint32_t shared_s(int w) { return 128 + 128 * w; }
   __device__ static constexpr uint32_t shared_p(int w) { return 384 + 64 * w; }
@@ -131,7 +131,7 @@ struct Cfg {
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
   enum { kQFull = 0, kKvFull = 1, kKvEmpty = 7, kSFull = 13, kSFree = 15, kPFull = 17, kODone = 19,
-         kClusterA = 21, kClusterC = 22, kRecv = 23, kOFinal = 25, kPFullB = 26, kODoneB = 28, kCount = 30,
+         kClusterA = 21, kClusterC = 22, kRecv = 23, kOFinal = 25, kCount = 26,
          kLoopFirst = kKvFull, kLoopEnd = kClusterA };    // the key loop's barriers exist twice (one set per pass)
 };
 
@@ -293,9 +293,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // one lane per barrier of the block
     if (lane < Bars::kCount) {
       uint32_t count = 1;
-      if (lane >= Bars::kKvEmpty && lane < Bars::kSFull) count = (MT == 1 || C::kHalfTiles) ? 1 : n_mt;   // arrivals per stage
-      else if ((lane >= Bars::kSFree && lane < Bars::kODone) || (lane >= Bars::kPFullB && lane < Bars::kODoneB))
-        count = 128;                                                                    // kSFree, kPFull: a softmax warpgroup
+      if (lane >= Bars::kKvEmpty && lane < Bars::kSFull) count = (MT == 1 || C::kTurns) ? 1 : n_mt;   // arrivals per stage
+      else if (lane >= Bars::kSFree && lane < Bars::kODone) count = 128;                // kSFree, kPFull: a softmax warpgroup
       else if (lane == Bars::kClusterA || lane == Bars::kClusterC) count = S;
       ptx::mbar_init(bar(lane), count);
       // slice merge: every slice sends this CTA its block of rows of query tile (lane - kRecv)
@@ -530,7 +529,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
           if (active) {
-            ptx::tmem_ld32(e_lane + (C::kHalfTiles ? C::half_o(mt) : C::o_col(mt, 0)) + c * 32, o);
+            ptx::tmem_ld32(e_lane + (C::kTurns ? C::turn_o(mt) : C::o_col(mt, 0)) + c * 32, o);
             ptx::tmem_wait_ld();
           }
 #pragma unroll
@@ -809,7 +808,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if constexpr (MT == 1) {
       if (has_work) {
         if (warp == 0) {
-          produce(kAhead);
+          produce(kAhead, p.paged ? 0 : -1);        // a paged tile is 16 small copies: two warps request them
+        } else if (warp == 2) {
+          if (p.paged) produce(kAhead, 1);
         } else if (warp == 1) {
           // =========================================================== tcgen05 issuers, shared-accumulator form
           // Key tile tl belongs to warpgroup tl & 1 (score buffer and P buffer of that warpgroup).  Warp 1
@@ -888,7 +889,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (classic) second_barrier_set();
     }
 
-    if constexpr (C::kHalfTiles) {
+    if constexpr (C::kTurns) {
       // =========================================================== two query tiles per CTA
       // Each query tile (stream) keeps the classic bookkeeping -- own accumulator, running reference, rescale
       // when it rises -- but the two tiles take turns on ONE score buffer, which leaves TMEM columns for a P
@@ -917,7 +918,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               }
               ptx::tc_fence_after();
               const uint64_t desc_q = desc_q0 + static_cast<uint64_t>(mt * ((kHalves * kHalfBytes) >> 4));
-              const uint32_t s_tmem = tmem_base + C::half_s();
+              const uint32_t s_tmem = tmem_base + C::turn_s();
               if (ptx::elect_one()) {
 #pragma unroll
                 for (int kd = 0; kd < D / 16; ++kd) {
@@ -943,8 +944,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               ok = bounded_wait(bar(Bars::kPFull + mt), tl & 1, abort_flag, 8);
               if (!ok) break;
               ptx::tc_fence_after();
-              const uint32_t p_tmem = tmem_base + C::half_p(mt);
-              const uint32_t o_tmem = tmem_base + C::half_o(mt);
+              const uint32_t p_tmem = tmem_base + C::turn_p(mt);
+              const uint32_t o_tmem = tmem_base + C::turn_o(mt);
               if (ptx::elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kBN / 16; ++kk)
@@ -959,7 +960,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
 
-    if (!C::kHalfTiles && classic && has_work) {
+    if (!C::kTurns && classic && has_work) {
       if (warp == 0) {
         produce(0);
       } else if (warp == 1) {
@@ -1192,14 +1193,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
 
-    if constexpr (C::kHalfTiles) {
+    if constexpr (C::kTurns) {
       classic = false;
       if (has_work && wg < n_mt) {
         // =========================================================== softmax, one query tile of two
         bool ok = true;
-        const uint32_t tS = t_lane + C::half_s();
-        const uint32_t tO = t_lane + C::half_o(mt);
-        const uint32_t tP = t_lane + C::half_p(mt);
+        const uint32_t tS = t_lane + C::turn_s();
+        const uint32_t tO = t_lane + C::turn_o(mt);
+        const uint32_t tP = t_lane + C::turn_p(mt);
         int last_tl = -1;
 #pragma unroll 1
         for (int tl = 0; tl < T && ok; ++tl) {
@@ -1296,7 +1297,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
 
-    if (!C::kHalfTiles && classic && has_work && (MT == 1 || wg < n_mt)) {
+    if (!C::kTurns && classic && has_work && (MT == 1 || wg < n_mt)) {
       // =========================================================== softmax, classic form
       bool ok = true;
       int last_tl = -1;
