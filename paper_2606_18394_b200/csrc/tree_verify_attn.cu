@@ -6,8 +6,9 @@
 //                 so all G heads of a KV group share every K/V tile that is loaded.
 //   warp 0      = TMA producer: Q tiles once, then K and V tiles (128 keys) through a ring of
 //                 shared-memory stages; paged caches are fetched one 16-row page per TMA box.
-//   warp 1      = tcgen05 issuer: S = Q K^T into TMEM, O += P V into TMEM (in the shared-accumulator
-//                 form of the key loop warp 1 issues the Q K^T and warp 3 the P V products).
+//   warp 1      = tcgen05 issuer: S = Q K^T into TMEM, O += P V into TMEM (outside the classic
+//                 form of the key loop warp 1 issues the Q K^T and warp 3 the P V products; warp 2 is
+//                 a second TMA producer where a paged cache or two query tiles call for one).
 //   warp 2      = TMEM allocation / release.
 //   warps 4..11 = two softmax warpgroups, one thread per row: the thread reads its 128 scores of a key
 //                 tile from TMEM, replaces the scores of keys the row must not see (key validity,
@@ -16,8 +17,9 @@
 //   key loop    = with one query tile per CTA: both warpgroups (alternate key tiles) add into one
 //                 accumulator against a reference fixed after the first tile; if a row overflows that
 //                 reference the CTA repeats the key range in the classic form (own accumulator and
-//                 running maximum per stream, accumulator rescaled when the maximum rises), which is
-//                 also the form used with two query tiles per CTA.  See "the key loop" below.
+//                 running maximum per stream, accumulator rescaled when the maximum rises).  With two
+//                 query tiles per CTA each warpgroup owns a tile with the classic bookkeeping, and the
+//                 tiles take turns on one score buffer.  See "the key loop" below.
 //   key slices  = when there are fewer work items than SMs the key range is cut into `nsplit`
 //                 slices.  After the key loop every CTA hands the normalised rows (bf16) and their
 //                 log-sum-exp to the rows' owner CTAs -- through distributed shared memory when the
@@ -82,34 +84,31 @@ template <int D, int MT>
 struct Cfg {
   static constexpr int kHalves = D / 64;
   static constexpr int kQBytes = MT * kHalves * kHalfBytes;
-  // P (probabilities, bf16) never touches shared memory: it is written over the first 64 columns of the
-  // score buffer it was computed from (two bf16 per 32-bit column) and read from there by the P V product.
+  // P (probabilities, bf16) never touches shared memory: it is written to TMEM (two bf16 per 32-bit column)
+  // and read from there by the P V product.
   static constexpr int kPBytes = 0;
   static constexpr int kStageBytes = kHalves * kHalfBytes;
   static constexpr int kStages = (D == 128) ? (MT == 1 ? 6 : 5) : 6;
   static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
-  // With one query tile per CTA two softmax warpgroups work on it as two independent streams: stream 0
-  // takes the even key tiles, stream 1 the odd ones, each with its own score buffer, P buffer, O
-  // accumulator and running maximum / sum.  Their phases interleave (one computes maxima while the
-  // other exponentiates), and the two partial results are combined once, after the key loop.
+  // Two softmax warpgroups in every form: with one query tile per CTA they share the tile's key tiles (even /
+  // odd), with two each takes one query tile.
   static constexpr int kStreams = MT == 1 ? 2 : 1;
   static constexpr int kBarBytes = 1024;
   static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
   static constexpr int kThreads = 128 + 128 * MT * kStreams;
-  // TMEM (512 columns):
-  //   MT == 1: stream i owns S [i*128, +128) and O [256 + i*128, +D); key tile t belongs to stream t & 1
-  //   MT == 2: query tile mt owns S [mt*256, +128) and O [mt*256+128, +D)
+  // TMEM (512 columns), three layouts (the key loop's forms are described in the kernel):
+  //   MT == 1, shared-accumulator pass: O [0, +D), warpgroup w: scores [128 + 128 w, +128), P [384 + 64 w, +64)
+  //   MT == 1, classic pass (fallback): stream i: scores / P [i*128, +128), O [256 + i*128, +D); key tile t
+  //            belongs to stream t & 1
+  //   MT == 2: O of query tile mt [mt*128, +D), ONE score buffer [256, +128) that the two query tiles use in
+  //            turn, P of query tile mt [384 + 64 mt, +64)
   static constexpr int kTmemCols = 512;
-  __device__ static constexpr uint32_t s_col(int mt, int t) { return MT == 1 ? (t & 1) * 128 : mt * 256; }
-  __device__ static constexpr uint32_t o_col(int mt, int t) { return MT == 1 ? 256 + (t & 1) * 128 : mt * 256 + 128; }
+  __device__ static constexpr uint32_t s_col(int mt, int t) { return (t & 1) * 128; }
+  __device__ static constexpr uint32_t o_col(int mt, int t) { return 256 + (t & 1) * 128; }
   // Each score buffer (and the P that replaces it) has its own barriers, so that neither side can run two
-  // phases ahead of the other on one barrier: buffer index and use count of key tile t of query tile mt.
-  __device__ static constexpr int s_buf(int mt, int t) { return MT == 1 ? (t & 1) : mt; }
-  __device__ static constexpr int s_use(int t) { return MT == 1 ? (t >> 1) : t; }
-  // MT == 1, shared-accumulator pass (see the kernel): one accumulator for both warpgroups, a score buffer
-  // and a separate P buffer (64 columns of packed bf16 pairs) per warpgroup.
-  // MT == 2, shared-score-buffer form (see the kernel): accumulators [mt*128, +D), ONE 128-column score buffer
-  // that the two query tiles use in turn, one P buffer (64 columns of packed bf16 pairs) per query tile.
+  // phases ahead of the other on one barrier: buffer index and use count of key tile t (classic pass).
+  __device__ static constexpr int s_buf(int mt, int t) { return t & 1; }
+  __device__ static constexpr int s_use(int t) { return t >> 1; }
   static constexpr bool kTurns = MT == 2;
   __device__ static constexpr uint32_t turn_o(int mt) { return mt * 128; }
   __device__ static constexpr uint32_t turn_s() { return 256; }
@@ -680,7 +679,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   };
 
   // ---------------- the key loop
-  // Two forms.  The classic form gives every stream its own accumulator and reference maximum, which may rise
+  // Three forms (the third, for two query tiles per CTA, is described where it starts).  The classic form
+  // gives every stream its own accumulator and reference maximum, which may rise
   // at any tile (the accumulator is rescaled); it is exact for any input.  With one query tile per CTA the
   // loop first runs in the shared-accumulator form: both warpgroups add into ONE accumulator against a per-row
   // reference that is fixed after the first key tile, which frees the TMEM columns for P buffers apart from
