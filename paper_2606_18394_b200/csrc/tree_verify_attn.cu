@@ -32,6 +32,7 @@
 #include <cuda_bf16.h>
 #include <cstdlib>
 #include <cstring>
+#include <type_traits>
 
 #include "jet_common.cuh"
 #include "sm100_ptx.cuh"
@@ -723,8 +724,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
     // =========================================================== TMA producer (warp 0)
     // K runs `ahead` key tiles in front of V in the ring (0: K_t, V_t alternate).
-    // only: -1 = this warp requests every tile, 0 = the K tiles only, 1 = the V tiles only (two producer warps).
-    auto produce = [&](const int ahead, const int only = -1) {
+    // only_c (a compile-time constant: a run-time role cost 4 % on long contiguous prefixes): -1 = this warp
+    // requests every tile, 0 = the K tiles only, 1 = the V tiles only (two producer warps).
+    auto produce = [&](const int ahead, auto only_c) {
+      constexpr int only = decltype(only_c)::value;
       if (tid == 0) JET_TR(27);
       bool ok = true;
       int issued = 0;
@@ -808,9 +811,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if constexpr (MT == 1) {
       if (has_work) {
         if (warp == 0) {
-          produce(kAhead, p.paged ? 0 : -1);        // a paged tile is 16 small copies: two warps request them
+          // a paged tile is 16 small copies: two warps request them
+          if (p.paged) produce(kAhead, std::integral_constant<int, 0>{});
+          else produce(kAhead, std::integral_constant<int, -1>{});
         } else if (warp == 2) {
-          if (p.paged) produce(kAhead, 1);
+          if (p.paged) produce(kAhead, std::integral_constant<int, 1>{});
         } else if (warp == 1) {
           // =========================================================== tcgen05 issuers, shared-accumulator form
           // Key tile tl belongs to warpgroup tl & 1 (score buffer and P buffer of that warpgroup).  Warp 1
@@ -899,9 +904,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       classic = false;
       if (has_work) {
         if (warp == 0) {
-          produce(0, 0);                     // K tiles
+          produce(0, std::integral_constant<int, 0>{});                     // K tiles
         } else if (warp == 2) {
-          produce(0, 1);                     // V tiles (a paged tile is 16 small copies: two warps request them)
+          produce(0, std::integral_constant<int, 1>{});                     // V tiles (a paged tile is 16 small copies: two warps request them)
         } else if (warp == 1) {
           bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
           int prev_mt = -1, prev_tl = 0;
@@ -962,7 +967,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
     if (!C::kTurns && classic && has_work) {
       if (warp == 0) {
-        produce(0);
+        produce(0, std::integral_constant<int, -1>{});
       } else if (warp == 1) {
         // =========================================================== tcgen05 issuer, classic form
         // A stream is a chain  S = Q K^T -> softmax -> O += P V -> next S  on its own score buffer (which the P
