@@ -10,6 +10,7 @@ from .generators import (  # noqa: F401
     chain_tree,
     f32_to_bf16_bits,
     make_attn_inputs,
+    make_draft_logits,
     make_logp,
     make_paged_cache,
     make_target_logits,

@@ -57,6 +57,20 @@ def make_logp(rng: np.random.Generator, N: int, V: int, sigma: float, peaked_p: 
     return (logits - lse).astype(np.float32)
 
 
+def make_draft_logits(rng: np.random.Generator, N: int, V: int, sigma: float, peaked_p: float | None = None,
+                      offset: float = 0.0):
+    """[N,V] float32 raw draft logits: N(0, sigma) + offset, not normalised; with ``peaked_p`` one random token
+    per depth is raised to about that probability (as in make_logp)."""
+    logits = (rng.standard_normal((N, V), dtype=np.float32) * np.float32(sigma)).astype(np.float64)
+    if peaked_p is not None:
+        for d in range(N):
+            t = int(rng.integers(0, V))
+            rest = np.delete(logits[d], t)
+            m = rest.max()
+            logits[d, t] = np.log(peaked_p / (1.0 - peaked_p)) + m + np.log(np.exp(rest - m).sum())
+    return (logits + offset).astype(np.float32)
+
+
 # ---------------------------------------------------------------- attention operands
 def make_attn_inputs(rng: np.random.Generator, B: int, Hq: int, Hkv: int, D: int, L: int):
     """q [B,Hq,D], k/v prefix [L,Hkv,D], tree_k/tree_v [B,Hkv,D]; N(0,1) rounded to bf16 bits."""

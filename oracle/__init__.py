@@ -13,10 +13,12 @@ from .jet_oracle import (  # noqa: F401
     gather_paged_prefix,
     kv_compact_ref,
     kv_compact_tail_ref,
+    log_softmax_ref,
     target_probs_ref,
     tree_accept_ref,
     tree_accept_sample_ref,
     tree_attn_ref,
     tree_attn_rows_ref,
+    tree_build_logits_ref,
     tree_build_ref,
 )

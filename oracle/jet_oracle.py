@@ -10,6 +10,8 @@ Each function follows one passage of the paper:
   its ``score_mode`` argument selects the alternative expansion scores of
   Appendix C (per-depth entropy alone, accumulated log-probability plus alpha
   times the per-depth entropy), with ``depth_entropy_ref`` as the entropy.
+  ``tree_build_logits_ref`` is the same fed with raw draft logits
+  (``log_softmax_ref`` first).
 * ``tree_attn_ref``    -- the tree-causal mask and masked attention equations
   of Section 3.2 (prefix visible to every node, a node sees Anc(v) + {v}).
 * ``tree_accept_ref``  -- the greedy acceptance rule of Section 3.3 and
@@ -53,7 +55,11 @@ large alpha the entropy-only tree), closed-form entropies (uniform, two-point),
 closed-form trees for monotone entropies (level order / comb) and by replaying
 the pop order against priorities recomputed from the paths; whether the entropy
 term is that of the node's own depth or a sum along the branch is a reading
-with no counterpart to check against: parity unpinned for that reading only.
+with no counterpart to check against: parity unpinned for that reading only.  ``log_softmax_ref`` is pinned against
+scipy's log_softmax, closed forms (uniform, two-point), rows summing to one and
+shift invariance; ``tree_build_logits_ref`` by the invariance of the tree under
+a per-row shift of the logits and by agreement with ``tree_build_ref`` on
+log-probabilities that scipy computed.
 """
 from __future__ import annotations
 
@@ -97,6 +103,29 @@ def depth_entropy_ref(logp: np.ndarray, N: int) -> np.ndarray:
         fin = np.isfinite(l)
         H[d] = np.float32(-np.sum(np.exp(l[fin]) * l[fin]))
     return H
+
+
+def log_softmax_ref(logits: np.ndarray):
+    """Draft log-probabilities from raw draft logits (Section 3.3: the tree is scored with log q): per row
+    lse = log sum_v exp(z_v), formed in float64 as max + log(sum(exp(z - max))), and
+    logp_v = float32(float64(z_v) - lse), rounded once.  Returns (logp [N,V] float32, lse [N] float64).
+    Entries of -inf stay -inf (probability 0)."""
+    z = np.asarray(logits, dtype=np.float64)
+    m = z.max(axis=1)
+    lse = m + np.log(np.exp(z - m[:, None]).sum(axis=1))
+    return (z - lse[:, None]).astype(np.float32), lse
+
+
+def tree_build_logits_ref(logits: np.ndarray, root_token: int, N: int, W: int, B: int,
+                          score_mode: str = "accum_logp", alpha: float = 0.0) -> dict:
+    """Algorithm 1 fed with raw draft logits: exactly log_softmax_ref followed by tree_build_ref (the
+    candidates are ranked by their rounded float32 log-probabilities, so two logits that round to the same
+    log-probability tie and the lower token id comes first, as in tree_build_ref).  Adds ``depth_lse``
+    (float32 rounding of each row's lse) to the result."""
+    logp, lse = log_softmax_ref(np.asarray(logits)[:N])
+    out = tree_build_ref(logp, root_token, N, W, B, score_mode=score_mode, alpha=alpha)
+    out["depth_lse"] = lse.astype(np.float32)
+    return out
 
 
 def tree_build_ref(logp: np.ndarray, root_token: int, N: int, W: int, B: int,
