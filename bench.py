@@ -156,7 +156,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0, tail=False):
+def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0, tail=False, draft_logits=False):
     """Seeded synthetic step inputs on the device.  Returns (VerifyStep, info dict)."""
     import torch
     from paper_2606_18394_b200.step import VerifyStep
@@ -202,7 +202,9 @@ def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0
         rest = logits.clone()
         rest[torch.arange(N, device=device), top] = -float("inf")
         logits[torch.arange(N, device=device), top] = np.log(0.7 / 0.3) + torch.logsumexp(rest, dim=1)
-        st.logp[b].copy_(torch.log_softmax(logits, dim=1).float())
+        # --draft-input logits: the raw logits themselves (jet_tree_build_logits normalises on the fly)
+        st.logp[b].copy_(logits.float() if draft_logits else torch.log_softmax(logits, dim=1).float())
+    st.draft_logits = draft_logits
     st.root_token.copy_(torch.arange(batch, device=device, dtype=torch.int32) + 1)
     st.logits.copy_(torch.randn(st.logits.shape, generator=gen, device=device, dtype=torch.float32) * c["sigma_target"])
     # plant the target arg-max along one random path of the tree that jet_tree_build produces
@@ -273,7 +275,8 @@ def bench_jet(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
     c = workload(args.config, args.budget, args.batch)
-    st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha, args.layout == "tail")
+    st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha, args.layout == "tail",
+                            args.draft_input == "logits")
     layers = c["layers"]
     if args.accept == "sample":
         st.accept_mode = "sample"
@@ -467,7 +470,8 @@ def bench_jet(args):
                    "paged": bool(c.get("paged")), "cuda_graph": not args.no_graph,
                    "l2": "every layer streams its own KV buffers; one step reads far more than the 126 MB L2",
                    "accepted_len": acc, "accept": args.accept, "tree_kv": args.layout,
-                   "score": args.score if args.score != "hybrid" else f"hybrid(alpha={args.score_alpha})"},
+                   "score": args.score if args.score != "hybrid" else f"hybrid(alpha={args.score_alpha})",
+                   "draft_input": args.draft_input},
         "attn_us_per_layer": attn_us,
         "e2e": {"value": e2e_ms_step * 1e3 / (layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,
@@ -497,7 +501,8 @@ def oracle_sample(c, x, attn_layers):
     import oracle
     B, N, W, layers = c["B"], c["N"], c["W"], c["layers"]
     t0 = time.perf_counter()
-    tree = oracle.tree_build_ref(x["logp"], x["root"], N, W, B)
+    build = oracle.tree_build_logits_ref if x.get("draft_logits") else oracle.tree_build_ref
+    tree = build(x["logp"], x["root"], N, W, B, score_mode=x.get("score_mode", "accum_logp"), alpha=x.get("alpha", 0.0))
     t_build = time.perf_counter() - t0
     t_attn = 0.0
     for layer in range(attn_layers):
@@ -540,7 +545,8 @@ def cpu_baseline(st, c, info):
         vs = [_bits(st.v_cache[l, 0, :L]) for l in range(nl)]
     x = dict(logp=st.logp[0].cpu().numpy(), root=int(st.root_token[0].item()), logits=st.logits[0].cpu().numpy(),
              planted=info["planted"][0], scale=st.scale, q=[_bits(st.q[l, 0]) for l in range(nl)], k=ks, v=vs,
-             tk=[_bits(st.tree_k[l, 0]) for l in range(nl)], tv=[_bits(st.tree_v[l, 0]) for l in range(nl)])
+             tk=[_bits(st.tree_k[l, 0]) for l in range(nl)], tv=[_bits(st.tree_v[l, 0]) for l in range(nl)],
+             draft_logits=st.draft_logits, score_mode=st.score_mode, alpha=st.score_alpha)
     secs, desc, per_layer_us = oracle_sample(c, x, attn_layers=nl)
     return {"value": per_layer_us, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle", "sample": desc,
             "seconds": secs, "host_cpus": os.cpu_count()}
@@ -604,6 +610,8 @@ def main():
     ap.add_argument("--score", choices=["accum_logp", "entropy", "hybrid"], default="accum_logp",
                     help="expansion score of the tree construction (hybrid: --score-alpha)")
     ap.add_argument("--score-alpha", type=float, default=1.0)
+    ap.add_argument("--draft-input", choices=["logp", "logits"], default="logp",
+                    help="the draft head's output as log-probabilities, or as raw logits (normalised on the fly)")
     ap.add_argument("--accept", choices=["greedy", "sample"], default="greedy",
                     help="acceptance rule of the step: greedy (the headline) or the non-greedy rule at temperature 1")
     args = ap.parse_args()

@@ -13,6 +13,7 @@
  * and their variants:
  *
  *   jet_tree_build_scored      entropy / hybrid expansion scores, per-sequence budgets
+ *   jet_tree_build_logits      the same fed with raw draft logits (log-softmax on the fly)
  *   jet_tree_verify_attn_tail  the tree's K/V rows live in the cache behind the prefix
  *   jet_kv_compact_tail        in-place commit for that layout
  *   jet_tree_accept_static     greedy acceptance on scratch built into the library
@@ -139,6 +140,37 @@ JET_API jet_status jet_tree_build_scored(const float* logp, int64_t logp_batch_s
                                  int32_t* token, float* score, uint32_t* anc_mask, int32_t* n_nodes,
                                  float* depth_entropy, void* workspace, size_t workspace_bytes,
                                  void* stream);
+
+/* ---------------------------------------------------------------------------
+ * jet_tree_build_logits -- jet_tree_build_scored fed with RAW draft logits z
+ * (Section 3.3: the draft head's one forward gives logits for N depths; the
+ * tree is scored with their log-probabilities).  Computes exactly what a
+ * log-softmax followed by jet_tree_build_scored computes, without the [N,V]
+ * log-probabilities ever existing in memory:
+ *   lse[b,d]  = log sum_t exp(z[b,d,t]), formed in fp64 as max + log(sum exp(z - max));
+ *   logp[b,d,t] = fl32(double(z[b,d,t]) - lse[b,d])   (one rounding);
+ * candidates are ranked by these fp32 log-probabilities (two logits that round
+ * to the same log-probability tie -> lowest token id), entropies are taken of
+ * them, scores add them.  The fp64 sums are formed in a fixed order (per 4096-
+ * entry slice, then over the slices), so results do not change from run to run;
+ * against another summation order lse can differ in its last bits, which moves
+ * a log-probability only if it sits within ~1e-15 (relative) of a rounding
+ * boundary.
+ *
+ *   logits       fp32 [batch, N, V], strides as for logp.  No NaN, no +inf; a
+ *                row must hold at least one finite entry (-inf = probability 0)
+ *   depth_lse    fp32 [batch, N] out, may be NULL: fl32(lse[b,d])
+ *   every other argument as for jet_tree_build_scored
+ * Workspace: jet_tree_build_logits_workspace_bytes.
+ */
+JET_API size_t jet_tree_build_logits_workspace_bytes(int batch, int N, int V, int W);
+
+JET_API jet_status jet_tree_build_logits(const float* logits, int64_t logits_batch_stride,
+                                 int64_t logits_depth_stride, const int32_t* root_token, int batch, int N,
+                                 int V, int W, int B, const int32_t* node_budget, int score_mode, float alpha,
+                                 int32_t* parent, int32_t* depth, int32_t* token, float* score,
+                                 uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy, float* depth_lse,
+                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
  * jet_tree_verify_attn -- the masked tree attention of Section 3.2 (tree-causal

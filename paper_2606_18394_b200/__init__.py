@@ -21,6 +21,8 @@ from .binding import (  # noqa: F401
     jet_tree_accept_static,
     jet_tree_accept_workspace_bytes,
     jet_tree_build,
+    jet_tree_build_logits,
+    jet_tree_build_logits_workspace_bytes,
     jet_tree_build_scored,
     jet_tree_build_scored_workspace_bytes,
     jet_tree_build_workspace_bytes,

@@ -32,6 +32,9 @@ _SIGNATURES = {
     "jet_tree_build_scored_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "jet_tree_build_scored": (_c.c_int32, [_vp, _i64, _i64, _vp, _i, _i, _i, _i, _i, _vp, _i, _f, _vp, _vp, _vp, _vp,
                                            _vp, _vp, _vp, _vp, _sz, _vp]),
+    "jet_tree_build_logits_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "jet_tree_build_logits": (_c.c_int32, [_vp, _i64, _i64, _vp, _i, _i, _i, _i, _i, _vp, _i, _f, _vp, _vp, _vp, _vp,
+                                           _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_tree_verify_attn_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "jet_tree_verify_attn": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp,
                                           _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -142,6 +145,27 @@ def jet_tree_build_scored(logp, root_token, batch, N, V, W, B, score_mode, alpha
                                       _p(n_nodes), _p(depth_entropy), _p(workspace), wb, _stream(stream))
     if check:
         _check(st, "jet_tree_build_scored")
+    return st
+
+
+def jet_tree_build_logits_workspace_bytes(batch, N, V, W) -> int:
+    return load().jet_tree_build_logits_workspace_bytes(batch, N, V, W)
+
+
+def jet_tree_build_logits(logits, root_token, batch, N, V, W, B, score_mode, alpha, parent, depth, token, score,
+                          anc_mask, n_nodes, depth_entropy, depth_lse, workspace, workspace_bytes=None,
+                          logits_batch_stride=None, logits_depth_stride=None, stream=None, check=True,
+                          node_budget=None):
+    bs = logits_batch_stride if logits_batch_stride is not None else logits.stride(0)
+    ds = logits_depth_stride if logits_depth_stride is not None else logits.stride(1)
+    wb = workspace_bytes if workspace_bytes is not None else (workspace.numel() * workspace.element_size()
+                                                              if workspace is not None else 0)
+    st = load().jet_tree_build_logits(_p(logits), bs, ds, _p(root_token), batch, N, V, W, B, _p(node_budget),
+                                      int(score_mode), float(alpha), _p(parent), _p(depth), _p(token), _p(score),
+                                      _p(anc_mask), _p(n_nodes), _p(depth_entropy), _p(depth_lse), _p(workspace), wb,
+                                      _stream(stream))
+    if check:
+        _check(st, "jet_tree_build_logits")
     return st
 
 

@@ -4,6 +4,11 @@
 // entropy alone; accumulated log-probability + alpha * per-depth entropy): the scan
 // also leaves per-slice sums of p * log p (fp64), the expansion kernel adds them up
 // per depth and uses the entropy in the queue's priority.
+// jet_tree_build_logits: the same fed with raw draft logits.  One more launch in front
+// (lse_partial_kernel: per-slice maximum and sum of exponentials in fp64); the scan then
+// forms every log-probability on the fly as float(double(z) - lse), so the [N,V]
+// log-probabilities never exist in memory and the second pass over the logits comes
+// out of L2.
 //
 // Two launches:
 //   topw_partial_kernel  grid (chunks, N, batch): every block scans one slice of one
@@ -29,23 +34,11 @@ constexpr int kTopChunk = kTopThreads * kTopElems;   // vocabulary slice per blo
 // many equal values all of them become candidates and the key order (value, then lowest index) decides.
 // kEntropy: the block also leaves sum(exp(l) * l) over its slice (fp64; entries of -inf contribute 0) for the
 // per-depth entropy; the reduction order is fixed, so the value does not change from run to run.
-template <bool kEntropy>
-__global__ void __launch_bounds__(kTopThreads)
-topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
-                    int V, int Wc, int nchunks, bool vec_ok,
-                    unsigned long long* __restrict__ cand, double* __restrict__ plogp_partial) {
-  grid_dependency_wait();
-  const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x, lane = tid & 31;
-  const float* row = logp + b * batch_stride + d * depth_stride;
-  const int base = chunk * kTopChunk;
-
-  // element e of this thread has vocabulary index idx_of(e); out-of-range elements are -inf and never candidates
-  float v[kTopElems];
-  const bool vec = vec_ok && base + kTopChunk <= V;
-  auto idx_of = [&](int e) -> int {
-    return vec ? base + ((e >> 2) * kTopThreads + tid) * 4 + (e & 3) : base + e * kTopThreads + tid;
-  };
+// Loads the 16 elements of a thread: element e has vocabulary index
+//   vec ? base + ((e >> 2) * kTopThreads + tid) * 4 + (e & 3) : base + e * kTopThreads + tid;
+// elements beyond V read as -inf.
+__device__ __forceinline__ void load_slice(const float* __restrict__ row, int base, int V, bool vec, int tid,
+                                           float (&v)[kTopElems]) {
   if (vec) {
     const float4* row4 = reinterpret_cast<const float4*>(row + base);
 #pragma unroll
@@ -59,6 +52,104 @@ topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_
       const int idx = base + i * kTopThreads + tid;
       v[i] = idx < V ? __ldg(row + idx) : -INFINITY;
     }
+  }
+}
+
+// Raw logits: every block leaves (m, z) of its slice, m = the slice's maximum and z = sum(exp(double(x) - m))
+// in fp64 with a fixed reduction order (a slice of -inf only: m = -inf, z = 0).
+__global__ void __launch_bounds__(kTopThreads)
+lse_partial_kernel(const float* __restrict__ logits, int64_t batch_stride, int64_t depth_stride, int V, int nchunks,
+                   bool vec_ok, double* __restrict__ lse_partial) {
+  grid_dependency_wait();
+  const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const float* row = logits + b * batch_stride + d * depth_stride;
+  const int base = chunk * kTopChunk;
+  float v[kTopElems];
+  load_slice(row, base, V, vec_ok && base + kTopChunk <= V, tid, v);
+  float m = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < kTopElems; ++i) m = fmaxf(m, v[i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  __shared__ float s_m[kTopThreads / 32];
+  __shared__ double s_z[kTopThreads / 32];
+  if (lane == 0) s_m[tid >> 5] = m;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < kTopThreads / 32; ++w) m = fmaxf(m, s_m[w]);
+  double z = 0.0;
+  if (m > -INFINITY) {
+    const double md = static_cast<double>(m);
+#pragma unroll
+    for (int i = 0; i < kTopElems; ++i)
+      if (v[i] > -INFINITY) z += exp(static_cast<double>(v[i]) - md);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+  if (lane == 0) s_z[tid >> 5] = z;
+  __syncthreads();
+  if (tid == 0) {
+    double total = 0.0;
+    for (int w = 0; w < kTopThreads / 32; ++w) total += s_z[w];
+    double* out = lse_partial + ((static_cast<size_t>(b) * gridDim.y + d) * nchunks + chunk) * 2;
+    out[0] = static_cast<double>(m);
+    out[1] = total;
+  }
+}
+
+// The row's log-sum-exp from the slices' (m, z): M = max m, lse = M + log(sum z * exp(m - M)), fp64, one warp,
+// fixed order (every block of a row gets the same bits).
+__device__ __forceinline__ double row_lse(const double* __restrict__ part, int nchunks, int lane) {
+  double M = -INFINITY;
+  for (int i = lane; i < nchunks; i += 32) M = fmax(M, part[2 * i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmax(M, __shfl_xor_sync(0xffffffffu, M, o));
+  double Z = 0.0;
+  for (int i = lane; i < nchunks; i += 32) {
+    const double m = part[2 * i], z = part[2 * i + 1];
+    if (z > 0.0) Z += z * exp(m - M);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, o);
+  return M + log(Z);
+}
+
+// kLogits: the row holds raw logits; lse_partial holds its slices' (m, z) and every element becomes the
+// log-probability float(double(x) - lse) before anything else looks at it (block 0 of the row also leaves
+// float(lse) in depth_lse_out if that is given).
+template <bool kEntropy, bool kLogits>
+__global__ void __launch_bounds__(kTopThreads)
+topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_t depth_stride,
+                    int V, int Wc, int nchunks, bool vec_ok,
+                    unsigned long long* __restrict__ cand, double* __restrict__ plogp_partial,
+                    const double* __restrict__ lse_partial, float* __restrict__ depth_lse_out) {
+  grid_dependency_wait();
+  const int chunk = blockIdx.x, d = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const float* row = logp + b * batch_stride + d * depth_stride;
+  const int base = chunk * kTopChunk;
+
+  // element e of this thread has vocabulary index idx_of(e); out-of-range elements are -inf and never candidates
+  float v[kTopElems];
+  const bool vec = vec_ok && base + kTopChunk <= V;
+  auto idx_of = [&](int e) -> int {
+    return vec ? base + ((e >> 2) * kTopThreads + tid) * 4 + (e & 3) : base + e * kTopThreads + tid;
+  };
+  load_slice(row, base, V, vec, tid, v);
+  if constexpr (kLogits) {
+    __shared__ double s_lse;
+    if (tid < 32) {
+      const double lse = row_lse(lse_partial + (static_cast<size_t>(b) * gridDim.y + d) * nchunks * 2, nchunks, lane);
+      if (lane == 0) {
+        s_lse = lse;
+        if (chunk == 0 && depth_lse_out) depth_lse_out[static_cast<size_t>(b) * gridDim.y + d] = static_cast<float>(lse);
+      }
+    }
+    __syncthreads();
+    const double lse = s_lse;
+#pragma unroll
+    for (int i = 0; i < kTopElems; ++i) v[i] = static_cast<float>(static_cast<double>(v[i]) - lse);
   }
 
   if constexpr (kEntropy) {
@@ -327,7 +418,7 @@ jet_status tree_build_launch(const float* logp, int64_t logp_batch_stride, int64
                              float alpha, int32_t* parent, int32_t* depth, int32_t* token, float* score,
                              uint32_t* anc_mask, int32_t* n_nodes, float* depth_entropy,
                              const int32_t* node_budget, void* workspace, size_t workspace_bytes, size_t need,
-                             void* stream) {
+                             void* stream, bool from_logits = false, float* depth_lse = nullptr) {
   if (!logp || !root_token || !parent || !depth || !token || !anc_mask || !n_nodes)
     return JET_ERR_INVALID_ARG;
   if (batch < 1 || batch > 65535 || N < 1 || N > JET_MAX_DEPTH || W < 1 || W > JET_MAX_WIDTH || V < 1 ||
@@ -344,16 +435,34 @@ jet_status tree_build_launch(const float* logp, int64_t logp_batch_stride, int64
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto* cand = static_cast<unsigned long long*>(workspace);
   auto* plogp = reinterpret_cast<double*>(static_cast<uint8_t*>(workspace) + cand_bytes(batch, N, V, W));
+  const double* no_lse = nullptr;
+  float* no_out = nullptr;
+  if (from_logits) {
+    double* lse_part = plogp + round_up(static_cast<size_t>(batch) * N * nchunks * sizeof(double), 256) / sizeof(double);
+    launch_dependent(lse_partial_kernel, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+        logp, logp_batch_stride, logp_depth_stride, V, nchunks, vec_ok, lse_part);
+    const double* lse_in = lse_part;
+    if (score_mode == JET_SCORE_ACCUM_LOGP)
+      launch_dependent(topw_partial_kernel<false, true>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+          logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, static_cast<double*>(nullptr),
+          lse_in, depth_lse);
+    else
+      launch_dependent(topw_partial_kernel<true, true>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+          logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, plogp, lse_in, depth_lse);
+  } else if (score_mode == JET_SCORE_ACCUM_LOGP) {
+    launch_dependent(topw_partial_kernel<false, false>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+        logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, static_cast<double*>(nullptr),
+        no_lse, no_out);
+  } else {
+    launch_dependent(topw_partial_kernel<true, false>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
+        logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, plogp, no_lse, no_out);
+  }
   if (score_mode == JET_SCORE_ACCUM_LOGP) {
-    launch_dependent(topw_partial_kernel<false>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
-        logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, static_cast<double*>(nullptr));
     launch_dependent(tree_expand_kernel<0>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
         root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
         static_cast<const double*>(nullptr), 0.0f, static_cast<float*>(nullptr), node_budget);
     return launch_status();
   }
-  launch_dependent(topw_partial_kernel<true>, dim3(nchunks, N, batch), dim3(kTopThreads), st,
-      logp, logp_batch_stride, logp_depth_stride, V, Wc, nchunks, vec_ok, cand, plogp);
   if (score_mode == JET_SCORE_ENTROPY)
     launch_dependent(tree_expand_kernel<1>, dim3(batch), dim3(kExpThreads), st, logp, logp_batch_stride, logp_depth_stride,
         root_token, N, Wc, B, nchunks, cand, parent, depth, token, score, anc_mask, n_nodes,
@@ -402,4 +511,23 @@ extern "C" jet_status jet_tree_build_scored(const float* logp, int64_t logp_batc
   return jet::tree_build_launch(logp, logp_batch_stride, logp_depth_stride, root_token, batch, N, V, W, B, score_mode,
                                 alpha, parent, depth, token, score, anc_mask, n_nodes, depth_entropy, node_budget,
                                 workspace, workspace_bytes, need, stream);
+}
+
+extern "C" size_t jet_tree_build_logits_workspace_bytes(int batch, int N, int V, int W) {
+  if (batch < 1 || N < 1 || V < 1 || W < 1) return 0;
+  return jet_tree_build_scored_workspace_bytes(batch, N, V, W) +
+         jet::round_up(static_cast<size_t>(batch) * N * jet::chunks_for(V) * 2 * sizeof(double), 256);
+}
+
+extern "C" jet_status jet_tree_build_logits(const float* logits, int64_t logits_batch_stride,
+                                            int64_t logits_depth_stride, const int32_t* root_token,
+                                            int batch, int N, int V, int W, int B, const int32_t* node_budget,
+                                            int score_mode, float alpha, int32_t* parent, int32_t* depth,
+                                            int32_t* token, float* score, uint32_t* anc_mask, int32_t* n_nodes,
+                                            float* depth_entropy, float* depth_lse, void* workspace,
+                                            size_t workspace_bytes, void* stream) {
+  const size_t need = jet_tree_build_logits_workspace_bytes(batch, N, V, W);
+  return jet::tree_build_launch(logits, logits_batch_stride, logits_depth_stride, root_token, batch, N, V, W, B,
+                                score_mode, alpha, parent, depth, token, score, anc_mask, n_nodes, depth_entropy,
+                                node_budget, workspace, workspace_bytes, need, stream, true, depth_lse);
 }

@@ -68,7 +68,11 @@ class VerifyStep:
         def ws(nbytes):
             return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=dev)
         self.ws_build = ws(max(jet.jet_tree_build_workspace_bytes(batch, N, V, W),
-                               jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W)))
+                               jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W),
+                               jet.jet_tree_build_logits_workspace_bytes(batch, N, V, W)))
+        # True: `logp` holds the draft head's RAW logits and the tree is built by jet_tree_build_logits
+        self.draft_logits = False
+        self.depth_lse = torch.zeros((batch, N), dtype=torch.float32, device=dev)
         # expansion score of the tree construction: "accum_logp" (default), "entropy" or "hybrid" (+ score_alpha)
         self.score_mode = "accum_logp"
         self.node_budget = None        # optional i32 [batch]: per-sequence budgets <= B
@@ -121,11 +125,16 @@ class VerifyStep:
 
     # ------------------------------------------------------------------ the four calls
     def tree_build(self):
-        if self.score_mode == "accum_logp" and self.node_budget is None:
+        mode = {"accum_logp": 0, "entropy": 1, "hybrid": 2}[self.score_mode]
+        if self.draft_logits:
+            jet.jet_tree_build_logits(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, mode,
+                                      self.score_alpha, self.parent, self.depth, self.token, self.score,
+                                      self.anc_mask, self.n_nodes, self.depth_entropy, self.depth_lse,
+                                      self.ws_build, node_budget=self.node_budget)
+        elif self.score_mode == "accum_logp" and self.node_budget is None:
             jet.jet_tree_build(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, self.parent,
                                self.depth, self.token, self.score, self.anc_mask, self.n_nodes, self.ws_build)
         else:
-            mode = {"accum_logp": 0, "entropy": 1, "hybrid": 2}[self.score_mode]
             jet.jet_tree_build_scored(self.logp, self.root_token, self.batch, self.N, self.V, self.W, self.B, mode,
                                       self.score_alpha, self.parent, self.depth, self.token, self.score,
                                       self.anc_mask, self.n_nodes, self.depth_entropy, self.ws_build,
@@ -191,4 +200,4 @@ class VerifyStep:
     LAUNCHES_PER_STEP_FIXED = 6      # tree_build 2, tree_accept 2, kv_compact 2
 
     def launches_per_step(self, attn_launches_per_layer):
-        return self.LAUNCHES_PER_STEP_FIXED + self.layers * attn_launches_per_layer
+        return self.LAUNCHES_PER_STEP_FIXED + (1 if self.draft_logits else 0) + self.layers * attn_launches_per_layer

@@ -72,6 +72,30 @@ def run_tree_build_scored(logp, root_token, N, W, B, score_mode, alpha, node_bud
                 n_nodes=n_nodes.cpu().numpy(), depth_entropy=ent.cpu().numpy())
 
 
+def run_tree_build_logits(logits, root_token, N, W, B, score_mode, alpha, node_budget=None):
+    """As run_tree_build_scored, through jet_tree_build_logits (raw logits in); also returns depth_lse [batch,N]."""
+    batch, _, V = logits.shape
+    d_logits = dev(logits)
+    d_root = dev(np.asarray(root_token, dtype=np.int32))
+    words = (B + 31) // 32
+    parent = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
+    depth = torch.full_like(parent, -7)
+    token = torch.full_like(parent, -7)
+    score = torch.full((batch, B), 123.0, dtype=torch.float32, device=DEV)
+    anc = torch.full((batch, B, words), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
+    n_nodes = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
+    ent = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
+    lse = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
+    ws = workspace(jet.jet_tree_build_logits_workspace_bytes(batch, N, V, W))
+    jet.jet_tree_build_logits(d_logits, d_root, batch, N, V, W, B, score_mode, alpha, parent, depth, token, score,
+                              anc, n_nodes, ent, lse, ws,
+                              node_budget=dev(np.asarray(node_budget, dtype=np.int32)) if node_budget is not None else None)
+    torch.cuda.synchronize()
+    return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
+                score=score.cpu().numpy(), anc_mask=anc.cpu().numpy().view(np.uint32),
+                n_nodes=n_nodes.cpu().numpy(), depth_entropy=ent.cpu().numpy(), depth_lse=lse.cpu().numpy())
+
+
 def run_tree_accept(logits, token, parent, depth, anc_mask, n_nodes, N):
     """logits [batch,B,V]; tree arrays [batch,B]; returns dict of numpy arrays."""
     batch, B, V = logits.shape
