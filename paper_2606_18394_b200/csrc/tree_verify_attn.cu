@@ -66,6 +66,12 @@ struct AttnParams {
   int tail;           // the tree's K/V rows sit in the cache behind the prefix (rows seq_len .. seq_len + n - 1)
   int batch, B, Hq, Hkv, G, words;
   int nsplit, n_mgroups, n_units;
+  // The code around the key loop runs once per launch, from a cold instruction cache: its cost is its
+  // instruction count.  What the host can work out arrives ready-made, and divisions by the two run-time
+  // divisors are multiplications by these reciprocals (udiv below).
+  int rows_per;       // ceil(128 / nsplit): rows of a query tile that one slice combines
+  int npt;            // 128 / G: nodes per query tile
+  uint32_t magic_S, magic_G;
   int via_global;     // key slices exchange their rows through the workspace instead of a cluster
   int* counters;      // via_global: [2][units * MT] arrival / departure counts, zero between calls
   uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D bf16 + log2-sum-exp (fp32) + pad]
@@ -75,8 +81,12 @@ struct AttnParams {
 #endif
 };
 
+// floor(x / d) for d <= 128 and x < 2^25, with magic = ceil(2^32 / d) (0 stands for d == 1).
+__host__ __device__ inline uint32_t udiv_magic(uint32_t d) { return d == 1 ? 0u : static_cast<uint32_t>(((1ull << 32) + d - 1) / d); }
+__device__ __forceinline__ uint32_t udiv(uint32_t x, uint32_t magic) { return magic ? __umulhi(x, magic) : x; }
+
 #ifdef JET_TRACE
-#define JET_TR(slot) do { if (p.trace) p.trace[blockIdx.x * 64 + (slot)] = clock64(); } while (0)
+#define JET_TR(slot) do { if (p.trace) p.trace[(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) * 64 + (slot)] = clock64(); } while (0)
 #else
 #define JET_TR(slot) do { } while (0)
 #endif
@@ -270,23 +280,18 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   uint32_t sBarLoop = sBar;        // base of the key loop's barrier set in use
   auto lbar = [&](int idx) { return sBarLoop + 8u * idx; };
   const int S = p.nsplit;                            // key slices = cluster size
-  const int split = blockIdx.x % S;                  // = rank in the cluster
-  const int rows_per = (kBM + S - 1) / S;            // rows of a query tile that one slice combines
-  const int own_lo = split * rows_per;
-  const int own_n = max(0, min(rows_per, kBM - own_lo));
-
-  // ---------------- work item: what the launch parameters alone decide
-  const int unit = blockIdx.x / S;
-  const int mgroup = unit % p.n_mgroups;
-  const int bg = unit / p.n_mgroups;
-  const int g = bg % p.Hkv;
-  const int b_rank = bg / p.Hkv;                 // position of the sequence in launch order
+  // ---------------- work item: what the launch parameters alone decide.  Grid = (query-tile groups x slices,
+  // KV heads, sequences); CTAs are dispatched x first, so a unit's slices are neighbours.
+  const int mgroup = static_cast<int>(udiv(blockIdx.x, p.magic_S));
+  const int split = static_cast<int>(blockIdx.x) - mgroup * S;    // = rank in the cluster
+  const int g = blockIdx.y;
+  const int b_rank = blockIdx.z;                 // position of the sequence in launch order
   constexpr bool sorted_launch = kSorted;
   const int G = p.G;
-  const int npt = kBM / G;                       // nodes per query tile
+  const int npt = p.npt;                         // nodes per query tile
   const int node_lo = mgroup * MT * npt;
   const int node_hi = min(p.B, node_lo + MT * npt);
-  const int n_mt = (node_hi - node_lo + npt - 1) / npt;     // query tiles of this CTA that hold nodes
+  const int n_mt = (MT == 2 && node_hi - node_lo > npt) ? 2 : 1;     // query tiles of this CTA that hold nodes
 
   // ---------------- set-up that touches no global memory (may overlap the previous kernel's tail)
   if (warp == 0) {
@@ -299,7 +304,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ptx::mbar_init(bar(lane), count);
       // slice merge: every slice sends this CTA its block of rows of query tile (lane - kRecv)
       if (S > 1 && lane >= Bars::kRecv && lane < Bars::kRecv + MT)
-        ptx::mbar_arrive_expect_tx(bar(lane), S * own_n * C::kRecvPitch);
+        ptx::mbar_arrive_expect_tx(bar(lane), S * max(0, min(p.rows_per, kBM - split * p.rows_per)) * C::kRecvPitch);
       ptx::fence_mbar_init();
     }
     if (lane == 31) {
@@ -390,8 +395,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int T_all = TP + TT;
   // key tiles of this slice; when they do not divide evenly the first slices take the extra tile, so that
   // the last slice, whose tree tile (masked) is the slowest kind, has the fewest
-  const int t_lo = static_cast<int>((static_cast<uint32_t>(T_all) * split + S - 1) / static_cast<uint32_t>(S));
-  const int t_hi = static_cast<int>((static_cast<uint32_t>(T_all) * (split + 1) + S - 1) / static_cast<uint32_t>(S));
+  int t_lo, t_hi;
+  if (T_all < (1 << 20)) {
+    t_lo = static_cast<int>(udiv(static_cast<uint32_t>(T_all) * split + S - 1, p.magic_S));
+    t_hi = static_cast<int>(udiv(static_cast<uint32_t>(T_all) * (split + 1) + S - 1, p.magic_S));
+  } else {
+    t_lo = static_cast<int>((static_cast<uint32_t>(T_all) * split + S - 1) / static_cast<uint32_t>(S));
+    t_hi = static_cast<int>((static_cast<uint32_t>(T_all) * (split + 1) + S - 1) / static_cast<uint32_t>(S));
+  }
   const int T = t_hi - t_lo;
   const bool has_work = node_lo < n && T > 0;    // otherwise: no live node here, or an empty key slice
   // A CTA without work never looks at its query rows, but they must have landed before the epilogue reuses
@@ -413,6 +424,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // part in every CTA-wide barrier and issue the bulk copies and the counter updates).
   auto epilogue = [&](auto sm_side) {
     constexpr bool kSm = decltype(sm_side)::value;
+    // The slice bookkeeping is worked out again here, from the CTA index read afresh, so that none of it
+    // occupies a register through the key loop (the softmax threads have none to spare).
+    uint32_t e_bx;
+    asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(e_bx));
+    const int e_mgroup = static_cast<int>(udiv(e_bx, p.magic_S));
+    const int split = static_cast<int>(e_bx) - e_mgroup * S;
+    const int rows_per = p.rows_per;                   // rows of a query tile that one slice combines
+    const int own_lo = split * rows_per;
+    const int own_n = max(0, min(rows_per, kBM - own_lo));
+    const int unit = (static_cast<int>(blockIdx.z) * p.Hkv + static_cast<int>(blockIdx.y)) * p.n_mgroups + e_mgroup;
     // =============================================================== epilogue
     // One round per query tile: its softmax threads stage their normalised rows (D bf16 + log2-sum-exp)
     // in shared memory.  With key slices every CTA then sends each owner slice its block of rows with
@@ -621,47 +642,32 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       for (int i = kSm ? tid - 128 : items; i < items; i += C::kThreads - 128) {
         const int rl = i / (D / 8), c8 = i - rl * (D / 8);
         const int R = mt * kBM + own_lo + rl;                  // row within the unit
-        const int v = node_lo + R / G, h = g * G + R % G;
+        const int vq = static_cast<int>(udiv(R, p.magic_G));
+        const int v = node_lo + vq, h = g * G + (R - vq * G);
         if (v >= p.B) continue;
         float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         float lse2 = -INFINITY;
         if (v < n) {
           const uint8_t* row0 = src_rows + rl * C::kRecvPitch;
-          // weights first (all loads independent) ...
-          float ls[kMaxSplit];
+          // (rolled loops: this code runs once per launch and costs what its instruction count costs)
           float mx = -INFINITY;
-#pragma unroll
-          for (int c = 0; c < kMaxSplit; ++c) {
-            ls[c] = c < S ? *reinterpret_cast<const float*>(row0 + c * src_stride + D * 2) : -INFINITY;
-            mx = fmaxf(mx, ls[c]);
-          }
+#pragma unroll 1
+          for (int c = 0; c < S; ++c) mx = fmaxf(mx, *reinterpret_cast<const float*>(row0 + c * src_stride + D * 2));
           float wsum = 0.0f;
           if (mx > -INFINITY) {
+#pragma unroll 1
+            for (int c = 0; c < S; ++c) {
+              const uint8_t* src = row0 + c * src_stride;
+              const float lc = *reinterpret_cast<const float*>(src + D * 2);
+              const float w = lc > -INFINITY ? exp2f(lc - mx) : 0.0f;        // absent slices get weight 0
+              wsum += w;
+              // a slice with weight 0 is not read (it may hold junk)
+              const uint4 x = w > 0.0f ? *reinterpret_cast<const uint4*>(src + c8 * 16) : make_uint4(0u, 0u, 0u, 0u);
+              const uint32_t v4[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-            for (int c = 0; c < kMaxSplit; ++c) {
-              ls[c] = ls[c] > -INFINITY ? exp2f(ls[c] - mx) : 0.0f;        // absent slices get weight 0
-              wsum += ls[c];
-            }
-            // ... then the rows, four slices at a time; a slice with weight 0 is not read (it may hold junk)
-#pragma unroll
-            for (int c0 = 0; c0 < kMaxSplit; c0 += 4) {
-              if (c0 < S) {
-                uint4 x[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const uint8_t* src = row0 + (c0 + k) * src_stride;
-                  x[k] = ls[c0 + k] > 0.0f ? *reinterpret_cast<const uint4*>(src + c8 * 16) : make_uint4(0u, 0u, 0u, 0u);
-                }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const float w = ls[c0 + k];
-                  const uint32_t v4[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
-                    acc[2 * q] += w * __uint_as_float(v4[q] << 16);
-                    acc[2 * q + 1] += w * __uint_as_float(v4[q] & 0xFFFF0000u);
-                  }
-                }
+              for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
+                acc[2 * q] += w * __uint_as_float(v4[q] << 16);
+                acc[2 * q + 1] += w * __uint_as_float(v4[q] & 0xFFFF0000u);
               }
             }
             const float inv = 1.0f / wsum;
@@ -1048,7 +1054,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int stream = MT == 1 ? wg : 0;                    // its share of the key tiles (tl % kStreams)
     const int r = (tid - 128) & 127;                        // row of the query tile = TMEM lane
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    const int v = node_lo + mt * npt + r / G;
+    const int v = node_lo + mt * npt + static_cast<int>(udiv(r, p.magic_G));
     const bool row_live = v < n;
     const uint32_t* mask_row = p.anc_mask + (static_cast<size_t>(b) * p.B + (row_live ? v : 0)) * p.words;
     const float sl2 = p.scale_log2;
@@ -1448,7 +1454,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     JET_TR(13);
     if (*abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
 #ifdef JET_TRACE
-    if (*abort_flag && p.trace) p.trace[blockIdx.x * 64 + 31] = *abort_flag;
+    if (*abort_flag && p.trace) p.trace[(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) * 64 + 31] = *abort_flag;
 #endif
   }
 }
@@ -1627,7 +1633,7 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   using C = Cfg<D, MT>;
   if (!configure_kernel<D, MT>()) return JET_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(pl.units * pl.nsplit);
+  cfg.gridDim = dim3(pl.n_mgroups * pl.nsplit, p.Hkv, p.batch);
   cfg.blockDim = dim3(C::kThreads);
   cfg.dynamicSmemBytes = C::kSmemBytes;
   cfg.stream = st;
@@ -1681,7 +1687,9 @@ extern "C" JET_API int jet_debug_max_clusters(int cluster) {
 
 extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                                        int max_seq_len) {
-  if (batch < 1 || B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0 || (D != 64 && D != 128)) return 0;
+  if (batch < 1 || batch > 65535 || B < 1 || Hq < 1 || Hkv < 1 || Hkv > 65535 || Hq % Hkv != 0 || max_seq_len < 0 ||
+      (D != 64 && D != 128))
+    return 0;
   return jet::workspace_need(jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len), D);
 }
 
@@ -1698,7 +1706,8 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
                      size_t workspace_bytes, void* stream) {
   if (!q || !seq_len || !anc_mask || !n_nodes || !out) return JET_ERR_INVALID_ARG;
   if (tail ? (!k_cache || !v_cache || max_seq_len < 1) : (!tree_k || !tree_v)) return JET_ERR_INVALID_ARG;
-  if (batch < 1 || B < 1 || B > JET_MAX_NODES || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || max_seq_len < 0)
+  if (batch < 1 || batch > 65535 || B < 1 || B > JET_MAX_NODES || Hq < 1 || Hkv < 1 || Hkv > 65535 || Hq % Hkv != 0 ||
+      max_seq_len < 0)        // (sequences and KV heads are grid dimensions)
     return JET_ERR_INVALID_ARG;
   if (max_seq_len > 0 && (!k_cache || !v_cache)) return JET_ERR_INVALID_ARG;
   const int G = Hq / Hkv;
@@ -1772,6 +1781,10 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
   p.nsplit = pl.nsplit;
   p.n_mgroups = pl.n_mgroups;
   p.n_units = pl.units;
+  p.rows_per = (kBM + pl.nsplit - 1) / pl.nsplit;
+  p.npt = kBM / G;
+  p.magic_S = udiv_magic(static_cast<uint32_t>(pl.nsplit));
+  p.magic_G = udiv_magic(static_cast<uint32_t>(G));
   p.via_global = pl.via_global;
   p.counters = static_cast<int*>(workspace);
   p.partials = static_cast<uint8_t*>(workspace) + kCounterBytes;
