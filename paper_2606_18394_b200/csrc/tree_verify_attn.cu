@@ -408,6 +408,23 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // A CTA without work never looks at its query rows, but they must have landed before the epilogue reuses
   // their memory (and before the CTA exits).
   if (!has_work && warp == 2) bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
+  // The first K tiles are requested here, straight after the lengths are known: the producer's own loop
+  // lies some two thousand cycles of cold code further on (register re-split, set-up of the ring), and
+  // the first Q K^T waits for exactly these tiles.  They are the first items of the ring in every form of
+  // the key loop (ring order starts K_0 .. K_ahead); the producers start behind them.  A paged tile needs
+  // its page ids first and is left to the producers.
+  const int n_early = (has_work && !p.paged) ? (MT == 1 ? min(2, T) : 1) : 0;
+  if (warp == 0 && lane == 0) {
+    for (int i = 0; i < n_early; ++i) {
+      const int t = t_lo + i;
+      const bool prefix = t < TP;
+      const CUtensorMap* map = prefix ? &tm_k : &tm_tk;
+      const int row0 = prefix ? t * kBN : (t - TP) * kBN;
+      const uint32_t full = bar(Bars::kKvFull + i);
+      ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+      for (int h = 0; h < kHalves; ++h) ptx::tma_load_4d(sKV + i * C::kStageBytes + h * kHalfBytes, map, full, h * 64, g, row0, b);
+    }
+  }
   if (tid == 0) JET_TR(1);
 
   // per-row state of the softmax threads, live until the epilogue
@@ -732,18 +749,19 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // K runs `ahead` key tiles in front of V in the ring (0: K_t, V_t alternate).
     // only_c (a compile-time constant: a run-time role cost 4 % on long contiguous prefixes): -1 = this warp
     // requests every tile, 0 = the K tiles only, 1 = the V tiles only (two producer warps).
-    auto produce = [&](const int ahead, auto only_c) {
+    // first: ring items already requested (K tiles 0 .. first - 1, see n_early).
+    auto produce = [&](const int ahead, auto only_c, const int first) {
       constexpr int only = decltype(only_c)::value;
       if (tid == 0) JET_TR(27);
       bool ok = true;
-      int issued = 0;
+      int issued = first;
       // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
       // fetched while the current tile's copies are issued, so the table look-up is off the critical path
       auto tile_page = [&](int t) -> int {
         if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= Lc) return 0;
         return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
       };
-      int kt = 0, vt = 0;                       // next K tile, next V tile
+      int kt = first, vt = 0;                   // next K tile, next V tile (first > 0 only without pages)
       int pk_cur = tile_page(t_lo), pk_next = tile_page(t_lo + 1);
       int pv_cur = pk_cur, pv_next = pk_next;
       if (tid == 0) JET_TR(28);
@@ -818,10 +836,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (has_work) {
         if (warp == 0) {
           // a paged tile is 16 small copies: two warps request them
-          if (p.paged) produce(kAhead, std::integral_constant<int, 0>{});
-          else produce(kAhead, std::integral_constant<int, -1>{});
+          if (p.paged) produce(kAhead, std::integral_constant<int, 0>{}, 0);
+          else produce(kAhead, std::integral_constant<int, -1>{}, n_early);
         } else if (warp == 2) {
-          if (p.paged) produce(kAhead, std::integral_constant<int, 1>{});
+          if (p.paged) produce(kAhead, std::integral_constant<int, 1>{}, 0);
         } else if (warp == 1) {
           // =========================================================== tcgen05 issuers, shared-accumulator form
           // Key tile tl belongs to warpgroup tl & 1 (score buffer and P buffer of that warpgroup).  Warp 1
@@ -910,9 +928,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       classic = false;
       if (has_work) {
         if (warp == 0) {
-          produce(0, std::integral_constant<int, 0>{});                     // K tiles
+          produce(0, std::integral_constant<int, 0>{}, n_early);            // K tiles
         } else if (warp == 2) {
-          produce(0, std::integral_constant<int, 1>{});                     // V tiles (a paged tile is 16 small copies: two warps request them)
+          produce(0, std::integral_constant<int, 1>{}, n_early);            // V tiles (a paged tile is 16 small copies: two warps request them)
         } else if (warp == 1) {
           bool ok = bounded_wait(bar(Bars::kQFull), 0, abort_flag, 4);
           int prev_mt = -1, prev_tl = 0;
@@ -973,7 +991,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
     if (!C::kTurns && classic && has_work) {
       if (warp == 0) {
-        produce(0, std::integral_constant<int, -1>{});
+        produce(0, std::integral_constant<int, -1>{}, 0);
       } else if (warp == 1) {
         // =========================================================== tcgen05 issuer, classic form
         // A stream is a chain  S = Q K^T -> softmax -> O += P V -> next S  on its own score buffer (which the P
