@@ -342,7 +342,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
           for (int c2 = 0; c2 < kMaxSorted / 32; ++c2) {
             if (c2 * 32 < p.batch) {
-              for (int j = 0; j < 32; ++j) {
+#pragma unroll 1
+              for (int j = 0; j < 32; ++j) {       // (rolled: this runs once per launch, from cold code)
                 const int other = __shfl_sync(0xffffffffu, len[c2], j), ob = c2 * 32 + j;
                 before += (ob < p.batch && (other > mine || (other == mine && ob < me))) ? 1 : 0;
               }
