@@ -202,7 +202,10 @@ JET_API jet_status jet_tree_build_logits(const float* logits, int64_t logits_bat
  *   device_status  i32[1], may be NULL: set to JET_ERR_TIMEOUT if a bounded
  *                wait inside the kernel expired (outputs are then undefined).
  * Limits: D in {64,128}; Hq % Hkv == 0 and Hq/Hkv a power of two <= 16;
- * page_size == 16 when paged; all base pointers 16-byte aligned.
+ * page_size == 16 when paged; all base pointers 16-byte aligned; batch and Hkv
+ * at most 65535 (they are grid dimensions).  max_seq_len is a bound, but a call
+ * with one sequence whose seq_len equals it exactly starts a little faster (the
+ * first key tiles are prefetched on that guess).
  * Workspace: unlike the other calls, the first 4096 bytes of this workspace hold
  * counters that must be ZERO when the call starts.  Zero them once after
  * allocating the workspace; every call that completes leaves them zero again.
