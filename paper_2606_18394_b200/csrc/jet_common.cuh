@@ -60,13 +60,14 @@ __device__ __forceinline__ float key_value(unsigned long long k) {
   return __uint_as_float((c & 0x80000000u) ? (c & 0x7FFFFFFFu) : ~c);
 }
 
+// Maximum of the warp's 64-bit keys with two 32-bit warp reductions (redux.sync): the largest high word, then
+// the largest low word among the lanes that hold it.  Needs no key with a zero low word other than the empty
+// key 0 (the keys made here never have one: the low word holds an inverted index).
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    unsigned long long other = __shfl_xor_sync(0xffffffffu, k, o);
-    k = other > k ? other : k;
-  }
-  return k;
+  const uint32_t hi = static_cast<uint32_t>(k >> 32), lo = static_cast<uint32_t>(k);
+  const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+  const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+  return (static_cast<unsigned long long>(mh) << 32) | ml;
 }
 
 }  // namespace jet
