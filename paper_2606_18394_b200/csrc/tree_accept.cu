@@ -46,6 +46,30 @@ argmax_partial_kernel(const float* __restrict__ logits, int64_t row_stride, int 
       if (x[i].z > best) { best = x[i].z; best_idx = idx + 2; }
       if (x[i].w > best) { best = x[i].w; best_idx = idx + 3; }
     }
+  } else if (vec_ok) {
+    // the row's last, partial slice: still 16-byte loads wherever four elements are in range
+    const float4* p4 = reinterpret_cast<const float4*>(p + base);
+    float4 x[kArgElems / 4];
+#pragma unroll
+    for (int i = 0; i < kArgElems / 4; ++i) {
+      const int idx = base + (i * kArgThreads + tid) * 4;
+      if (idx + 3 < V) {
+        x[i] = __ldcs(p4 + i * kArgThreads + tid);
+      } else {
+        x[i].x = idx < V ? __ldcs(p + idx) : -INFINITY;
+        x[i].y = idx + 1 < V ? __ldcs(p + idx + 1) : -INFINITY;
+        x[i].z = idx + 2 < V ? __ldcs(p + idx + 2) : -INFINITY;
+        x[i].w = -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kArgElems / 4; ++i) {
+      const int idx = base + (i * kArgThreads + tid) * 4;     // ascending in i
+      if (idx < V && (best_idx == 0xFFFFFFFFu || x[i].x > best)) { best = x[i].x; best_idx = idx; }
+      if (idx + 1 < V && x[i].y > best) { best = x[i].y; best_idx = idx + 1; }
+      if (idx + 2 < V && x[i].z > best) { best = x[i].z; best_idx = idx + 2; }
+      if (idx + 3 < V && x[i].w > best) { best = x[i].w; best_idx = idx + 3; }
+    }
   } else {
 #pragma unroll 4
     for (int i = 0; i < kArgElems; ++i) {
