@@ -92,9 +92,9 @@ class VerifyStep:
 
     @property
     def attn_max_len(self):
-        if self.paged:
-            return self.max_seq_len + (self.B if self.tail else 0)
-        return self.rows_per_seq
+        # the bound on the cached keys that the attention call is given: the caller's max_seq_len itself (not
+        # the rows a sequence owns, which include room for the commit) -- a call whose bound is exact starts faster
+        return self.max_seq_len + (self.B if self.tail else 0)
 
     def place_tree(self):
         """Tail layout: writes tree_k / tree_v to the cache rows seq_len0[b] + v (what the model's K/V
