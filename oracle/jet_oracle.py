@@ -57,7 +57,9 @@ the pop order against priorities recomputed from the paths; whether the entropy
 term is that of the node's own depth or a sum along the branch is a reading
 with no counterpart to check against: parity unpinned for that reading only.  ``log_softmax_ref`` is pinned against
 scipy's log_softmax, closed forms (uniform, two-point), rows summing to one and
-shift invariance; ``tree_build_logits_ref`` by the invariance of the tree under
+shift invariance; the two helpers ``bf16_bits_to_f64`` (fixed bit patterns whose values the bfloat16
+format itself gives) and ``gather_paged_prefix`` (a cache whose rows hold their own page and offset)
+have pins of their own; ``tree_build_logits_ref`` by the invariance of the tree under
 a per-row shift of the logits and by agreement with ``tree_build_ref`` on
 log-probabilities that scipy computed.
 """

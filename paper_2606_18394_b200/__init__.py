@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     JET_ERR_UNSUPPORTED,
     JET_ERR_WORKSPACE,
     JET_OK,
+    JET_STATIC_ACCEPT_SCRATCH_BYTES,
     JetError,
     exported_symbols,
     jet_kv_compact,

@@ -20,6 +20,7 @@ JET_ERR_UNSUPPORTED = -2
 JET_ERR_WORKSPACE = -3
 JET_ERR_CUDA = -4
 JET_ERR_TIMEOUT = -5
+JET_STATIC_ACCEPT_SCRATCH_BYTES = 1 << 20     # jet.h: built-in scratch of jet_tree_accept_static
 
 _c = ctypes
 _vp, _i, _i64, _f, _sz = _c.c_void_p, _c.c_int, _c.c_int64, _c.c_float, _c.c_size_t

@@ -9,6 +9,7 @@
 //                          builds the match bit-set, tests every node's ancestor mask
 //                          against it, picks the deepest accepted node and writes the
 //                          path and the output tokens.
+#include <atomic>
 #include "jet_common.cuh"
 
 namespace jet {
@@ -223,16 +224,21 @@ extern "C" jet_status jet_tree_accept_static(const float* logits, int64_t logits
   if (need > JET_STATIC_ACCEPT_SCRATCH_BYTES) return JET_ERR_WORKSPACE;   // beyond the built-in scratch
 
   // Device address of the built-in array, looked up once per device with that device current.
-  // (In host code the array's name is only a handle; kernels must be given this address.)
-  static unsigned long long* scratch_of_device[kMaxDevices] = {};
+  // (In host code the array's name is only a handle; kernels must be given this address.)  The cache is
+  // one atomic pointer per device: host threads that make their first call together each look the address
+  // up and store the same value.
+  static std::atomic<unsigned long long*> scratch_of_device[kMaxDevices];
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return JET_ERR_CUDA;
-  unsigned long long* scratch = scratch_of_device[dev];
+  unsigned long long* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
   if (!scratch) {
     void* addr = nullptr;
-    if (cudaGetSymbolAddress(&addr, g_accept_scratch) != cudaSuccess || !addr) return JET_ERR_CUDA;
+    if (cudaGetSymbolAddress(&addr, g_accept_scratch) != cudaSuccess || !addr) {
+      cudaGetLastError();
+      return JET_ERR_CUDA;
+    }
     scratch = static_cast<unsigned long long*>(addr);
-    scratch_of_device[dev] = scratch;
+    scratch_of_device[dev].store(scratch, std::memory_order_release);
   }
   // Nothing in the scratch has to start at zero: every entry that accept_path_kernel reads was
   // written by argmax_partial_kernel of the same call.

@@ -29,21 +29,57 @@ def workspace(nbytes):
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=DEV)
 
 
+# ---------------------------------------------------------------------------------------------------
+# Canary margins.  Every output tensor of a call is carved out of a larger buffer whose bytes in front
+# of and behind the tensor hold a sentinel; after the call the margins must be untouched.  (An
+# out-of-bounds store would otherwise land in the allocator's slack unseen.)
+# ---------------------------------------------------------------------------------------------------
+_MARGIN = 512            # bytes on either side (keeps the 256-byte alignment of the tensor itself)
+_SENTINEL = 0xA5
+_guards = []
+
+
+def guarded_full(shape, fill, dtype):
+    """A tensor like torch.full(shape, fill, dtype) on the device, with sentinel margins around it."""
+    shape = tuple(int(x) for x in (shape if isinstance(shape, (tuple, list)) else (shape,)))
+    item = torch.empty((), dtype=dtype).element_size()
+    nbytes = int(np.prod(shape, dtype=np.int64)) * item
+    padded = (nbytes + 255) // 256 * 256
+    raw = torch.full((_MARGIN + padded + _MARGIN,), _SENTINEL, dtype=torch.uint8, device=DEV)
+    body = raw[_MARGIN:_MARGIN + nbytes].view(dtype).view(shape)
+    body.fill_(fill)
+    _guards.append((raw, nbytes))
+    return body
+
+
+def check_guards():
+    """Asserts that no call wrote outside its output tensors; forgets the registered buffers."""
+    torch.cuda.synchronize()
+    try:
+        for raw, nbytes in _guards:
+            front = raw[:_MARGIN]
+            back = raw[_MARGIN + nbytes:]
+            assert bool((front == _SENTINEL).all()), "bytes in front of an output tensor were overwritten"
+            assert bool((back == _SENTINEL).all()), "bytes behind an output tensor were overwritten"
+    finally:
+        _guards.clear()
+
+
 def run_tree_build(logp, root_token, N, W, B, with_score=True):
     """logp [batch,N,V] fp32 numpy; returns dict of numpy arrays."""
     batch, _, V = logp.shape
     d_logp = dev(logp)
     d_root = dev(np.asarray(root_token, dtype=np.int32))
     words = (B + 31) // 32
-    parent = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
-    depth = torch.full_like(parent, -7)
-    token = torch.full_like(parent, -7)
-    score = torch.full((batch, B), 123.0, dtype=torch.float32, device=DEV) if with_score else None
-    anc = torch.full((batch, B, words), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
-    n_nodes = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
+    parent = guarded_full((batch, B), -7, torch.int32)
+    depth = guarded_full((batch, B), -7, torch.int32)
+    token = guarded_full((batch, B), -7, torch.int32)
+    score = guarded_full((batch, B), 123.0, torch.float32) if with_score else None
+    anc = guarded_full((batch, B, words), 0x5A5A5A5A, torch.int32)
+    n_nodes = guarded_full((batch,), -7, torch.int32)
     ws = workspace(jet.jet_tree_build_workspace_bytes(batch, N, V, W))
     jet.jet_tree_build(d_logp, d_root, batch, N, V, W, B, parent, depth, token, score, anc, n_nodes, ws)
-    torch.cuda.synchronize()
+    check_guards()
     return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
                 score=score.cpu().numpy() if with_score else None,
                 anc_mask=anc.cpu().numpy().view(np.uint32), n_nodes=n_nodes.cpu().numpy())
@@ -55,18 +91,18 @@ def run_tree_build_scored(logp, root_token, N, W, B, score_mode, alpha, node_bud
     d_logp = dev(logp)
     d_root = dev(np.asarray(root_token, dtype=np.int32))
     words = (B + 31) // 32
-    parent = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
-    depth = torch.full_like(parent, -7)
-    token = torch.full_like(parent, -7)
-    score = torch.full((batch, B), 123.0, dtype=torch.float32, device=DEV)
-    anc = torch.full((batch, B, words), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
-    n_nodes = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
-    ent = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
+    parent = guarded_full((batch, B), -7, torch.int32)
+    depth = guarded_full((batch, B), -7, torch.int32)
+    token = guarded_full((batch, B), -7, torch.int32)
+    score = guarded_full((batch, B), 123.0, torch.float32)
+    anc = guarded_full((batch, B, words), 0x5A5A5A5A, torch.int32)
+    n_nodes = guarded_full((batch,), -7, torch.int32)
+    ent = guarded_full((batch, N), -1.0, torch.float32)
     ws = workspace(jet.jet_tree_build_scored_workspace_bytes(batch, N, V, W))
     jet.jet_tree_build_scored(d_logp, d_root, batch, N, V, W, B, score_mode, alpha, parent, depth, token, score,
                               anc, n_nodes, ent, ws,
                               node_budget=dev(np.asarray(node_budget, dtype=np.int32)) if node_budget is not None else None)
-    torch.cuda.synchronize()
+    check_guards()
     return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
                 score=score.cpu().numpy(), anc_mask=anc.cpu().numpy().view(np.uint32),
                 n_nodes=n_nodes.cpu().numpy(), depth_entropy=ent.cpu().numpy())
@@ -78,19 +114,19 @@ def run_tree_build_logits(logits, root_token, N, W, B, score_mode, alpha, node_b
     d_logits = dev(logits)
     d_root = dev(np.asarray(root_token, dtype=np.int32))
     words = (B + 31) // 32
-    parent = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
-    depth = torch.full_like(parent, -7)
-    token = torch.full_like(parent, -7)
-    score = torch.full((batch, B), 123.0, dtype=torch.float32, device=DEV)
-    anc = torch.full((batch, B, words), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
-    n_nodes = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
-    ent = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
-    lse = torch.full((batch, N), -1.0, dtype=torch.float32, device=DEV)
+    parent = guarded_full((batch, B), -7, torch.int32)
+    depth = guarded_full((batch, B), -7, torch.int32)
+    token = guarded_full((batch, B), -7, torch.int32)
+    score = guarded_full((batch, B), 123.0, torch.float32)
+    anc = guarded_full((batch, B, words), 0x5A5A5A5A, torch.int32)
+    n_nodes = guarded_full((batch,), -7, torch.int32)
+    ent = guarded_full((batch, N), -1.0, torch.float32)
+    lse = guarded_full((batch, N), -1.0, torch.float32)
     ws = workspace(jet.jet_tree_build_logits_workspace_bytes(batch, N, V, W))
     jet.jet_tree_build_logits(d_logits, d_root, batch, N, V, W, B, score_mode, alpha, parent, depth, token, score,
                               anc, n_nodes, ent, lse, ws,
                               node_budget=dev(np.asarray(node_budget, dtype=np.int32)) if node_budget is not None else None)
-    torch.cuda.synchronize()
+    check_guards()
     return dict(parent=parent.cpu().numpy(), depth=depth.cpu().numpy(), token=token.cpu().numpy(),
                 score=score.cpu().numpy(), anc_mask=anc.cpu().numpy().view(np.uint32),
                 n_nodes=n_nodes.cpu().numpy(), depth_entropy=ent.cpu().numpy(), depth_lse=lse.cpu().numpy())
@@ -100,15 +136,15 @@ def run_tree_accept(logits, token, parent, depth, anc_mask, n_nodes, N):
     """logits [batch,B,V]; tree arrays [batch,B]; returns dict of numpy arrays."""
     batch, B, V = logits.shape
     d_logits = dev(logits)
-    tgt = torch.full((batch, B), -7, dtype=torch.int32, device=DEV)
-    acc = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
-    path = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
-    toks = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
+    tgt = guarded_full((batch, B), -7, torch.int32)
+    acc = guarded_full((batch,), -7, torch.int32)
+    path = guarded_full((batch, N + 1), -7, torch.int32)
+    toks = guarded_full((batch, N + 1), -7, torch.int32)
     ws = workspace(jet.jet_tree_accept_workspace_bytes(batch, B, V))
     jet.jet_tree_accept(d_logits, V, dev(token.astype(np.int32)), dev(parent.astype(np.int32)),
                         dev(depth.astype(np.int32)), dev(anc_mask.view(np.int32)),
                         dev(np.asarray(n_nodes, dtype=np.int32)), batch, B, V, N, tgt, acc, path, toks, ws)
-    torch.cuda.synchronize()
+    check_guards()
     return dict(tgt=tgt.cpu().numpy(), accept_len=acc.cpu().numpy(), path=path.cpu().numpy(),
                 out_tokens=toks.cpu().numpy())
 
@@ -117,10 +153,10 @@ def run_tree_accept_sample(logits, temperature, draft_logp, token, parent, depth
                            u_sample):
     """logits [batch,B,V], draft_logp [batch,N,V], u_accept [batch,B], u_sample [batch]; returns numpy arrays."""
     batch, B, V = logits.shape
-    alpha = torch.full((batch, B), -7.0, dtype=torch.float32, device=DEV)
-    acc = torch.full((batch,), -7, dtype=torch.int32, device=DEV)
-    path = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
-    toks = torch.full((batch, N + 1), -7, dtype=torch.int32, device=DEV)
+    alpha = guarded_full((batch, B), -7.0, torch.float32)
+    acc = guarded_full((batch,), -7, torch.int32)
+    path = guarded_full((batch, N + 1), -7, torch.int32)
+    toks = guarded_full((batch, N + 1), -7, torch.int32)
     ws = workspace(jet.jet_tree_accept_sample_workspace_bytes(batch, B, V))
     jet.jet_tree_accept_sample(dev(logits), V, float(temperature), dev(draft_logp.astype(np.float32)), N * V, V,
                                dev(token.astype(np.int32)), dev(parent.astype(np.int32)),
@@ -128,7 +164,7 @@ def run_tree_accept_sample(logits, temperature, draft_logp, token, parent, depth
                                dev(np.asarray(n_nodes, dtype=np.int32)), dev(u_accept.astype(np.float32)),
                                dev(np.asarray(u_sample, dtype=np.float32)), batch, B, V, N, alpha, acc, path,
                                toks, ws)
-    torch.cuda.synchronize()
+    check_guards()
     return dict(alpha=alpha.cpu().numpy(), accept_len=acc.cpu().numpy(), path=path.cpu().numpy(),
                 out_tokens=toks.cpu().numpy())
 
@@ -152,7 +188,7 @@ def run_kv_compact(tree_k, tree_v, k_cache, v_cache, page_table, path, accept_le
     jet.jet_kv_compact(dev(tree_k.view(np.int16)), dev(tree_v.view(np.int16)), dk, dv, layer_stride,
                        batch_stride, pt, max_pages, page_size, dev(path.astype(np.int32)),
                        dev(np.asarray(accept_len, dtype=np.int32)), d_seq, layers, batch, B, Hkv, D, N)
-    torch.cuda.synchronize()
+    check_guards()
     return (dk.cpu().numpy().view(np.uint16), dv.cpu().numpy().view(np.uint16), d_seq.cpu().numpy())
 
 
@@ -177,15 +213,15 @@ def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_
         pt = dev(page_table.astype(np.int32))
         max_pages, page_size, num_pages = page_table.shape[1], k_cache.shape[1], k_cache.shape[0]
         kv_batch_stride = 0
-    out = torch.full((batch, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
-    lse = torch.full((batch, Hq, B), float("nan"), dtype=torch.float32, device=DEV) if want_lse else None
-    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = guarded_full((batch, B, Hq, D), float("nan"), torch.bfloat16)
+    lse = guarded_full((batch, Hq, B), float("nan"), torch.float32) if want_lse else None
+    status = guarded_full((1,), 0, torch.int32)
     ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
     ws.zero_()          # the attention workspace starts with counters that must be zero
     jet.jet_tree_verify_attn(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
                              d_tk, d_tv, dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
                              batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
-    torch.cuda.synchronize()
+    check_guards()
     return (bf16_to_f64(out), lse.cpu().numpy().astype(np.float64) if want_lse else None,
             int(status.cpu()[0]))
 
@@ -202,15 +238,15 @@ def run_tree_attn_tail(q, k_cache, v_cache, page_table, seq_len, anc_mask, n_nod
         pt = dev(page_table.astype(np.int32))
         max_pages, page_size, num_pages = page_table.shape[1], k_cache.shape[1], k_cache.shape[0]
         kv_batch_stride = 0
-    out = torch.full((batch, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
-    lse = torch.full((batch, Hq, B), float("nan"), dtype=torch.float32, device=DEV)
-    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = guarded_full((batch, B, Hq, D), float("nan"), torch.bfloat16)
+    lse = guarded_full((batch, Hq, B), float("nan"), torch.float32)
+    status = guarded_full((1,), 0, torch.int32)
     ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
     ws.zero_()
     jet.jet_tree_verify_attn_tail(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
                                   dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
                                   batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
-    torch.cuda.synchronize()
+    check_guards()
     return bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), int(status.cpu()[0])
 
 
@@ -233,5 +269,5 @@ def run_kv_compact_tail(k_cache, v_cache, page_table, path, accept_len, seq_len,
     jet.jet_kv_compact_tail(d_k, d_v, layer_stride, kv_batch_stride, pt, max_pages, page_size,
                             dev(path.astype(np.int32)), dev(np.asarray(accept_len, dtype=np.int32)), d_seq,
                             layers, batch, B, Hkv, D, N)
-    torch.cuda.synchronize()
+    check_guards()
     return (d_k.cpu().numpy().view(np.uint16), d_v.cpu().numpy().view(np.uint16), d_seq.cpu().numpy())

@@ -89,6 +89,31 @@ def test_argmax_ties_take_lowest_index_across_slices():
     assert got["accept_len"][0] == 3
 
 
+def test_subnormal_logits_are_compared_by_value():
+    """The arg-max is an IEEE fp32 compare without flush-to-zero: a subnormal beats +-0 and a more negative
+    subnormal loses to -0.0; -0.0 == +0.0 still tie to the lowest index."""
+    tiny = np.float32(1e-40)
+    assert 0 < tiny < np.finfo(np.float32).tiny
+    B, V, N = 6, 20000, 5
+    parent, depth, token = chain_tree(B)
+    logits = np.zeros((1, B, V), dtype=np.float32)
+    logits[0, 0, 15000] = tiny                                  # subnormal > 0: wins over index 0
+    logits[0, 1, :] = -tiny
+    logits[0, 1, 9000] = -0.0                                   # -0.0 > -1e-40
+    logits[0, 2, :] = -0.0
+    logits[0, 2, 8200] = 0.0                                    # +0.0 == -0.0: index 0 wins
+    logits[0, 3, :] = -2 * tiny
+    logits[0, 3, [17000, 300]] = -tiny                          # equal subnormal maxima in two slices -> 300
+    logits[0, 4, :] = -np.inf
+    logits[0, 4, 19999] = -np.finfo(np.float32).max
+    logits[0, 5, [1, 2]] = [tiny, 2 * tiny]
+    token = np.array([1, 15000, 9000, 0, 300, 19999], dtype=np.int32)
+    anc = anc_from_parent(parent, B, B)
+    got = _compare(logits, token[None], parent[None], depth[None], anc[None], np.array([B]), N)
+    assert got["tgt"][0].tolist() == [15000, 9000, 0, 300, 19999, 2]
+    assert got["accept_len"][0] == 5
+
+
 def test_star_and_duplicate_sibling_tokens():
     B, V, N = 9, 50, 2
     parent, depth, token = star_tree(B)

@@ -69,6 +69,29 @@ def test_ties_signed_zero_and_minus_inf():
     _compare(flat, [0], 2, 4, 19)
 
 
+def test_subnormal_log_probabilities_are_not_flushed():
+    """IEEE fp32 without flush-to-zero: a subnormal increment under a zero parent score stays subnormal in
+    `score`, and subnormals rank among each other and against +-0 by value."""
+    tiny = np.float32(1e-40)                                  # subnormal (smallest normal is 1.18e-38)
+    assert tiny > 0 and tiny < np.finfo(np.float32).tiny
+    N, V, W, B = 3, 9000, 4, 40
+    logp = np.full((1, N, V), -3.0, dtype=np.float32)
+    # depth 0: four candidates -1e-40 < -0.0 == +0.0 ... ranked by value, ties to the lowest id
+    logp[0, 0, [8500, 40, 4100, 7]] = [-tiny, -0.0, 0.0, -2 * tiny]
+    # depth 1: subnormals in different 4096-entry slices, and a value one ulp below the largest
+    logp[0, 1, [5, 4097, 8999]] = [-3 * tiny, -tiny, -2 * tiny]
+    logp[0, 2, [100, 200]] = [-tiny, -tiny]                   # equal subnormals: lowest id first
+    ref = tree_build_ref(logp[0], 0, N, W, B)
+    assert ref["token"][1:5].tolist() == [40, 4100, 8500, 7]
+    assert (np.abs(ref["score"][1:ref["n_nodes"]]) < np.finfo(np.float32).tiny).any()   # the oracle keeps subnormals
+    _compare(logp, [0], N, W, B)
+    # a subnormal against a normal neighbour: the sum must round as IEEE does, not from a flushed operand
+    logp2 = np.full((1, 2, 64), -np.inf, dtype=np.float32)
+    logp2[0, 0, :3] = [-np.finfo(np.float32).tiny, -tiny, -5.0]
+    logp2[0, 1, :3] = [-tiny, -np.finfo(np.float32).tiny * np.float32(0.5), -1.0]
+    _compare(logp2, [1], 2, 3, 13)
+
+
 def test_unaligned_rows_take_the_scalar_path():
     import torch
     import jet_harness as H

@@ -192,3 +192,40 @@ def test_parent_consistent_relabelling_permutes_rows():
     b, _ = tree_attn_ref(x["q"][inv], x["k_prefix"], x["v_prefix"], x["tree_k"][inv], x["tree_v"][inv],
                          anc_from_parent(parent2, B, B), B, 0.4)
     np.testing.assert_allclose(b[new_of_old], a, rtol=1e-12, atol=1e-14)
+
+
+def test_bf16_widening_of_fixed_bit_patterns():
+    """bf16_bits_to_f64 against values the bfloat16 format itself fixes (1 sign, 8 exponent, 7 mantissa bits):
+    a wrong shift, a dropped sign or a mantissa taken as the exponent fails one of these."""
+    bits = np.array([0x3F80, 0xC000, 0x0000, 0x8000, 0x7F80, 0xFF80, 0x3FC0, 0x4049, 0x0001, 0x0080, 0x7F7F, 0x3B80],
+                    dtype=np.uint16)
+    want = [1.0, -2.0, 0.0, -0.0, np.inf, -np.inf, 1.5, 3.140625, 2.0 ** -133, 2.0 ** -126,
+            (2.0 - 2.0 ** -7) * 2.0 ** 127, 2.0 ** -8]
+    got = bf16_bits_to_f64(bits)
+    assert got.dtype == np.float64
+    np.testing.assert_array_equal(got, np.array(want, dtype=np.float64))
+    assert np.signbit(got[3]) and not np.signbit(got[2])
+    assert np.isnan(bf16_bits_to_f64(np.array([0x7FC0], dtype=np.uint16)))[0]
+    # arrays that are not bit patterns pass through as values
+    np.testing.assert_array_equal(bf16_bits_to_f64(np.array([0.5, -3.0])), [0.5, -3.0])
+
+
+def test_paged_gather_on_a_cache_with_known_rows():
+    """gather_paged_prefix on a cache whose every row holds its own (page, offset): position j must come
+    from page table[j // page_size], offset j % page_size -- a swapped division or a page taken as a row
+    shows at once."""
+    from oracle import gather_paged_prefix
+    num_pages, page_size = 5, 4
+    cache = np.zeros((num_pages, page_size, 2, 3), dtype=np.int64)
+    for pg in range(num_pages):
+        for off in range(page_size):
+            cache[pg, off] = 100 * pg + off
+    table = np.array([3, 0, 4, 1])
+    got = gather_paged_prefix(cache, table, 10)
+    want = [300, 301, 302, 303, 0, 1, 2, 3, 400, 401]
+    assert got.shape == (10, 2, 3)
+    for j in range(10):
+        assert (got[j] == want[j]).all(), j
+    assert gather_paged_prefix(cache, table, 0).shape == (0, 2, 3)
+    # a prefix that ends inside a page stops there
+    assert gather_paged_prefix(cache, table, 5)[-1, 0, 0] == 0
