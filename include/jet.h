@@ -15,6 +15,7 @@
  *   jet_tree_build_scored      entropy / hybrid expansion scores, per-sequence budgets
  *   jet_tree_build_logits      the same fed with raw draft logits (log-softmax on the fly)
  *   jet_tree_verify_attn_tail  the tree's K/V rows live in the cache behind the prefix
+ *   jet_tree_verify_attn_ex, jet_tree_verify_attn_tail_ex   the same with a flags word
  *   jet_kv_compact_tail        in-place commit for that layout
  *   jet_tree_accept_static     greedy acceptance on scratch built into the library
  *   jet_tree_accept_sample     non-greedy (min(1, p/q)) acceptance with a correction draw
@@ -240,6 +241,52 @@ JET_API jet_status jet_tree_verify_attn_tail(const void* q, const void* k_cache,
                                      int Hq, int Hkv, int D, int64_t kv_batch_stride, float softmax_scale,
                                      void* out, float* lse, int32_t* device_status, void* workspace,
                                      size_t workspace_bytes, void* stream);
+
+/* jet_tree_verify_attn_ex / jet_tree_verify_attn_tail_ex -- the two attention calls
+ * with a `flags` word (0 = exactly the plain calls).  The operation is that of
+ * Section 3.2 / Appendix E as above; the flag only tells the kernel what it may
+ * read EARLY.
+ *
+ * The kernel is launched so that it may begin while the kernel before it in the
+ * stream is still finishing (programmatic dependent launch); normally it touches
+ * no global memory until that kernel has completed.  Within a decoding step most
+ * of its inputs are much older than that: the cached prefix was committed by
+ * earlier steps, lengths and page table were set when the step began.
+ *
+ *   JET_ATTN_STABLE_PREFIX   the caller promises that seq_len, n_nodes, page_table
+ *       and every cache row at a position below seq_len[b] were written by work
+ *       that had finished before the kernel DIRECTLY PRECEDING this call in the
+ *       stream could let its successor start (for the kernels of this library,
+ *       which signal only after their own dependency wait, and for ordinary
+ *       launches: "not written by the directly preceding launch, nor by
+ *       anything running concurrently on another stream").  The kernel then
+ *       reads the lengths and streams the prefix K/V tiles into shared memory
+ *       before its dependency wait, i.e. under the preceding kernel's tail.
+ *       q, tree_k / tree_v (tail layout: the rows at and behind seq_len[b]),
+ *       anc_mask and every output are still read / written only behind the wait.
+ *       A broken promise gives undefined attention outputs (stale reads), no
+ *       fault.  In a layer stack: set it for every layer but the first when the
+ *       tree (n_nodes) was built by the launch right before the first layer.
+ * Any other bit: JET_ERR_INVALID_ARG.
+ */
+#define JET_ATTN_STABLE_PREFIX 1u
+
+JET_API jet_status jet_tree_verify_attn_ex(const void* q, const void* k_cache, const void* v_cache,
+                                   const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                   int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                   const void* tree_k, const void* tree_v, const uint32_t* anc_mask,
+                                   const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D,
+                                   int64_t kv_batch_stride, float softmax_scale, void* out, float* lse,
+                                   int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                   void* stream, uint32_t flags);
+
+JET_API jet_status jet_tree_verify_attn_tail_ex(const void* q, const void* k_cache, const void* v_cache,
+                                        const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                        int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                        const uint32_t* anc_mask, const int32_t* n_nodes, int batch, int B,
+                                        int Hq, int Hkv, int D, int64_t kv_batch_stride, float softmax_scale,
+                                        void* out, float* lse, int32_t* device_status, void* workspace,
+                                        size_t workspace_bytes, void* stream, uint32_t flags);
 
 /* ---------------------------------------------------------------------------
  * jet_tree_accept -- greedy acceptance (Section 3.3, Appendix E): a node is

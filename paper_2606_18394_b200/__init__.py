@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     JET_ERR_TIMEOUT,
     JET_ERR_UNSUPPORTED,
     JET_ERR_WORKSPACE,
+    JET_ATTN_STABLE_PREFIX,
     JET_OK,
     JET_STATIC_ACCEPT_SCRATCH_BYTES,
     JetError,
@@ -28,7 +29,9 @@ from .binding import (  # noqa: F401
     jet_tree_build_scored_workspace_bytes,
     jet_tree_build_workspace_bytes,
     jet_tree_verify_attn,
+    jet_tree_verify_attn_ex,
     jet_tree_verify_attn_tail,
+    jet_tree_verify_attn_tail_ex,
     jet_tree_verify_attn_workspace_bytes,
     load,
     status_string,

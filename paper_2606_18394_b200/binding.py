@@ -20,6 +20,7 @@ JET_ERR_UNSUPPORTED = -2
 JET_ERR_WORKSPACE = -3
 JET_ERR_CUDA = -4
 JET_ERR_TIMEOUT = -5
+JET_ATTN_STABLE_PREFIX = 1                     # jet.h: flag of the *_ex attention calls
 JET_STATIC_ACCEPT_SCRATCH_BYTES = 1 << 20     # jet.h: built-in scratch of jet_tree_accept_static
 
 _c = ctypes
@@ -41,6 +42,12 @@ _SIGNATURES = {
                                           _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_tree_verify_attn_tail": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp,
                                                _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "jet_tree_verify_attn_ex": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp,
+                                             _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp,
+                                             _c.c_uint32]),
+    "jet_tree_verify_attn_tail_ex": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp,
+                                                  _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp,
+                                                  _c.c_uint32]),
     "jet_kv_compact_tail": (_c.c_int32, [_vp, _vp, _i64, _i64, _vp, _i, _i, _vp, _vp, _vp, _i, _i, _i, _i,
                                          _i, _i, _vp]),
     "jet_tree_accept_workspace_bytes": (_sz, [_i, _i, _i]),
@@ -202,6 +209,38 @@ def jet_tree_verify_attn_tail(q, k_cache, v_cache, page_table, max_pages_per_seq
                                           _p(out), _p(lse), _p(device_status), _p(workspace), wb, _stream(stream))
     if check:
         _check(st, "jet_tree_verify_attn_tail")
+    return st
+
+
+def jet_tree_verify_attn_ex(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len,
+                            max_seq_len, tree_k, tree_v, anc_mask, n_nodes, batch, B, Hq, Hkv, D,
+                            kv_batch_stride, softmax_scale, out, lse, device_status, workspace, flags,
+                            workspace_bytes=None, stream=None, check=True):
+    wb = workspace_bytes if workspace_bytes is not None else (workspace.numel() * workspace.element_size()
+                                                              if workspace is not None else 0)
+    st = load().jet_tree_verify_attn_ex(_p(q), _p(k_cache), _p(v_cache), _p(page_table), max_pages_per_seq,
+                                        page_size, num_pages, _p(seq_len), max_seq_len, _p(tree_k), _p(tree_v),
+                                        _p(anc_mask), _p(n_nodes), batch, B, Hq, Hkv, D, kv_batch_stride,
+                                        softmax_scale, _p(out), _p(lse), _p(device_status), _p(workspace), wb,
+                                        _stream(stream), int(flags))
+    if check:
+        _check(st, "jet_tree_verify_attn_ex")
+    return st
+
+
+def jet_tree_verify_attn_tail_ex(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages,
+                                 seq_len, max_seq_len, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride,
+                                 softmax_scale, out, lse, device_status, workspace, flags, workspace_bytes=None,
+                                 stream=None, check=True):
+    wb = workspace_bytes if workspace_bytes is not None else (workspace.numel() * workspace.element_size()
+                                                              if workspace is not None else 0)
+    st = load().jet_tree_verify_attn_tail_ex(_p(q), _p(k_cache), _p(v_cache), _p(page_table), max_pages_per_seq,
+                                             page_size, num_pages, _p(seq_len), max_seq_len, _p(anc_mask),
+                                             _p(n_nodes), batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
+                                             _p(out), _p(lse), _p(device_status), _p(workspace), wb,
+                                             _stream(stream), int(flags))
+    if check:
+        _check(st, "jet_tree_verify_attn_tail_ex")
     return st
 
 

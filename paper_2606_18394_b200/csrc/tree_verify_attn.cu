@@ -73,6 +73,7 @@ struct AttnParams {
   int npt;            // 128 / G: nodes per query tile
   uint32_t magic_S, magic_G;
   int len_hint;       // the caller's bound on the cached keys (max_seq_len); 0 = none
+  int stable;         // JET_ATTN_STABLE_PREFIX: lengths, page table and prefix rows may be read before the dependency wait
   int via_global;     // key slices exchange their rows through the workspace instead of a cluster
   int* counters;      // via_global: [2][units * MT] arrival / departure counts, zero between calls
   uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D bf16 + log2-sum-exp (fp32) + pad]
@@ -137,7 +138,7 @@ struct Cfg {
   static constexpr int kBlockBytes = kBM * kRecvPitch;                   // the 128 staged rows of one stream
   static constexpr int kStageOff = 0;
   static constexpr int kRecvOff = (kBlockBytes + 1023) / 1024 * 1024;
-  static_assert(kRecvOff + (kBM + kMaxSplit) * kRecvPitch + 2048 <= kTileBytes, "merge buffers must fit in the tile memory");
+  static_assert(kRecvOff + (kBM + kMaxSplit) * kRecvPitch + 4096 <= kTileBytes, "merge buffers must fit in the tile memory");
 };
 
 struct Bars {       // offsets (in 8-byte units) inside the barrier block
@@ -261,6 +262,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   constexpr int kStages = C::kStages;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) JET_TR(0);
+#ifdef JET_TRACE
+  if (tid == 0 && p.trace) {
+    unsigned long long gt;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+    p.trace[(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) * 64 + 62] = static_cast<long long>(gt);
+  }
+#endif
 
   // ---------------- shared memory carve-up (1024-byte aligned for the 128-byte swizzle)
   extern __shared__ uint8_t smem_raw[];
@@ -356,7 +364,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       // SMs the long sequences start early and the short ones fill the tail): this warp finds the sequence of
       // rank b_rank by counting and leaves it in shared memory.  Beyond kMaxSorted sequences the order stays
       // as given (many small items balance by themselves, and the count is quadratic).
-      ptx::grid_dep_wait();
+      if (!p.stable) ptx::grid_dep_wait();
       int len[kMaxSorted / 32];
 #pragma unroll
       for (int c = 0; c < kMaxSorted / 32; ++c) len[c] = c * 32 + lane < p.batch ? __ldg(p.seq_len + c * 32 + lane) : -1;
@@ -395,15 +403,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (via_cluster) ptx::cluster_arrive();
   const uint32_t tmem_base = *tmem_slot;
   if (tid == 0) JET_TR(42);
-  ptx::grid_dep_wait();      // inputs may be written by the preceding kernel in the stream
-  ptx::grid_dep_launch();    // the next kernel may start its own set-up as SMs become free
-  if (tid == 0) JET_TR(43);
+  // Inputs may be written by the preceding kernel of the stream: nothing in global memory is touched before
+  // the dependency wait.  Exception (p.stable, the caller's promise): the lengths, the page table and the
+  // prefix rows of the caches are older than that kernel, so the K/V producers read them at once -- under the
+  // preceding kernel's tail -- and only the warps that need the query rows, the tree's own K/V rows, the
+  // ancestor masks or the outputs wait, each where it first needs them.  The next kernel of the stream may be
+  // scheduled once this CTA has passed its own wait (so a chain of such kernels never runs more than one ahead).
+  const bool early = p.stable != 0;
+  if (!early || warp == 3) {
+    ptx::grid_dep_wait();
+    ptx::grid_dep_launch();
+  }
+  if (tid == 96) JET_TR(43);
 
   // ---------------- work item, continued: what depends on device data
   const int b = sorted_launch ? *seq_slot : b_rank;
-  // The query rows depend on nothing but the work item: warp 2 (idle after the TMEM allocation) requests them
-  // now, under the look-up of the sequence's lengths.
-  if (warp == 2 && lane == 0) {
+  // The query rows depend on nothing but the work item: warp 3 (idle until the first P V product) requests
+  // them now, under the look-up of the sequence's lengths.
+  if (warp == 3 && lane == 0) {
     JET_TR(46);
     ptx::mbar_arrive_expect_tx(bar(Bars::kQFull), n_mt * kHalves * kHalfBytes);
     for (int mt = 0; mt < n_mt; ++mt)
@@ -435,13 +452,18 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const bool has_work = node_lo < n && T > 0;    // otherwise: no live node here, or an empty key slice
   // A CTA without work never looks at its query rows, but they must have landed before the epilogue reuses
   // their memory (and before the CTA exits).
-  if (!has_work && warp == 2) bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
+  if (!has_work && warp == 3) bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
   // The first K tiles are requested here, straight after the lengths are known: the producer's own loop
   // lies some two thousand cycles of cold code further on (register re-split, set-up of the ring), and
   // the first Q K^T waits for exactly these tiles.  They are the first items of the ring in every form of
   // the key loop (ring order starts K_0 .. K_ahead); the producers start behind them.  A paged tile needs
   // its page ids first and is left to the producers.
-  const int n_early = (has_work && !p.paged) ? (MT == 1 ? min(2, T) : 1) : 0;
+  int n_early = (has_work && !p.paged) ? (MT == 1 ? min(2, T) : 1) : 0;
+  if (early) {         // before the dependency wait only tiles that lie wholly inside the prefix may be read
+    int k = 0;
+    while (k < n_early && (t_lo + k + 1) * kBN <= L) ++k;
+    n_early = k;
+  }
   if (warp == 0 && lane == 0) {
     for (int i = 0; i < n_early; ++i) {
       const int t = t_lo + i;
@@ -469,6 +491,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // part in every CTA-wide barrier and issue the bulk copies and the counter updates).
   auto epilogue = [&](auto sm_side) {
     constexpr bool kSm = decltype(sm_side)::value;
+    if (!kSm && early) ptx::grid_dep_wait();      // (the softmax warps passed theirs before their first tile)
     // The slice bookkeeping is worked out again here, from the CTA index read afresh, so that none of it
     // occupies a register through the key loop (the softmax threads have none to spare).
     uint32_t e_bx;
@@ -681,33 +704,56 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       }
       const uint32_t src_stride = rows_per * C::kRecvPitch;     // distance between the blocks of consecutive slices
-      // the softmax warpgroups combine the blocks: one item = 8 output values of one row
-      const int items = rows_ok ? own_n * (D / 8) : 0;
-#pragma unroll 1
-      for (int i = kSm ? tid - 128 : items; i < items; i += C::kThreads - 128) {
-        const int rl = i / (D / 8), c8 = i - rl * (D / 8);
-        const int R = mt * kBM + own_lo + rl;                  // row within the unit
-        const int vq = static_cast<int>(udiv(R, p.magic_G));
-        const int v = node_lo + vq, h = g * G + (R - vq * G);
-        if (v >= p.B) continue;
-        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        float lse2 = -INFINITY;
-        if (v < n) {
-          const uint8_t* row0 = src_rows + rl * C::kRecvPitch;
-          // (rolled loops: this code runs once per launch and costs what its instruction count costs)
-          float mx = -INFINITY;
-#pragma unroll 1
-          for (int c = 0; c < S; ++c) mx = fmaxf(mx, *reinterpret_cast<const float*>(row0 + c * src_stride + D * 2));
-          float wsum = 0.0f;
-          if (mx > -INFINITY) {
-#pragma unroll 1
+      // The softmax warpgroups combine the blocks in two steps, so that no thread runs a chain of exponentials:
+      // first one thread per row turns the S log-sum-exps into normalised slice weights (shared memory),
+      // then one item = 8 output values of one row is a short run of independent multiply-adds.
+      if constexpr (kSm) {
+        float* wts = reinterpret_cast<float*>(smem_gen + C::kTileBytes - 4096);      // [own_n][S], then 1/sum [own_n]
+        const int n_rows = rows_ok ? own_n : 0;
+        {
+          const int rl = tid - 128;
+          if (rl < n_rows) {
+            const int R = mt * kBM + own_lo + rl;                  // row within the unit
+            const int vq = static_cast<int>(udiv(R, p.magic_G));
+            const int v = node_lo + vq, h = g * G + (R - vq * G);
+            const uint8_t* lse0 = src_rows + rl * C::kRecvPitch + D * 2;
+            float mx = -INFINITY;
+            if (v < n) {
+#pragma unroll 4
+              for (int c = 0; c < S; ++c) mx = fmaxf(mx, *reinterpret_cast<const float*>(lse0 + c * src_stride));
+            }
+            float wsum = 0.0f;
+#pragma unroll 4
             for (int c = 0; c < S; ++c) {
-              const uint8_t* src = row0 + c * src_stride;
-              const float lc = *reinterpret_cast<const float*>(src + D * 2);
-              const float w = lc > -INFINITY ? exp2f(lc - mx) : 0.0f;        // absent slices get weight 0
+              const float lc = *reinterpret_cast<const float*>(lse0 + c * src_stride);
+              // absent slices (log-sum-exp -inf) and rows of padding nodes get weight 0 and are never read
+              const float w = (mx > -INFINITY && lc > -INFINITY) ? exp2f(lc - mx) : 0.0f;
+              wts[rl * S + c] = w;
               wsum += w;
-              // a slice with weight 0 is not read (it may hold junk)
-              const uint4 x = w > 0.0f ? *reinterpret_cast<const uint4*>(src + c8 * 16) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            wts[own_n * S + rl] = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+            if (p.lse && v < p.B)
+              p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] =
+                  wsum > 0.0f ? (mx + log2f(wsum)) * 0.6931471805599453f : -INFINITY;
+          }
+        }
+        ptx::named_sync(2, 256);
+        const int items = n_rows * (D / 8);
+#pragma unroll 1
+        for (int i = tid - 128; i < items; i += 256) {
+          const int rl = i / (D / 8), c8 = i - rl * (D / 8);
+          const int R = mt * kBM + own_lo + rl;
+          const int vq = static_cast<int>(udiv(R, p.magic_G));
+          const int v = node_lo + vq, h = g * G + (R - vq * G);
+          if (v >= p.B) continue;
+          float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+          const uint8_t* src = src_rows + rl * C::kRecvPitch + c8 * 16;
+          const float* wrow = wts + rl * S;
+#pragma unroll 3
+          for (int c = 0; c < S; ++c) {
+            const float w = wrow[c];
+            if (w > 0.0f) {                        // (a slice with weight 0 may hold junk)
+              const uint4 x = *reinterpret_cast<const uint4*>(src + c * src_stride);
               const uint32_t v4[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
               for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
@@ -715,16 +761,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 acc[2 * q + 1] += w * __uint_as_float(v4[q] & 0xFFFF0000u);
               }
             }
-            const float inv = 1.0f / wsum;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) acc[k] *= inv;
-            lse2 = mx + log2f(wsum);
           }
+          const float inv = wts[own_n * S + rl];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) acc[k] *= inv;
+          *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+              make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                         pack_bf16(acc[6], acc[7]));
         }
-        *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
-            make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
-                       pack_bf16(acc[6], acc[7]));
-        if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
       }
     }
 
@@ -782,6 +826,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       constexpr int only = decltype(only_c)::value;
       if (tid == 0) JET_TR(27);
       bool ok = true;
+      bool waited = !early;          // this warp has passed the dependency wait
       int issued = first;
       // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
       // fetched while the current tile's copies are issued, so the table look-up is off the critical path
@@ -800,6 +845,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (only >= 0 && kv != only) {          // the other producer warp's tile
           if (take_k) ++kt; else ++vt;
           continue;
+        }
+        if (!waited && (t + 1) * kBN > L) {      // not wholly inside the prefix: may hold rows the preceding kernel writes
+          ptx::grid_dep_wait();
+          waited = true;
         }
         if (issued >= kStages) {
           ok = bounded_wait(lbar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
@@ -1092,6 +1141,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     epilogue(std::false_type{});
   } else {
     ptx::setmaxnreg_inc<kRegsSoftmax>();
+    if (early) ptx::grid_dep_wait();        // ancestor masks, outputs and the workspace belong behind the wait
     constexpr int kChunks = kBN / 32;                       // 32-key chunks per row and tile
     static_assert(kChunks == 4, "the register-resident row is written out for four 32-key chunks");
     constexpr int kStreams = C::kStreams;
@@ -1498,6 +1548,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   if (tid == 0) {
     JET_TR(13);
+#ifdef JET_TRACE
+    if (p.trace) {
+      unsigned long long gt;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+      p.trace[(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) * 64 + 61] = static_cast<long long>(gt);
+    }
+#endif
     if (*abort_flag && p.status) *p.status = JET_ERR_TIMEOUT;
 #ifdef JET_TRACE
     if (*abort_flag && p.trace) p.trace[(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) * 64 + 31] = *abort_flag;
@@ -1749,8 +1806,9 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
                      int max_seq_len, const void* tree_k, const void* tree_v, bool tail, const uint32_t* anc_mask,
                      const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D, int64_t kv_batch_stride,
                      float softmax_scale, void* out, float* lse, int32_t* device_status, void* workspace,
-                     size_t workspace_bytes, void* stream) {
+                     size_t workspace_bytes, void* stream, uint32_t flags) {
   if (!q || !seq_len || !anc_mask || !n_nodes || !out) return JET_ERR_INVALID_ARG;
+  if (flags & ~static_cast<uint32_t>(JET_ATTN_STABLE_PREFIX)) return JET_ERR_INVALID_ARG;
   if (tail ? (!k_cache || !v_cache || max_seq_len < 1) : (!tree_k || !tree_v)) return JET_ERR_INVALID_ARG;
   if (batch < 1 || batch > 65535 || B < 1 || B > JET_MAX_NODES || Hq < 1 || Hkv < 1 || Hkv > 65535 || Hq % Hkv != 0 ||
       max_seq_len < 0)        // (sequences and KV heads are grid dimensions)
@@ -1833,6 +1891,7 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
   p.magic_G = udiv_magic(static_cast<uint32_t>(G));
   // (measured: a gain of 3-9 % with one query tile per KV head, none to a small loss with two or more)
   p.len_hint = (!paged && !tail && batch == 1 && pl.n_mgroups == 1 && max_seq_len > 0 && max_seq_len < (1 << 26)) ? max_seq_len : 0;
+  p.stable = (flags & JET_ATTN_STABLE_PREFIX) ? 1 : 0;
   p.via_global = pl.via_global;
   p.counters = static_cast<int*>(workspace);
   p.partials = static_cast<uint8_t*>(workspace) + kCounterBytes;
@@ -1865,7 +1924,20 @@ extern "C" jet_status jet_tree_verify_attn(const void* q, const void* k_cache, c
                                            void* stream) {
   return jet::attn_call(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len, max_seq_len,
                         tree_k, tree_v, false, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
-                        out, lse, device_status, workspace, workspace_bytes, stream);
+                        out, lse, device_status, workspace, workspace_bytes, stream, 0u);
+}
+
+extern "C" jet_status jet_tree_verify_attn_ex(const void* q, const void* k_cache, const void* v_cache,
+                                              const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                              int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                              const void* tree_k, const void* tree_v, const uint32_t* anc_mask,
+                                              const int32_t* n_nodes, int batch, int B, int Hq, int Hkv, int D,
+                                              int64_t kv_batch_stride, float softmax_scale, void* out, float* lse,
+                                              int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                              void* stream, uint32_t flags) {
+  return jet::attn_call(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len, max_seq_len,
+                        tree_k, tree_v, false, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
+                        out, lse, device_status, workspace, workspace_bytes, stream, flags);
 }
 
 extern "C" jet_status jet_tree_verify_attn_tail(const void* q, const void* k_cache, const void* v_cache,
@@ -1877,5 +1949,18 @@ extern "C" jet_status jet_tree_verify_attn_tail(const void* q, const void* k_cac
                                                 void* workspace, size_t workspace_bytes, void* stream) {
   return jet::attn_call(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len, max_seq_len,
                         nullptr, nullptr, true, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
-                        out, lse, device_status, workspace, workspace_bytes, stream);
+                        out, lse, device_status, workspace, workspace_bytes, stream, 0u);
+}
+
+extern "C" jet_status jet_tree_verify_attn_tail_ex(const void* q, const void* k_cache, const void* v_cache,
+                                                   const int32_t* page_table, int max_pages_per_seq, int page_size,
+                                                   int64_t num_pages, const int32_t* seq_len, int max_seq_len,
+                                                   const uint32_t* anc_mask, const int32_t* n_nodes, int batch,
+                                                   int B, int Hq, int Hkv, int D, int64_t kv_batch_stride,
+                                                   float softmax_scale, void* out, float* lse,
+                                                   int32_t* device_status, void* workspace, size_t workspace_bytes,
+                                                   void* stream, uint32_t flags) {
+  return jet::attn_call(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len, max_seq_len,
+                        nullptr, nullptr, true, anc_mask, n_nodes, batch, B, Hq, Hkv, D, kv_batch_stride, softmax_scale,
+                        out, lse, device_status, workspace, workspace_bytes, stream, flags);
 }

@@ -89,6 +89,10 @@ class VerifyStep:
         self.alpha = torch.zeros((batch, B), dtype=torch.float32, device=dev)
         self.accept_mode = "greedy"
         self.scale = 1.0 / math.sqrt(D)
+        # Within a step the lengths, the page table and the cached prefix are older than any launch of the
+        # layer stack, so every layer but the first (whose predecessor in the stream builds the tree and
+        # writes n_nodes) lets the attention kernel read them before its dependency wait.
+        self.stable_prefix = True
 
     @property
     def attn_max_len(self):
@@ -140,19 +144,25 @@ class VerifyStep:
                                       self.anc_mask, self.n_nodes, self.depth_entropy, self.ws_build,
                                       node_budget=self.node_budget)
 
-    def verify_attn(self, layer):
+    def verify_attn(self, layer, first_in_stack=None):
+        """Attention of one layer.  first_in_stack: the launch before this call wrote the tree (default:
+        layer == 0), so nothing may be read early."""
+        if first_in_stack is None:
+            first_in_stack = layer == 0
+        flags = jet.JET_ATTN_STABLE_PREFIX if (self.stable_prefix and not first_in_stack) else 0
         if self.tail:
-            jet.jet_tree_verify_attn_tail(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
-                                          self.max_pages, self.page_size, self.num_pages, self.seq_len,
-                                          self.attn_max_len, self.anc_mask, self.n_nodes, self.batch, self.B,
-                                          self.Hq, self.Hkv, self.D, self.kv_batch_stride, self.scale,
-                                          self.out[layer], None, self.status, self.ws_attn)
+            jet.jet_tree_verify_attn_tail_ex(self.q[layer], self.k_cache[layer], self.v_cache[layer],
+                                             self.page_table, self.max_pages, self.page_size, self.num_pages,
+                                             self.seq_len, self.attn_max_len, self.anc_mask, self.n_nodes,
+                                             self.batch, self.B, self.Hq, self.Hkv, self.D, self.kv_batch_stride,
+                                             self.scale, self.out[layer], None, self.status, self.ws_attn, flags)
             return
-        jet.jet_tree_verify_attn(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
-                                 self.max_pages, self.page_size, self.num_pages, self.seq_len, self.attn_max_len,
-                                 self.tree_k[layer], self.tree_v[layer], self.anc_mask, self.n_nodes, self.batch,
-                                 self.B, self.Hq, self.Hkv, self.D, self.kv_batch_stride, self.scale,
-                                 self.out[layer], None, self.status, self.ws_attn)
+        jet.jet_tree_verify_attn_ex(self.q[layer], self.k_cache[layer], self.v_cache[layer], self.page_table,
+                                    self.max_pages, self.page_size, self.num_pages, self.seq_len,
+                                    self.attn_max_len, self.tree_k[layer], self.tree_v[layer], self.anc_mask,
+                                    self.n_nodes, self.batch, self.B, self.Hq, self.Hkv, self.D,
+                                    self.kv_batch_stride, self.scale, self.out[layer], None, self.status,
+                                    self.ws_attn, flags)
 
     def tree_accept(self):
         jet.jet_tree_accept(self.logits, self.V, self.token, self.parent, self.depth, self.anc_mask, self.n_nodes,

@@ -193,7 +193,7 @@ def run_kv_compact(tree_k, tree_v, k_cache, v_cache, page_table, path, accept_le
 
 
 def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_mask, n_nodes, scale,
-                  max_seq_len=None, want_lse=True):
+                  max_seq_len=None, want_lse=True, flags=0):
     """q [batch,B,Hq,D], tree_k/v [batch,B,Hkv,D] bf16 bits; cache contiguous [batch,Lmax,Hkv,D] or paged
     [num_pages,16,Hkv,D] (with page_table [batch,max_pages]).  Returns (out fp64, lse fp64, status)."""
     batch, B, Hq, D = q.shape
@@ -218,15 +218,23 @@ def run_tree_attn(q, k_cache, v_cache, page_table, seq_len, tree_k, tree_v, anc_
     status = guarded_full((1,), 0, torch.int32)
     ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
     ws.zero_()          # the attention workspace starts with counters that must be zero
-    jet.jet_tree_verify_attn(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
-                             d_tk, d_tv, dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
-                             batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
+    d_len, d_anc, d_n = dev(seq_len), dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32))
+    torch.cuda.synchronize()      # (with flags: every input is older than the launch before the call)
+    if flags:
+        jet.jet_tree_verify_attn_ex(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, d_len, max_seq_len,
+                                    d_tk, d_tv, d_anc, d_n, batch, B, Hq, Hkv, D, kv_batch_stride, float(scale),
+                                    out, lse, status, ws, flags)
+    else:
+        jet.jet_tree_verify_attn(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, d_len, max_seq_len,
+                                 d_tk, d_tv, d_anc, d_n, batch, B, Hq, Hkv, D, kv_batch_stride, float(scale),
+                                 out, lse, status, ws)
     check_guards()
     return (bf16_to_f64(out), lse.cpu().numpy().astype(np.float64) if want_lse else None,
             int(status.cpu()[0]))
 
 
-def run_tree_attn_tail(q, k_cache, v_cache, page_table, seq_len, anc_mask, n_nodes, scale, max_seq_len, Hkv):
+def run_tree_attn_tail(q, k_cache, v_cache, page_table, seq_len, anc_mask, n_nodes, scale, max_seq_len, Hkv,
+                       flags=0):
     """As run_tree_attn for a cache that already holds the tree rows behind each prefix."""
     batch, B, Hq, D = q.shape
     seq_len = np.asarray(seq_len, dtype=np.int32)
@@ -243,9 +251,16 @@ def run_tree_attn_tail(q, k_cache, v_cache, page_table, seq_len, anc_mask, n_nod
     status = guarded_full((1,), 0, torch.int32)
     ws = workspace(jet.jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len))
     ws.zero_()
-    jet.jet_tree_verify_attn_tail(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, dev(seq_len), max_seq_len,
-                                  dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32)),
-                                  batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out, lse, status, ws)
+    d_len, d_anc, d_n = dev(seq_len), dev(anc_mask.view(np.int32)), dev(np.asarray(n_nodes, dtype=np.int32))
+    torch.cuda.synchronize()
+    if flags:
+        jet.jet_tree_verify_attn_tail_ex(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, d_len, max_seq_len,
+                                         d_anc, d_n, batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out,
+                                         lse, status, ws, flags)
+    else:
+        jet.jet_tree_verify_attn_tail(d_q, d_k, d_v, pt, max_pages, page_size, num_pages, d_len, max_seq_len,
+                                      d_anc, d_n, batch, B, Hq, Hkv, D, kv_batch_stride, float(scale), out,
+                                      lse, status, ws)
     check_guards()
     return bf16_to_f64(out), lse.cpu().numpy().astype(np.float64), int(status.cpu()[0])
 

@@ -27,6 +27,26 @@ def _contiguous_case(rng, B, n, Hq, Hkv, D, L, extra=24):
     return x, anc, kc, vc, rows
 
 
+@pytest.mark.parametrize("L", [0, 127, 128, 129, 1000])
+@pytest.mark.parametrize("B,n", [(16, 16), (33, 20), (64, 64)])
+def test_contiguous_tail_with_early_prefix_reads(L, B, n):
+    """JET_ATTN_STABLE_PREFIX in the tail layout: the tiles that hold tree rows (at and behind seq_len) must
+    still be read behind the dependency wait; results equal those of the plain call bit for bit."""
+    import jet_harness as H
+    rng = np.random.default_rng(L * 100 + B)
+    Hq, Hkv, D = 8, 2, 128
+    x, anc, kc, vc, rows = _contiguous_case(rng, B, n, Hq, Hkv, D, L)
+    scale = 1.0 / np.sqrt(D)
+    plain, lse_p, st_p = H.run_tree_attn_tail(x["q"][None], kc, vc, None, [L], anc[None], [n], scale, rows, Hkv)
+    early, lse_e, st_e = H.run_tree_attn_tail(x["q"][None], kc, vc, None, [L], anc[None], [n], scale, rows, Hkv,
+                                              flags=1)
+    assert st_p == 0 and st_e == 0
+    assert np.array_equal(plain, early) and np.array_equal(lse_p, lse_e)
+    ref, _ = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, n, scale)
+    err = np.abs(early[0] - ref)
+    assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR
+
+
 @pytest.mark.parametrize("L", [0, 1, 100, 127, 128, 129, 300, 1000])
 @pytest.mark.parametrize("B,n", [(1, 1), (16, 16), (33, 20), (64, 64)])
 def test_contiguous_tail_against_oracle(L, B, n):

@@ -14,11 +14,15 @@ pytestmark = pytest.mark.gpu
 
 MAX_ERR, MEAN_ERR, LSE_ERR = 2e-2, 2e-3, 1e-3
 NAN_BITS = np.uint16(0x7FC0)
+# (Where the stated bound comes from: every probability is rounded to bf16, 2^-9 relative, before it multiplies
+# V entries of size up to ~4.5, the row sum keeps the unrounded values, and the output is rounded to bf16 --
+# 2^-8 * 4.5 = 1.8e-2 in the worst case of a row that sees one or two keys.  With thousands of keys the errors
+# average out; the full-size tests hold the kernel to 4e-3 / 4e-4 there.)
 
 
 def _check(out, lse, ref, rlse, n):
     assert not np.isnan(out).any()
-    err = np.abs(out - ref)
+    err = np.abs(out - ref)[:n]                 # live rows only: the zero rows of padding nodes would dilute the mean
     assert err.max() <= MAX_ERR, err.max()
     assert err.mean() <= MEAN_ERR, err.mean()
     assert (out[n:] == 0).all()
@@ -32,7 +36,7 @@ def _tree(kind, n, rng):
             "star": lambda: star_tree(n), "binary": lambda: binary_tree(n)}[kind]()
 
 
-def _run_contiguous(B, Hq, Hkv, D, L, seed, n=None, kind="random", junk_rows=40, scale=None):
+def _run_contiguous(B, Hq, Hkv, D, L, seed, n=None, kind="random", junk_rows=40, scale=None, flags=0):
     import jet_harness as H
     rng = np.random.default_rng(seed)
     n = n or B
@@ -48,10 +52,33 @@ def _run_contiguous(B, Hq, Hkv, D, L, seed, n=None, kind="random", junk_rows=40,
     tk, tv = x["tree_k"].copy(), x["tree_v"].copy()
     tk[n:], tv[n:] = NAN_BITS, NAN_BITS                       # padding nodes hold junk too
     out, lse, st = H.run_tree_attn(x["q"][None], kc, vc, None, [L], tk[None], tv[None], anc[None], [n], scale,
-                                   max_seq_len=L + junk_rows)
+                                   max_seq_len=L + junk_rows, flags=flags)
     assert st == 0
     _check(out[0], lse[0], ref, rlse, n)
     return out[0], ref
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,D,L", [(32, 8, 2, 128, 0), (32, 8, 2, 128, 127), (33, 8, 2, 128, 128),
+                                          (64, 8, 2, 128, 1000), (64, 32, 8, 128, 4096), (16, 32, 8, 128, 4097),
+                                          (256, 8, 2, 128, 700), (40, 4, 2, 64, 700)])
+def test_stable_prefix_flag_reads_early_and_computes_the_same(B, Hq, Hkv, D, L):
+    """JET_ATTN_STABLE_PREFIX only moves reads of the lengths and of whole prefix tiles in front of the dependency
+    wait; prefixes that end inside a tile, empty prefixes and junk behind the prefix give the same results."""
+    plain, _ = _run_contiguous(B, Hq, Hkv, D, L, 900 + B + L)
+    early, _ = _run_contiguous(B, Hq, Hkv, D, L, 900 + B + L, flags=1)
+    assert np.array_equal(plain, early)
+
+
+def test_unknown_attention_flags_are_rejected():
+    import torch
+    import jet_harness as H
+    import paper_2606_18394_b200 as jet
+    t = torch.zeros(1 << 16, dtype=torch.bfloat16, device=H.DEV)
+    i32 = torch.ones(64, dtype=torch.int32, device=H.DEV)
+    ws = H.workspace(1 << 20)
+    st = jet.jet_tree_verify_attn_ex(t, t, t, None, 0, 0, 0, i32, 16, t, t, i32, i32, 1, 8, 8, 2, 128, 0, 0.1, t, None,
+                                     None, ws, 2, check=False)
+    assert st == jet.JET_ERR_INVALID_ARG
 
 
 @pytest.mark.parametrize("seed", range(2))
@@ -344,8 +371,9 @@ def test_batched_paged_full_size_sampled_rows():
         assert (out[b, n:] == 0).all()
 
 
+@pytest.mark.parametrize("flags", [0, 1])
 @pytest.mark.parametrize("batch,B,Hq,Hkv,D", [(3, 16, 8, 2, 64), (5, 64, 8, 2, 128), (32, 64, 32, 8, 128)])
-def test_batched_paged_ragged(batch, B, Hq, Hkv, D):
+def test_batched_paged_ragged(batch, B, Hq, Hkv, D, flags):
     import jet_harness as H
     rng = np.random.default_rng(4000 + batch)
     if batch == 32:
@@ -370,7 +398,7 @@ def test_batched_paged_ragged(batch, B, Hq, Hkv, D):
         ancs.append(anc_from_parent(parent, int(n_nodes[b]), B))
     scale = 1.0 / np.sqrt(D)
     out, lse, st = H.run_tree_attn(np.stack(qs), kp, vp, table, seq, np.stack(tks), np.stack(tvs), np.stack(ancs),
-                                   n_nodes, scale)
+                                   n_nodes, scale, flags=flags)
     assert st == 0
     check = range(batch) if batch <= 5 else (0, 7, 31)
     for b in check:
