@@ -32,12 +32,26 @@ from jet_inputs import CONFIGS, plant_path  # noqa: E402
 METRIC = "tree_verify_us_per_layer"
 UNIT = "us/layer"
 
-# DRAM bytes (read + write) of one tree_attn_kernel launch on the benchmark workload, from the ncu
-# capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"qwen3_8b": 17659392}     # profiles/tree_attn_kernel_qwen3_8b.md
-# Workloads too large to capture whole: DRAM traffic of a smaller capture of the same kernel as a fraction of
-# that capture's algorithmic bytes (the traffic is the K/V stream and grows in proportion).
-NCU_TRAFFIC_RATIO = {"batched_paged": 0.997}     # profiles/tree_attn_kernel_batched_paged.md
+# DRAM traffic of one tree_attn_kernel launch per workload comes from a small tracked file written from ncu
+# captures (bytes per launch, or -- for workloads too large to capture whole -- the ratio DRAM bytes /
+# algorithmic bytes of a smaller capture of the same kernel), together with the commit it was captured at.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+MIN_TIMED_SECONDS = 0.5       # every timed region of the attention launches is repeated up to this length
+
+
+def ncu_traffic(workload_name, bytes_alg):
+    """(traffic bytes per launch or None, note) for the named workload."""
+    try:
+        table = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        return None, "no capture on file"
+    e = table.get(workload_name)
+    if not e:
+        return None, "no capture on file"
+    note = f"ncu capture at commit {e.get('commit', '?')}: {e.get('source', '')}"
+    if "bytes_per_launch" in e:
+        return int(e["bytes_per_launch"]), note
+    return int(e["ratio_to_algorithmic_bytes"] * bytes_alg), note + " (scaled by the algorithmic bytes)"
 
 
 def workload(name, budget=None, batch=None):
@@ -259,6 +273,153 @@ def rank_seed(base, rank):
     return 1000 * base + rank
 
 
+def time_attention(st, layers, stream, steps, use_graph, sampler=None):
+    """The attention launches alone: `layers` launches per repetition, each on its own KV buffers (cold),
+    replayed as a graph like the step itself, CUDA events on the launching stream.  At least `steps`
+    repetitions, and as many more as it takes to fill MIN_TIMED_SECONDS.  Returns (us per launch, how, reps)."""
+    import torch
+    with torch.cuda.stream(stream):
+        st.seq_len.copy_(st.seq_len0)
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            for layer in range(layers):
+                st.verify_attn(layer)
+            stream.synchronize()
+            with torch.cuda.graph(graph, stream=stream):
+                for layer in range(layers):
+                    st.verify_attn(layer)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(3):
+                graph.replay()
+            a1.record(stream)
+            stream.synchronize()
+            per_replay_s = max(a0.elapsed_time(a1) * 1e-3 / 3, 1e-6)
+            reps = max(steps, int(MIN_TIMED_SECONDS / per_replay_s) + 1)
+            if sampler is not None:
+                sampler.start()
+            a0.record(stream)
+            for _ in range(reps):
+                graph.replay()
+            a1.record(stream)
+            stream.synchronize()
+            return (a0.elapsed_time(a1) * 1e3 / (reps * layers),
+                    f"CUDA events around {reps} replays of a graph of the {layers} attention launches", reps)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(layers * steps)]
+        for rep_i in range(2):                       # first repetition warms up
+            if rep_i == 1 and sampler is not None:
+                sampler.start()
+            i = 0
+            for _ in range(steps):
+                for layer in range(layers):
+                    a, b_ = evs[i]
+                    a.record(stream)
+                    st.verify_attn(layer)
+                    b_.record(stream)
+                    i += 1
+            stream.synchronize()
+        return (statistics.mean(a.elapsed_time(b_) for a, b_ in evs) * 1e3, "CUDA events around every attention call",
+                steps)
+
+
+def attention_roofline(c, info, attn_us, clocks, workload_name, timing):
+    """The roofline object of the attention kernel for one workload."""
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peaks, peak_src = json.load(open(peaks_path)), "measured"
+    else:
+        peaks, peak_src = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+    bytes_alg = attn_algorithmic_bytes(c, info["seq_lens"], info["n_nodes"])
+    flops_alg = attn_algorithmic_flops(c, info["seq_lens"], info["depth"])
+    t_bytes = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    t_flops = flops_alg / (peaks["bf16_tflops"] * 1e12)
+    if t_bytes >= t_flops:
+        roof = {"bound": "hbm", "achieved": bytes_alg / (attn_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        # a tensor-bound kernel timed in a long region under the power cap (reason flag, or the sampled SM clock well
+        # below its maximum) is held against the sustained GEMM figure (seconds-long loop), otherwise against the
+        # burst figure; the fraction of the burst figure is reported beside it
+        slowed = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
+        capped = ("sw_power_cap" in (clocks.get("reasons") or []) or slowed) and "bf16_tflops_sustained" in peaks
+        achieved = flops_alg / (attn_us * 1e-6) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved,
+                "peak": peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "peak_kind": "sustained (power cap or SM clock below 90 % of its maximum during the timed region)" if capped else "burst",
+                "frac_of_burst_peak": achieved / peaks["bf16_tflops"]}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"], roof["traffic_note"] = ncu_traffic(workload_name, bytes_alg)
+    roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us, timing=timing,
+                algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
+                roofline_us=max(t_bytes, t_flops) * 1e6)
+    if clocks.get("sm_mhz"):
+        # a latency-bound launch scales with the SM clock: the product lets runs at different clocks be compared
+        roof["us_x_sm_mhz"] = attn_us * clocks["sm_mhz"]
+    return roof
+
+
+def sweep_point(name, c, seed, device, steps, sampler_args, layers=None):
+    """One more workload for the recorded line: the attention launches alone (no tree construction,
+    acceptance or commit timed), on enough layers that the K/V of one repetition is several times the L2."""
+    import torch
+    from paper_2606_18394_b200.step import VerifyStep
+    c = dict(c)
+    batch, B, N, W, Hq, Hkv, D = c["batch"], c["B"], c["N"], c["W"], c["Hq"], c["Hkv"], c["D"]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    rng = np.random.default_rng(seed)
+    if c.get("paged"):
+        seq = rng.integers(c["L_range"][0], c["L_range"][1] + 1, size=batch).astype(np.int32)
+    else:
+        seq = np.full(batch, c["L"], dtype=np.int32)
+    kv_bytes = int(2 * int(seq.sum()) * Hkv * D * 2)
+    layers = layers or max(2, min(c["layers"], int(600e6 // kv_bytes) + 1))
+    c["layers"] = layers
+    V = 4096                         # the draft vocabulary plays no part in the attention launches
+    if c.get("paged"):
+        need = [(int(L) + N + 1 + 15) // 16 for L in seq]
+        num_pages = sum(need) + 3
+        perm = rng.permutation(num_pages)
+        table = np.zeros((batch, max(need)), dtype=np.int32)
+        pos = 0
+        for b, cnt in enumerate(need):
+            table[b, :cnt] = perm[pos:pos + cnt]
+            pos += cnt
+        st = VerifyStep(batch=batch, layers=layers, Hq=Hq, Hkv=Hkv, D=D, B=B, N=N, W=W, V=V,
+                        max_seq_len=int(seq.max()), page_size=16, num_pages=num_pages, max_pages=max(need),
+                        device=device)
+        st.page_table.copy_(torch.from_numpy(table))
+    else:
+        st = VerifyStep(batch=batch, layers=layers, Hq=Hq, Hkv=Hkv, D=D, B=B, N=N, W=W, V=V,
+                        max_seq_len=int(c["L"]), device=device)
+    st.seq_len0.copy_(torch.from_numpy(seq))
+    for t in (st.q, st.tree_k, st.tree_v):
+        t.copy_(torch.randn(t.shape, generator=gen, device=device, dtype=torch.float32))
+    for layer in range(layers):
+        st.k_cache[layer].copy_(torch.randn(st.k_cache[layer].shape, generator=gen, device=device, dtype=torch.float32))
+        st.v_cache[layer].copy_(torch.randn(st.v_cache[layer].shape, generator=gen, device=device, dtype=torch.float32))
+    logits = torch.randn(st.logp.shape, generator=gen, device=device, dtype=torch.float32) * 3.0
+    top = torch.randint(0, V, (batch, N), generator=gen, device=device)
+    logits.scatter_(2, top[:, :, None], 14.0)          # one confident token per depth, so the trees grow deep
+    st.logp.copy_(torch.log_softmax(logits.double(), dim=2).float())
+    st.root_token.fill_(1)
+    st.seq_len.copy_(st.seq_len0)
+    st.tree_build()
+    torch.cuda.synchronize()
+    info = dict(seq_lens=[int(x) for x in seq], depth=st.depth.cpu().numpy(), n_nodes=st.n_nodes.cpu().numpy())
+    stream = torch.cuda.Stream()
+    sampler = ClockSampler(*sampler_args)
+    attn_us, timing, reps = time_attention(st, layers, stream, steps, True, sampler)
+    clocks = sampler.stop()
+    assert int(st.status.item()) == 0, "a bounded device wait expired"
+    roof = attention_roofline(c, info, attn_us, clocks, name, timing)
+    point = {"workload": name, "batch": batch, "tree_nodes": B, "prefix": info["seq_lens"] if c.get("paged") else c["L"],
+             "layers_timed": layers, "us_per_launch": attn_us, "launches": reps * layers, "clocks": clocks, "roofline": roof}
+    del st
+    torch.cuda.empty_cache()
+    return point
+
+
 def bench_jet(args):
     import torch
     import torch.distributed as dist
@@ -311,6 +472,29 @@ def bench_jet(args):
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
     ms_step = max_over_ranks(ms_total, device, world) / args.steps
+    # The K steps above may last only a few milliseconds, at whatever clock the GPU happened to run; the same step
+    # is timed again over a region of MIN_TIMED_SECONDS with its own clock samples (reported as "sustained").
+    sustained = None
+    if ms_total * 1e-3 < MIN_TIMED_SECONDS:
+        more = int(MIN_TIMED_SECONDS / max(ms_step * 1e-3, 1e-6)) + 1
+        sus_sampler = ClockSampler(local_rank, gpu_uuid)
+        if rank == 0:
+            sus_sampler.start()
+        barrier()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(more):
+                run()
+            e1.record(stream)
+        stream.synchronize()
+        barrier()
+        sus_ms = max_over_ranks(e0.elapsed_time(e1), device, world) / more
+        sus_clocks = sus_sampler.stop() if rank == 0 else None
+        if rank == 0:
+            sustained = {"steps": more, "ms_per_step": sus_ms, "value": sus_ms * 1e3 / (layers * world), "unit": UNIT,
+                         "clocks": sus_clocks}
+            if sus_clocks.get("sm_mhz"):
+                sustained["value_x_sm_mhz"] = sustained["value"] * sus_clocks["sm_mhz"]
     assert int(st.status.item()) == 0, "a bounded device wait expired"
     acc = st.accept_len.cpu().numpy().tolist()
     if args.accept == "greedy":
@@ -318,46 +502,16 @@ def bench_jet(args):
     else:
         assert all(0 <= a <= c["N"] for a in acc), acc
 
-    # ---------------- the attention launches alone (the dominant kernel): `layers` launches per repetition, each
-    #                  on its own KV buffers (cold), replayed as a graph like the step itself; CUDA events on the
-    #                  launching stream around `steps` repetitions.  Without a graph: events around every call.
-    with torch.cuda.stream(stream):
-        st.seq_len.copy_(st.seq_len0)
-        if not args.no_graph:
-            attn_graph = torch.cuda.CUDAGraph()
-            for layer in range(layers):
-                st.verify_attn(layer)
-            stream.synchronize()
-            with torch.cuda.graph(attn_graph, stream=stream):
-                for layer in range(layers):
-                    st.verify_attn(layer)
-            for _ in range(3):
-                attn_graph.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            for _ in range(args.steps):
-                attn_graph.replay()
-            a1.record(stream)
-            stream.synchronize()
-            attn_us = a0.elapsed_time(a1) * 1e3 / (args.steps * layers)
-            attn_timing = f"CUDA events around {args.steps} replays of a graph of the {layers} attention launches"
-        else:
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                   for _ in range(layers * args.steps)]
-            for rep in range(2):                       # first repetition warms up
-                i = 0
-                for _ in range(args.steps):
-                    for layer in range(layers):
-                        a, b_ = evs[i]
-                        a.record(stream)
-                        st.verify_attn(layer)
-                        b_.record(stream)
-                        i += 1
-                stream.synchronize()
-            attn_us = statistics.mean(a.elapsed_time(b_) for a, b_ in evs) * 1e3
-            attn_timing = "CUDA events around every attention call"
+    # ---------------- the attention launches alone (the dominant kernel), in a region of its own with its own
+    #                  clock samples (this is the denominator of roofline.achieved)
+    attn_sampler = ClockSampler(local_rank, gpu_uuid)
+    attn_us, attn_timing, attn_reps = time_attention(st, layers, stream, args.steps, not args.no_graph,
+                                                     attn_sampler if rank == 0 else None)
+    attn_clocks = attn_sampler.stop() if rank == 0 else None
     assert int(st.status.item()) == 0, "a bounded device wait expired"
+    # the same launches issued call by call (no graph): what a caller that does not capture pays per call,
+    # host-side argument checks and tensor-map encoding included
+    attn_us_eager, _, _ = time_attention(st, layers, stream, max(2, min(args.steps, 10)), False, None)
 
     # ---------------- end to end: host buffers in, result out, every step
     pinned = {k: getattr(st, k).cpu().pin_memory() for k in ("logp", "root_token", "logits", "q", "tree_k", "tree_v")}
@@ -427,36 +581,21 @@ def bench_jet(args):
         return
 
     # ---------------- roofline of the dominant kernel (one attention call = one tree_attn_kernel launch)
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peaks, peak_src = json.load(open(peaks_path)), "measured"
-    else:
-        peaks, peak_src = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
-    bytes_alg = attn_algorithmic_bytes(c, info["seq_lens"], info["n_nodes"])
-    flops_alg = attn_algorithmic_flops(c, info["seq_lens"], info["depth"])
-    t_bytes = bytes_alg / (peaks["hbm_gbs"] * 1e9)
-    t_flops = flops_alg / (peaks["bf16_tflops"] * 1e12)
-    if t_bytes >= t_flops:
-        roof = {"bound": "hbm", "achieved": bytes_alg / (attn_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    else:
-        # a tensor-bound kernel timed in a long region under the power cap (reason flag, or the sampled SM clock well
-        # below its maximum) is held against the sustained GEMM figure (seconds-long loop), otherwise against the
-        # burst figure; the fraction of the burst figure is reported beside it
-        slowed = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
-        capped = ("sw_power_cap" in (clocks.get("reasons") or []) or slowed) and "bf16_tflops_sustained" in peaks
-        achieved = flops_alg / (attn_us * 1e-6) / 1e12
-        roof = {"bound": "tensor", "achieved": achieved,
-                "peak": peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "peak_kind": "sustained (power cap or SM clock below 90 % of its maximum during the timed region)" if capped else "burst",
-                "frac_of_burst_peak": achieved / peaks["bf16_tflops"]}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(args.config)
-    if roof["traffic"] is None and args.config in NCU_TRAFFIC_RATIO:
-        roof["traffic"] = int(NCU_TRAFFIC_RATIO[args.config] * bytes_alg)
-        roof["traffic_note"] = "scaled from a smaller ncu capture of the same kernel by the algorithmic bytes"
-    roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us, timing=attn_timing,
-                algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
-                roofline_us=max(t_bytes, t_flops) * 1e6)
+    roof = attention_roofline(c, info, attn_us, attn_clocks, args.config, attn_timing)
+    roof["clocks"] = attn_clocks
+    roof["us_per_call_without_graph"] = attn_us_eager
+
+    # ---------------- the rest of the metric's range (64 .. 256-node trees at the same layer shape, and the batched
+    #                  serving shape): attention launches only, each point timed for MIN_TIMED_SECONDS
+    sweep = []
+    if args.config == "qwen3_8b" and not args.no_sweep and world == 1:
+        base = dict(CONFIGS["qwen3_8b"])
+        for nodes in (128, 256):
+            cc = dict(base, B=nodes, N=12)
+            sweep.append(sweep_point(f"qwen3_8b_b{nodes}", cc, rank_seed(5, rank) + nodes, device, 3,
+                                     (local_rank, gpu_uuid)))
+        sweep.append(sweep_point("batched_paged", dict(CONFIGS["batched_paged"]), rank_seed(6, rank), device, 3,
+                                 (local_rank, gpu_uuid)))
 
     cpu = cpu_baseline(st, c, info) if not args.no_cpu_baseline else None
 
@@ -480,6 +619,10 @@ def bench_jet(args):
         "gpu_launches": args.steps * st.launches_per_step(1),
         "clocks": clocks, "roofline": roof,
     }
+    if sustained is not None:
+        line["sustained"] = sustained
+    if sweep:
+        line["sweep"] = sweep
     if cpu is not None:
         line["cpu_baseline"] = cpu
     print(json.dumps(line), flush=True)
@@ -605,6 +748,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="batch, for configurations that list several")
     ap.add_argument("--no-graph", action="store_true", help="issue the calls directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the extra attention-only points of the default run")
     ap.add_argument("--layout", choices=["separate", "tail"], default="separate",
                     help="tree K/V in their own buffers, or in the cache behind each prefix")
     ap.add_argument("--score", choices=["accum_logp", "entropy", "hybrid"], default="accum_logp",
