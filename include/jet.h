@@ -210,7 +210,23 @@ JET_API jet_status jet_tree_build_logits(const float* logits, int64_t logits_bat
  * Workspace: unlike the other calls, the first 4096 bytes of this workspace hold
  * counters that must be ZERO when the call starts.  Zero them once after
  * allocating the workspace; every call that completes leaves them zero again.
- * (A call that reported JET_ERR_TIMEOUT may leave them dirty: zero them again.)
+ * (A call that reported JET_ERR_TIMEOUT may leave them dirty: zero them again.
+ * Counters that are not zero on entry are the caller's error: the key slices of
+ * a work item then never see each other arrive, every CTA gives up after its
+ * bounded wait, device_status reads JET_ERR_TIMEOUT and the outputs are
+ * undefined; nothing faults and the next call on a zeroed workspace is correct.)
+ * When a sequence has fewer work items than the GPU has SMs, its key range is cut
+ * into slices that run as separate CTAs and hand each other their partial rows
+ * through this workspace inside the one launch.  That exchange assumes that all
+ * CTAs of the launch are resident at once: the plan is sized from the device's SM
+ * count, so give the call the whole GPU (no other kernel holding SMs at the same
+ * time through another stream, MPS or a green context).  If some CTAs cannot
+ * start until others finish, the waiting ones give up after about a second with
+ * JET_ERR_TIMEOUT instead of hanging.
+ * Test hooks, read from the environment once per process and meant for the
+ * test-suite only: JET_FORCE_MT / JET_FORCE_SPLIT force a launch plan (query
+ * tiles per CTA; key slices, with ",g" through the workspace),
+ * JET_TEST_POLL_LIMIT shortens the bounded wait of the workspace exchange.
  */
 JET_API size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                             int max_seq_len);

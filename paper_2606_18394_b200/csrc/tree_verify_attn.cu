@@ -73,6 +73,7 @@ struct AttnParams {
   int npt;            // 128 / G: nodes per query tile
   uint32_t magic_S, magic_G;
   int len_hint;       // the caller's bound on the cached keys (max_seq_len); 0 = none
+  uint32_t poll_limit;  // workspace merge: polls of the arrival count before the CTA gives up (about a second)
   int stable;         // JET_ATTN_STABLE_PREFIX: lengths, page table and prefix rows may be read before the dependency wait
   int via_global;     // key slices exchange their rows through the workspace instead of a cluster
   int* counters;      // via_global: [2][units * MT] arrival / departure counts, zero between calls
@@ -678,7 +679,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           JET_TR(29);
           bool seen = ptx::atom_add_acq_rel_gpu(arrive, 1) + 1 >= S;
           JET_TR(30);
-          for (uint32_t i = 0; i < (1u << 22) && !seen; ++i) {
+          for (uint32_t i = 0; i < p.poll_limit && !seen; ++i) {
             if (ptx::ld_acquire_gpu(arrive) >= S) { seen = true; break; }
             __nanosleep(32);
             if (*abort_flag) break;
@@ -1892,6 +1893,14 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
   // (measured: a gain of 3-9 % with one query tile per KV head, none to a small loss with two or more)
   p.len_hint = (!paged && !tail && batch == 1 && pl.n_mgroups == 1 && max_seq_len > 0 && max_seq_len < (1 << 26)) ? max_seq_len : 0;
   p.stable = (flags & JET_ATTN_STABLE_PREFIX) ? 1 : 0;
+  // Test hook (read once per process): JET_TEST_POLL_LIMIT shortens the bounded spin of the workspace merge so
+  // that a test can make it run out within milliseconds.
+  static const uint32_t poll_limit = [] {
+    const char* e = getenv("JET_TEST_POLL_LIMIT");
+    const long v = e ? atol(e) : 0;
+    return v > 0 ? static_cast<uint32_t>(v) : (1u << 22);
+  }();
+  p.poll_limit = poll_limit;
   p.via_global = pl.via_global;
   p.counters = static_cast<int*>(workspace);
   p.partials = static_cast<uint8_t*>(workspace) + kCounterBytes;

@@ -556,3 +556,60 @@ print("ok")
     env = dict(os.environ, JET_FORCE_MT="2")
     res = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=300)
     assert res.returncode == 0 and "ok" in res.stdout, res.stdout + res.stderr
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_library_usable():
+    """Failure made on the host: the workspace's arrival counter of the first work item is preset to a value from
+    which the key slices can never count up to their number (a dirty workspace is a caller error the header
+    describes).  With the poll limit of the workspace exchange shortened (test hook), every CTA of that work
+    item gives up within milliseconds: the call returns, device_status reads JET_ERR_TIMEOUT, nothing hangs or
+    faults, and the next call on a re-zeroed workspace is correct (TMEM was released, no barrier left armed)."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import sys, os
+sys.path.insert(0, os.getcwd()); sys.path.insert(0, os.path.join(os.getcwd(), "tests"))
+import numpy as np, torch
+import jet_harness as H
+import paper_2606_18394_b200 as jet
+from jet_inputs import make_attn_inputs, random_tree
+from oracle import anc_from_parent, tree_attn_ref
+B, Hq, Hkv, D, L = 32, 8, 2, 128, 600
+rng = np.random.default_rng(3)
+x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+parent, _, _ = random_tree(B, rng)
+anc = anc_from_parent(parent, B, B)
+scale = 1.0 / np.sqrt(D)
+ref, _ = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, B, scale)
+nbytes = jet.jet_tree_verify_attn_workspace_bytes(1, B, Hq, Hkv, D, L)
+assert nbytes > 4096, "the forced plan must exchange through the workspace"
+ws = torch.zeros(nbytes, dtype=torch.uint8, device=H.DEV)
+d = dict(q=H.dev_bf16(x["q"][None]), k=H.dev_bf16(x["k_prefix"][None]), v=H.dev_bf16(x["v_prefix"][None]),
+         tk=H.dev_bf16(x["tree_k"][None]), tv=H.dev_bf16(x["tree_v"][None]), anc=H.dev(anc[None].view(np.int32)),
+         n=H.dev(np.array([B], np.int32)), seq=H.dev(np.array([L], np.int32)))
+def call(out, status):
+    return jet.jet_tree_verify_attn(d["q"], d["k"], d["v"], None, 0, 0, 0, d["seq"], L, d["tk"], d["tv"], d["anc"],
+                                    d["n"], 1, B, Hq, Hkv, D, L * Hkv * D, float(scale), out, None, status, ws,
+                                    check=False)
+status = torch.zeros(1, dtype=torch.int32, device=H.DEV)
+out = torch.full((1, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=H.DEV)
+ws[:4096].view(torch.int32)[0] = -1000          # the first work item's arrival count can never reach its slice count
+assert call(out, status) == jet.JET_OK          # the call itself is asynchronous and has nothing to report yet
+torch.cuda.synchronize()                        # returns: every wait was bounded
+assert int(status.item()) == jet.JET_ERR_TIMEOUT, int(status.item())
+# second call, workspace zeroed again: correct, and the status word is only ever set, never cleared, by the library
+ws.zero_(); status.zero_()
+out2 = torch.full((1, B, Hq, D), float("nan"), dtype=torch.bfloat16, device=H.DEV)
+assert call(out2, status) == jet.JET_OK
+torch.cuda.synchronize()
+assert int(status.item()) == 0
+err = np.abs(H.bf16_to_f64(out2)[0] - ref)
+assert not np.isnan(H.bf16_to_f64(out2)).any() and err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
+assert int(ws[:4096].view(torch.int32).abs().sum().item()) == 0
+print("ok")
+'''
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, JET_FORCE_MT="1", JET_FORCE_SPLIT="2,g", JET_TEST_POLL_LIMIT="2000")
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0 and "ok" in res.stdout, res.stdout[-2000:] + res.stderr[-3000:]
