@@ -386,6 +386,15 @@ JET_API jet_status jet_tree_accept_static(const float* logits, int64_t logits_ro
  *   u_accept     fp32 [batch, B]; u_sample fp32 [batch]
  *   alpha        optional out fp32 [batch, B] (0 for padding rows, 1 for the root)
  *   accept_len   i32 [batch]; path, out_tokens i32 [batch, N+1], -1 padded
+ * What distribution comes out: on a CHAIN whose tokens were drawn from q the
+ * emitted tokens follow the target distribution exactly (the guarantee of
+ * speculative sampling).  On a BRANCHED tree the rule above is applied to every
+ * sibling on its own and the deepest passing branch wins, which is the per-branch
+ * rule the paper states but does not preserve the target distribution (two
+ * siblings with p == q both pass, and the one with the lower node index is always
+ * the one emitted; the residual after several rejected siblings is the single-draft
+ * one).  A caller that needs exact target sampling at temperature > 0 verifies
+ * chains (W = 1) with this call, or uses greedy acceptance on trees.
  * Precision: fp32 throughout, cumulative masses in fp64; a draw or a test that
  * falls within rounding of its threshold may differ from an fp64 evaluation.
  * temperature must be positive and finite.

@@ -210,24 +210,13 @@ topw_partial_kernel(const float* __restrict__ logp, int64_t batch_stride, int64_
   }
   // many equal values: warp 0 alone walks the candidates in rank order
   if (tid >= 32) return;
-  constexpr int kHeld = 8;                       // candidates a lane keeps in registers (usual case)
-  unsigned long long held[kHeld];
-  const bool in_regs = count <= 32 * kHeld;
-  if (in_regs) {
-#pragma unroll
-    for (int i = 0; i < kHeld; ++i) held[i] = lane + 32 * i < count ? s_cand[lane + 32 * i] : 0ull;
-  }
+  // (more than kTopThreads candidates here, too many for registers: every round scans shared memory)
   unsigned long long prev = ~0ull;
   for (int r = 0; r < Wc; ++r) {
     unsigned long long best = 0ull;
-    if (in_regs) {
-#pragma unroll
-      for (int i = 0; i < kHeld; ++i) if (held[i] < prev && held[i] > best) best = held[i];
-    } else {
-      for (int i = lane; i < count; i += 32) {
-        const unsigned long long k = s_cand[i];
-        if (k < prev && k > best) best = k;
-      }
+    for (int i = lane; i < count; i += 32) {
+      const unsigned long long k = s_cand[i];
+      if (k < prev && k > best) best = k;
     }
     best = warp_max_u64(best);
     if (lane == 0) out[r] = best;

@@ -30,6 +30,7 @@
 // TMEM is released and JET_ERR_TIMEOUT is reported.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <type_traits>
@@ -1594,13 +1595,30 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Everything the host side caches about the GPU is kept per device (a process may drive several).
+constexpr int kMaxDevices = 64;
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return 0;
+  }
+  return dev;
+}
+
 int sm_count() {
-  static int n = [] {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
-    return v;
-  }();
+  static std::atomic<int> cache[kMaxDevices];
+  const int dev = current_device();
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+      cudaGetLastError();
+      v = 148;
+    }
+    n = v;
+    cache[dev].store(n, std::memory_order_relaxed);
+  }
   return n;
 }
 
@@ -1616,7 +1634,9 @@ constexpr size_t kCounterBytes = 4096;     // head of the workspace: arrival / d
 
 template <int D, int MT>
 bool configure_kernel() {
-  static int state = 0;     // 0 = not yet, 1 = ok, -1 = failed
+  static std::atomic<int> states[kMaxDevices];      // per device: 0 = not yet, 1 = ok, -1 = failed
+  std::atomic<int>& state_ref = states[current_device()];
+  int state = state_ref.load(std::memory_order_acquire);
   if (state == 0) {
     auto set = [](auto kernel) {
       return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D, MT>::kSmemBytes) ==
@@ -1627,6 +1647,7 @@ bool configure_kernel() {
                 ? 1
                 : -1;
     if (state < 0) cudaGetLastError();
+    state_ref.store(state, std::memory_order_release);
   }
   return state > 0;
 }
@@ -1635,9 +1656,10 @@ bool configure_kernel() {
 // cluster must fit inside one GPC).  Asked of the driver once per cluster size and cached.
 template <int D, int MT>
 int max_active_clusters(int cluster) {
-  static int cache[kMaxSplit + 1] = {};      // 0 = unknown, -1 = none
+  static std::atomic<int> caches[kMaxDevices][kMaxSplit + 1];      // per device: 0 = unknown, -1 = none
   if (cluster < 1 || cluster > kMaxSplit) return 0;
-  if (cache[cluster] == 0) {
+  std::atomic<int>* cache = caches[current_device()];
+  if (cache[cluster].load(std::memory_order_relaxed) == 0) {
     int n = 0;
     if (configure_kernel<D, MT>()) {
       cudaLaunchConfig_t cfg = {};
@@ -1656,9 +1678,10 @@ int max_active_clusters(int cluster) {
         n = 0;
       }
     }
-    cache[cluster] = n > 0 ? n : -1;
+    cache[cluster].store(n > 0 ? n : -1, std::memory_order_relaxed);
   }
-  return cache[cluster] > 0 ? cache[cluster] : 0;
+  const int have = cache[cluster].load(std::memory_order_relaxed);
+  return have > 0 ? have : 0;
 }
 
 int max_active_clusters_for(int D, int mt, int cluster) {

@@ -129,6 +129,34 @@ def test_star_with_every_child_rejected_draws_from_the_residual():
     assert (ref["cdf"][t - 1] if t else 0.0) - tol <= target <= ref["cdf"][t] + tol
 
 
+def test_two_siblings_follow_the_per_branch_reading():
+    """Branched tree, the documented reading: every sibling is tested on its own, the deepest passing branch wins
+    (lowest node index first).  With q == p both siblings always pass and the first one is emitted; the GPU and
+    the oracle agree on every draw."""
+    import jet_harness as H
+    rng = np.random.default_rng(17)
+    V, N, B = 4099, 2, 3
+    p_logits = (rng.standard_normal(V) * 2.0).astype(np.float32)
+    z = p_logits.astype(np.float64)
+    logp0 = (z - (z.max() + np.log(np.exp(z - z.max()).sum()))).astype(np.float32)     # q == p at depth 0
+    logp = np.stack([logp0, make_logp(rng, 1, V, 2.0)[0]])[None]
+    order = np.argsort(-p_logits)
+    token = np.array([[7, int(order[1]), int(order[0])]], np.int32)     # two children of the root
+    parent = np.array([[-1, 0, 0]], np.int32)
+    depth = np.array([[0, 1, 1]], np.int32)
+    anc = anc_from_parent(parent[0], B, B)[None]
+    logits = np.stack([p_logits, (rng.standard_normal(V) * 2).astype(np.float32),
+                       (rng.standard_normal(V) * 2).astype(np.float32)])[None]
+    for _ in range(20):
+        u = rng.random((1, B)).astype(np.float32) * 0.98
+        u_s = rng.random(1).astype(np.float32)
+        got = H.run_tree_accept_sample(logits, 1.0, logp, token, parent, depth, anc, np.array([B]), N, u, u_s)
+        ref = tree_accept_sample_ref(logits[0], 1.0, logp[0], token[0], parent[0], depth[0], B, N, u[0], u_s[0])
+        assert got["accept_len"][0] == ref["accept_len"] == 1
+        assert np.array_equal(got["path"][0], ref["path"]) and got["path"][0, 1] == 1
+        assert got["out_tokens"][0, 0] == ref["out_tokens"][0] == token[0, 1]
+
+
 def test_padding_nodes_and_argument_errors():
     import torch
     import jet_harness as H

@@ -168,3 +168,30 @@ def test_deepest_accepted_node_matches_brute_force_over_leaves():
         assert (r["accept_len"], r["end_node"]) == (best_len, best_end)
         assert list(r["path"][: best_len + 1]) == [int(x) for x in r["path"][: best_len + 1]]
         assert r["path"][0] == 0 and r["path"][best_len] == best_end
+
+
+def test_branched_tree_applies_the_rule_per_branch_and_is_not_target_distributed():
+    """The reading taken for several siblings (the paper gives the per-branch rule only): every sibling is tested
+    on its own against the same target distribution and the deepest passing branch wins, lowest index first.
+    That is exact on chains (tests above) and NOT distribution-preserving on branched trees -- the header of the
+    library says so.  Pinned here so that the behaviour cannot drift unnoticed: with q == p two siblings both
+    pass whatever the random numbers are, so the first emitted token is always the lower-indexed sibling's,
+    where the target would emit it with probability p only."""
+    rng = np.random.default_rng(5)
+    V = 5
+    p_logits = np.log(np.array([0.4, 0.3, 0.15, 0.1, 0.05])).astype(np.float32)
+    q_logp = _log_softmax(p_logits[None].astype(np.float64))          # q == p at depth 0
+    token = np.array([0, 1, 0], np.int32)                              # root, two children: tokens 1 and 0
+    parent = np.array([-1, 0, 0], np.int32)
+    depth = np.array([0, 1, 1], np.int32)
+    logits = np.stack([p_logits, rng.normal(size=V).astype(np.float32), rng.normal(size=V).astype(np.float32)])
+    firsts = set()
+    for _ in range(200):
+        r = tree_accept_sample_ref(logits, 1.0, q_logp, token, parent, depth, 3, 1, rng.random(3), rng.random())
+        assert r["accept_len"] == 1 and r["path"][1] == 1              # sibling with the lower node index
+        firsts.add(int(r["out_tokens"][0]))
+    assert firsts == {1}                                               # always token 1; the target gives it 0.3
+    # a sibling that fails its own test does not stop the other one
+    q2 = _log_softmax(np.log(np.array([[0.02, 0.9, 0.02, 0.03, 0.03]])))    # token 1 over-proposed: alpha = 0.3 / 0.9
+    r = tree_accept_sample_ref(logits, 1.0, q2, token, parent, depth, 3, 1, np.array([0.0, 0.9, 0.5]), 0.3)
+    assert r["accept_len"] == 1 and r["path"][1] == 2 and r["out_tokens"][0] == 0
