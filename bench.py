@@ -596,6 +596,10 @@ def bench_jet(args):
                                      (local_rank, gpu_uuid)))
         sweep.append(sweep_point("batched_paged", dict(CONFIGS["batched_paged"]), rank_seed(6, rank), device, 3,
                                  (local_rank, gpu_uuid)))
+        # the draft head's own block-causal attention: a chain of 16 rows (one per draft depth, width 1) over the
+        # same context length, at the head's shape; timed over 36 distinct KV buffers so every launch is cold
+        sweep.append(sweep_point("draft_head_block16", dict(base, B=16, N=15, W=1), rank_seed(7, rank), device, 3,
+                                 (local_rank, gpu_uuid)))
 
     cpu = cpu_baseline(st, c, info) if not args.no_cpu_baseline else None
 

@@ -132,6 +132,37 @@ def test_moe_30b_batch_8_with_per_sequence_node_counts(B):
         assert (out[b, n:] == 0).all() and np.isneginf(lse[b][:, n:]).all()
 
 
+@pytest.mark.parametrize("L", [0, 37, 512, 4096])
+@pytest.mark.parametrize("rows", [16, 9])
+def test_draft_head_block_causal_shape(L, rows):
+    """The draft head's own attention (Section 3.2, training details of the appendix): a block of up to 16 rows,
+    one per draft depth, each attending to the context (the injected target features of the prefix) and to the
+    earlier rows of its block -- a chain-shaped tree of 16 nodes at the head's shape (32 / 8 heads, head_dim 128),
+    with no, a short and a long context.  Full comparison with the oracle."""
+    import jet_harness as H
+    from jet_inputs import chain_tree
+    from oracle import tree_attn_ref
+    B, Hq, Hkv, D = 16, 32, 8, 128
+    rng = np.random.default_rng(7600 + L + rows)
+    x = make_attn_inputs(rng, B, Hq, Hkv, D, L)
+    parent, _, _ = chain_tree(rows)
+    anc = anc_from_parent(parent, rows, B)
+    scale = 1.0 / np.sqrt(D)
+    ref, rlse = tree_attn_ref(x["q"], x["k_prefix"], x["v_prefix"], x["tree_k"], x["tree_v"], anc, rows, scale)
+    kc = x["k_prefix"][None] if L else None
+    vc = x["v_prefix"][None] if L else None
+    for flags in (0, 1):
+        out, lse, st = H.run_tree_attn(x["q"][None], kc, vc, None, [L], x["tree_k"][None], x["tree_v"][None],
+                                       anc[None], [rows], scale, max_seq_len=L, flags=flags)
+        assert st == 0 and not np.isnan(out).any()
+        err = np.abs(out[0] - ref)[:rows]
+        assert err.max() <= MAX_ERR and err.mean() <= MEAN_ERR, (err.max(), err.mean())
+        if L >= 4096:
+            assert err.max() <= TIGHT_MAX and err.mean() <= TIGHT_MEAN
+        assert (out[0, rows:] == 0).all()
+        assert np.abs(lse[0][:, :rows] - rlse[:, :rows]).max() <= LSE_ERR
+
+
 def _trees(rng, batch, N, W, B, V):
     trees = [tree_build_ref(make_logp(rng, N, V, 3.0, peaked_p=0.7), 1 + b, N, W, B) for b in range(batch)]
     stack = lambda k: np.stack([t[k] for t in trees])
