@@ -620,7 +620,7 @@ def bench_jet(args):
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,
                 "note": "all inputs come from pinned host memory every step; the target logits are copied on a second "
                         "stream while the tree is built and attended, the acceptance waits for them"},
-        "gpu_launches": args.steps * st.launches_per_step(1),
+        "gpu_launches": args.steps * st.launches_per_step(),
         "clocks": clocks, "roofline": roof,
     }
     if sustained is not None:

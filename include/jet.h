@@ -223,13 +223,25 @@ JET_API jet_status jet_tree_build_logits(const float* logits, int64_t logits_bat
  * time through another stream, MPS or a green context).  If some CTAs cannot
  * start until others finish, the waiting ones give up after about a second with
  * JET_ERR_TIMEOUT instead of hanging.
+ * (For shapes with few query rows per KV head -- one 128-row query tile, e.g.
+ * up to 32 nodes at 4 query heads per KV head -- the slices only WRITE their rows
+ * in the first launch and a second, small launch combines them: then nothing
+ * waits inside a kernel, the counters are unused and the residency assumption
+ * falls away; jet_tree_verify_attn_launches tells which form a shape gets.
+ * JET_FORCE_SPLIT="<slices>,g" / ",h" selects the one- / two-launch form.)
  * Test hooks, read from the environment once per process and meant for the
  * test-suite only: JET_FORCE_MT / JET_FORCE_SPLIT force a launch plan (query
- * tiles per CTA; key slices, with ",g" through the workspace),
+ * tiles per CTA; key slices, with ",g" / ",h" through the workspace in one / two launches),
  * JET_TEST_POLL_LIMIT shortens the bounded wait of the workspace exchange.
  */
 JET_API size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                             int max_seq_len);
+
+/* Kernel launches one attention call of this shape enqueues: 1, or 2 when the key range of a work item is cut
+ * into slices whose partial rows a second, small kernel combines (0 for an invalid shape).  For callers that
+ * count launches (CUDA-graph sizing, launch statistics); same arguments as the workspace query.
+ */
+JET_API int jet_tree_verify_attn_launches(int batch, int B, int Hq, int Hkv, int D, int max_seq_len);
 
 JET_API jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
                                 const int32_t* page_table, int max_pages_per_seq, int page_size,

@@ -30,6 +30,7 @@ from .binding import (  # noqa: F401
     jet_tree_build_workspace_bytes,
     jet_tree_verify_attn,
     jet_tree_verify_attn_ex,
+    jet_tree_verify_attn_launches,
     jet_tree_verify_attn_tail,
     jet_tree_verify_attn_tail_ex,
     jet_tree_verify_attn_workspace_bytes,

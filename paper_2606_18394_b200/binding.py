@@ -38,6 +38,7 @@ _SIGNATURES = {
     "jet_tree_build_logits": (_c.c_int32, [_vp, _i64, _i64, _vp, _i, _i, _i, _i, _i, _vp, _i, _f, _vp, _vp, _vp, _vp,
                                            _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_tree_verify_attn_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "jet_tree_verify_attn_launches": (_i, [_i, _i, _i, _i, _i, _i]),
     "jet_tree_verify_attn": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp,
                                           _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_tree_verify_attn_tail": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp,
@@ -179,6 +180,10 @@ def jet_tree_build_logits(logits, root_token, batch, N, V, W, B, score_mode, alp
 
 def jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len) -> int:
     return load().jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len)
+
+
+def jet_tree_verify_attn_launches(batch, B, Hq, Hkv, D, max_seq_len) -> int:
+    return load().jet_tree_verify_attn_launches(batch, B, Hq, Hkv, D, max_seq_len)
 
 
 def jet_tree_verify_attn(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len,

@@ -76,7 +76,8 @@ struct AttnParams {
   int len_hint;       // the caller's bound on the cached keys (max_seq_len); 0 = none
   uint32_t poll_limit;  // workspace merge: polls of the arrival count before the CTA gives up (about a second)
   int stable;         // JET_ATTN_STABLE_PREFIX: lengths, page table and prefix rows may be read before the dependency wait
-  int via_global;     // key slices exchange their rows through the workspace instead of a cluster
+  int via_global;     // key slices exchange their rows through the workspace instead of a cluster: 1 = inside this
+                      // launch (arrival counters, bounded spin), 2 = a second launch combines them
   int* counters;      // via_global: [2][units * MT] arrival / departure counts, zero between calls
   uint8_t* partials;  // via_global: [units * nsplit * MT][128 rows][D bf16 + log2-sum-exp (fp32) + pad]
   float scale_log2;   // softmax_scale * log2(e)
@@ -674,6 +675,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           uint4* dst4 = reinterpret_cast<uint4*>(slots + (static_cast<size_t>(split) * MT + mt) * kBlockBytes);
           for (int i = tid; i < static_cast<int>(kBlockBytes / 16); i += C::kThreads) __stcg(dst4 + i, src4[i]);
         }
+        // Two launches: this one ends here; the merge kernel that follows it in the stream starts when every
+        // CTA of this launch has exited, i.e. when every block is in place -- no counter, no spin, and no need
+        // for the slices to be resident together.
+        if (p.via_global == 2) continue;
         ptx::cta_sync();
         if (!kSm && tid == 0) {
           // the last slice to arrive knows from its own count that everybody has published
@@ -1564,6 +1569,88 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
 }
 
+// ------------------------------------------------------------------------------------------ merge kernel
+// Second launch of the two-launch slice merge: every key slice of a work item has left its 128 normalised rows
+// (D bf16 values + log2-sum-exp, fp32) in the workspace; one thread combines 8 output values of one row over the
+// S slices with softmax weights of the slice sums and writes them (bf16), the first thread of a row also its
+// log-sum-exp.  All loads of a thread are independent of each other: one round trip to L2.
+struct MergeParams {
+  const uint8_t* partials;
+  const int32_t* n_nodes;
+  __nv_bfloat16* out;
+  float* lse;
+  int B, Hq, Hkv, G, S, MT, n_mgroups, npt;
+  uint32_t magic_G;
+};
+
+template <int D>
+__global__ void __launch_bounds__(256) tree_attn_merge_kernel(const MergeParams p) {
+  constexpr int kPitch = D * 2 + 16;
+  constexpr int kItemsPerRow = D / 8;
+  constexpr int kRowsPerCta = 256 / kItemsPerRow;
+  constexpr int kBlocksPerTile = kBM / kRowsPerCta;
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
+  int bx = static_cast<int>(blockIdx.x);
+  const int rb = bx % kBlocksPerTile;
+  bx /= kBlocksPerTile;
+  const int mt = bx % p.MT, mgroup = bx / p.MT;
+  const int g = blockIdx.y, b = blockIdx.z;
+  const int row = rb * kRowsPerCta + static_cast<int>(threadIdx.x) / kItemsPerRow;
+  const int c8 = static_cast<int>(threadIdx.x) % kItemsPerRow;
+  const int R = mt * kBM + row;                              // row within the work item
+  const int vq = static_cast<int>(udiv(R, p.magic_G));
+  const int v = mgroup * p.MT * p.npt + vq, h = g * p.G + (R - vq * p.G);
+  if (v >= p.B) return;
+  const int n = min(p.n_nodes[b], p.B);
+  const int unit = (b * p.Hkv + g) * p.n_mgroups + mgroup;
+  const int S = p.S;
+  const size_t stride = static_cast<size_t>(p.MT) * kBM * kPitch;       // distance between consecutive slices
+  const uint8_t* row0 = p.partials + (static_cast<size_t>(unit) * S * p.MT + mt) * (static_cast<size_t>(kBM) * kPitch) +
+                        static_cast<size_t>(row) * kPitch;
+  // every load of the thread is issued before any is used (the slots are valid memory for any row)
+  float lc[kMaxSplit];
+  uint4 x[kMaxSplit];
+#pragma unroll
+  for (int c = 0; c < kMaxSplit; ++c) {
+    if (c < S) {
+      lc[c] = __ldcg(reinterpret_cast<const float*>(row0 + c * stride + D * 2));
+      x[c] = __ldcg(reinterpret_cast<const uint4*>(row0 + c * stride + c8 * 16));
+    } else {
+      lc[c] = -INFINITY;
+      x[c] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  float lse2 = -INFINITY;
+  float mx = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < kMaxSplit; ++c) mx = fmaxf(mx, lc[c]);
+  if (v < n && mx > -INFINITY) {
+    float wsum = 0.0f;
+#pragma unroll
+    for (int c = 0; c < kMaxSplit; ++c) {
+      const float w = lc[c] > -INFINITY ? exp2f(lc[c] - mx) : 0.0f;       // absent slices get weight 0 ...
+      wsum += w;
+      const uint32_t v4[4] = {x[c].x, x[c].y, x[c].z, x[c].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
+        const float lo = __uint_as_float(v4[q] << 16), hi = __uint_as_float(v4[q] & 0xFFFF0000u);
+        acc[2 * q] += w > 0.0f ? w * lo : 0.0f;                          // ... and whatever they hold is not used
+        acc[2 * q + 1] += w > 0.0f ? w * hi : 0.0f;
+      }
+    }
+    const float inv = 1.0f / wsum;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] *= inv;
+    lse2 = mx + log2f(wsum);
+  }
+  *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
+      make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
+                 pack_bf16(acc[6], acc[7]));
+  if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
+}
+
 // ------------------------------------------------------------------------------------------ host
 using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1708,7 +1795,11 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   // "slices,g" (g = merge through the workspace); a forced choice the device cannot hold is ignored.
   static const int force_mt = [] { const char* e = getenv("JET_FORCE_MT"); return e ? atoi(e) : 0; }();
   static const int force_ns = [] { const char* e = getenv("JET_FORCE_SPLIT"); return e ? atoi(e) : 0; }();
-  static const int force_via = [] { const char* e = getenv("JET_FORCE_SPLIT"); return (e && strstr(e, ",g")) ? 1 : 0; }();
+  // ",g": exchange inside the launch (counters and a bounded spin); ",h": exchange finished by a second launch
+  static const int force_via = [] {
+    const char* e = getenv("JET_FORCE_SPLIT");
+    return (e && strstr(e, ",g")) ? 1 : ((e && strstr(e, ",h")) ? 2 : 0);
+  }();
   for (int mt = 1; mt <= (rows > kBM ? 2 : 1); ++mt) {
     if (force_mt && mt != force_mt && !(force_mt == 2 && rows <= kBM)) continue;
     Plan pl;
@@ -1734,9 +1825,15 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
       if (resident > 0) consider(ns, 0, static_cast<double>((pl.units + resident - 1) / resident), ns == 1 ? 6.0 : 8.0);
       // (b) independent CTAs that merge through the workspace: all of them must be resident at once
       //     (a cluster has to fit into one GPC, which can leave a third of the SMs idle)
+      //     -- either inside the launch (arrival counters, bounded spin), or with a second small launch that
+      //     combines the blocks once the first has ended (nothing waits inside a kernel)
       if (ns > 1 && static_cast<long>(pl.units) * ns <= sm_count() &&
-          static_cast<size_t>(pl.units) * mt * 2 * sizeof(int) <= kCounterBytes)
-        consider(ns, 1, 1.0, 10.0);
+          static_cast<size_t>(pl.units) * mt * 2 * sizeof(int) <= kCounterBytes) {
+        // measured (Qwen3-8B layer shape, prefix 4096 / 16384): with one query tile per KV head (few rows, many
+        // slices) the two-launch form is 1-3 % faster, with more query tiles the single launch is (2.6 % at 64 nodes)
+        const int via = force_via ? force_via : (pl.n_mgroups == 1 ? 2 : 1);
+        consider(ns, via, 1.0, 10.0);
+      }
     }
   }
   if (best_cost < 0.0) {        // the occupancy query failed: plain launch without slices
@@ -1785,6 +1882,17 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
     cudaGetLastError();
     return JET_ERR_CUDA;
   }
+  if (pl.via_global == 2) {
+    MergeParams m;
+    m.partials = p.partials;
+    m.n_nodes = p.n_nodes;
+    m.out = p.out;
+    m.lse = p.lse;
+    m.B = p.B; m.Hq = p.Hq; m.Hkv = p.Hkv; m.G = p.G; m.S = pl.nsplit; m.MT = MT; m.n_mgroups = pl.n_mgroups; m.npt = p.npt;
+    m.magic_G = p.magic_G;
+    constexpr int kRowsPerCta = 256 / (D / 8);
+    launch_dependent(tree_attn_merge_kernel<D>, dim3((kBM / kRowsPerCta) * MT * pl.n_mgroups, p.Hkv, p.batch), dim3(256), st, m);
+  }
   return launch_status();
 }
 
@@ -1818,6 +1926,13 @@ extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq,
       (D != 64 && D != 128))
     return 0;
   return jet::workspace_need(jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len), D);
+}
+
+extern "C" int jet_tree_verify_attn_launches(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
+  if (batch < 1 || batch > 65535 || B < 1 || Hq < 1 || Hkv < 1 || Hkv > 65535 || Hq % Hkv != 0 || max_seq_len < 0 ||
+      (D != 64 && D != 128))
+    return 0;
+  return jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len).via_global == 2 ? 2 : 1;
 }
 
 namespace jet {

@@ -209,5 +209,8 @@ class VerifyStep:
 
     LAUNCHES_PER_STEP_FIXED = 6      # tree_build 2, tree_accept 2, kv_compact 2
 
-    def launches_per_step(self, attn_launches_per_layer):
+    def launches_per_step(self, attn_launches_per_layer=None):
+        if attn_launches_per_layer is None:       # what the library says one attention call of this shape enqueues
+            attn_launches_per_layer = jet.jet_tree_verify_attn_launches(self.batch, self.B, self.Hq, self.Hkv, self.D,
+                                                                        self.attn_max_len)
         return self.LAUNCHES_PER_STEP_FIXED + (1 if self.draft_logits else 0) + self.layers * attn_launches_per_layer

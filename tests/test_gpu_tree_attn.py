@@ -234,7 +234,8 @@ def test_rows_without_a_key_in_their_first_tile_and_very_negative_scores():
     assert np.abs(got_lse - rlse).max() <= 1e-3 * np.abs(rlse).max()
 
 
-@pytest.mark.parametrize("mt,force", [("1", "2"), ("1", "2,g"), ("1", "4"), ("2", "1"), ("2", "2"), ("2", "4,g")])
+@pytest.mark.parametrize("mt,force", [("1", "2"), ("1", "2,g"), ("1", "2,h"), ("1", "4"), ("2", "1"), ("2", "2"),
+                                      ("2", "4,g"), ("2", "4,h")])
 def test_adversarial_scores_under_forced_slicings(mt, force):
     """The launch plan decides where the key slices begin, and with it which rows meet an empty first tile.  The
     library reads JET_FORCE_MT / JET_FORCE_SPLIT once per process, so the adversarial-score tests run again in
@@ -272,10 +273,12 @@ def test_small_budgets_at_the_full_prefix(B):
 
 
 @pytest.mark.parametrize("mt,split", [("1", "1"), ("1", "3"), ("1", "6"), ("1", "9,g"), ("1", "16,g"), ("1", "18,g"),
-                                      ("2", "1"), ("2", "2"), ("2", "4,g")])
+                                      ("1", "9,h"), ("1", "4,h"), ("1", "18,h"), ("2", "1"), ("2", "2"), ("2", "4,g"),
+                                      ("2", "4,h")])
 def test_every_kind_of_launch_plan(mt, split):
     """The planner picks one plan per shape; the others (query tiles per CTA, number of key slices, merge through
-    a cluster or through the workspace) must compute the same thing.  Runs the benchmark-shape test, the tile
+    a cluster, through the workspace inside the launch (",g") or through the workspace with a second launch
+    (",h")) must compute the same thing.  Runs the benchmark-shape test, the tile
     boundary tests and the tree-shape tests in a child process under a forced plan (a forced plan the device
     cannot hold is ignored by the library, i.e. falls back to the planner's)."""
     import os
