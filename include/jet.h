@@ -18,6 +18,7 @@
  *   jet_tree_verify_attn_ex, jet_tree_verify_attn_tail_ex   the same with a flags word
  *   jet_kv_compact_tail        in-place commit for that layout
  *   jet_tree_accept_static     greedy acceptance on scratch built into the library
+ *   jet_tree_accept_hidden     greedy acceptance from the final hidden states (LM head inside, arg-max only)
  *   jet_tree_accept_sample     non-greedy (min(1, p/q)) acceptance with a correction draw
  *
  * Conventions shared by every call
@@ -342,6 +343,39 @@ JET_API jet_status jet_tree_accept(const float* logits, int64_t logits_row_strid
                            int32_t* tgt_argmax, int32_t* accept_len, int32_t* path,
                            int32_t* out_tokens, void* workspace, size_t workspace_bytes,
                            void* stream);
+
+/* ---------------------------------------------------------------------------
+ * jet_tree_accept_hidden -- greedy acceptance (Section 3.3, Appendix E: "the target
+ * model's greedy prediction" at every node) straight from the target's FINAL HIDDEN
+ * STATES: the LM head is applied inside the call and only the arg-max of every row
+ * is kept, so the [batch*B, V] logits are neither written nor read.
+ *
+ *   logit[r, t] = sum_k hidden[r, k] * lm_head_weight[t, k]   bf16 operands, fp32
+ *                 accumulation (tensor cores, accumulation order unspecified);
+ *   tgt_argmax[r] = arg max_t logit[r, t], ties -> lowest t, -0.0 == +0.0;
+ * then exactly jet_tree_accept's path selection.  Because the sums are formed in
+ * fp32 in an unspecified order, two tokens whose exact logits differ by less than
+ * the rounding of a K-term fp32 sum (about K * 2^-24 * sum_k |hidden * weight|) may
+ * come out in either order; everything else matches an exact evaluation.
+ *
+ *   hidden          bf16 [batch*B, d], rows contiguous (row r = sequence r / B, node r % B);
+ *                   rows of padding nodes may hold anything
+ *   lm_head_weight  bf16 [V, d], rows contiguous (the usual [vocab, hidden] layout)
+ *   d               hidden size, a multiple of 64
+ *   every other argument as for jet_tree_accept; device_status as for the attention call
+ * Cost: one pass over the weights (V * d * 2 bytes from HBM) for up to 512 rows; more
+ * rows stream them once per group of 512.
+ * Workspace: jet_tree_accept_hidden_workspace_bytes (one 64-bit key per row; need not
+ * be initialised).
+ */
+JET_API size_t jet_tree_accept_hidden_workspace_bytes(int batch, int B);
+
+JET_API jet_status jet_tree_accept_hidden(const void* hidden, const void* lm_head_weight, int d,
+                                  const int32_t* token, const int32_t* parent, const int32_t* depth,
+                                  const uint32_t* anc_mask, const int32_t* n_nodes, int batch, int B,
+                                  int V, int N, int32_t* tgt_argmax, int32_t* accept_len, int32_t* path,
+                                  int32_t* out_tokens, int32_t* device_status, void* workspace,
+                                  size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
  * jet_tree_accept_static -- the same operation as jet_tree_accept for callers that cannot

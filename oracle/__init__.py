@@ -13,6 +13,7 @@ from .jet_oracle import (  # noqa: F401
     gather_paged_prefix,
     kv_compact_ref,
     kv_compact_tail_ref,
+    lm_head_argmax_ref,
     log_softmax_ref,
     target_probs_ref,
     tree_accept_ref,

@@ -22,6 +22,8 @@ Each function follows one passage of the paper:
   K/V rows of the accepted path are copied behind the prefix;
   ``kv_compact_tail_ref`` is the same commit for a cache that already holds the
   tree's rows behind the prefix (the serving layout of Appendix E).
+* ``lm_head_argmax_ref`` -- that greedy prediction taken from the target's final hidden
+  states (logit = hidden . LM-head row, arg-max per row, ties to the lowest id).
 * ``tree_accept_sample_ref`` -- the non-greedy acceptance rule of Section 3.3
   (Eq. nongreedy_specdec): along every branch a draft token is accepted with
   probability min(1, p/q); a correction token is sampled from the target where
@@ -59,7 +61,9 @@ with no counterpart to check against: parity unpinned for that reading only.  ``
 scipy's log_softmax, closed forms (uniform, two-point), rows summing to one and
 shift invariance; the two helpers ``bf16_bits_to_f64`` (fixed bit patterns whose values the bfloat16
 format itself gives) and ``gather_paged_prefix`` (a cache whose rows hold their own page and offset)
-have pins of their own; ``tree_build_logits_ref`` by the invariance of the tree under
+have pins of their own; ``lm_head_argmax_ref`` is pinned by brute-force integer sums on small
+integer-valued inputs (every product and sum exact), one-hot hidden states that select a weight column,
+ties to the lowest id and the sign flip that turns the arg-max into the arg-min; ``tree_build_logits_ref`` by the invariance of the tree under
 a per-row shift of the logits and by agreement with ``tree_build_ref`` on
 log-probabilities that scipy computed.
 """
@@ -91,6 +95,24 @@ def gather_paged_prefix(cache: np.ndarray, page_table_row: np.ndarray, L: int) -
     if not rows:
         return np.zeros((0,) + cache.shape[2:], dtype=cache.dtype)
     return np.stack(rows, axis=0)
+
+
+# --------------------------------------------------------------------------
+# O0  target prediction from hidden states (Section 3.3 / Appendix E: "the target model's greedy prediction")
+# --------------------------------------------------------------------------
+def lm_head_argmax_ref(hidden, weight):
+    """The target's greedy prediction of every row from its final hidden state.
+
+    ``hidden`` [R, d] and ``weight`` [V, d] are bfloat16 bit patterns (uint16) or numbers; they are widened
+    exactly to float64 and logit[r, t] = sum_k hidden[r, k] * weight[t, k] is formed in float64 (a library
+    matrix product).  Returns a dict: ``logits`` [R, V] float64; ``tgt`` [R] = arg-max per row, ties to the
+    lowest token id; ``abs_dot`` [R, V] = sum_k |hidden[r, k] * weight[t, k]|, the scale of the rounding error
+    that a K-term fp32 evaluation of the same sum may make (about K * 2**-24 of it), which the GPU parity test
+    uses to tell a genuine disagreement from two tokens whose exact logits are closer than that."""
+    h = bf16_bits_to_f64(hidden)
+    w = bf16_bits_to_f64(weight)
+    logits = h @ w.T
+    return dict(logits=logits, tgt=np.argmax(logits, axis=1).astype(np.int32), abs_dot=np.abs(h) @ np.abs(w).T)
 
 
 # --------------------------------------------------------------------------

@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     jet_kv_compact,
     jet_kv_compact_tail,
     jet_tree_accept,
+    jet_tree_accept_hidden,
+    jet_tree_accept_hidden_workspace_bytes,
     jet_tree_accept_sample,
     jet_tree_accept_sample_workspace_bytes,
     jet_tree_accept_static,

@@ -54,6 +54,9 @@ _SIGNATURES = {
     "jet_tree_accept_workspace_bytes": (_sz, [_i, _i, _i]),
     "jet_tree_accept": (_c.c_int32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp,
                                      _vp, _vp, _sz, _vp]),
+    "jet_tree_accept_hidden_workspace_bytes": (_sz, [_i, _i]),
+    "jet_tree_accept_hidden": (_c.c_int32, [_vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp,
+                                            _vp, _vp, _sz, _vp]),
     "jet_tree_accept_static": (_c.c_int32, [_vp, _i64, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp,
                                             _vp, _vp]),
     "jet_tree_accept_sample_workspace_bytes": (_sz, [_i, _i, _i]),
@@ -274,6 +277,24 @@ def jet_tree_accept(logits, logits_row_stride, token, parent, depth, anc_mask, n
                                 _p(out_tokens), _p(workspace), wb, _stream(stream))
     if check:
         _check(st, "jet_tree_accept")
+    return st
+
+
+def jet_tree_accept_hidden_workspace_bytes(batch, B) -> int:
+    return load().jet_tree_accept_hidden_workspace_bytes(batch, B)
+
+
+def jet_tree_accept_hidden(hidden, lm_head_weight, d, token, parent, depth, anc_mask, n_nodes, batch, B, V, N,
+                           tgt_argmax, accept_len, path, out_tokens, device_status, workspace, workspace_bytes=None,
+                           stream=None, check=True):
+    """Greedy acceptance from the final hidden states: the LM head runs inside the call, only arg-maxima are kept."""
+    wb = workspace_bytes if workspace_bytes is not None else (workspace.numel() * workspace.element_size()
+                                                              if workspace is not None else 0)
+    st = load().jet_tree_accept_hidden(_p(hidden), _p(lm_head_weight), d, _p(token), _p(parent), _p(depth),
+                                       _p(anc_mask), _p(n_nodes), batch, B, V, N, _p(tgt_argmax), _p(accept_len),
+                                       _p(path), _p(out_tokens), _p(device_status), _p(workspace), wb, _stream(stream))
+    if check:
+        _check(st, "jet_tree_accept_hidden")
     return st
 
 
