@@ -420,6 +420,77 @@ def sweep_point(name, c, seed, device, steps, sampler_args, layers=None):
     return point
 
 
+def lm_head_point(c, seed, device, sampler_args, d_model=4096):
+    """jet_tree_accept_hidden at the workload's shape: the LM head applied inside the acceptance call, only the
+    per-row arg-max kept (no [rows, V] logits in memory).  A weight stream: V * d * 2 bytes from HBM per call;
+    several weight copies are cycled so that no call finds its weights in L2."""
+    import torch
+    import paper_2606_18394_b200 as jet
+    batch, B, N, V = c["batch"], c["B"], c["N"], c["V"]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    rows = batch * B
+    hidden = torch.randn((rows, d_model), generator=gen, device=device, dtype=torch.float32).bfloat16()
+    copies = 3
+    weights = [(torch.randn((V, d_model), generator=gen, device=device, dtype=torch.float32) * 0.02).bfloat16()
+               for _ in range(copies)]
+    i32 = lambda *shape: torch.zeros(shape, dtype=torch.int32, device=device)
+    token, parent, depth = i32(batch, B), i32(batch, B), i32(batch, B)
+    parent[:, 0] = -1                                   # a star: every node hangs off the root
+    depth[:, 1:] = 1
+    anc = i32(batch, B, (B + 31) // 32)
+    anc[:, :, 0] = 1
+    for v in range(1, B):
+        anc[:, v, v // 32] |= (1 << (v % 32)) if v % 32 != 31 else -(1 << 31)
+    n_nodes = torch.full((batch,), B, dtype=torch.int32, device=device)
+    tgt, acc, path, toks, status = i32(batch, B), i32(batch), i32(batch, N + 1), i32(batch, N + 1), i32(1)
+    ws = torch.empty(max(jet.jet_tree_accept_hidden_workspace_bytes(batch, B), 256), dtype=torch.uint8, device=device)
+
+    def call(w):
+        jet.jet_tree_accept_hidden(hidden, w, d_model, token, parent, depth, anc, n_nodes, batch, B, V, N, tgt, acc, path,
+                                   toks, status, ws)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        for w in weights:
+            call(w)
+        stream.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            for w in weights:
+                call(w)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(3):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        reps = max(3, int(MIN_TIMED_SECONDS / max(e0.elapsed_time(e1) * 1e-3 / 3, 1e-6)) + 1)
+        sampler = ClockSampler(*sampler_args)
+        sampler.start()
+        e0.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, "a bounded device wait expired"
+    us = e0.elapsed_time(e1) * 1e3 / (reps * copies)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peaks, src = (json.load(open(peaks_path)), "measured") if os.path.exists(peaks_path) else ({"hbm_gbs": 6650.0}, "fallback")
+    bytes_alg = V * d_model * 2 + rows * d_model * 2 + rows * 4
+    traffic, note = ncu_traffic("lm_head_accept", bytes_alg)
+    roof = {"bound": "hbm", "achieved": bytes_alg / (us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "kernel": "lm_head_argmax_kernel", "peak_source": src, "us_per_launch": us, "algorithmic_bytes": bytes_alg,
+            "algorithmic_flops": 2 * rows * d_model * V, "traffic": traffic, "traffic_note": note,
+            "timing": f"CUDA events around {reps} replays of a graph of {copies} calls (memset + GEMM/arg-max + path kernel each)"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    del weights
+    torch.cuda.empty_cache()
+    return {"workload": "lm_head_accept", "rows": rows, "hidden_size": d_model, "vocab": V, "us_per_call": us,
+            "launches": reps * copies * 2, "clocks": clocks, "roofline": roof,
+            "note": "replaces jet_tree_accept's scan of fp32 logits when the caller hands over hidden states instead"}
+
+
 def bench_jet(args):
     import torch
     import torch.distributed as dist
@@ -600,6 +671,7 @@ def bench_jet(args):
         # same context length, at the head's shape; timed over 36 distinct KV buffers so every launch is cold
         sweep.append(sweep_point("draft_head_block16", dict(base, B=16, N=15, W=1), rank_seed(7, rank), device, 3,
                                  (local_rank, gpu_uuid)))
+        sweep.append(lm_head_point(c, rank_seed(8, rank), device, (local_rank, gpu_uuid)))
 
     cpu = cpu_baseline(st, c, info) if not args.no_cpu_baseline else None
 
