@@ -403,7 +403,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // The barriers of every CTA of the cluster must exist before any CTA arrives on them remotely:
   // arrive on the hardware cluster barrier now, wait for it only when the slices are merged.
   const bool via_cluster = S > 1 && !p.via_global;
-  if (via_cluster) ptx::cluster_arrive();
   const uint32_t tmem_base = *tmem_slot;
   if (tid == 0) JET_TR(42);
   // Inputs may be written by the preceding kernel of the stream: nothing in global memory is touched before
@@ -515,15 +514,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int e_r = (tid - 128) & 127;                           // its row within the query tile
     uint8_t* stage = smem_gen + C::kStageOff;
     bool merge_ok = true;
-    if (via_cluster) {
-      __syncwarp();
-      ptx::cluster_wait();     // pairs with cluster_arrive above: every CTA's barriers are initialised
-      // A: every CTA of the cluster has left its key loop, so its tile memory may be overwritten
-      merge_ok = cluster_rendezvous(bar(Bars::kClusterA), S, abort_flag, 12);
-      if (tid == 128) JET_TR(7);
-    } else {
-      ptx::cta_sync();
-    }
+    ptx::cta_sync();
     // Staging of a row: normalised, D bf16 values followed by the row's log2-sum-exp (fp32).  Rows this CTA
     // computed nothing for (empty key slice, tile without nodes) get log2-sum-exp = -inf ("absent").
     const uint32_t e_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
@@ -540,8 +531,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int mt = 0; mt < n_mt; ++mt) {      // n_mt is the same in every CTA of the cluster
       if (mt > 0) {
         // C: everybody has combined the previous tile's rows, so both buffers are free again
-        if (via_cluster) merge_ok = cluster_rendezvous(bar(Bars::kClusterC), S, abort_flag, 13) && merge_ok;
-        else ptx::cta_sync();
+        if (via_cluster) {
+          __syncwarp();
+          ptx::cluster_sync_all();
+        } else {
+          ptx::cta_sync();
+        }
       }
       if constexpr (MT == 1) {
         // Both warpgroups stage half of every row (64 columns each), folding the two streams' accumulators
@@ -637,30 +632,48 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         *reinterpret_cast<float*>(dst + D * 2) = own_lse2;
       }
-      if (via_cluster) ptx::fence_proxy_async_smem();
-      ptx::cta_sync();
-      const uint8_t* src_rows = stage;         // S == 1: the staged rows themselves
-      bool rows_ok = merge_ok;
       if (via_cluster) {
-        if (!kSm && tid < S && merge_ok) {
-          const int dst_lo = tid * rows_per;
-          const int dst_n = max(0, min(rows_per, kBM - dst_lo));
-          if (dst_n > 0)
-            ptx::bulk_copy_to_cluster(
-                ptx::map_to_rank(smem_base + C::kRecvOff + static_cast<uint32_t>(split * rows_per * C::kRecvPitch), tid),
-                smem_base + C::kStageOff + static_cast<uint32_t>(dst_lo * C::kRecvPitch),
-                static_cast<uint32_t>(dst_n * C::kRecvPitch), ptx::map_to_rank(bar(Bars::kRecv + mt), tid));
-        }
+        // The slices of the work item form a thread-block cluster: once every CTA has staged its rows (the
+        // hardware cluster barrier, release / acquire, makes them visible cluster-wide), each CTA PULLS its own
+        // block of rows out of every slice's shared memory into a buffer of its own -- all loads of a thread in
+        // flight at once, one round trip over the SM-to-SM network -- and combines the copies.  No remote
+        // writes, no arrival counters; a CTA must only not exit (or restage) before its peers have read it:
+        // the cluster barriers behind the loop.  (The first version pushed the blocks with bulk copies credited
+        // to the owners' mbarriers behind a cluster-wide rendezvous; the pull is 1 - 3 us per launch faster.)
+        __syncwarp();
+        ptx::cluster_sync_all();
         if (tid == 128 && mt == 0) JET_TR(8);
-        // all blocks of this CTA's rows have arrived (always waited for, so that the CTA never exits
-        // while copies into its memory are in flight)
-        rows_ok = bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14) && merge_ok;
+        if constexpr (kSm) {
+          // gather: 16-byte chunk e of this CTA's row block, from slice c, for every (e, c) pair of the thread --
+          // at most 16 pairs (fewer slices mean more rows per CTA and the other way round)
+          constexpr int kChunksPerRow = C::kRecvPitch / 16;
+          const int per_slice = own_n * kChunksPerRow;
+          const int pairs = ((per_slice + 255) / 256) * S;
+          const uint32_t local = smem_base + C::kStageOff + static_cast<uint32_t>(own_lo * C::kRecvPitch);
+          uint8_t* recv = smem_gen + C::kRecvOff;
+          uint4 got[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            const int j = static_cast<int>(udiv(static_cast<uint32_t>(q), p.magic_S)), c = q - j * S;
+            const int e = tid - 128 + 256 * j;
+            if (q < pairs && e < per_slice) got[q] = ptx::ld_cluster_v4(ptx::map_to_rank(local + static_cast<uint32_t>(e * 16), c));
+          }
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            const int j = static_cast<int>(udiv(static_cast<uint32_t>(q), p.magic_S)), c = q - j * S;
+            const int e = tid - 128 + 256 * j;
+            if (q < pairs && e < per_slice)
+              *reinterpret_cast<uint4*>(recv + static_cast<size_t>(c) * rows_per * C::kRecvPitch + e * 16) = got[q];
+          }
+          ptx::named_sync(2, 256);
+        }
         if (tid == 128 && mt == 0) JET_TR(9);
-        src_rows = smem_gen + C::kRecvOff;
-        // This CTA's own bulk copies read its staged rows asynchronously: it may only exit once every
-        // peer has received them.  Arrive on the hardware cluster barrier now, wait for it at the end.
-        if (mt == n_mt - 1) ptx::cluster_arrive();
-      } else if (S > 1) {
+      } else {
+        ptx::cta_sync();
+      }
+      const uint8_t* src_rows = via_cluster ? smem_gen + C::kRecvOff : stage;         // S == 1: the staged rows themselves
+      bool rows_ok = merge_ok;
+      if (S > 1 && !via_cluster) {
         // Exchange through the workspace: publish this CTA's staged rows, count the slices of the unit
         // that have published (bounded spin), then fetch this CTA's block of rows from every slice.
         constexpr uint32_t kBlockBytes = kBM * C::kRecvPitch;
@@ -1545,7 +1558,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (tid == 128) JET_TR(12);
   if (via_cluster) {
     __syncwarp();
-    ptx::cluster_wait();     // every CTA of the cluster has received all of its blocks
+    ptx::cluster_sync_all();     // every CTA of the cluster has read this CTA's staged rows
   }
   ptx::tc_fence_before();
   ptx::cta_sync();
