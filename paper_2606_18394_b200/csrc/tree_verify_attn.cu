@@ -1822,9 +1822,10 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
     const double shared = 1.0 + 0.75 / pl.n_mgroups;
     const double tile_cost = mt == 1 ? shared : (shared > 2.2 ? shared : 2.2);
     const double fixed_scale = mt == 1 ? 1.0 : 1.6;
-    auto consider = [&](int ns, int via_global, double waves, double fixed) {
+    auto consider = [&](int ns, int via_global, double waves, double fixed, double given_cost = -1.0) {
       if (force_ns && (ns != force_ns || (ns > 1 && via_global != force_via))) return;
-      const double cost = waves * (((tiles + ns - 1) / ns) * tile_cost + fixed * fixed_scale);
+      const double cost = given_cost >= 0.0 ? given_cost
+                                            : waves * (((tiles + ns - 1) / ns) * tile_cost + fixed * fixed_scale);
       if (best_cost < 0.0 || cost < best_cost) {
         best = pl;
         best.nsplit = ns;
@@ -1845,7 +1846,15 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
         // measured (Qwen3-8B layer shape, prefix 4096 / 16384): with one query tile per KV head (few rows, many
         // slices) the two-launch form is 1-3 % faster, with more query tiles the single launch is (2.6 % at 64 nodes)
         const int via = force_via ? force_via : (pl.n_mgroups == 1 ? 2 : 1);
-        consider(ns, via, 1.0, 10.0);
+        if (via == 2 && mt == 1 && pl.n_mgroups == 1) {
+          // One query tile per KV head: few work items, so the launch is a handful of tiles per CTA plus the
+          // merge.  Fitted to a sweep of 6 .. 18 slices at prefixes 2048 .. 16384 (budgets 16 and 32): 0.6 us per
+          // key tile of a CTA, 0.1 us per slice for the second launch, 0.25 us more per slice beyond 12 (in the
+          // planner's unit of 0.8 us: 0.75, 0.125, 0.31).  9 - 11 slices win up to prefix 8192, 13 - 18 beyond.
+          consider(ns, via, 1.0, 0.0, ((tiles + ns - 1) / ns) * 0.75 + 0.125 * ns + 0.31 * (ns > 12 ? ns - 12 : 0) + 9.7);
+        } else {
+          consider(ns, via, 1.0, 10.0);
+        }
       }
     }
   }
