@@ -507,6 +507,8 @@ def bench_jet(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
     c = workload(args.config, args.budget, args.batch)
+    if args.layers:
+        c["layers"] = args.layers
     st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha, args.layout == "tail",
                             args.draft_input == "logits")
     layers = c["layers"]
@@ -683,6 +685,7 @@ def bench_jet(args):
                    "Hkv": c["Hkv"], "head_dim": c["D"], "prefix": info["seq_lens"] if c.get("paged") else c["L"],
                    "tree_nodes": c["B"], "max_depth": c["N"], "width": c["W"], "vocab": c["V"],
                    "paged": bool(c.get("paged")), "cuda_graph": not args.no_graph,
+                   "layers_overridden": bool(args.layers),
                    "l2": "every layer streams its own KV buffers; one step reads far more than the 126 MB L2",
                    "accepted_len": acc, "accept": args.accept, "tree_kv": args.layout,
                    "score": args.score if args.score != "hybrid" else f"hybrid(alpha={args.score_alpha})",
@@ -822,6 +825,8 @@ def main():
     ap.add_argument("--config", default="qwen3_8b", choices=list(CONFIGS))
     ap.add_argument("--budget", type=int, default=None, help="tree budget, for the sweep configurations")
     ap.add_argument("--batch", type=int, default=None, help="batch, for configurations that list several")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="override the workload's layer count (small captures under a profiler; not a bench value)")
     ap.add_argument("--no-graph", action="store_true", help="issue the calls directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the extra attention-only points of the default run")
