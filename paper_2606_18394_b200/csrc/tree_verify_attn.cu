@@ -21,10 +21,11 @@
 //                 query tiles per CTA each warpgroup owns a tile with the classic bookkeeping, and the
 //                 tiles take turns on one score buffer.  See "the key loop" below.
 //   key slices  = when there are fewer work items than SMs the key range is cut into `nsplit`
-//                 slices.  After the key loop every CTA hands the normalised rows (bf16) and their
-//                 log-sum-exp to the rows' owner CTAs -- through distributed shared memory when the
-//                 slices form a thread-block cluster, else through the workspace -- and the owners
-//                 combine the slices and write the output.  There is no second launch.
+//                 slices.  After the key loop every CTA stages its normalised rows (bf16) and their
+//                 log-sum-exp; the rows' owner CTAs collect them -- by loads from their peers' shared
+//                 memory when the slices form a thread-block cluster, else through the workspace -- combine
+//                 the slices and write the output.  With few rows and many slices the combination is left
+//                 to a second, small launch (tree_attn_merge_kernel) instead.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
 // loops (still taking part in the CTA-wide and cluster barriers), outstanding TMA loads are drained,
 // TMEM is released and JET_ERR_TIMEOUT is reported.
