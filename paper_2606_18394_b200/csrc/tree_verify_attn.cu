@@ -725,70 +725,82 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       }
       const uint32_t src_stride = rows_per * C::kRecvPitch;     // distance between the blocks of consecutive slices
-      // The softmax warpgroups combine the blocks in two steps, so that no thread runs a chain of exponentials:
-      // first one thread per row turns the S log-sum-exps into normalised slice weights (shared memory),
-      // then one item = 8 output values of one row is a short run of independent multiply-adds.
+      // The softmax warpgroups combine the blocks: one item = 8 output values of one row.  A thread first issues
+      // every load of its item (the S log-sum-exps of the row and its 16 bytes of every slice), then forms the
+      // softmax weights of the slice sums and the weighted sum -- one round trip to shared memory, no chain of
+      // dependent loads, no table of weights and no barrier between two passes.
       if constexpr (kSm) {
-        float* wts = reinterpret_cast<float*>(smem_gen + C::kTileBytes - 4096);      // [own_n][S], then 1/sum [own_n]
-        const int n_rows = rows_ok ? own_n : 0;
-        {
-          const int rl = tid - 128;
-          if (rl < n_rows) {
-            const int R = mt * kBM + own_lo + rl;                  // row within the unit
-            const int vq = static_cast<int>(udiv(R, p.magic_G));
-            const int v = node_lo + vq, h = g * G + (R - vq * G);
-            const uint8_t* lse0 = src_rows + rl * C::kRecvPitch + D * 2;
-            float mx = -INFINITY;
-            if (v < n) {
-#pragma unroll 4
-              for (int c = 0; c < S; ++c) mx = fmaxf(mx, *reinterpret_cast<const float*>(lse0 + c * src_stride));
-            }
-            float wsum = 0.0f;
-#pragma unroll 4
-            for (int c = 0; c < S; ++c) {
-              const float lc = *reinterpret_cast<const float*>(lse0 + c * src_stride);
-              // absent slices (log-sum-exp -inf) and rows of padding nodes get weight 0 and are never read
-              const float w = (mx > -INFINITY && lc > -INFINITY) ? exp2f(lc - mx) : 0.0f;
-              wts[rl * S + c] = w;
-              wsum += w;
-            }
-            wts[own_n * S + rl] = wsum > 0.0f ? 1.0f / wsum : 0.0f;
-            if (p.lse && v < p.B)
-              p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] =
-                  wsum > 0.0f ? (mx + log2f(wsum)) * 0.6931471805599453f : -INFINITY;
-          }
-        }
-        ptx::named_sync(2, 256);
-        const int items = n_rows * (D / 8);
+        const int items = rows_ok ? own_n * (D / 8) : 0;
 #pragma unroll 1
         for (int i = tid - 128; i < items; i += 256) {
           const int rl = i / (D / 8), c8 = i - rl * (D / 8);
-          const int R = mt * kBM + own_lo + rl;
+          const int R = mt * kBM + own_lo + rl;                  // row within the unit
           const int vq = static_cast<int>(udiv(R, p.magic_G));
           const int v = node_lo + vq, h = g * G + (R - vq * G);
           if (v >= p.B) continue;
+          const uint8_t* src = src_rows + rl * C::kRecvPitch;
           float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-          const uint8_t* src = src_rows + rl * C::kRecvPitch + c8 * 16;
-          const float* wrow = wts + rl * S;
-#pragma unroll 3
-          for (int c = 0; c < S; ++c) {
-            const float w = wrow[c];
-            if (w > 0.0f) {                        // (a slice with weight 0 may hold junk)
-              const uint4 x = *reinterpret_cast<const uint4*>(src + c * src_stride);
+          float lse2 = -INFINITY;
+          if (S == 1) {
+            // no slices: the staged row is the result
+            const float lc = *reinterpret_cast<const float*>(src + D * 2);
+            const uint4 x = *reinterpret_cast<const uint4*>(src + c8 * 16);
+            if (v < n && lc > -INFINITY) {
               const uint32_t v4[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
-                acc[2 * q] += w * __uint_as_float(v4[q] << 16);
-                acc[2 * q + 1] += w * __uint_as_float(v4[q] & 0xFFFF0000u);
+              for (int q = 0; q < 4; ++q) {
+                acc[2 * q] = __uint_as_float(v4[q] << 16);
+                acc[2 * q + 1] = __uint_as_float(v4[q] & 0xFFFF0000u);
               }
+              lse2 = lc;
+            }
+          } else {
+            // (four slices at a time: their loads are issued together, then used)
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < S; c0 += 4) {
+              float l4[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                l4[k] = c0 + k < S ? *reinterpret_cast<const float*>(src + (c0 + k) * src_stride + D * 2) : -INFINITY;
+              mx = fmaxf(fmaxf(mx, fmaxf(l4[0], l4[1])), fmaxf(l4[2], l4[3]));
+            }
+            if (v < n && mx > -INFINITY) {
+              float wsum = 0.0f;
+#pragma unroll 1
+              for (int c0 = 0; c0 < S; c0 += 4) {
+                float l4[4];
+                uint4 x4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const bool in = c0 + k < S;
+                  l4[k] = in ? *reinterpret_cast<const float*>(src + (c0 + k) * src_stride + D * 2) : -INFINITY;
+                  x4[k] = in ? *reinterpret_cast<const uint4*>(src + (c0 + k) * src_stride + c8 * 16) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  // absent slices (log-sum-exp -inf) get weight 0, and whatever their rows hold is not used
+                  const float w = l4[k] > -INFINITY ? exp2f(l4[k] - mx) : 0.0f;
+                  wsum += w;
+                  const uint32_t v4[4] = {x4[k].x, x4[k].y, x4[k].z, x4[k].w};
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {      // bf16 pair -> fp32: the bits are the upper half of the float
+                    const float lo = __uint_as_float(v4[q] << 16), hi = __uint_as_float(v4[q] & 0xFFFF0000u);
+                    acc[2 * q] += w > 0.0f ? w * lo : 0.0f;
+                    acc[2 * q + 1] += w > 0.0f ? w * hi : 0.0f;
+                  }
+                }
+              }
+              const float inv = 1.0f / wsum;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) acc[k] *= inv;
+              lse2 = mx + log2f(wsum);
             }
           }
-          const float inv = wts[own_n * S + rl];
-#pragma unroll
-          for (int k = 0; k < 8; ++k) acc[k] *= inv;
           *reinterpret_cast<uint4*>(p.out + ((static_cast<size_t>(b) * p.B + v) * p.Hq + h) * D + c8 * 8) =
               make_uint4(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]), pack_bf16(acc[4], acc[5]),
                          pack_bf16(acc[6], acc[7]));
+          if (p.lse && c8 == 0) p.lse[(static_cast<size_t>(b) * p.Hq + h) * p.B + v] = lse2 * 0.6931471805599453f;
         }
       }
     }
