@@ -303,6 +303,17 @@ def time_attention(st, layers, stream, steps, use_graph, sampler=None):
                 graph.replay()
             a1.record(stream)
             stream.synchronize()
+            # per-replay samples for a median and a minimum beside the mean (50 replays, one event pair each)
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(50)]
+            for x, y in pairs:
+                x.record(stream)
+                graph.replay()
+                y.record(stream)
+            stream.synchronize()
+            per = sorted(x.elapsed_time(y) * 1e3 / layers for x, y in pairs)
+            time_attention.last_samples = {"median_us_per_launch": per[len(per) // 2], "min_us_per_launch": per[0],
+                                           "samples": len(per),
+                                           "note": "one event pair per graph replay: includes the replay's launch gap"}
             return (a0.elapsed_time(a1) * 1e3 / (reps * layers),
                     f"CUDA events around {reps} replays of a graph of the {layers} attention launches", reps)
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -319,11 +330,17 @@ def time_attention(st, layers, stream, steps, use_graph, sampler=None):
                     b_.record(stream)
                     i += 1
             stream.synchronize()
+        time_attention.last_samples = None
         return (statistics.mean(a.elapsed_time(b_) for a, b_ in evs) * 1e3, "CUDA events around every attention call",
                 steps)
 
 
-def attention_roofline(c, info, attn_us, clocks, workload_name, timing):
+time_attention.last_samples = None
+# Nominal peaks (context beside the measured ones): HBM3e 8 TB/s, dense bf16 2.25 PFLOP/s.
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+
+
+def attention_roofline(c, info, attn_us, clocks, workload_name, timing, samples=None):
     """The roofline object of the attention kernel for one workload."""
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(peaks_path):
@@ -348,6 +365,10 @@ def attention_roofline(c, info, attn_us, clocks, workload_name, timing):
                 "peak_kind": "sustained (power cap or SM clock below 90 % of its maximum during the timed region)" if capped else "burst",
                 "frac_of_burst_peak": achieved / peaks["bf16_tflops"]}
     roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["frac_of_nominal"] = roof["achieved"] / (NOMINAL["hbm_gbs"] if roof["bound"] == "hbm" else NOMINAL["bf16_tflops"])
+    samples = samples if samples is not None else time_attention.last_samples
+    if samples:
+        roof["per_replay"] = samples
     roof["traffic"], roof["traffic_note"] = ncu_traffic(workload_name, bytes_alg)
     roof.update(kernel="tree_attn_kernel", peak_source=peak_src, us_per_launch=attn_us, timing=timing,
                 algorithmic_bytes=bytes_alg, algorithmic_flops=flops_alg,
@@ -581,6 +602,7 @@ def bench_jet(args):
     attn_us, attn_timing, attn_reps = time_attention(st, layers, stream, args.steps, not args.no_graph,
                                                      attn_sampler if rank == 0 else None)
     attn_clocks = attn_sampler.stop() if rank == 0 else None
+    attn_samples = time_attention.last_samples
     assert int(st.status.item()) == 0, "a bounded device wait expired"
     # the same launches issued call by call (no graph): what a caller that does not capture pays per call,
     # host-side argument checks and tensor-map encoding included
@@ -654,7 +676,7 @@ def bench_jet(args):
         return
 
     # ---------------- roofline of the dominant kernel (one attention call = one tree_attn_kernel launch)
-    roof = attention_roofline(c, info, attn_us, attn_clocks, args.config, attn_timing)
+    roof = attention_roofline(c, info, attn_us, attn_clocks, args.config, attn_timing, attn_samples)
     roof["clocks"] = attn_clocks
     roof["us_per_call_without_graph"] = attn_us_eager
 
@@ -669,6 +691,11 @@ def bench_jet(args):
                                      (local_rank, gpu_uuid)))
         sweep.append(sweep_point("batched_paged", dict(CONFIGS["batched_paged"]), rank_seed(6, rank), device, 3,
                                  (local_rank, gpu_uuid)))
+        # the long-generation regime of the same layer shape (prefix 16384): an HBM-bound and a tensor-bound budget
+        for nodes in (64, 256):
+            cc = dict(CONFIGS["sweep_16k"], B=nodes, N=12 if nodes > 64 else 8)
+            sweep.append(sweep_point(f"sweep_16k_b{nodes}", cc, rank_seed(9, rank) + nodes, device, 3,
+                                     (local_rank, gpu_uuid)))
         # the draft head's own block-causal attention: a chain of 16 rows (one per draft depth, width 1) over the
         # same context length, at the head's shape; timed over 36 distinct KV buffers so every launch is cold
         sweep.append(sweep_point("draft_head_block16", dict(base, B=16, N=15, W=1), rank_seed(7, rank), device, 3,
