@@ -170,7 +170,34 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0, tail=False, draft_logits=False):
+def plant_hidden(st, b, token, parent, depth, n_nodes, length, rng):
+    """The planted path for accept_mode "hidden": the hidden state of every node on the path points along the
+    LM-head row of the token that must win there (logit ~ 8 * |row| ~ 10 against ~ N(0, 0.16) for every other
+    token), the end node's along a token none of its children carries.  Returns the effective path length."""
+    import torch
+    B, V = st.B, st.V
+    max_depth = int(depth[:n_nodes].max())
+    eff = min(length, max_depth)
+    cands = [v for v in range(n_nodes) if depth[v] == eff]
+    end = int(cands[int(rng.integers(0, len(cands)))])
+
+    def point(row, tok):
+        w = st.lm_head[tok].float()
+        st.hidden[b * B + row].copy_((8.0 * w / w.norm()).bfloat16())
+    u = end
+    while parent[u] != -1:
+        point(int(parent[u]), int(token[u]))
+        u = int(parent[u])
+    child_tokens = {int(token[cn]) for cn in range(n_nodes) if parent[cn] == end}
+    t = int(rng.integers(0, V))
+    while t in child_tokens:
+        t = (t + 1) % V
+    point(end, t)
+    return eff
+
+
+def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0, tail=False, draft_logits=False,
+                 target_hidden=False, d_model=4096):
     """Seeded synthetic step inputs on the device.  Returns (VerifyStep, info dict)."""
     import torch
     from paper_2606_18394_b200.step import VerifyStep
@@ -230,9 +257,18 @@ def build_inputs(c, name, seed, device, score_mode="accum_logp", score_alpha=0.0
     n_nodes = st.n_nodes.cpu().numpy()
     rng = np.random.default_rng(seed + 1)
     planted = []
+    if target_hidden:
+        # the acceptance is fed with final hidden states (N(0,1)) and LM-head weights (N(0, 0.02^2)) instead of logits
+        st.enable_lm_head(d_model)
+        st.accept_mode = "hidden"
+        st.hidden.copy_(torch.randn(st.hidden.shape, generator=gen, device=device, dtype=torch.float32))
+        st.lm_head.copy_(torch.randn(st.lm_head.shape, generator=gen, device=device, dtype=torch.float32) * 0.02)
     for b in range(batch):
-        rows = st.logits[b].cpu().numpy()
         want = c.get("plant", int(rng.integers(1, N + 1)))
+        if target_hidden:
+            planted.append(plant_hidden(st, b, token[b], parent[b], depth[b], int(n_nodes[b]), want, rng))
+            continue
+        rows = st.logits[b].cpu().numpy()
         _, eff = plant_path(rows, token[b], parent[b], depth[b], int(n_nodes[b]), want, rng)
         st.logits[b].copy_(torch.from_numpy(rows))
         planted.append(eff)
@@ -531,9 +567,10 @@ def bench_jet(args):
     if args.layers:
         c["layers"] = args.layers
     st, info = build_inputs(c, args.config, rank_seed(2, rank), device, args.score, args.score_alpha, args.layout == "tail",
-                            args.draft_input == "logits")
+                            args.draft_input == "logits", args.target_input == "hidden")
     layers = c["layers"]
     if args.accept == "sample":
+        assert args.target_input == "logits", "the non-greedy rule needs the target logits"
         st.accept_mode = "sample"
         g = torch.Generator(device=device).manual_seed(rank_seed(3, rank))
         st.u_accept.copy_(torch.rand(st.u_accept.shape, generator=g, device=device))
@@ -609,49 +646,69 @@ def bench_jet(args):
     attn_us_eager, _, _ = time_attention(st, layers, stream, max(2, min(args.steps, 10)), False, None)
 
     # ---------------- end to end: host buffers in, result out, every step
-    pinned = {k: getattr(st, k).cpu().pin_memory() for k in ("logp", "root_token", "logits", "q", "tree_k", "tree_v")}
+    big = "hidden" if st.accept_mode == "hidden" else "logits"      # the acceptance's input, needed last
+    pinned = {k: getattr(st, k).cpu().pin_memory() for k in ("logp", "root_token", big, "q", "tree_k", "tree_v")}
     host_out = {k: torch.empty_like(getattr(st, k), device="cpu").pin_memory()
                 for k in ("accept_len", "out_tokens", "path")}
     h2d = sum(v.numel() * v.element_size() for v in pinned.values())
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
 
-    # The target logits (the largest input) are only needed by the acceptance at the end of the step: their
-    # copy runs on a second stream under tree construction and attention.
+    # The inputs arrive in the order the step needs them, on a copy stream of their own: draft log-probs first, then
+    # q / tree K / tree V of the first quarter of the layers, the second ... and last the acceptance's input (the
+    # largest, or the hidden states).  The step is cut into graphs at the same places (tree construction, four
+    # groups of layers, acceptance + commit); each group starts as soon as its inputs are on the device, so the
+    # copies of later layers run under the attention of earlier ones.
     copy_stream = torch.cuda.Stream()
-    logits_done, back_done, small_done = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+    n_groups = 1 if st.tail else min(4, layers)          # (in-cache tree layout: the tree rows are placed after all copies)
+    bounds = [round(i * layers / n_groups) for i in range(n_groups + 1)]
+    ev_small, ev_big, back_done = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+    ev_group = [torch.cuda.Event() for _ in range(n_groups)]
+
+    def part_build():
+        st.seq_len.copy_(st.seq_len0)
+        st.tree_build()
+
+    def part_group(i):
+        for layer in range(bounds[i], bounds[i + 1]):
+            st.verify_attn(layer)
+    parts = [part_build] + [(lambda i=i: part_group(i)) for i in range(n_groups)] + [st.run_back]
     if not args.no_graph:
         with torch.cuda.stream(stream):
-            g_front, g_back = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-            st.run_front()
-            st.run_back()
+            for f in parts:
+                f()
             stream.synchronize()
-            with torch.cuda.graph(g_front, stream=stream):
-                st.run_front()
-            with torch.cuda.graph(g_back, stream=stream):
-                st.run_back()
+            graphs = []
+            for f in parts:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    f()
+                graphs.append(g)
             stream.synchronize()
-        front, back = g_front.replay, g_back.replay
-    else:
-        front, back = st.run_front, st.run_back
+        parts = [g.replay for g in graphs]
     back_done.record(stream)
 
     def e2e_step():
-        for k, v in pinned.items():
-            if k != "logits":
-                getattr(st, k).copy_(v, non_blocking=True)
-        # the logits copy starts when the copies above are done (side by side they would share the link and hold
-        # the front of the step back) and when the acceptance of the step before has read the logits
-        small_done.record(stream)
-        copy_stream.wait_event(small_done)
+        # the copies of this step may start once the step before has finished with the buffers
         copy_stream.wait_event(back_done)
         with torch.cuda.stream(copy_stream):
-            st.logits.copy_(pinned["logits"], non_blocking=True)
-            logits_done.record(copy_stream)
-        if st.tail:
-            st.place_tree()                # the tree's K/V arrive in staging buffers and are put behind the prefixes
-        front()
-        stream.wait_event(logits_done)
-        back()
+            for k in ("logp", "root_token"):
+                getattr(st, k).copy_(pinned[k], non_blocking=True)
+            ev_small.record(copy_stream)
+            for i in range(n_groups):
+                for k in ("q", "tree_k", "tree_v"):
+                    getattr(st, k)[bounds[i]:bounds[i + 1]].copy_(pinned[k][bounds[i]:bounds[i + 1]], non_blocking=True)
+                ev_group[i].record(copy_stream)
+            getattr(st, big).copy_(pinned[big], non_blocking=True)
+            ev_big.record(copy_stream)
+        stream.wait_event(ev_small)
+        parts[0]()
+        for i in range(n_groups):
+            stream.wait_event(ev_group[i])
+            if st.tail and i == 0:
+                st.place_tree()            # the tree's K/V arrive in staging buffers and are put behind the prefixes
+            parts[1 + i]()
+        stream.wait_event(ev_big)
+        parts[-1]()
         back_done.record(stream)
         for k, v in host_out.items():
             v.copy_(getattr(st, k), non_blocking=True)
@@ -716,12 +773,13 @@ def bench_jet(args):
                    "l2": "every layer streams its own KV buffers; one step reads far more than the 126 MB L2",
                    "accepted_len": acc, "accept": args.accept, "tree_kv": args.layout,
                    "score": args.score if args.score != "hybrid" else f"hybrid(alpha={args.score_alpha})",
-                   "draft_input": args.draft_input},
+                   "draft_input": args.draft_input, "target_input": args.target_input},
         "attn_us_per_layer": attn_us,
         "e2e": {"value": e2e_ms_step * 1e3 / (layers * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,
-                "note": "all inputs come from pinned host memory every step; the target logits are copied on a second "
-                        "stream while the tree is built and attended, the acceptance waits for them"},
+                "note": "all inputs come from pinned host memory every step, on a copy stream, in the order the step needs "
+                        "them (log-probs, then q / tree K / tree V per quarter of the layers, then the acceptance's input); "
+                        "every part of the step starts when its inputs have arrived"},
         "gpu_launches": args.steps * st.launches_per_step(),
         "clocks": clocks, "roofline": roof,
     }
@@ -792,7 +850,13 @@ def cpu_baseline(st, c, info):
     else:
         ks = [_bits(st.k_cache[l, 0, :L]) for l in range(nl)]
         vs = [_bits(st.v_cache[l, 0, :L]) for l in range(nl)]
-    x = dict(logp=st.logp[0].cpu().numpy(), root=int(st.root_token[0].item()), logits=st.logits[0].cpu().numpy(),
+    if st.accept_mode == "hidden":
+        import oracle
+        B = st.B
+        logits0 = oracle.lm_head_argmax_ref(_bits(st.hidden[:B]), _bits(st.lm_head))["logits"].astype(np.float32)
+    else:
+        logits0 = st.logits[0].cpu().numpy()
+    x = dict(logp=st.logp[0].cpu().numpy(), root=int(st.root_token[0].item()), logits=logits0,
              planted=info["planted"][0], scale=st.scale, q=[_bits(st.q[l, 0]) for l in range(nl)], k=ks, v=vs,
              tk=[_bits(st.tree_k[l, 0]) for l in range(nl)], tv=[_bits(st.tree_v[l, 0]) for l in range(nl)],
              draft_logits=st.draft_logits, score_mode=st.score_mode, alpha=st.score_alpha)
@@ -864,6 +928,9 @@ def main():
     ap.add_argument("--score-alpha", type=float, default=1.0)
     ap.add_argument("--draft-input", choices=["logp", "logits"], default="logp",
                     help="the draft head's output as log-probabilities, or as raw logits (normalised on the fly)")
+    ap.add_argument("--target-input", choices=["logits", "hidden"], default="logits",
+                    help="what the acceptance is fed with: the target's fp32 logits (the workload as stated), or its final "
+                         "hidden states, with the LM head applied inside the call (jet_tree_accept_hidden)")
     ap.add_argument("--accept", choices=["greedy", "sample"], default="greedy",
                     help="acceptance rule of the step: greedy (the headline) or the non-greedy rule at temperature 1")
     args = ap.parse_args()

@@ -194,17 +194,6 @@ __device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, volatile uint
   return ptx::cta_sync_and((ok ? 1 : 0) != 0);
 }
 
-// Cluster-wide rendezvous built from one mbarrier per CTA (count = cluster size): after a CTA-wide
-// barrier one thread arrives on the barrier of every CTA of the cluster, then everybody waits for
-// all `nsplit` arrivals on the local one.
-__device__ __forceinline__ bool cluster_rendezvous(uint32_t local_bar, int nsplit, volatile uint32_t* abort_flag,
-                                                uint32_t site) {
-  ptx::cta_sync();
-  if (threadIdx.x == 0)
-    for (int c = 0; c < nsplit; ++c) ptx::mbar_arrive_remote(ptx::map_to_rank(local_bar, c));
-  return bounded_wait_cluster(local_bar, abort_flag, site);
-}
-
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 pk = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&pk);
@@ -313,7 +302,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       uint32_t count = 1;
       if (lane >= Bars::kKvEmpty && lane < Bars::kSFull) count = (MT == 1 || C::kTurns) ? 1 : n_mt;   // arrivals per stage
       else if (lane >= Bars::kSFree && lane < Bars::kODone) count = 128;                // kSFree, kPFull: a softmax warpgroup
-      else if (lane == Bars::kClusterA || lane == Bars::kClusterC) count = S;
       ptx::mbar_init(bar(lane), count);
       // slice merge: every slice sends this CTA its block of rows of query tile (lane - kRecv)
       if (S > 1 && lane >= Bars::kRecv && lane < Bars::kRecv + MT)

@@ -88,6 +88,12 @@ class VerifyStep:
         self.u_sample = torch.zeros((batch,), dtype=torch.float32, device=dev)
         self.alpha = torch.zeros((batch, B), dtype=torch.float32, device=dev)
         self.accept_mode = "greedy"
+        # accept_mode "hidden": the acceptance takes the target's final hidden states and applies the LM head itself
+        # (enable_lm_head allocates them); no [batch, B, V] logits are needed then
+        self.hidden = None
+        self.lm_head = None
+        self.d_model = 0
+        self.ws_accept_hidden = None
         self.scale = 1.0 / math.sqrt(D)
         # Within a step the lengths, the page table and the cached prefix are older than any launch of the
         # layer stack, so every layer but the first (whose predecessor in the stream builds the tree and
@@ -169,6 +175,19 @@ class VerifyStep:
                             self.batch, self.B, self.V, self.N, self.tgt, self.accept_len, self.path,
                             self.out_tokens, self.ws_accept)
 
+    def enable_lm_head(self, d_model):
+        """Buffers for accept_mode = "hidden": hidden states [batch * B, d_model] and LM-head weights [V, d_model]."""
+        self.d_model = d_model
+        self.hidden = torch.zeros((self.batch * self.B, d_model), dtype=torch.bfloat16, device=self.device)
+        self.lm_head = torch.zeros((self.V, d_model), dtype=torch.bfloat16, device=self.device)
+        self.ws_accept_hidden = torch.empty(max(jet.jet_tree_accept_hidden_workspace_bytes(self.batch, self.B), 256),
+                                            dtype=torch.uint8, device=self.device)
+
+    def tree_accept_hidden(self):
+        jet.jet_tree_accept_hidden(self.hidden, self.lm_head, self.d_model, self.token, self.parent, self.depth,
+                                   self.anc_mask, self.n_nodes, self.batch, self.B, self.V, self.N, self.tgt,
+                                   self.accept_len, self.path, self.out_tokens, self.status, self.ws_accept_hidden)
+
     def tree_accept_sample(self):
         jet.jet_tree_accept_sample(self.logits, self.V, self.temperature, self.logp, self.N * self.V, self.V,
                                    self.token, self.parent, self.depth, self.anc_mask, self.n_nodes, self.u_accept,
@@ -198,6 +217,8 @@ class VerifyStep:
         """Acceptance against the target logits and the commit."""
         if self.accept_mode == "sample":
             self.tree_accept_sample()
+        elif self.accept_mode == "hidden":
+            self.tree_accept_hidden()
         else:
             self.tree_accept()
         self.kv_compact()
