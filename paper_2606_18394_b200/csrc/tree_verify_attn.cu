@@ -1994,7 +1994,7 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < workspace_need(pl, D)) return JET_ERR_WORKSPACE;
 
   // ---- tensor maps (bf16, 128-byte swizzle, 64-element inner box)
-  CUtensorMap tq, tk, tv, ttk, ttv;
+  CUtensorMap tq = {}, tk = {}, tv = {}, ttk = {}, ttv = {};     // (maps a call does not use stay zeroed)
   const uint64_t eb = 2;
   {
     const uint64_t dims[4] = {static_cast<uint64_t>(D), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
