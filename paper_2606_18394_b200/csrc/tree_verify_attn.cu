@@ -32,6 +32,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <type_traits>
@@ -51,6 +52,7 @@ constexpr int kBM = 128;               // query rows per tile
 constexpr int kBN = 128;               // keys per tile
 constexpr int kHalfBytes = 128 * 128;  // one [128 rows x 64 bf16] swizzled block
 constexpr int kMaxSplit = 20;          // most key slices (a cluster holds at most 16; more only through the workspace)
+constexpr int kMaxCluster = 16;        // largest thread-block cluster the hardware launches (non-portable size)
 constexpr int kMaxSorted = 128;          // batches up to this size are launched longest prefix first
 constexpr float kSharedSumFloor = 8.6736174e-19f;  // 2^-60: a row that saw keys but summed to less has lost them to underflow
 constexpr float kSharedSumLimit = 1.2089258e24f;   // 2^80: tile sums a fixed reference may reach before the CTA falls back
@@ -492,7 +494,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int rows_per = p.rows_per;                   // rows of a query tile that one slice combines
     const int own_lo = split * rows_per;
     const int own_n = max(0, min(rows_per, kBM - own_lo));
-    const int unit = (static_cast<int>(blockIdx.z) * p.Hkv + static_cast<int>(blockIdx.y)) * p.n_mgroups + e_mgroup;
+    // (indexed by the sequence itself, not by its rank in launch order: the merge kernel of the two-launch form
+    //  addresses the slots by sequence)
+    const int unit = (b * p.Hkv + static_cast<int>(blockIdx.y)) * p.n_mgroups + e_mgroup;
     // =============================================================== epilogue
     // One round per query tile: its softmax threads stage their normalised rows (D bf16 + log2-sum-exp)
     // in shared memory.  With key slices every CTA then sends each owner slice its block of rows with
@@ -1758,7 +1762,7 @@ bool configure_kernel() {
 template <int D, int MT>
 int max_active_clusters(int cluster) {
   static std::atomic<int> caches[kMaxDevices][kMaxSplit + 1];      // per device: 0 = unknown, -1 = none
-  if (cluster < 1 || cluster > kMaxSplit) return 0;
+  if (cluster < 1 || cluster > kMaxCluster) return 0;       // (the occupancy query does not refuse larger ones)
   std::atomic<int>* cache = caches[current_device()];
   if (cache[cluster].load(std::memory_order_relaxed) == 0) {
     int n = 0;
@@ -1902,6 +1906,11 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   const cudaError_t err = sorted ? cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, true>, tq, tk, tv, ttk, ttv, p)
                                  : cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, false>, tq, tk, tv, ttk, ttv, p);
   if (err != cudaSuccess) {
+#ifdef JET_TRACE
+    fprintf(stderr, "attention launch failed: %s (grid %d x %d x %d, cluster %d, %d slices, merge form %d, D %d, MT %d)\n",
+            cudaGetErrorString(err), pl.n_mgroups * pl.nsplit, p.Hkv, p.batch, pl.via_global ? 1 : pl.nsplit, pl.nsplit,
+            pl.via_global, D, MT);
+#endif
     cudaGetLastError();
     return JET_ERR_CUDA;
   }
