@@ -817,6 +817,18 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int lead = min(ahead + 1, T);
     return lead + tl + min(tl, T - lead);
   };
+  // Where a tile sits in shared memory: .x = stage, .y = parity of this use of the stage's barriers.
+  //  * One producer warp: all tiles go through ONE ring in issue order (ring item i -> stage i % kStages).
+  //  * Two producer warps (warp 0 requests the K tiles, warp 2 the V tiles): each warp has stages of its own, K tile
+  //    t in stage t % kKStages, V tile t in stage kKStages + t % kVStages.  A parity wait tells "one phase further"
+  //    from "two phases further" only for a thread that saw the phase before itself; with one shared ring a warp
+  //    that runs past the other warp's tiles can be two uses of a stage ahead of the consumers (a slow load is
+  //    enough), takes the stale parity for its turn and overwrites a tile that has not been read.  With stages
+  //    of its own every wait of a warp follows its own previous wait on the same barrier.
+  constexpr int kKStages = (kStages + 1) / 2, kVStages = kStages - kKStages;
+  auto ring_pos = [&](int item) { return make_int2(item % kStages, (item / kStages) & 1); };
+  auto k_pos_split = [&](int tl) { return make_int2(tl % kKStages, (tl / kKStages) & 1); };
+  auto v_pos_split = [&](int tl) { return make_int2(kKStages + tl % kVStages, (tl / kVStages) & 1); };
   // The barriers of the classic pass when it follows a shared-accumulator pass: a fresh set.
   auto second_barrier_set = [&]() {
     sBarLoop = sBar + 8u * Bars::kCount;
@@ -866,17 +878,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll 1
       for (; issued < 2 * T; ++issued) {
         const bool take_k = kt < T && kt <= vt + ahead;
-        const int t = t_lo + (take_k ? kt : vt), kv = take_k ? 0 : 1, stage = issued % kStages;
+        const int t = t_lo + (take_k ? kt : vt), kv = take_k ? 0 : 1;
         if (only >= 0 && kv != only) {          // the other producer warp's tile
           if (take_k) ++kt; else ++vt;
           continue;
         }
+        // stage and how often it has been used before (see ring_pos / k_pos_split)
+        const int nth = take_k ? kt : vt;
+        const int stage = only < 0 ? issued % kStages : (take_k ? nth % kKStages : kKStages + nth % kVStages);
+        const int use = only < 0 ? issued / kStages : (take_k ? nth / kKStages : nth / kVStages);
         if (!waited && (t + 1) * kBN > L) {      // not wholly inside the prefix: may hold rows the preceding kernel writes
           ptx::grid_dep_wait();
           waited = true;
         }
-        if (issued >= kStages) {
-          ok = bounded_wait(lbar(Bars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
+        if (use >= 1) {
+          ok = bounded_wait(lbar(Bars::kKvEmpty + stage), (use - 1) & 1, abort_flag, 1);
           if (!ok) break;
         }
         const uint32_t dst = sKV + stage * C::kStageBytes;
@@ -914,11 +930,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (lane == 0 && issued == 0) JET_TR(14);
       }
       if (__any_sync(0xffffffffu, *abort_flag != 0u)) {
-        // drain: every load that was issued must land before the CTA may exit
+        // drain: every load that this warp issued must land before the CTA may exit
         for (int s = 0; s < kStages; ++s) {
-          if (issued > s) {
-            const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
-            bounded_wait(lbar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
+          if (only < 0) {
+            if (issued > s) {
+              const int last = ((issued - 1 - s) / kStages) * kStages + s;     // last item issued to stage s
+              bounded_wait(lbar(Bars::kKvFull + s), (last / kStages) & 1, abort_flag, 2);
+            }
+          } else {
+            const bool k_stage = s < kKStages;
+            const int n = k_stage ? kt : vt, ring = k_stage ? kKStages : kVStages, r = k_stage ? s : s - kKStages;
+            if ((only == 0) == k_stage && n > r) {
+              const int last = ((n - 1 - r) / ring) * ring + r;                // last tile of this kind in stage s
+              bounded_wait(lbar(Bars::kKvFull + s), (last / ring) & 1, abort_flag, 2);
+            }
           }
         }
         bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
@@ -956,9 +981,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll 1
           for (int tl = 0; tl < T && ok; ++tl) {
             const int w = tl & 1, j = tl >> 1;
-            const int item = tl < lead ? tl : 2 * tl - lead + 1;
-            const int stage = item % kStages;
-            const uint32_t par = (item / kStages) & 1;
+            const int2 pos = p.paged ? k_pos_split(tl) : ring_pos(tl < lead ? tl : 2 * tl - lead + 1);
+            const int stage = pos.x;
+            const uint32_t par = pos.y;
             if (tl == 12 && lane == 0) JET_TR(61);
             if (j > 0) {
               ok = bounded_wait(bar(Bars::kSFree + w), (j - 1) & 1, abort_flag, 20);
@@ -987,9 +1012,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll 1
           for (int tl = 0; tl < T && ok; ++tl) {
             const int w = tl & 1, j = tl >> 1;
-            const int item = v_item(tl, kAhead);
-            const int stage = item % kStages;
-            const uint32_t par = (item / kStages) & 1;
+            const int2 pos = p.paged ? v_pos_split(tl) : ring_pos(v_item(tl, kAhead));
+            const int stage = pos.x;
+            const uint32_t par = pos.y;
             if (tl == 8 && lane == 0) JET_TR(58);
             ok = bounded_wait(bar(Bars::kKvFull + stage), par, abort_flag, 7);
             if (!ok) break;
@@ -1038,8 +1063,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           int prev_mt = -1, prev_tl = 0;
 #pragma unroll 1
           for (int tl = 0; tl < T && ok; ++tl) {
-            const int item = 2 * tl, stage = item % kStages;
-            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 5);
+            const int2 pos = k_pos_split(tl);
+            const int stage = pos.x;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), pos.y, abort_flag, 5);
             if (!ok) break;
             const uint64_t desc_k = desc_k0 + static_cast<uint64_t>((stage * C::kStageBytes) >> 4);
             for (int mt = 0; mt < n_mt && ok; ++mt) {
@@ -1067,8 +1093,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           bool ok = true;
 #pragma unroll 1
           for (int tl = 0; tl < T && ok; ++tl) {
-            const int item = 2 * tl + 1, stage = item % kStages;
-            ok = bounded_wait(bar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 7);
+            const int2 pos = v_pos_split(tl);
+            const int stage = pos.x;
+            ok = bounded_wait(bar(Bars::kKvFull + stage), pos.y, abort_flag, 7);
             if (!ok) break;
             const uint64_t desc_v = desc_v0 + static_cast<uint64_t>((stage * C::kStageBytes) >> 4);
             for (int mt = 0; mt < n_mt && ok; ++mt) {
@@ -1198,11 +1225,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // Masked keys get P = 0 exactly, but 0 * NaN is NaN: the V rows of keys beyond the valid ones (stale
     // cache rows, rows of padding nodes) are cleared before the P V product may read them.  `item` = the V
     // tile's position in the ring.  Returns false if the wait for the tile gave up.
-    auto clear_v_tail = [&](int t, int item) -> bool {
+    auto clear_v_tail = [&](int t, int2 pos) -> bool {
       const int valid = t < TP ? min(kBN, Lc - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
       if (valid >= kBN) return true;
-      const int stage = item % kStages;
-      if (!bounded_wait(lbar(Bars::kKvFull + stage), (item / kStages) & 1, abort_flag, 10)) return false;
+      const int stage = pos.x;
+      if (!bounded_wait(lbar(Bars::kKvFull + stage), pos.y, abort_flag, 10)) return false;
       uint8_t* vt = gen_kv + stage * C::kStageBytes;
       const int chunks = (kBN - valid) * 8;                // 16-byte chunks per 64-column block
       for (int h = 0; h < kHalves; ++h)
@@ -1289,7 +1316,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           l += tile_sum;
           if (tid == 128 && j == 4) JET_TR(17);
           if (!full_tile) {
-            ok = clear_v_tail(t, v_item(tl, kAhead));
+            ok = clear_v_tail(t, p.paged ? v_pos_split(tl) : ring_pos(v_item(tl, kAhead)));
             if (!ok) break;
           }
           ptx::tmem_wait_st();                     // P is in TMEM
@@ -1414,7 +1441,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           }
           l = l * factor + tile_sum;
           if (!full_tile) {
-            ok = clear_v_tail(t, 2 * tl + 1);
+            ok = clear_v_tail(t, v_pos_split(tl));
             if (!ok) break;
           }
           ptx::tmem_wait_st();                     // P (and a rescaled O) are in TMEM
@@ -1538,7 +1565,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         l = l * factor + tile_sum;
         if (!full_tile) {
-          ok = clear_v_tail(t, 2 * tl + 1);
+          ok = clear_v_tail(t, ring_pos(2 * tl + 1));
           if (!ok) break;
         }
         ptx::tmem_wait_st();                     // P (and a rescaled O) are in TMEM

@@ -10,15 +10,19 @@ Tolerance: the arithmetic bound |err| <= 2^-8 (|ref| + max |v|) + 2e-3 element-w
 bf16 before they weigh V entries of size up to 4.5, output rounded to bf16), mean |err| <= 2.5e-3 over the live
 rows, log-sum-exp within 2e-3.
 
-Two cases are pinned by name because a randomized run found faults with them: small trees in a ragged batch
-(one query tile per KV head, key slices combined by the second launch, sequences launched longest first), and
-17 key tiles with few work items (a plan with a cluster of 17 CTAs, which the hardware does not launch).
+Cases pinned by name because randomized runs found faults with them:
+  * a paged cache with one query tile per CTA at scale: K and V tiles come from two producer warps there; with one
+    shared ring of stages a warp could run two uses of a stage ahead of the consumers when a load was slow and
+    overwrite a tile that had not been read (the warps now have stages of their own);
+  * small trees in a ragged batch: one query tile per KV head, key slices combined by the second launch,
+    sequences launched longest first -- the partial rows were addressed by launch rank instead of by sequence;
+  * 17 key tiles with few work items: a plan with a cluster of 17 CTAs, which the hardware does not launch.
 """
 import numpy as np
 import pytest
 
 from jet_inputs import binary_tree, chain_tree, make_attn_inputs, make_paged_cache, random_tree, star_tree
-from oracle import anc_from_parent, tree_attn_ref
+from oracle import anc_from_parent, gather_paged_prefix, tree_attn_ref, tree_attn_rows_ref
 
 pytestmark = pytest.mark.gpu
 
@@ -135,3 +139,39 @@ def test_seventeen_key_tiles_with_few_work_items(paged):
     rng = np.random.default_rng(5200)
     seq = np.asarray([1973, 1000, 1571], np.int32)
     _run_case(rng, 64, 2, 1, 3, 32, seq, np.asarray([28, 18, 23]), paged, 1, 0.125, False)
+
+
+@pytest.mark.parametrize("G,Hkv,batch,B,L,ragged,flags", [
+    (4, 8, 2, 384, 9000, False, 1),       # 12 query tiles per KV head, two key slices in clusters of two, three waves
+    (1, 4, 16, 96, 4100, False, 0),       # one query tile per KV head, two slices combined by the second launch
+    (1, 8, 32, 128, 3988, True, 0),       # 256 work items, two waves, sequences launched longest first
+    (1, 8, 32, 16, 4100, False, 1),
+    (4, 8, 32, 16, 4096, False, 1),
+])
+def test_paged_cache_one_query_tile_per_cta_at_scale(G, Hkv, batch, B, L, ragged, flags):
+    """Sampled rows of the first, last, shortest and longest sequence against the oracle (D = 128)."""
+    import jet_harness as H
+    D, Hq = 128, G * Hkv
+    rng = np.random.default_rng(5300 + batch * B)
+    seq = (rng.integers(L // 5, L + 1, size=batch) if ragged else np.full(batch, L)).astype(np.int32)
+    n_nodes = np.full(batch, B)
+    qs, tks, tvs, ancs = [], [], [], []
+    for b in range(batch):
+        x = make_attn_inputs(rng, B, Hq, Hkv, D, 0)
+        parent = random_tree(B, rng)[0]
+        qs.append(x["q"]); tks.append(x["tree_k"]); tvs.append(x["tree_v"]); ancs.append(anc_from_parent(parent, B, B))
+    kp, vp, table = make_paged_cache(rng, seq, 16, Hkv, D, reserve=0)
+    scale = 1.0 / np.sqrt(D)
+    for _ in range(3):                    # (the fault depended on timing: a few launches)
+        out, lse, st = H.run_tree_attn(np.stack(qs), kp, vp, table, seq, np.stack(tks), np.stack(tvs), np.stack(ancs),
+                                       n_nodes, scale, flags=flags)
+        assert st == 0 and not np.isnan(out).any()
+    for b in sorted({0, batch - 1, int(np.argmin(seq)), int(np.argmax(seq))}):
+        kpre = gather_paged_prefix(kp, table[b], int(seq[b]))
+        vpre = gather_paged_prefix(vp, table[b], int(seq[b]))
+        rows = [(int(rng.integers(0, B)), int(rng.integers(0, Hq))) for _ in range(10)] + [(0, 0), (B - 1, Hq - 1)]
+        ref, rlse = tree_attn_rows_ref(qs[b], kpre, vpre, tks[b], tvs[b], ancs[b], B, scale, rows)
+        got = np.stack([out[b, v, h] for v, h in rows])
+        err = np.abs(got - ref)
+        assert (err <= 2.0 ** -8 * (np.abs(ref) + V_MAX) + 2e-3).all(), (b, float(err.max()))
+        assert np.abs(np.array([lse[b, h, v] for v, h in rows]) - rlse).max() <= 2e-3
