@@ -1016,10 +1016,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int stage = pos.x;
             const uint32_t par = pos.y;
             if (tl == 8 && lane == 0) JET_TR(58);
-            ok = bounded_wait(bar(Bars::kKvFull + stage), par, abort_flag, 7);
+            // P first: once P of this tile exists its Q K^T is complete, i.e. every K tile up to this one has landed.
+            // In the shared ring the stages of V tiles 1 and 2 were first used by K tiles 0 and 2, whose phases this
+            // warp has not seen; behind the P wait the parity of the V tile's phase cannot be mistaken for theirs.
+            ok = bounded_wait(bar(Bars::kPFull + w), j & 1, abort_flag, 8);
             if (!ok) break;
             if (tl == 8 && lane == 0) JET_TR(59);
-            ok = bounded_wait(bar(Bars::kPFull + w), j & 1, abort_flag, 8);
+            ok = bounded_wait(bar(Bars::kKvFull + stage), par, abort_flag, 7);
             if (!ok) break;
             if (tl == 8 && lane == 0) JET_TR(60);
             ptx::tc_fence_after();
