@@ -153,7 +153,9 @@ struct Bars {       // offsets (in 8-byte units) inside the barrier block
          kLoopFirst = kKvFull, kLoopEnd = kClusterA };    // the key loop's barriers exist twice (one set per pass)
 };
 
-// Every wait is bounded: at most kWaitRounds suspensions of kWaitHintNs each (about a second).
+// Every wait is bounded: at most kWaitRounds suspensions of at most kWaitHintNs each -- a second at the longest; the
+// hardware may end a suspension early, and waits that did run out were seen to do so after some tens of
+// milliseconds, still far beyond anything a launch of well under a millisecond waits for.
 // Register split (setmaxnreg): warps 0-3 (producer, MMA issuer, helpers) keep kRegsControl registers per
 // thread, the softmax warpgroups get kRegsSoftmax; 128 * kRegsControl + 256 * kRegsSoftmax must not exceed
 // the 384 * 168 registers the CTA is launched with.
