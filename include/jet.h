@@ -327,6 +327,12 @@ JET_API jet_status jet_tree_verify_attn_tail_ex(const void* q, const void* k_cac
  *                V entries.  Arg-max ties -> lowest index.  No NaN.
  *   token, parent, depth   i32 [batch, B]  (from jet_tree_build)
  *   anc_mask, n_nodes      as produced by jet_tree_build
+ *                The tree arrays are not validated (they live in device memory).
+ *                Arrays that do not describe a tree give a meaningless result,
+ *                but never a store outside the outputs: n_nodes is clipped to B,
+ *                a depth outside 0 .. N is clamped / its node left out of path
+ *                and out_tokens, a parent outside the tree never matches.  The
+ *                same holds for the _static, _hidden and _sample forms.
  *   tgt_argmax   i32 [batch, B] out (-1 on padding rows)
  *   accept_len   i32 [batch] out: a = number of accepted draft nodes (root not
  *                counted); end node v* = deepest accepted node, ties -> lowest

@@ -110,7 +110,7 @@ accept_path_kernel(const unsigned long long* __restrict__ partial, int nchunks,
   __shared__ int s_end;
 
   const int b = blockIdx.x, v = threadIdx.x, lane = v & 31, warp = v >> 5;
-  const int n = n_nodes[b];
+  const int n = min(n_nodes[b], B);
   const int words = (B + 31) / 32;
   const size_t o = static_cast<size_t>(b) * B;
   const bool live = v < n;              // blockDim.x >= B, n <= B
@@ -155,12 +155,14 @@ accept_path_kernel(const unsigned long long* __restrict__ partial, int nchunks,
   if (v < words) s_end_row[v] = anc_mask[(o + end) * words + v];
   __syncthreads();
 
-  const int a = s_tgt[end] >= 0 ? depth[o + end] : 0;
+  // (clamped: the arrays of a tree are the caller's and are not validated; a depth outside 0 .. N must not turn
+  //  into a store outside the N + 1 entries of this sequence's outputs)
+  const int a = s_tgt[end] >= 0 ? min(max(depth[o + end], 0), N) : 0;
   int32_t* my_path = path + static_cast<size_t>(b) * (N + 1);
   int32_t* my_tok = out_tokens + static_cast<size_t>(b) * (N + 1);
   for (int i = v; i <= N; i += blockDim.x)
     if (i > a) { my_path[i] = -1; my_tok[i] = -1; }
-  if (live && ((s_end_row[v >> 5] >> (v & 31)) & 1u) && my_depth <= N) {
+  if (live && ((s_end_row[v >> 5] >> (v & 31)) & 1u) && my_depth >= 0 && my_depth <= N) {
     my_path[my_depth] = v;
     if (my_depth >= 1) my_tok[my_depth - 1] = my_token;
   }

@@ -147,7 +147,7 @@ accept_sample_kernel(const float2* __restrict__ partial, int nchunks, const floa
   float alpha = 1.0f;
   bool ok = live && v == 0;
   if (live) { my_parent = parent[o + v]; my_depth = depth[o + v]; my_token = token[o + v]; }
-  if (live && v > 0 && my_parent >= 0 && my_parent < n && my_token >= 0 && my_token < V) {
+  if (live && v > 0 && my_parent >= 0 && my_parent < n && my_token >= 0 && my_token < V && my_depth >= 1 && my_depth <= N) {
     const float lq = lp[static_cast<int64_t>(my_depth - 1) * logp_depth_stride + my_token];
     if (lq > -INFINITY) {
       const float x = logits[static_cast<int64_t>(o + my_parent) * row_stride + my_token];
@@ -181,7 +181,9 @@ accept_sample_kernel(const float2* __restrict__ partial, int nchunks, const floa
   if (v < words) s_end_row[v] = anc_mask[(o + end) * words + v];
   if (live && my_parent == end) s_has_child = 1;          // benign race: every writer stores 1
   __syncthreads();
-  const int a = n > 0 ? depth[o + end] : 0;
+  // (clamped: the arrays of a tree are the caller's and are not validated; a depth outside 0 .. N must not turn
+  //  into a store outside the N + 1 entries of this sequence's outputs)
+  const int a = n > 0 ? min(max(depth[o + end], 0), N) : 0;
   const bool residual = s_has_child != 0;
 
   // ---- correction token: inverse CDF over the vocabulary of r(x) = max(0, p(x) - q(x)) (or p(x)).
@@ -332,7 +334,7 @@ accept_sample_kernel(const float2* __restrict__ partial, int nchunks, const floa
   int32_t* my_tok = out_tokens + static_cast<size_t>(b) * (N + 1);
   for (int i = v; i <= N; i += kSampleThreads)
     if (i > a) { my_path[i] = -1; my_tok[i] = -1; }
-  if (live && ((s_end_row[v >> 5] >> (v & 31)) & 1u) && my_depth <= N) {
+  if (live && ((s_end_row[v >> 5] >> (v & 31)) & 1u) && my_depth >= 0 && my_depth <= N) {
     my_path[my_depth] = v;
     if (my_depth >= 1) my_tok[my_depth - 1] = my_token;
   }

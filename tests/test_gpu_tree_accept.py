@@ -123,3 +123,25 @@ def test_star_and_duplicate_sibling_tokens():
     anc = anc_from_parent(parent, B, B)
     got = _compare(logits[None], token[None], parent[None], depth[None], anc[None], np.array([B]), N)
     assert got["path"][0].tolist() == [0, 1, -1]
+
+
+def test_tree_arrays_that_are_not_a_tree_stay_inside_the_outputs():
+    """The tree arrays are the caller's and are not validated.  Whatever they hold -- depths outside 0 .. N, parents
+    outside the tree, node counts beyond the budget, arbitrary mask bits -- every store of the call must stay inside
+    its output tensors (sentinel margins around them are checked) and the call must end without an error."""
+    import jet_harness as H
+    rng = np.random.default_rng(77)
+    batch, B, V, N = 3, 70, 1000, 6
+    logits = rng.standard_normal((batch, B, V)).astype(np.float32)
+    token = rng.integers(-5, V + 5, size=(batch, B)).astype(np.int32)
+    parent = rng.integers(-5, 2 * B, size=(batch, B)).astype(np.int32)
+    depth = rng.integers(-1000, 1000, size=(batch, B)).astype(np.int32)
+    anc = rng.integers(0, 2 ** 32, size=(batch, B, (B + 31) // 32), dtype=np.uint64).astype(np.uint32)
+    n_nodes = np.array([B + 100, B, 1], np.int32)
+    got = H.run_tree_accept(logits, token, parent, depth, anc, n_nodes, N)       # checks the margins
+    assert ((got["accept_len"] >= 0) & (got["accept_len"] <= N)).all()
+    u = rng.random((batch, B)).astype(np.float32)
+    logp = np.log(np.full((batch, N, V), 1.0 / V, np.float32))
+    got = H.run_tree_accept_sample(logits, 1.0, logp, token, parent, depth, anc, np.minimum(n_nodes, B), N, u,
+                                   rng.random(batch).astype(np.float32))
+    assert ((got["accept_len"] >= 0) & (got["accept_len"] <= N)).all()
