@@ -21,7 +21,9 @@ kv_compact_kernel(const uint4* __restrict__ tree_k, const uint4* __restrict__ tr
   if (node < 0 || node >= B) return;
   const int64_t pos = static_cast<int64_t>(seq_len[b]) + i;
   int64_t dst_row;
+  if (pos < 0) return;
   if (page_table) {
+    if (pos / page_size >= max_pages) return;        // (a length beyond the table is the caller's error: no access outside it)
     const int page = page_table[static_cast<size_t>(b) * max_pages + pos / page_size];
     dst_row = static_cast<int64_t>(page) * page_size + pos % page_size;
     dst_row = layer * layer_stride16 + dst_row * row16;
@@ -54,7 +56,10 @@ kv_compact_tail_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
   const int64_t L = seq_len[b];
   auto row_of = [&](int64_t pos) -> int64_t {
     if (page_table) {
-      const int page = page_table[static_cast<size_t>(b) * max_pages + pos / page_size];
+      // (the index is kept inside the table: a length beyond it is the caller's error and must not become an access
+      //  outside the table)
+      const int64_t slot = min(max(pos / page_size, static_cast<int64_t>(0)), static_cast<int64_t>(max_pages - 1));
+      const int page = page_table[static_cast<size_t>(b) * max_pages + slot];
       return layer * layer_stride16 + (static_cast<int64_t>(page) * page_size + pos % page_size) * row16;
     }
     return layer * layer_stride16 + b * batch_stride16 + pos * row16;

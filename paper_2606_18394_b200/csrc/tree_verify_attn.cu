@@ -870,7 +870,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       // paged cache: lane i holds the page of the tile's i-th 16-row block; the ids of the next tile are
       // fetched while the current tile's copies are issued, so the table look-up is off the critical path
       auto tile_page = [&](int t) -> int {
-        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= Lc) return 0;
+        // (the last test: a sequence length beyond what the table covers -- the caller's error -- must not become a
+        //  read outside the table)
+        if (!p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= Lc || t * 8 + lane >= p.max_pages) return 0;
         return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
       };
       int kt = first, vt = 0;                   // next K tile, next V tile (first > 0 only without pages)
