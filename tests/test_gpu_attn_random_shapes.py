@@ -4,7 +4,7 @@ Every case draws head layout (G = 1 .. 16, 1 .. 4 KV heads, D 64 / 128), batch (
 ragged prefix lengths (0 .. 2600, contiguous or paged), live node counts, tree shape, softmax scale and the
 stable-prefix flag, so that the launch planner is exercised far from the benchmark shapes: every merge form of
 the key slices, one and two query tiles per CTA, sorted launch order with slices, clusters up to the largest
-size.  All rows of every sequence are compared.
+size.  All rows of every sequence are compared.  120 further cases use the in-cache layout (tree rows behind the prefix).
 
 Tolerance: the arithmetic bound |err| <= 2^-8 (|ref| + max |v|) + 2e-3 element-wise (probabilities rounded to
 bf16 before they weigh V entries of size up to 4.5, output rounded to bf16), mean |err| <= 2.5e-3 over the live
@@ -111,6 +111,60 @@ def test_random_configurations(block):
         D, G, Hkv, batch, B, seq, n_nodes, paged, flags, scale, wide = _draw(rng)
         try:
             _run_case(rng, D, G, Hkv, batch, B, seq, n_nodes, paged, flags, scale, wide)
+        except AssertionError as e:
+            raise AssertionError(f"case {block}/{it}: D={D} G={G} Hkv={Hkv} batch={batch} B={B} seq={seq.tolist()} "
+                                 f"n={n_nodes.tolist()} paged={paged} flags={flags} scale={scale}: {e}") from e
+
+
+def _run_case_in_cache(rng, D, G, Hkv, batch, B, seq, n_nodes, paged, flags, scale):
+    """The same comparison for the in-cache layout: node v of sequence b sits at cache position seq[b] + v."""
+    import jet_harness as H
+    Hq = G * Hkv
+    xs, qs, ancs = [], [], []
+    for b in range(batch):
+        x = make_attn_inputs(rng, B, Hq, Hkv, D, int(seq[b]))
+        parent = random_tree(int(n_nodes[b]), rng)[0]
+        xs.append(x); qs.append(x["q"]); ancs.append(anc_from_parent(parent, int(n_nodes[b]), B))
+    if paged:
+        kp, vp, table = make_paged_cache(rng, seq, 16, Hkv, D, reserve=B)
+        kp[:], vp[:] = NAN_BITS, NAN_BITS
+        for b in range(batch):
+            n, L = int(n_nodes[b]), int(seq[b])
+            rows_k = np.concatenate([xs[b]["k_prefix"], xs[b]["tree_k"][:n]])
+            rows_v = np.concatenate([xs[b]["v_prefix"], xs[b]["tree_v"][:n]])
+            for pos in range(L + n):
+                kp[table[b, pos // 16], pos % 16] = rows_k[pos]
+                vp[table[b, pos // 16], pos % 16] = rows_v[pos]
+        out, lse, st = H.run_tree_attn_tail(np.stack(qs), kp, vp, table, seq, np.stack(ancs), n_nodes, scale,
+                                            table.shape[1] * 16, Hkv, flags=flags)
+    else:
+        rows = int(seq.max()) + B + 7
+        kc = np.full((batch, rows, Hkv, D), NAN_BITS, np.uint16)
+        vc = np.full_like(kc, NAN_BITS)
+        for b in range(batch):
+            n, L = int(n_nodes[b]), int(seq[b])
+            kc[b, :L], vc[b, :L] = xs[b]["k_prefix"], xs[b]["v_prefix"]
+            kc[b, L:L + n], vc[b, L:L + n] = xs[b]["tree_k"][:n], xs[b]["tree_v"][:n]
+        out, lse, st = H.run_tree_attn_tail(np.stack(qs), kc, vc, None, seq, np.stack(ancs), n_nodes, scale, rows, Hkv,
+                                            flags=flags)
+    assert st == 0 and not np.isnan(out).any()
+    for b in range(batch):
+        n = int(n_nodes[b])
+        ref, rlse = tree_attn_ref(qs[b], xs[b]["k_prefix"], xs[b]["v_prefix"], xs[b]["tree_k"], xs[b]["tree_v"], ancs[b],
+                                  n, scale)
+        err = np.abs(out[b] - ref)[:n]
+        assert (err <= 2.0 ** -8 * (np.abs(ref[:n]) + V_MAX) + 2e-3).all(), (b, float(err.max()))
+        assert (out[b, n:] == 0).all()
+        assert np.abs(lse[b][:, :n] - rlse[:, :n]).max() <= 2e-3
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_random_configurations_in_cache_layout(block):
+    for it in range(30):
+        rng = np.random.default_rng(99991 * (block + 1) + it)
+        D, G, Hkv, batch, B, seq, n_nodes, paged, flags, scale, _ = _draw(rng)
+        try:
+            _run_case_in_cache(rng, D, G, Hkv, batch, B, seq, n_nodes, paged, flags, scale)
         except AssertionError as e:
             raise AssertionError(f"case {block}/{it}: D={D} G={G} Hkv={Hkv} batch={batch} B={B} seq={seq.tolist()} "
                                  f"n={n_nodes.tolist()} paged={paged} flags={flags} scale={scale}: {e}") from e
