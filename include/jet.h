@@ -230,6 +230,10 @@ JET_API jet_status jet_tree_build_logits(const float* logits, int64_t logits_bat
  * waits inside a kernel, the counters are unused and the residency assumption
  * falls away; jet_tree_verify_attn_launches tells which form a shape gets.
  * JET_FORCE_SPLIT="<slices>,g" / ",h" selects the one- / two-launch form.)
+ * Stream capture: the first call for a shape family on a device configures the
+ * kernel (shared-memory size, cluster attribute) and asks the driver how many
+ * clusters fit; make it outside any stream capture (one warm-up call per head
+ * size and query-tile grouping is enough), later calls can be captured.
  * Test hooks, read from the environment once per process and meant for the
  * test-suite only: JET_FORCE_MT / JET_FORCE_SPLIT force a launch plan (query
  * tiles per CTA; key slices, with ",g" / ",h" through the workspace in one / two launches),
