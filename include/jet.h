@@ -237,7 +237,11 @@ JET_API jet_status jet_tree_build_logits(const float* logits, int64_t logits_bat
  * Test hooks, read from the environment once per process and meant for the
  * test-suite only: JET_FORCE_MT / JET_FORCE_SPLIT force a launch plan (query
  * tiles per CTA; key slices, with ",g" / ",h" through the workspace in one / two launches),
- * JET_TEST_POLL_LIMIT shortens the bounded wait of the workspace exchange.
+ * JET_TEST_POLL_LIMIT shortens the bounded wait of the workspace exchange,
+ * JET_FORCE_PAIR=1 runs pairs of consecutive query tiles of a work item as CTA
+ * pairs that share every K/V tile (D = 128, one query tile per CTA, an even
+ * number of query tiles per KV head; built and kept for measurement: slower than
+ * the default form, which the planner therefore always prefers).
  */
 JET_API size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, int Hkv, int D,
                                             int max_seq_len);
@@ -247,6 +251,16 @@ JET_API size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq, in
  * count launches (CUDA-graph sizing, launch statistics); same arguments as the workspace query.
  */
 JET_API int jet_tree_verify_attn_launches(int batch, int B, int Hq, int Hkv, int D, int max_seq_len);
+
+/* The launch plan of one attention call of this shape on the calling thread's current device, for tests and for
+ * reading timings: plan (HOST pointer, 5 entries) receives
+ *   [0] query tiles of 128 rows per CTA (1 or 2)         [1] groups of such tiles per (sequence, KV head)
+ *   [2] key slices per work item                         [3] how the slices are combined: 0 = no slices, 1 = inside
+ *       a thread-block cluster, 2 = through the workspace in the one launch, 3 = by a second launch
+ *   [4] 1 if consecutive query tiles run as CTA pairs (tcgen05 cta_group::2; only with JET_FORCE_PAIR=1).
+ * Returns 1, or 0 for an invalid shape.  Same arguments as the workspace query.
+ */
+JET_API int jet_tree_verify_attn_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len, int32_t* plan);
 
 JET_API jet_status jet_tree_verify_attn(const void* q, const void* k_cache, const void* v_cache,
                                 const int32_t* page_table, int max_pages_per_seq, int page_size,

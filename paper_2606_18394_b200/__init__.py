@@ -33,6 +33,7 @@ from .binding import (  # noqa: F401
     jet_tree_verify_attn,
     jet_tree_verify_attn_ex,
     jet_tree_verify_attn_launches,
+    jet_tree_verify_attn_plan,
     jet_tree_verify_attn_tail,
     jet_tree_verify_attn_tail_ex,
     jet_tree_verify_attn_workspace_bytes,

@@ -39,6 +39,7 @@ _SIGNATURES = {
                                            _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_tree_verify_attn_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "jet_tree_verify_attn_launches": (_i, [_i, _i, _i, _i, _i, _i]),
+    "jet_tree_verify_attn_plan": (_i, [_i, _i, _i, _i, _i, _i, _vp]),
     "jet_tree_verify_attn": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp,
                                           _i, _i, _i, _i, _i, _i64, _f, _vp, _vp, _vp, _vp, _sz, _vp]),
     "jet_tree_verify_attn_tail": (_c.c_int32, [_vp, _vp, _vp, _vp, _i, _i, _i64, _vp, _i, _vp, _vp,
@@ -187,6 +188,15 @@ def jet_tree_verify_attn_workspace_bytes(batch, B, Hq, Hkv, D, max_seq_len) -> i
 
 def jet_tree_verify_attn_launches(batch, B, Hq, Hkv, D, max_seq_len) -> int:
     return load().jet_tree_verify_attn_launches(batch, B, Hq, Hkv, D, max_seq_len)
+
+
+def jet_tree_verify_attn_plan(batch, B, Hq, Hkv, D, max_seq_len) -> dict:
+    """The launch plan of a shape: query tiles per CTA, tile groups, key slices, merge form, CTA pairs."""
+    out = (_c.c_int32 * 5)()
+    if not load().jet_tree_verify_attn_plan(batch, B, Hq, Hkv, D, max_seq_len, _c.cast(out, _c.c_void_p)):
+        raise JetError(JET_ERR_INVALID_ARG, "jet_tree_verify_attn_plan")
+    forms = {0: "none", 1: "cluster", 2: "workspace", 3: "second launch"}
+    return dict(query_tiles_per_cta=out[0], tile_groups=out[1], key_slices=out[2], merge=forms[out[3]], pair=bool(out[4]))
 
 
 def jet_tree_verify_attn(q, k_cache, v_cache, page_table, max_pages_per_seq, page_size, num_pages, seq_len,

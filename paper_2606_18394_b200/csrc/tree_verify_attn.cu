@@ -99,20 +99,24 @@ __device__ __forceinline__ uint32_t udiv(uint32_t x, uint32_t magic) { return ma
 #define JET_TR(slot) do { } while (0)
 #endif
 
-template <int D, int MT>
+// kPair: two CTAs (a cluster of two, consecutive query tiles of one work item) share every K/V tile -- each
+// loads half of it, and the products run as tcgen05 pair instructions (see "CTA pairs" in the kernel).
+template <int D, int MT, bool kPair = false>
 struct Cfg {
+  static_assert(!kPair || (D == 128 && MT == 1), "the CTA-pair form exists for one 128-wide query tile per CTA");
   static constexpr int kHalves = D / 64;
   static constexpr int kQBytes = MT * kHalves * kHalfBytes;
   // P (probabilities, bf16) never touches shared memory: it is written to TMEM (two bf16 per 32-bit column)
   // and read from there by the P V product.
   static constexpr int kPBytes = 0;
-  static constexpr int kStageBytes = kHalves * kHalfBytes;
-  static constexpr int kStages = (D == 128) ? (MT == 1 ? 6 : 5) : 6;
+  // (a pair's stage holds half a tile: 64 keys x D of K, or 128 keys x 64 columns of V)
+  static constexpr int kStageBytes = kPair ? kHalfBytes : kHalves * kHalfBytes;
+  static constexpr int kStages = kPair ? 10 : (D == 128) ? (MT == 1 ? 6 : 5) : 6;
   static constexpr int kTileBytes = kQBytes + kPBytes + kStages * kStageBytes;
   // Two softmax warpgroups in every form: with one query tile per CTA they share the tile's key tiles (even /
   // odd), with two each takes one query tile.
   static constexpr int kStreams = MT == 1 ? 2 : 1;
-  static constexpr int kBarBytes = 1024;
+  static constexpr int kBarBytes = kPair ? 2048 : 1024;
   static constexpr int kSmemBytes = kTileBytes + kBarBytes + 1024;
   static constexpr int kThreads = 128 + 128 * MT * kStreams;
   // TMEM (512 columns), three layouts (the key loop's forms are described in the kernel):
@@ -153,6 +157,17 @@ struct Bars {       // offsets (in 8-byte units) inside the barrier block
          kLoopFirst = kKvFull, kLoopEnd = kClusterA };    // the key loop's barriers exist twice (one set per pass)
 };
 
+// Barriers of the CTA-pair form.  Fixed ones first, then one set of key-loop barriers per pass (a pair
+// runs up to three passes over its keys, each on a fresh set: an arrival of the pass before that is still in
+// flight can then never land in a later phase).  kKvFull: this CTA's half of a stage has landed; kKvReady (used
+// in the even CTA): both halves are in place; kKvEmpty: the products that read the stage are complete.
+struct PBars {
+  enum { kQFull = 0, kQReady = 1, kRecv = 2, kFixed = 4,
+         kSFull = 0, kSFree = 2, kPFull = 4, kODone = 6, kOFinal = 8, kKvFull = 9, kKvReady = 19, kKvEmpty = 29,
+         kSet = 39, kPasses = 3, kCount = kFixed + kPasses * kSet };
+};
+static_assert(PBars::kKvReady - PBars::kKvFull == Cfg<128, 1, true>::kStages && PBars::kCount * 8 <= 1024, "pair barrier layout");
+
 // Every wait is bounded: at most kWaitRounds suspensions of at most kWaitHintNs each -- a second at the longest; the
 // hardware may end a suspension early, and waits that did run out were seen to do so after some tens of
 // milliseconds, still far beyond anything a launch of well under a millisecond waits for.
@@ -184,6 +199,18 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, vola
                                              uint32_t site) {
   if (__all_sync(0xffffffffu, ptx::mbar_test(bar, parity))) return true;
   return bounded_wait_slow(bar, parity, abort_flag, site);
+}
+
+// Warp-level wait on a barrier that threads of another CTA of the cluster arrive on (acquire at cluster scope).
+__device__ __forceinline__ bool bounded_wait_cl(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                uint32_t site) {
+  bool ok = false;
+  for (uint32_t i = 0; i < kWaitRounds; ++i) {
+    if (ptx::mbar_try_wait_cluster(bar, parity, kWaitHintNs)) { ok = true; break; }
+    if (*abort_flag) break;
+  }
+  if (!ok && *abort_flag == 0u) *abort_flag = 1u + site;
+  return __all_sync(0xffffffffu, ok);
 }
 
 // The same for a barrier that other CTAs of the cluster arrive on / copy into (acquire at cluster
@@ -249,12 +276,14 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&x)[32], float sl2, fl
 }
 
 // kSorted: the sequences of a batch are launched longest prefix first (see the set-up of warp 3).
-template <int D, int MT, bool kSorted = false>
-__global__ void __launch_bounds__(Cfg<D, MT>::kThreads, 1)
+// tm_k64 / tm_tk64: the K maps with boxes of 64 rows (a pair CTA's half of a key tile); unused otherwise.
+template <int D, int MT, bool kSorted = false, bool kPair = false>
+__global__ void __launch_bounds__(Cfg<D, MT, kPair>::kThreads, 1)
 tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tk,
-                 const __grid_constant__ CUtensorMap tm_tv, const AttnParams p) {
-  using C = Cfg<D, MT>;
+                 const __grid_constant__ CUtensorMap tm_tv, const __grid_constant__ CUtensorMap tm_k64,
+                 const __grid_constant__ CUtensorMap tm_tk64, const AttnParams p) {
+  using C = Cfg<D, MT, kPair>;
   constexpr int kHalves = C::kHalves;
   constexpr int kStages = C::kStages;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -276,20 +305,28 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t sBar = sKV + kStages * C::kStageBytes;
   uint8_t* gen_kv = smem_gen + C::kQBytes;
   uint8_t* gen_bar = gen_kv + kStages * C::kStageBytes;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + 2 * Bars::kCount * 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bar + (kPair ? 1024 : 2 * Bars::kCount * 8));
   volatile uint32_t* abort_flag = tmem_slot + 1;
   volatile int* seq_slot = reinterpret_cast<volatile int*>(tmem_slot + 2);     // sequence of this CTA when launch order is sorted
   volatile uint32_t* redo_flag = tmem_slot + 3;          // the shared-accumulator pass met a row it cannot hold
-  float* ref_s = reinterpret_cast<float*>(gen_bar + 512);  // [128] the rows' common reference (shared-accumulator pass)
-  static_assert(2 * Bars::kCount * 8 + 16 <= 512 && 512 + 128 * 4 <= C::kBarBytes, "barrier block layout");
+  // pair form: redo flag of pass i at redo_flag[i]; pair_slot[pass][rank] = what each CTA of the pair reported
+  volatile uint32_t* pair_slot = tmem_slot + 8;
+  float* ref_s = reinterpret_cast<float*>(gen_bar + (kPair ? 1536 : 512));  // [128] the rows' common reference (shared-accumulator pass)
+  static_assert(2 * Bars::kCount * 8 + 16 <= 512 && 512 + 128 * 4 <= 1024, "barrier block layout");
+  constexpr int kRecvBar = kPair ? static_cast<int>(PBars::kRecv) : static_cast<int>(Bars::kRecv);
   auto bar = [&](int idx) { return sBar + 8u * idx; };
   uint32_t sBarLoop = sBar;        // base of the key loop's barrier set in use
   auto lbar = [&](int idx) { return sBarLoop + 8u * idx; };
   const int S = p.nsplit;                            // key slices = cluster size
   // ---------------- work item: what the launch parameters alone decide.  Grid = (query-tile groups x slices,
   // KV heads, sequences); CTAs are dispatched x first, so a unit's slices are neighbours.
-  const int mgroup = static_cast<int>(udiv(blockIdx.x, p.magic_S));
-  const int split = static_cast<int>(blockIdx.x) - mgroup * S;    // = rank in the cluster
+  // CTA pairs: blockIdx.x = (pair of query tiles x slices) x 2 + rank; the two CTAs of a pair (a cluster of
+  // two) take the query tiles 2k and 2k + 1 of the work item and the same key slice.
+  const uint32_t prank = kPair ? (blockIdx.x & 1u) : 0u;
+  const uint32_t bx_item = kPair ? (blockIdx.x >> 1) : blockIdx.x;
+  const int mgroup_item = static_cast<int>(udiv(bx_item, p.magic_S));
+  const int split = static_cast<int>(bx_item) - mgroup_item * S;    // = rank in the cluster of slices
+  const int mgroup = kPair ? 2 * mgroup_item + static_cast<int>(prank) : mgroup_item;
   const int g = blockIdx.y;
   const int b_rank = blockIdx.z;                 // position of the sequence in launch order
   constexpr bool sorted_launch = kSorted;
@@ -298,9 +335,31 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int node_lo = mgroup * MT * npt;
   const int node_hi = min(p.B, node_lo + MT * npt);
   const int n_mt = (MT == 2 && node_hi - node_lo > npt) ? 2 : 1;     // query tiles of this CTA that hold nodes
+  // last node (exclusive) of the pair's two query tiles: both CTAs of a pair walk the same key tiles
+  const int node_hi_item = kPair ? min(p.B, (mgroup_item * 2 + 2) * npt) : node_hi;
 
   // ---------------- set-up that touches no global memory (may overlap the previous kernel's tail)
-  if (warp == 0) {
+  if (kPair && warp == 0) {
+    for (int i = lane; i < PBars::kCount; i += 32) {
+      uint32_t count = 1;
+      if (i == PBars::kQReady) count = 2;                       // one arrival per CTA of the pair
+      if (i >= PBars::kFixed) {
+        const int k = (i - PBars::kFixed) % PBars::kSet;
+        if (k >= PBars::kSFree && k < PBars::kODone) count = 8;       // kSFree, kPFull: the four warps of a warpgroup, both CTAs
+        else if (k >= PBars::kKvReady && k < PBars::kKvEmpty) count = 2;
+      }
+      ptx::mbar_init(bar(i), count);
+      if (S > 1 && i == PBars::kRecv)
+        ptx::mbar_arrive_expect_tx(bar(i), S * max(0, min(p.rows_per, kBM - split * p.rows_per)) * C::kRecvPitch);
+    }
+    ptx::fence_mbar_init();
+    if (lane == 31) {
+      redo_flag[0] = 0u;
+      redo_flag[1] = 0u;
+      redo_flag[2] = 0u;
+      *abort_flag = 0u;
+    }
+  } else if (warp == 0) {
     // one lane per barrier of the block
     if (lane < Bars::kCount) {
       uint32_t count = 1;
@@ -317,8 +376,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       *abort_flag = 0u;
     }
   } else if (warp == 2) {
-    ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
-    ptx::tmem_relinquish();
+    if constexpr (kPair) {
+      ptx::tmem_alloc2(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
+      ptx::tmem_relinquish2();
+    } else {
+      ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
+      ptx::tmem_relinquish();
+    }
     if (lane == 0) JET_TR(44);
   } else if (warp == 3) {
     if (lane == 0) {
@@ -327,13 +391,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ptx::prefetch_tmap(&tm_v);
       ptx::prefetch_tmap(&tm_tk);
       ptx::prefetch_tmap(&tm_tv);
+      if constexpr (kPair) {
+        ptx::prefetch_tmap(&tm_k64);
+        ptx::prefetch_tmap(&tm_tk64);
+      }
     }
     // A single sequence's length is very often exactly the caller's bound.  On that guess this slice's first
     // key tiles are asked into L2 now -- before the grid dependency wait, under the previous kernel's tail: L2
     // is where that kernel's writes arrive, so a line prefetched early cannot go stale -- and the copies
     // proper (issued once the real lengths are known) find them there.  A wrong guess costs a few tiles of
     // traffic and nothing else.
-    if (!sorted_launch && lane == 0 && p.len_hint > 0) {
+    if (!kPair && !sorted_launch && lane == 0 && p.len_hint > 0) {
       // (the CTA index is read afresh so that nothing here lengthens a live range of the main path)
       uint32_t bx, by, bz;
       asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(bx));
@@ -391,6 +459,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (tid == 0) JET_TR(40);
   ptx::tc_fence_before();
   ptx::cta_sync();
+  // (a pair's barriers take arrivals from the other CTA: both sets exist before either CTA goes on)
+  if constexpr (kPair) ptx::cluster_sync_all();
   ptx::tc_fence_after();
   if (tid == 0) JET_TR(41);
   // The barriers of every CTA of the cluster must exist before any CTA arrives on them remotely:
@@ -426,7 +496,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   const int L = p.seq_len[b];
   const int n = min(p.n_nodes[b], p.B);
-  const int ntree = min(n, node_hi);                         // tree keys any row here can see
+  const int ntree = min(n, node_hi_item);                    // tree keys any row here can see
   // Keys that come out of the cache: the prefix, and with p.tail also the tree's own rows behind it (then
   // there are no separate tree tiles: key j >= L is tree node j - L).
   const int Lc = p.tail ? L + ntree : L;
@@ -444,7 +514,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     t_hi = static_cast<int>((static_cast<uint32_t>(T_all) * (split + 1) + S - 1) / static_cast<uint32_t>(S));
   }
   const int T = t_hi - t_lo;
-  const bool has_work = node_lo < n && T > 0;    // otherwise: no live node here, or an empty key slice
+  // otherwise: no live node here (pair: in neither of its query tiles), or an empty key slice
+  const bool has_work = (kPair ? mgroup_item * 2 * npt : node_lo) < n && T > 0;
   // A CTA without work never looks at its query rows, but they must have landed before the epilogue reuses
   // their memory (and before the CTA exits).
   if (!has_work && warp == 3) bounded_wait(bar(Bars::kQFull), 0, abort_flag, 3);
@@ -453,7 +524,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   // the first Q K^T waits for exactly these tiles.  They are the first items of the ring in every form of
   // the key loop (ring order starts K_0 .. K_ahead); the producers start behind them.  A paged tile needs
   // its page ids first and is left to the producers.
-  int n_early = (has_work && !p.paged) ? (MT == 1 ? min(2, T) : 1) : 0;
+  int n_early = (has_work && !p.paged && !kPair) ? (MT == 1 ? min(2, T) : 1) : 0;
   if (early) {         // before the dependency wait only tiles that lie wholly inside the prefix may be read
     int k = 0;
     while (k < n_early && (t_lo + k + 1) * kBN <= L) ++k;
@@ -491,8 +562,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // occupies a register through the key loop (the softmax threads have none to spare).
     uint32_t e_bx;
     asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(e_bx));
-    const int e_mgroup = static_cast<int>(udiv(e_bx, p.magic_S));
-    const int split = static_cast<int>(e_bx) - e_mgroup * S;
+    const uint32_t e_item = kPair ? (e_bx >> 1) : e_bx;
+    const int e_mgroup_item = static_cast<int>(udiv(e_item, p.magic_S));
+    const int split = static_cast<int>(e_item) - e_mgroup_item * S;
+    const int e_mgroup = kPair ? 2 * e_mgroup_item + static_cast<int>(e_bx & 1u) : e_mgroup_item;
     const int rows_per = p.rows_per;                   // rows of a query tile that one slice combines
     const int own_lo = split * rows_per;
     const int own_n = max(0, min(rows_per, kBM - own_lo));
@@ -706,8 +779,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (!kSm && tid < S && published && own_n > 0)
           ptx::bulk_load_global(smem_base + C::kRecvOff + static_cast<uint32_t>(tid * rows_per * C::kRecvPitch),
                                 slots + (static_cast<size_t>(tid) * MT + mt) * kBlockBytes + own_lo * C::kRecvPitch,
-                                static_cast<uint32_t>(own_n * C::kRecvPitch), bar(Bars::kRecv + mt));
-        rows_ok = published && (own_n == 0 || bounded_wait_cluster(bar(Bars::kRecv + mt), abort_flag, 14));
+                                static_cast<uint32_t>(own_n * C::kRecvPitch), bar(kRecvBar + mt));
+        rows_ok = published && (own_n == 0 || bounded_wait_cluster(bar(kRecvBar + mt), abort_flag, 14));
         if (own_n == 0) ptx::cta_sync();
         if (tid == 128 && mt == 0) JET_TR(9);
         src_rows = smem_gen + C::kRecvOff;
@@ -849,6 +922,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     ptx::cta_sync();
   };
 
+  // End of a pass of the pair form (every thread of both CTAs calls it): each CTA tells the other whether a row
+  // overflowed its reference (bit 0) and whether a wait gave up (bit 1); both go on with the same verdict.
+  auto pair_verdict = [&](int pass) -> uint32_t {
+    ptx::cta_sync();
+    if (tid == 0) {
+      const uint32_t mine = (redo_flag[pass] ? 1u : 0u) | (*abort_flag ? 2u : 0u);
+      pair_slot[pass * 2 + prank] = mine;
+      ptx::st_cluster_u32(ptx::map_to_rank(ptx::smem_u32(const_cast<uint32_t*>(pair_slot + pass * 2 + prank)), prank ^ 1u), mine);
+    }
+    __syncwarp();
+    ptx::cluster_sync_all();
+    return pair_slot[pass * 2] | pair_slot[pass * 2 + 1];
+  };
+
   if (warp < 4) {
     // Warps 0-3 need few registers; what they give up goes to the softmax warpgroups, which hold a whole
     // score row (128 values) per thread.
@@ -963,7 +1050,183 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const uint64_t desc_k0 = ptx::smem_desc_sw128(sKV, 0);
     const uint64_t desc_v0 = ptx::smem_desc_sw128(sKV, kHalfBytes);
 
-    if constexpr (MT == 1) {
+    if constexpr (kPair) {
+      // =========================================================== CTA pairs, warps 0-3
+      // The two CTAs of a pair hold the query tiles 2k and 2k + 1 of one work item and walk the same key tiles
+      // in the shared-accumulator form.  Every product is ONE pair instruction (M = 256) issued by the even CTA:
+      // each CTA's 128 query rows (or its P rows in TMEM) meet all 128 keys of the tile, of which each CTA has
+      // loaded only half -- for Q K^T 64 of the keys, for P V 64 of V's columns -- so a CTA writes and reads
+      // half the shared-memory bytes per key tile that it would alone.  Roles per CTA:
+      //   warp 0  TMA producer of this CTA's halves (kKvFull, local)
+      //   warp 2  forwarder: tells the even CTA that a half has landed (one remote arrival per stage on its
+      //           kKvReady; the V half of a tile that is not full is announced by the softmax warpgroup that
+      //           clears its tail instead)
+      //   warp 1 / warp 3 of the even CTA: issue Q K^T / P V; their commits arrive on the barriers of both CTAs
+      //   softmax warpgroups: as in the shared-accumulator form; kSFree / kPFull arrivals (one per warp) go to
+      //           the even CTA's barriers.
+      // A fixed reference can overflow; the pair then repeats the key range: a pass that only finds every row's
+      // true maximum, and the shared-accumulator pass again with that maximum as the reference (exact).
+      constexpr uint32_t idesc_qk2 = ptx::umma_idesc_bf16(2 * kBM, kBN, false);
+      constexpr uint32_t idesc_pv2 = ptx::umma_idesc_bf16(2 * kBM, D, true);
+      constexpr int kKBlock = 64 * 128;          // one [64 keys x 64 bf16] swizzled block of a K half-tile
+      int mode = 0;                              // 0: reference from the first key tile, 1: row maxima only, 2: given reference
+#pragma unroll 1
+      for (int pass = 0; pass < PBars::kPasses && has_work; ++pass) {
+        sBarLoop = sBar + 8u * (PBars::kFixed + pass * PBars::kSet);
+        const int n_items = mode == 1 ? T : 2 * T;
+        if (warp == 0 || warp == 2) {
+          // ---- producer (warp 0) and forwarder (warp 2) walk the ring in the same order
+          const bool producer = warp == 0;
+          bool ok = true;
+          bool waited = !early || !producer;
+          auto tile_page = [&](int t) -> int {
+            if (!producer || !p.paged || t >= TP || lane >= 8 || t * kBN + lane * 16 >= Lc) return 0;
+            return __ldg(p.page_table + static_cast<size_t>(b) * p.max_pages + t * 8 + lane);
+          };
+          if (!producer && pass == 0) {
+            ok = bounded_wait(bar(PBars::kQFull), 0, abort_flag, 3);
+            if (ok && lane == 0) ptx::mbar_arrive_peer(ptx::map_to_rank(bar(PBars::kQReady), 0));
+          }
+          int kt = 0, vt = 0, issued = 0;
+          int pk_cur = tile_page(t_lo), pk_next = tile_page(t_lo + 1);
+          int pv_cur = pk_cur, pv_next = pk_next;
+#pragma unroll 1
+          for (; issued < n_items && ok; ++issued) {
+            const bool take_k = mode == 1 || (kt < T && kt <= vt + kAhead);
+            const int t = t_lo + (take_k ? kt : vt), stage = issued % kStages;
+            const uint32_t full = lbar(PBars::kKvFull + stage);
+            if (producer) {
+              if (!waited && (t + 1) * kBN > L) {
+                ptx::grid_dep_wait();
+                waited = true;
+              }
+              if (issued >= kStages) {
+                ok = bounded_wait(lbar(PBars::kKvEmpty + stage), ((issued / kStages) - 1) & 1, abort_flag, 1);
+                if (!ok) break;
+              }
+              const uint32_t dst = sKV + stage * C::kStageBytes;
+              if (t < TP && p.paged) {
+                const int npages = min(8, (Lc - t * kBN + 15) / 16);
+                if (take_k) {           // this CTA's 64 keys = pages 4 rank .. 4 rank + 3 of the tile
+                  const int mine = max(0, min(4, npages - 4 * static_cast<int>(prank)));
+                  const int pg = __shfl_sync(0xffffffffu, pk_cur, (4 * static_cast<int>(prank) + lane) & 7);
+                  if (lane == 0) ptx::mbar_arrive_expect_tx(full, mine * kHalves * 2048);
+                  __syncwarp();
+                  if (lane < mine) {
+                    for (int h = 0; h < kHalves; ++h)
+                      ptx::tma_load_3d(dst + h * kKBlock + lane * 2048, &tm_k, full, h * 64, g, pg * 16);
+                  }
+                } else {                // all keys, this CTA's 64 columns
+                  if (lane == 0) ptx::mbar_arrive_expect_tx(full, npages * 2048);
+                  __syncwarp();
+                  if (lane < npages) ptx::tma_load_3d(dst + lane * 2048, &tm_v, full, static_cast<int>(prank) * 64, g, pv_cur * 16);
+                }
+              } else if (lane == 0) {
+                const bool prefix = t < TP;
+                const int row0 = prefix ? t * kBN : (t - TP) * kBN;
+                ptx::mbar_arrive_expect_tx(full, C::kStageBytes);
+                if (take_k) {
+                  for (int h = 0; h < kHalves; ++h)
+                    ptx::tma_load_4d(dst + h * kKBlock, prefix ? &tm_k64 : &tm_tk64, full, h * 64, g,
+                                     row0 + 64 * static_cast<int>(prank), b);
+                } else {
+                  ptx::tma_load_4d(dst, prefix ? &tm_v : &tm_tv, full, static_cast<int>(prank) * 64, g, row0, b);
+                }
+              }
+            } else {
+              ok = bounded_wait(full, (issued / kStages) & 1, abort_flag, 22);
+              if (!ok) break;
+              bool left_to_softmax = false;         // a V tile that is not full: announced once its tail is cleared
+              if (!take_k) {
+                const int valid = t < TP ? min(kBN, Lc - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
+                left_to_softmax = valid < kBN;
+              }
+              if (!left_to_softmax && lane == 0) ptx::mbar_arrive_peer(ptx::map_to_rank(lbar(PBars::kKvReady + stage), 0));
+            }
+            if (take_k) {
+              ++kt;
+              pk_cur = pk_next;
+              pk_next = tile_page(t + 2);
+            } else {
+              ++vt;
+              pv_cur = pv_next;
+              pv_next = tile_page(t + 2);
+            }
+            __syncwarp();
+          }
+          if (producer && __any_sync(0xffffffffu, *abort_flag != 0u)) {
+            // drain: every load that was issued must land before the CTA may exit
+            for (int st = 0; st < kStages; ++st) {
+              if (issued > st) {
+                const int last = ((issued - 1 - st) / kStages) * kStages + st;     // last item issued to stage st
+                bounded_wait(lbar(PBars::kKvFull + st), (last / kStages) & 1, abort_flag, 2);
+              }
+            }
+            bounded_wait(bar(PBars::kQFull), 0, abort_flag, 3);
+          }
+        } else if (prank == 0 && warp == 1) {
+          // ---- Q K^T of both CTAs' query tiles against the whole key tile
+          bool ok = pass > 0 || bounded_wait(bar(PBars::kQReady), 0, abort_flag, 4);
+          const int lead = min(kAhead + 1, T);
+#pragma unroll 1
+          for (int tl = 0; tl < T && ok; ++tl) {
+            const int w = tl & 1, j = tl >> 1;
+            const int item = mode == 1 ? tl : (tl < lead ? tl : 2 * tl - lead + 1);
+            const int stage = item % kStages;
+            if (j > 0) {
+              ok = bounded_wait(lbar(PBars::kSFree + w), (j - 1) & 1, abort_flag, 20);
+              if (!ok) break;
+            }
+            ok = bounded_wait_cl(lbar(PBars::kKvReady + stage), (item / kStages) & 1, abort_flag, 5);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint64_t desc_k = desc_k0 + static_cast<uint64_t>(stage * (C::kStageBytes >> 4));
+            const uint32_t s_tmem = tmem_base + C::shared_s(w);
+            if (ptx::elect_one()) {
+#pragma unroll
+              for (int kd = 0; kd < D / 16; ++kd) {
+                const uint64_t off_q = static_cast<uint64_t>(((kd / 4) * kHalfBytes + (kd % 4) * 32) >> 4);
+                const uint64_t off_k = static_cast<uint64_t>(((kd / 4) * kKBlock + (kd % 4) * 32) >> 4);
+                ptx::umma_ss2(s_tmem, desc_q0 + off_q, desc_k + off_k, idesc_qk2, kd > 0 ? 1u : 0u);
+              }
+              ptx::umma_commit2(lbar(PBars::kSFull + w), 3);
+              ptx::umma_commit2(lbar(PBars::kKvEmpty + stage), 3);
+            }
+          }
+        } else if (prank == 0 && warp == 3 && mode != 1) {
+          // ---- O += P V of both CTAs
+          bool ok = true;
+#pragma unroll 1
+          for (int tl = 0; tl < T && ok; ++tl) {
+            const int w = tl & 1, j = tl >> 1;
+            const int item = v_item(tl, kAhead);
+            const int stage = item % kStages;
+            ok = bounded_wait(lbar(PBars::kPFull + w), j & 1, abort_flag, 8);        // (P first, as in the single-CTA form)
+            if (!ok) break;
+            ok = bounded_wait_cl(lbar(PBars::kKvReady + stage), (item / kStages) & 1, abort_flag, 7);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            const uint64_t desc_v = desc_v0 + static_cast<uint64_t>(stage * (C::kStageBytes >> 4));
+            const uint32_t p_tmem = tmem_base + C::shared_p(w);
+            const uint32_t o_tmem = tmem_base + C::shared_o();
+            if (ptx::elect_one()) {
+#pragma unroll
+              for (int kk = 0; kk < kBN / 16; ++kk)
+                ptx::umma_ts2(o_tmem, p_tmem + kk * 8, desc_v + static_cast<uint64_t>((kk * 2048) >> 4), idesc_pv2,
+                              (tl == 0 && kk == 0) ? 0u : 1u);
+              ptx::umma_commit2(lbar(PBars::kODone + w), 3);
+              ptx::umma_commit2(lbar(PBars::kKvEmpty + stage), 3);
+              if (tl == T - 1) ptx::umma_commit2(lbar(PBars::kOFinal), 3);
+            }
+          }
+        }
+        const uint32_t verdict = pair_verdict(pass);
+        if ((verdict & 2u) || pass == 2 || (pass == 0 && !(verdict & 1u))) break;
+        mode = pass + 1;
+      }
+      classic = false;
+      shared_result = true;
+    } else if constexpr (MT == 1) {
       if (has_work) {
         if (warp == 0) {
           // a paged tile is 16 small copies: two warps request them
@@ -1125,7 +1388,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
 
-    if (!C::kTurns && classic && has_work) {
+    if (!kPair && !C::kTurns && classic && has_work) {
       if (warp == 0) {
         produce(0, std::integral_constant<int, -1>{}, 0);
       } else if (warp == 1) {
@@ -1246,7 +1509,154 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       return true;
     };
 
-    if constexpr (MT == 1) {
+    if constexpr (kPair) {
+      // =========================================================== CTA pairs, softmax warpgroups
+      // The shared-accumulator form on this CTA's own query tile; arrivals that the issuing warps wait for go to
+      // the even CTA's barriers, one per warp.
+      auto arrive_pair = [&](uint32_t local_bar) {
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_peer(ptx::map_to_rank(local_bar, 0));
+      };
+      // This CTA's half of a V tile (all keys, 64 columns): rows of keys beyond the valid ones are cleared, then
+      // the warpgroup announces the half to the even CTA in the forwarder's place.
+      auto clear_v_half = [&](int t, int item) -> bool {
+        const int valid = t < TP ? min(kBN, Lc - t * kBN) : min(kBN, ntree - (t - TP) * kBN);
+        if (valid >= kBN) return true;
+        const int stage = item % kStages;
+        const bool landed = bounded_wait(lbar(PBars::kKvFull + stage), (item / kStages) & 1, abort_flag, 10);
+        if (landed) {
+          uint8_t* vt = gen_kv + stage * C::kStageBytes;
+          const int chunks = (kBN - valid) * 8;
+          for (int i = r; i < chunks; i += 128) *reinterpret_cast<uint4*>(vt + valid * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+          ptx::fence_proxy_async_all();
+        }
+        ptx::named_sync(3 + wg, 128);
+        if (landed && r == 0) ptx::mbar_arrive_remote(ptx::map_to_rank(lbar(PBars::kKvReady + stage), 0));
+        return landed;
+      };
+      float m_ref = 0.0f;
+      int mode = 0;
+      const uint32_t tS = t_lane + C::shared_s(wg);
+      const uint32_t tP = t_lane + C::shared_p(wg);
+#pragma unroll 1
+      for (int pass = 0; pass < PBars::kPasses && has_work; ++pass) {
+        sBarLoop = sBar + 8u * (PBars::kFixed + pass * PBars::kSet);
+        bool ok = true;
+        bool synced = false;
+        bool saw_key = false;
+        float m_run = -INFINITY;
+        l = 0.0f;
+        if (tid == 128) JET_TR(5 + pass);
+#pragma unroll 1
+        for (int tl = wg; tl < T && ok; tl += 2) {
+          const int t = t_lo + tl, j = tl >> 1;
+          const bool full_tile = t < TP && (L - t * kBN) >= kBN;
+          ok = bounded_wait(lbar(PBars::kSFull + wg), j & 1, abort_flag, 9);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          if (tid == 128 && pass == 0 && j < 4) JET_TR(19 + 2 * j);
+          if (tid == 128 && pass == 0 && j == 8) JET_TR(36);
+          if (tid == 128 && pass == 0 && j == 16) JET_TR(37);
+          uint32_t xa[32], xb[32], xc[32], xd[32];
+          uint32_t b0 = 0xFFFFFFFFu, b1 = 0xFFFFFFFFu, b2 = 0xFFFFFFFFu, b3 = 0xFFFFFFFFu;
+          if (!full_tile) { b0 = chunk_bits(t, 0); b1 = chunk_bits(t, 1); b2 = chunk_bits(t, 2); b3 = chunk_bits(t, 3); }
+          saw_key = saw_key || (b0 | b1 | b2 | b3) != 0u;
+          ptx::tmem_ld32(tS, xa);
+          ptx::tmem_ld32(tS + 32, xb);
+          ptx::tmem_ld32(tS + 64, xc);
+          ptx::tmem_ld32(tS + 96, xd);
+          ptx::tmem_wait_ld();
+          ptx::tc_fence_before();
+          arrive_pair(lbar(PBars::kSFree + wg));            // the scores are in registers
+          if (tid == 128 && pass == 0 && j == 8) JET_TR(52);
+          if (!full_tile) {
+            mask_chunk(xa, b0);
+            mask_chunk(xb, b1);
+            mask_chunk(xc, b2);
+            mask_chunk(xd, b3);
+          }
+          if (mode == 1 || (mode == 0 && j == 0 && wg == 0)) {
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            max_chunk(xa, mx);
+            max_chunk(xb, mx);
+            max_chunk(xc, mx);
+            max_chunk(xd, mx);
+            m_run = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
+          }
+          if (mode == 1) continue;
+          if (mode == 0 && j == 0) {
+            // the reference of a row: its maximum over the first key tile (0 if it sees no key there)
+            if (wg == 0) {
+              m_ref = (m_run == -INFINITY) ? -0.0f : m_run * sl2;
+              if (T > 1) {
+                ref_s[r] = m_ref;
+                ptx::named_arrive(1, 256);
+              }
+            } else {
+              ptx::named_sync(1, 256);
+              m_ref = ref_s[r];
+            }
+            synced = true;
+          }
+          if (j > 0) {
+            ok = bounded_wait(lbar(PBars::kODone + wg), (j - 1) & 1, abort_flag, 21);
+            if (!ok) break;
+          }
+          if (tid == 128 && pass == 0 && j == 8) JET_TR(53);
+          float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          exp_chunk(xa, sl2, m_ref, sum, tP);
+          exp_chunk(xb, sl2, m_ref, sum, tP + 16);
+          exp_chunk(xc, sl2, m_ref, sum, tP + 32);
+          exp_chunk(xd, sl2, m_ref, sum, tP + 48);
+          const float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+          if (row_live && !(tile_sum <= kSharedSumLimit)) redo_flag[pass] = 1u;
+          l += tile_sum;
+          if (tid == 128 && pass == 0 && j == 8) JET_TR(54);
+          if (!full_tile) {
+            ok = clear_v_half(t, v_item(tl, kAhead));
+            if (!ok) break;
+          }
+          ptx::tmem_wait_st();                     // P is in TMEM
+          ptx::tc_fence_before();
+          arrive_pair(lbar(PBars::kPFull + wg));
+          if (tid == 128 && pass == 0 && j < 4) JET_TR(20 + 2 * j);
+          if (tid == 128 && pass == 0 && j == 8) JET_TR(55);
+        }
+        if (mode == 0) {
+          // (see the shared-accumulator form: a row without a reference of its own may have lost its keys to underflow)
+          if (row_live && saw_key && __float_as_uint(m_ref) == 0x80000000u && !(l >= kSharedSumFloor)) redo_flag[pass] = 1u;
+          if (T > 1 && !synced) {
+            if (wg == 0) ptx::named_arrive(1, 256);
+            else ptx::named_sync(1, 256);
+          }
+        } else if (mode == 1) {
+          // the row's true maximum over all keys of the slice, from both warpgroups
+          if (wg == 1) ref_s[r] = m_run;
+          ptx::named_sync(1, 256);
+          if (wg == 0) {
+            const float m = fmaxf(m_run, ref_s[r]);
+            m_ref = (m == -INFINITY) ? 0.0f : m * sl2;
+            ref_s[r] = m_ref;
+          }
+          ptx::named_sync(1, 256);
+          if (wg == 1) m_ref = ref_s[r];
+        }
+        if (mode != 1) {
+          if (ok) ok = bounded_wait(lbar(PBars::kOFinal), 0, abort_flag, 11);      // the last P V is complete
+          if (ok) ptx::tc_fence_after();
+        }
+        row_ok = ok;
+        const uint32_t verdict = pair_verdict(pass);
+#ifdef JET_TRACE
+        if (tid == 128 && p.trace) p.trace[(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) * 64 + 56 + pass] = 100 + verdict;
+#endif
+        if ((verdict & 2u) || pass == 2 || (pass == 0 && !(verdict & 1u))) break;
+        mode = pass + 1;
+      }
+      m_ref_common = m_ref;
+      classic = false;
+      shared_result = true;
+    } else if constexpr (MT == 1) {
       if (has_work) {
         // =========================================================== softmax, shared-accumulator form
         // Warpgroup wg takes key tiles wg, wg + 2, ...  A thread reads its whole score row from TMEM, hands
@@ -1463,7 +1873,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
 
-    if (!C::kTurns && classic && has_work && (MT == 1 || wg < n_mt)) {
+    if (!kPair && !C::kTurns && classic && has_work && (MT == 1 || wg < n_mt)) {
       // =========================================================== softmax, classic form
       bool ok = true;
       int last_tl = -1;
@@ -1601,7 +2011,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   ptx::tc_fence_before();
   ptx::cta_sync();
-  if (warp == 2) {
+  if constexpr (kPair) {
+    ptx::cluster_sync_all();       // the pair's TMEM is released together, once both CTAs are done with theirs
+    if (warp == 2) {
+      ptx::tc_fence_after();
+      ptx::tmem_dealloc2(tmem_base, C::kTmemCols);
+    }
+  } else if (warp == 2) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, C::kTmemCols);
   }
@@ -1767,22 +2183,23 @@ struct Plan {
   int units;       // work items before key slicing
   int nsplit;      // key slices
   int via_global;  // 1: slices exchange rows through the workspace (no cluster), 0: through a cluster
+  int pair;        // 1: CTA pairs (clusters of two CTAs with consecutive query tiles share the K/V tiles)
 };
 
 constexpr size_t kCounterBytes = 4096;     // head of the workspace: arrival / departure counters
 
-template <int D, int MT>
+template <int D, int MT, bool kPair = false>
 bool configure_kernel() {
   static std::atomic<int> states[kMaxDevices];      // per device: 0 = not yet, 1 = ok, -1 = failed
   std::atomic<int>& state_ref = states[current_device()];
   int state = state_ref.load(std::memory_order_acquire);
   if (state == 0) {
     auto set = [](auto kernel) {
-      return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D, MT>::kSmemBytes) ==
+      return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D, MT, kPair>::kSmemBytes) ==
                  cudaSuccess &&
              cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
     };
-    state = (set(tree_attn_kernel<D, MT, false>) && set(tree_attn_kernel<D, MT, true>))
+    state = (set(tree_attn_kernel<D, MT, false, kPair>) && set(tree_attn_kernel<D, MT, true, kPair>))
                 ? 1
                 : -1;
     if (state < 0) cudaGetLastError();
@@ -1837,6 +2254,11 @@ int max_active_clusters_for(int D, int mt, int cluster) {
 //   fixed cost of a CTA                6 (no slices), 8 (slices merged inside a cluster), 10 (through the
 //                                      workspace); 1.6 times that with two query tiles (two merge rounds)
 // and the CTAs run in waves of what the device holds at once.
+// Measured: a key tile costs a pair CTA 1800 cycles against 1475 for a CTA on its own (the hand-overs cross two SMs),
+// so the planner never prefers the pair form; JET_FORCE_PAIR=1 selects it.
+constexpr double kPairTile = 1.22;    // a pair CTA's key tile against a single CTA's
+constexpr double kPairFixed = 1.0;    // what a pair adds per CTA (cluster barriers at set-up, end of pass, teardown)
+
 Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   const int G = Hq / Hkv;
   const int rows = B * G;
@@ -1848,6 +2270,8 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   static const int force_mt = [] { const char* e = getenv("JET_FORCE_MT"); return e ? atoi(e) : 0; }();
   static const int force_ns = [] { const char* e = getenv("JET_FORCE_SPLIT"); return e ? atoi(e) : 0; }();
   // ",g": exchange inside the launch (counters and a bounded spin); ",h": exchange finished by a second launch
+  // JET_FORCE_PAIR: 1 = CTA pairs wherever the shape allows them, -1 = never
+  static const int force_pair = [] { const char* e = getenv("JET_FORCE_PAIR"); return e ? atoi(e) : 0; }();
   static const int force_via = [] {
     const char* e = getenv("JET_FORCE_SPLIT");
     return (e && strstr(e, ",g")) ? 1 : ((e && strstr(e, ",h")) ? 2 : 0);
@@ -1861,21 +2285,28 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
     const double shared = 1.0 + 0.75 / pl.n_mgroups;
     const double tile_cost = mt == 1 ? shared : (shared > 2.2 ? shared : 2.2);
     const double fixed_scale = mt == 1 ? 1.0 : 1.6;
-    auto consider = [&](int ns, int via_global, double waves, double fixed, double given_cost = -1.0) {
+    // CTA pairs: one 128-wide query tile per CTA, an even number of them per work item
+    const bool pair_ok = D == 128 && mt == 1 && pl.n_mgroups % 2 == 0;
+    auto consider = [&](int ns, int via_global, double waves, double fixed, double given_cost = -1.0, int pair = 0) {
       if (force_ns && (ns != force_ns || (ns > 1 && via_global != force_via))) return;
+      if (force_pair && (force_pair > 0) != (pair != 0) && (pair || pair_ok)) return;
       const double cost = given_cost >= 0.0 ? given_cost
-                                            : waves * (((tiles + ns - 1) / ns) * tile_cost + fixed * fixed_scale);
+                                            : waves * (((tiles + ns - 1) / ns) * tile_cost * (pair ? kPairTile : 1.0) +
+                                                       (fixed + (pair ? kPairFixed : 0.0)) * fixed_scale);
       if (best_cost < 0.0 || cost < best_cost) {
         best = pl;
         best.nsplit = ns;
         best.via_global = via_global;
+        best.pair = pair;
         best_cost = cost;
       }
     };
+
     for (int ns = 1; ns <= kMaxSplit && ns <= tiles; ++ns) {
       // (a) the slices of a unit form a thread-block cluster and merge through distributed shared memory
       const int resident = max_active_clusters_for(D, mt, ns);
       if (resident > 0) consider(ns, 0, static_cast<double>((pl.units + resident - 1) / resident), ns == 1 ? 6.0 : 8.0);
+      if (pair_ok && ns == 1) consider(1, 0, static_cast<double>((pl.units + sm_count() - 1) / sm_count()), 6.0, -1.0, 1);
       // (b) independent CTAs that merge through the workspace: all of them must be resident at once
       //     (a cluster has to fit into one GPC, which can leave a third of the SMs idle)
       //     -- either inside the launch (arrival counters, bounded spin), or with a second small launch that
@@ -1893,6 +2324,7 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
           consider(ns, via, 1.0, 0.0, ((tiles + ns - 1) / ns) * 0.75 + 0.125 * ns + 0.31 * (ns > 12 ? ns - 12 : 0) + 9.7);
         } else {
           consider(ns, via, 1.0, 10.0);
+          if (pair_ok) consider(ns, via, 1.0, 10.0, -1.0, 1);
         }
       }
     }
@@ -1903,6 +2335,7 @@ Plan make_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
     best.units = batch * Hkv * best.n_mgroups;
     best.nsplit = 1;
     best.via_global = 0;
+    best.pair = 0;
   }
   return best;
 }
@@ -1912,11 +2345,12 @@ size_t workspace_need(const Plan& pl, int D) {
   return kCounterBytes + static_cast<size_t>(pl.units) * pl.nsplit * pl.mt * kBM * (D * 2 + 16);
 }
 
-template <int D, int MT>
+template <int D, int MT, bool kPair = false>
 jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& ttk,
-                  const CUtensorMap& ttv, const AttnParams& p, const Plan& pl, cudaStream_t st) {
-  using C = Cfg<D, MT>;
-  if (!configure_kernel<D, MT>()) return JET_ERR_CUDA;
+                  const CUtensorMap& ttv, const CUtensorMap& tk64, const CUtensorMap& ttk64, const AttnParams& p,
+                  const Plan& pl, cudaStream_t st) {
+  using C = Cfg<D, MT, kPair>;
+  if (!configure_kernel<D, MT, kPair>()) return JET_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.n_mgroups * pl.nsplit, p.Hkv, p.batch);
   cfg.blockDim = dim3(C::kThreads);
@@ -1925,7 +2359,7 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   cudaLaunchAttribute attrs[2];
   int na = 0;
   attrs[na].id = cudaLaunchAttributeClusterDimension;
-  attrs[na].val.clusterDim.x = pl.via_global ? 1 : pl.nsplit;
+  attrs[na].val.clusterDim.x = kPair ? 2 : (pl.via_global ? 1 : pl.nsplit);
   attrs[na].val.clusterDim.y = 1;
   attrs[na].val.clusterDim.z = 1;
   ++na;
@@ -1937,8 +2371,9 @@ jet_status launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
   cfg.attrs = attrs;
   cfg.numAttrs = na;
   const bool sorted = p.batch > 1 && p.batch <= kMaxSorted;
-  const cudaError_t err = sorted ? cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, true>, tq, tk, tv, ttk, ttv, p)
-                                 : cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, false>, tq, tk, tv, ttk, ttv, p);
+  const cudaError_t err =
+      sorted ? cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, true, kPair>, tq, tk, tv, ttk, ttv, tk64, ttk64, p)
+             : cudaLaunchKernelEx(&cfg, tree_attn_kernel<D, MT, false, kPair>, tq, tk, tv, ttk, ttv, tk64, ttk64, p);
   if (err != cudaSuccess) {
 #ifdef JET_TRACE
     fprintf(stderr, "attention launch failed: %s (grid %d x %d x %d, cluster %d, %d slices, merge form %d, D %d, MT %d)\n",
@@ -1994,6 +2429,19 @@ extern "C" size_t jet_tree_verify_attn_workspace_bytes(int batch, int B, int Hq,
   return jet::workspace_need(jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len), D);
 }
 
+extern "C" int jet_tree_verify_attn_plan(int batch, int B, int Hq, int Hkv, int D, int max_seq_len, int32_t* plan) {
+  if (!plan || batch < 1 || batch > 65535 || B < 1 || Hq < 1 || Hkv < 1 || Hkv > 65535 || Hq % Hkv != 0 || max_seq_len < 0 ||
+      (D != 64 && D != 128))
+    return 0;
+  const jet::Plan pl = jet::make_plan(batch, B, Hq, Hkv, D, max_seq_len);
+  plan[0] = pl.mt;
+  plan[1] = pl.n_mgroups;
+  plan[2] = pl.nsplit;
+  plan[3] = pl.nsplit > 1 ? (pl.via_global == 0 ? 1 : pl.via_global + 1) : 0;     // 0 none, 1 cluster, 2 workspace in one launch, 3 second launch
+  plan[4] = pl.pair;
+  return 1;
+}
+
 extern "C" int jet_tree_verify_attn_launches(int batch, int B, int Hq, int Hkv, int D, int max_seq_len) {
   if (batch < 1 || batch > 65535 || B < 1 || Hq < 1 || Hkv < 1 || Hkv > 65535 || Hq % Hkv != 0 || max_seq_len < 0 ||
       (D != 64 && D != 128))
@@ -2037,7 +2485,7 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < workspace_need(pl, D)) return JET_ERR_WORKSPACE;
 
   // ---- tensor maps (bf16, 128-byte swizzle, 64-element inner box)
-  CUtensorMap tq = {}, tk = {}, tv = {}, ttk = {}, ttv = {};     // (maps a call does not use stay zeroed)
+  CUtensorMap tq = {}, tk = {}, tv = {}, ttk = {}, ttv = {}, tk64 = {}, ttk64 = {};     // (maps a call does not use stay zeroed; the last two: K with boxes of 64 rows, for CTA pairs)
   const uint64_t eb = 2;
   {
     const uint64_t dims[4] = {static_cast<uint64_t>(D), static_cast<uint64_t>(G), static_cast<uint64_t>(Hkv),
@@ -2051,12 +2499,15 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
                               static_cast<uint64_t>(batch)};
     const uint64_t str[3] = {D * eb, static_cast<uint64_t>(Hkv) * D * eb, static_cast<uint64_t>(B) * Hkv * D * eb};
     const uint32_t box[4] = {64, 1, kBN, 1};
+    const uint32_t box64[4] = {64, 1, 64, 1};
     if (!make_map(&ttk, tree_k, 4, dims, str, box) || !make_map(&ttv, tree_v, 4, dims, str, box))
       return JET_ERR_CUDA;
+    if (pl.pair && !make_map(&ttk64, tree_k, 4, dims, str, box64)) return JET_ERR_CUDA;
   }
   if (max_seq_len == 0) {
     tk = ttk;   // never dereferenced: there are no prefix tiles
     tv = ttv;
+    tk64 = ttk64;
   } else if (paged) {
     const uint64_t dims[3] = {static_cast<uint64_t>(D), static_cast<uint64_t>(Hkv),
                               static_cast<uint64_t>(num_pages) * 16};
@@ -2071,9 +2522,13 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
                               static_cast<uint64_t>(max_seq_len), static_cast<uint64_t>(batch)};
     const uint64_t str[3] = {D * eb, static_cast<uint64_t>(Hkv) * D * eb, bstride * eb};
     const uint32_t box[4] = {64, 1, kBN, 1};
+    const uint32_t box64[4] = {64, 1, 64, 1};
     if (!make_map(&tk, k_cache, 4, dims, str, box) || !make_map(&tv, v_cache, 4, dims, str, box))
       return JET_ERR_CUDA;
+    if (pl.pair && !make_map(&tk64, k_cache, 4, dims, str, box64)) return JET_ERR_CUDA;
   }
+  if (!pl.pair || paged) tk64 = tk;        // (unused: a paged tile is fetched page by page)
+  if (!pl.pair || tail) ttk64 = tail ? tk64 : ttk;
 
   AttnParams p;
   p.page_table = page_table;
@@ -2095,7 +2550,7 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
   p.magic_S = udiv_magic(static_cast<uint32_t>(pl.nsplit));
   p.magic_G = udiv_magic(static_cast<uint32_t>(G));
   // (measured: a gain of 3-9 % with one query tile per KV head, none to a small loss with two or more)
-  p.len_hint = (!paged && !tail && batch == 1 && pl.n_mgroups == 1 && max_seq_len > 0 && max_seq_len < (1 << 26)) ? max_seq_len : 0;
+  p.len_hint = (!pl.pair && !paged && !tail && batch == 1 && pl.n_mgroups == 1 && max_seq_len > 0 && max_seq_len < (1 << 26)) ? max_seq_len : 0;
   p.stable = (flags & JET_ATTN_STABLE_PREFIX) ? 1 : 0;
   // Test hook (read once per process): JET_TEST_POLL_LIMIT shortens the bounded spin of the workspace merge so
   // that a test can make it run out within milliseconds.
@@ -2118,10 +2573,11 @@ jet_status attn_call(const void* q, const void* k_cache, const void* v_cache, co
     ttv = tv;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (D == 128) return pl.mt == 1 ? launch<128, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
-                                  : launch<128, 2>(tq, tk, tv, ttk, ttv, p, pl, st);
-  return pl.mt == 1 ? launch<64, 1>(tq, tk, tv, ttk, ttv, p, pl, st)
-                    : launch<64, 2>(tq, tk, tv, ttk, ttv, p, pl, st);
+  if (pl.pair) return launch<128, 1, true>(tq, tk, tv, ttk, ttv, tk64, ttk64, p, pl, st);
+  if (D == 128) return pl.mt == 1 ? launch<128, 1>(tq, tk, tv, ttk, ttv, tk64, ttk64, p, pl, st)
+                                  : launch<128, 2>(tq, tk, tv, ttk, ttv, tk64, ttk64, p, pl, st);
+  return pl.mt == 1 ? launch<64, 1>(tq, tk, tv, ttk, ttv, tk64, ttk64, p, pl, st)
+                    : launch<64, 2>(tq, tk, tv, ttk, ttv, tk64, ttk64, p, pl, st);
 }
 
 }  // namespace

@@ -294,6 +294,41 @@ def test_every_kind_of_launch_plan(mt, split):
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
 
+def test_cta_pair_form():
+    """The CTA-pair form of the key loop (consecutive query tiles of a work item on two SMs that share every K/V
+    tile through tcgen05 cta_group::2): never the planner's choice, so it is forced in a child process, where the
+    plan query must report it and the benchmark-shape, tile-boundary, tree-shape, padding, adversarial-score and
+    ragged paged batch tests must pass with it."""
+    import os
+    import subprocess
+    import sys
+    if os.environ.get("JET_FORCE_SPLIT") or os.environ.get("JET_FORCE_MT") or os.environ.get("JET_FORCE_PAIR"):
+        pytest.skip("already inside a forced run")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, JET_FORCE_MT="1", JET_FORCE_PAIR="1")
+    code = ("import paper_2606_18394_b200 as jet\n"
+            "p = jet.jet_tree_verify_attn_plan(1, 64, 32, 8, 128, 4096)\n"
+            "assert p['pair'] and p['query_tiles_per_cta'] == 1, p\n"
+            "q = jet.jet_tree_verify_attn_plan(1, 16, 32, 8, 128, 4096)\n"
+            "assert not q['pair'], q\n")           # one query tile per KV head: nothing to pair
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    r = subprocess.run([sys.executable, "-m", "pytest", __file__, "-m", "gpu", "-x", "-q", "-k",
+                        "qwen3_8b_config or tile_boundaries or tree_shapes or padding_nodes or very_negative or "
+                        "far_above or batched_paged_ragged or sweep_16k"],
+                       env=env, capture_output=True, text=True, cwd=root, timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_the_planner_never_picks_the_pair_form():
+    import paper_2606_18394_b200 as jet
+    import os
+    if os.environ.get("JET_FORCE_PAIR"):
+        pytest.skip("inside a forced run")
+    for B, L in ((64, 4096), (128, 4096), (256, 16384), (512, 32768)):
+        assert not jet.jet_tree_verify_attn_plan(1, B, 32, 8, 128, L)["pair"]
+
+
 def test_sweep_16k_sampled_rows():
     """Long prefix (sweep shape, B=128): the oracle checks a seeded sample of (node, head) rows."""
     import jet_harness as H
