@@ -26,6 +26,9 @@
 //                 memory when the slices form a thread-block cluster, else through the workspace -- combine
 //                 the slices and write the output.  With few rows and many slices the combination is left
 //                 to a second, small launch (tree_attn_merge_kernel) instead.
+//   CTA pairs   = an optional form (JET_FORCE_PAIR=1; measured slower, never the planner's choice): two CTAs with
+//                 consecutive query tiles of a work item form a cluster, each loads half of every K/V tile and
+//                 the products run as tcgen05 cta_group::2 instructions.  See "CTA pairs" in the kernel.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
 // loops (still taking part in the CTA-wide and cluster barriers), outstanding TMA loads are drained,
 // TMEM is released and JET_ERR_TIMEOUT is reported.
